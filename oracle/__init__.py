@@ -1,0 +1,175 @@
+"""CPU oracle for the Re-SpS speculative step -- TEST INFRASTRUCTURE, NOT THE PRODUCT.
+
+Thin numpy/ctypes wrapper over ``resps_oracle.cpp`` (single-threaded fp64 C++).
+Only tests, the smoke check and the benchmark's CPU-baseline leg may import this
+package; the CUDA library never does, and the two share no code.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from dataclasses import dataclass
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "resps_oracle.cpp")
+_LIB = os.path.join(_HERE, "libresps_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with g++ (-O2, no OpenMP, no SIMD flags)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".tmp{os.getpid()}"
+        subprocess.check_call(["g++", "-O2", "-std=c++17", "-shared", "-fPIC", _SRC, "-o", tmp])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+    return _lib
+
+
+def _p(a: np.ndarray):
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _c(a, dtype):
+    a = np.ascontiguousarray(a, dtype=dtype)
+    return a
+
+
+def topk_lse(row: np.ndarray, k: int):
+    """Top-k (value desc, id asc) and log-sum-exp of one fp32 row."""
+    row = _c(row, np.float32)
+    V = row.shape[0]
+    val = np.empty(k, np.float32)
+    idx = np.empty(k, np.int32)
+    lse = ctypes.c_double()
+    rc = _load().oracle_topk_lse(_p(row), V, k, _p(val), _p(idx), ctypes.byref(lse))
+    if rc != 0:
+        raise ValueError(f"oracle_topk_lse rc={rc}")
+    return val, idx, lse.value
+
+
+@dataclass
+class Tree:
+    tokens: np.ndarray        # int32 [n]
+    parent: np.ndarray        # int32 [n], root -1
+    depth: np.ndarray         # int32 [n]
+    position_ids: np.ndarray  # int32 [n]
+    mask: np.ndarray          # uint64 [n, 2]
+    retrieve: np.ndarray      # int32 [n_leaves, ret_stride]
+    n_nodes: int
+    n_leaves: int
+    cand_score: np.ndarray    # float64 [n_cand]
+    cand_token: np.ndarray    # int32 [n_cand]
+    cand_parent: np.ndarray   # int32 [n_cand], -1 = root
+    frontier: np.ndarray      # int32 [d, k]: candidates expanded after each level
+    min_gap: float
+
+
+def tree_expand(root_token: int, logits: np.ndarray, TT: int, d: int, k: int, L: int,
+                max_tt: int = 128, ret_stride: int | None = None) -> Tree:
+    """Draft-tree construction. ``logits`` is fp32 [>=d][>=k][V]; level 0 uses slot 0."""
+    logits = _c(logits, np.float32)
+    assert logits.ndim == 3 and logits.shape[0] >= d and (d == 1 or logits.shape[1] >= k)
+    V = logits.shape[2]
+    ld_level = logits.shape[1] * V
+    ld_row = V
+    if ret_stride is None:
+        ret_stride = d + 1
+    n_cand = k + (d - 1) * k * k
+    tokens = np.full(max_tt, -1, np.int32)
+    parent = np.full(max_tt, -1, np.int32)
+    depth = np.full(max_tt, -1, np.int32)
+    pos = np.full(max_tt, -1, np.int32)
+    mask = np.zeros((max_tt, 2), np.uint64)
+    retrieve = np.full((max_tt, ret_stride), -1, np.int32)
+    n_leaves = ctypes.c_int32()
+    n_nodes = ctypes.c_int32()
+    cand = np.zeros(n_cand, np.float64)
+    ctok = np.zeros(n_cand, np.int32)
+    cpar = np.zeros(n_cand, np.int32)
+    frontier = np.zeros((d, k), np.int32)
+    gap = ctypes.c_double()
+    rc = _load().oracle_tree_expand(
+        ctypes.c_int32(int(root_token)), _p(logits), ctypes.c_int64(ld_level), ctypes.c_int64(ld_row),
+        V, TT, d, k, L, max_tt, ret_stride, _p(tokens), _p(parent), _p(depth), _p(pos), _p(mask),
+        _p(retrieve), ctypes.byref(n_leaves), ctypes.byref(n_nodes), _p(cand), _p(ctok), _p(cpar),
+        _p(frontier), ctypes.byref(gap))
+    if rc != 0:
+        raise ValueError(f"oracle_tree_expand rc={rc}")
+    n = n_nodes.value
+    return Tree(tokens[:n], parent[:n], depth[:n], pos[:n], mask[:n], retrieve[:n_leaves.value],
+                n, n_leaves.value, cand, ctok, cpar, frontier, gap.value)
+
+
+def tree_attention(q: np.ndarray, k_cache: np.ndarray, v_cache: np.ndarray, L: int,
+                   mask: np.ndarray, scale: float, want_lse: bool = False):
+    """q: uint16(bf16 bits) [n][Hq][D]; caches uint16 [Hkv][cap][D]; mask uint64 [n][2].
+    Returns fp64 [n][Hq][D] (and lse [n][Hq])."""
+    q = _c(q, np.uint16)
+    k_cache = _c(k_cache, np.uint16)
+    v_cache = _c(v_cache, np.uint16)
+    mask = _c(mask, np.uint64)
+    n, Hq, D = q.shape
+    Hkv, cap, D2 = k_cache.shape
+    assert D2 == D and v_cache.shape == k_cache.shape and mask.shape == (n, 2)
+    assert L + n <= cap
+    out = np.empty((n, Hq, D), np.float64)
+    lse = np.empty((n, Hq), np.float64) if want_lse else None
+    rc = _load().oracle_tree_attention(
+        n, Hq, Hkv, D, L, _p(q), _p(k_cache), _p(v_cache), ctypes.c_int64(cap * D),
+        ctypes.c_int64(D), _p(mask), ctypes.c_double(scale), _p(out),
+        _p(lse) if want_lse else None)
+    if rc != 0:
+        raise ValueError(f"oracle_tree_attention rc={rc}")
+    return (out, lse) if want_lse else out
+
+
+@dataclass
+class Accept:
+    target_argmax: np.ndarray  # int32 [n]
+    path: np.ndarray           # int32 [a+1]
+    accept_len: int
+    out_tokens: np.ndarray     # int32 [a+1]
+
+
+def verify_accept(target_logits: np.ndarray, tokens: np.ndarray, parent: np.ndarray,
+                  path_cap: int = 17) -> Accept:
+    target_logits = _c(target_logits, np.float32)
+    tokens = _c(tokens, np.int32)
+    parent = _c(parent, np.int32)
+    n, V = target_logits.shape
+    assert tokens.shape[0] >= n and parent.shape[0] >= n
+    tgt = np.empty(n, np.int32)
+    path = np.empty(path_cap, np.int32)
+    out = np.empty(path_cap, np.int32)
+    a = ctypes.c_int32()
+    rc = _load().oracle_verify_accept(n, V, _p(target_logits), ctypes.c_int64(V), _p(tokens),
+                                      _p(parent), path_cap, _p(tgt), _p(path), ctypes.byref(a),
+                                      _p(out))
+    if rc != 0:
+        raise ValueError(f"oracle_verify_accept rc={rc}")
+    return Accept(tgt, path[:a.value + 1].copy(), a.value, out[:a.value + 1].copy())
+
+
+def kv_compact(k_cache: np.ndarray, v_cache: np.ndarray, L: int, path: np.ndarray) -> int:
+    """In-place on the given uint16 [Hkv][cap][D] arrays (via an internal copy). Returns L'."""
+    assert k_cache.dtype == np.uint16 and v_cache.dtype == np.uint16
+    assert k_cache.flags.c_contiguous and v_cache.flags.c_contiguous
+    Hkv, cap, D = k_cache.shape
+    path = _c(path, np.int32)
+    a = path.shape[0] - 1
+    rc = _load().oracle_kv_compact(Hkv, D, L, _p(path), a, _p(k_cache), _p(v_cache),
+                                   ctypes.c_int64(cap * D), ctypes.c_int64(D),
+                                   ctypes.c_int64(k_cache.size))
+    if rc != 0:
+        raise ValueError(f"oracle_kv_compact rc={rc}")
+    return L + a + 1
