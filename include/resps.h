@@ -1,0 +1,203 @@
+/*
+ * resps.h -- C ABI of libresps: the per-step speculative-sampling hot path that
+ * Re-SpS controls by re-choosing (TT, d, k) at every step.
+ *
+ * One speculative step is
+ *   resps_tree_expand     draft-tree construction
+ *   resps_tree_attention  tree-masked verification attention (once per layer)
+ *   resps_verify_accept   per-node target argmax + longest accepted path
+ *   resps_kv_compact      in-place KV-cache compaction of the accepted path
+ *
+ * General conventions
+ *  - Every pointer named d_* or documented as DEVICE points to memory of the
+ *    current CUDA device; every other pointer is HOST memory.
+ *  - The caller owns every buffer it passes.  A context owns only its private
+ *    device workspace (partial results, counters, a status word).
+ *  - No hot call allocates, synchronises or reads device memory on the host:
+ *    each only enqueues kernels on `stream`.  The per-step values (TT, d, k,
+ *    prefix length, node counts) are read by the kernels from device memory,
+ *    so they may change between calls -- or between replays of a captured CUDA
+ *    graph -- without re-capture or recompilation.
+ *  - A context serialises its workspace: calls on the same context must be
+ *    ordered on one stream (or otherwise not overlap on the GPU).
+ *  - Return value: RESPS_OK (0) or a negative RESPS_ERR_* code.  Argument
+ *    errors are detected on the host before anything is enqueued.  Conditions
+ *    only visible on the device (a step whose k exceeds the logits extent, a
+ *    prefix that overruns the cache, ...) set bits in the context's device
+ *    status word, which resps_status() copies back; the affected sequence is
+ *    then processed with its parameters clamped into range.
+ *  - Limits follow the paper's action space (Appendix A): TT <= 128, k <= 32,
+ *    d <= 16.  TT, d, k are upper limits (the action space of Eq. 2): a tree
+ *    has n = min(TT, 1 + k + (d-1) k^2) nodes, never an error.
+ */
+#ifndef RESPS_H_
+#define RESPS_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define RESPS_MAX_TT 128
+#define RESPS_MAX_K 32
+#define RESPS_MAX_DEPTH 16
+
+enum {
+    RESPS_OK = 0,
+    RESPS_ERR_INVALID_ARG = -1,       /* null pointer, non-positive size, misaligned buffer   */
+    RESPS_ERR_UNSUPPORTED_SHAPE = -2, /* head_dim not 64/128, Hq % Hkv != 0, limits exceeded  */
+    RESPS_ERR_CAPACITY = -3,          /* host-known: max_tt > kv_capacity, batch > max_batch  */
+    RESPS_ERR_CUDA = -4,              /* a CUDA runtime call or launch failed                 */
+    RESPS_ERR_NO_DEVICE = -5          /* no usable sm_100 device                              */
+};
+
+/* Bits of the device status word (resps_status). */
+enum {
+    RESPS_STATUS_STEP_CLAMPED = 1,   /* a step's tt/d/k was outside the supplied extents       */
+    RESPS_STATUS_KV_OVERFLOW = 2,    /* prefix_len + n exceeds kv_capacity (the KV-cache       */
+                                     /* overflow the paper's results section warns of); skipped */
+    RESPS_STATUS_WAIT_TIMEOUT = 4    /* a bounded device-side wait gave up                     */
+};
+
+typedef struct resps_ctx resps_ctx;      /* opaque */
+typedef struct CUstream_st* resps_stream; /* a cudaStream_t */
+
+/* Model shape and library limits, fixed per context. */
+typedef struct {
+    int32_t n_q_heads;  /* Hq                                               */
+    int32_t n_kv_heads; /* Hkv, divides Hq                                  */
+    int32_t head_dim;   /* D: 64 or 128                                     */
+    int32_t vocab;      /* V                                                */
+    int32_t max_batch;  /* sequences per call                               */
+    int32_t max_tt;     /* <= RESPS_MAX_TT; row stride of all per-node arrays */
+    int32_t max_k;      /* <= RESPS_MAX_K                                   */
+    int32_t max_depth;  /* <= RESPS_MAX_DEPTH; retrieve / path rows hold max_depth+1 entries */
+} resps_shape;
+
+/* Per-sequence, per-step parameters (Eq. 2: the action (TT, d, k)); lives in DEVICE memory. */
+typedef struct {
+    int32_t tt;         /* total tree tokens including the root, >= 1       */
+    int32_t d;          /* draft levels (node depths 1..d), >= 1            */
+    int32_t k;          /* expansion top-k, 1 <= k <= min(V, max_k)         */
+    int32_t prefix_len; /* L: tokens already in the KV cache                */
+} resps_step;
+
+/* Creates a context on the current device and allocates its workspace (the only
+ * allocation the library performs).  Errors: INVALID_ARG, UNSUPPORTED_SHAPE,
+ * NO_DEVICE, CUDA. */
+int resps_create(resps_ctx** out, const resps_shape* shape);
+/* Frees the workspace.  The caller must have synchronised all work using it. */
+int resps_destroy(resps_ctx* ctx);
+/* Static string for a return code. */
+const char* resps_strerror(int code);
+/* Synchronises `stream`, copies the device status word to *status and clears it. */
+int resps_status(resps_ctx* ctx, resps_stream stream, int32_t* status);
+/* Bytes of device workspace held by the context. */
+int64_t resps_workspace_bytes(const resps_ctx* ctx);
+
+/*
+ * Draft-tree construction (Section 3.2, "Draft Tree Expansion" and "Confidence-Based
+ * Candidate Reranking"; Algorithm 2, tree-building loop and rerank).
+ *
+ * For every sequence b < batch, with (TT, d, k, L) = d_steps[b]:
+ *   level 0: the k most probable tokens of row logits[b][0][0] become candidates 0..k-1
+ *     (children of the root) with score log p;
+ *   level j = 1..d-1: row logits[b][j][p] is the draft distribution after the p-th
+ *     frontier node; its k most probable tokens become candidates
+ *     c = k + (j-1) k^2 + p k + r with score = score(parent) + log p; the k best
+ *     candidates of the level (score desc, candidate index asc) form the next frontier;
+ *   rerank: the min(TT-1, n_cand) best of all candidates are kept and, in ascending
+ *     candidate order, become nodes 1..n-1 behind the root (node 0).
+ * Token order inside a row: value desc, token id asc.  log p = x - logsumexp(row).
+ *
+ * d_draft_logits  DEVICE fp32, element (b, level, slot, v) at
+ *                 b*ld_b + level*ld_level + slot*ld_row + v; extents n_levels x n_slots
+ *                 (level 0 uses slot 0 only).  16-byte aligned base and strides that are
+ *                 multiples of 4 elements select the vectorised path.
+ * d_root_token    DEVICE int32 [batch]
+ * Outputs, DEVICE, row stride max_tt per sequence, entries >= n untouched:
+ *   tokens, parent (root -1), depth, position_ids (= L + depth)   int32 [batch][max_tt]
+ *   mask       uint64 [batch][max_tt][2]: bit j <=> node j is the node or an ancestor
+ *   retrieve   int32 [batch][max_tt][max_depth+1]: one row per leaf in ascending leaf
+ *              order, root-to-leaf node indices, -1 padded; rows >= n_leaves untouched
+ *   n_leaves, n_nodes  int32 [batch]
+ * A step with d > n_levels or k > n_slots (or k > V, or tt > max_tt) is clamped and
+ * RESPS_STATUS_STEP_CLAMPED is set.
+ */
+int resps_tree_expand(resps_ctx* ctx, const resps_step* d_steps, int batch,
+                      const float* d_draft_logits, int64_t ld_b, int64_t ld_level, int64_t ld_row,
+                      int n_levels, int n_slots, const int32_t* d_root_token,
+                      int32_t* d_tokens, int32_t* d_parent, int32_t* d_depth,
+                      int32_t* d_position_ids, uint64_t* d_mask, int32_t* d_retrieve,
+                      int32_t* d_n_leaves, int32_t* d_n_nodes, resps_stream stream);
+
+/*
+ * Tree-masked verification attention for one layer (Section 3.2, "Verification Phase":
+ * the target model scores all tree tokens in a single pass; Appendix D: attention masks
+ * follow the tree).
+ *
+ * For sequence b with L = d_steps[b].prefix_len and n = d_n_nodes[b], node t < n, head h:
+ *   O[t,h] = sum_j softmax_j(scale * q[t,h] . K[g,j]) V[g,j],   g = h / (Hq/Hkv),
+ * over cache slots j in [0, L) and slots L+i for every set bit i of mask[b][t].
+ * The tree tokens' K/V must already be stored at slots L .. L+n-1.  No other slot
+ * influences the result.
+ *
+ * d_q, d_o     DEVICE bf16 [batch][max_tt][Hq][D]; rows >= n are neither read nor written
+ * d_lse        DEVICE fp32 [batch][max_tt][Hq] or NULL: natural-log sum of exp of the scaled scores
+ * d_k_cache, d_v_cache  DEVICE bf16; element (b, g, slot, e) at
+ *              b*kv_stride_seq + g*kv_stride_head + slot*kv_stride_tok + e  (elements);
+ *              16-byte aligned, strides multiples of 8 elements
+ * kv_capacity  slots per (sequence, head); a sequence with L + n > kv_capacity is skipped
+ *              and RESPS_STATUS_KV_OVERFLOW set
+ * d_mask       as written by resps_tree_expand
+ * Accumulation is fp32; the result is rounded to bf16 once.
+ */
+int resps_tree_attention(resps_ctx* ctx, const resps_step* d_steps, const int32_t* d_n_nodes,
+                         int batch, const void* d_q, void* d_o, float* d_lse,
+                         const void* d_k_cache, const void* d_v_cache, int64_t kv_stride_seq,
+                         int64_t kv_stride_head, int64_t kv_stride_tok, int64_t kv_capacity,
+                         const uint64_t* d_mask, float softmax_scale, resps_stream stream);
+
+/*
+ * Greedy verification and acceptance (Section 3.1: greedy decoding; Section 3.2,
+ * "Acceptance Criterion" at temperature 0 -- a draft token is accepted iff it equals the
+ * target's argmax after its parent; Algorithm 2, "get accepted tokens").
+ *
+ * d_target_logits  DEVICE fp32, element (b, i, v) at b*ld_b + i*ld_row + v: the target
+ *                  distribution after tree node i
+ * d_tokens, d_parent  from resps_tree_expand
+ * Outputs, DEVICE:
+ *   d_target_argmax int32 [batch][max_tt]   argmax per node, ties -> lowest id
+ *   d_accept_path   int32 [batch][max_depth+1]  node indices, path[0] = 0, unused -1
+ *   d_accept_len    int32 [batch]           a = accepted draft tokens
+ *   d_out_tokens    int32 [batch][max_depth+1]  the a accepted tokens then the bonus token
+ *                                           (target argmax at the last accepted node), unused -1
+ *   d_steps_next    resps_step [batch] or NULL: copy of d_steps with prefix_len += a+1
+ *                   (may alias d_steps)
+ */
+int resps_verify_accept(resps_ctx* ctx, const resps_step* d_steps, const int32_t* d_n_nodes,
+                        int batch, const float* d_target_logits, int64_t ld_b, int64_t ld_row,
+                        const int32_t* d_tokens, const int32_t* d_parent,
+                        int32_t* d_target_argmax, int32_t* d_accept_path, int32_t* d_accept_len,
+                        int32_t* d_out_tokens, resps_step* d_steps_next, resps_stream stream);
+
+/*
+ * In-place KV-cache compaction (Appendix D, "input update": rejected tokens are discarded
+ * from the cache).  For every bound layer, KV head and j = 0..a:
+ *   slot L+j  <-  slot L+path[j]     (K and V),   L = d_steps[b].prefix_len (before the step).
+ * Slots beyond L+a are left as they are.
+ *
+ * d_k_caches, d_v_caches  DEVICE arrays of n_layers DEVICE pointers (bf16 caches laid out as
+ *                         in resps_tree_attention)
+ */
+int resps_kv_compact(resps_ctx* ctx, const resps_step* d_steps, int batch,
+                     const int32_t* d_accept_path, const int32_t* d_accept_len,
+                     void* const* d_k_caches, void* const* d_v_caches, int n_layers,
+                     int64_t kv_stride_seq, int64_t kv_stride_head, int64_t kv_stride_tok,
+                     resps_stream stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RESPS_H_ */

@@ -1,0 +1,184 @@
+"""ctypes binding of libresps.so: the same entry points as include/resps.h, taking torch
+tensors (device memory) and doing argument marshalling only -- every step of the path runs
+in the library's CUDA kernels.  There is no CPU fallback: if the shared library cannot be
+loaded, importing a symbol from here raises."""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libresps.so")
+
+RESPS_OK = 0
+RESPS_ERR_INVALID_ARG = -1
+RESPS_ERR_UNSUPPORTED_SHAPE = -2
+RESPS_ERR_CAPACITY = -3
+RESPS_ERR_CUDA = -4
+RESPS_ERR_NO_DEVICE = -5
+RESPS_STATUS_STEP_CLAMPED = 1
+RESPS_STATUS_KV_OVERFLOW = 2
+RESPS_STATUS_WAIT_TIMEOUT = 4
+
+EXPORTS = ("resps_create", "resps_destroy", "resps_strerror", "resps_status",
+           "resps_workspace_bytes", "resps_tree_expand", "resps_tree_attention",
+           "resps_verify_accept", "resps_kv_compact")
+
+
+class RespsShape(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in
+                ("n_q_heads", "n_kv_heads", "head_dim", "vocab", "max_batch", "max_tt", "max_k",
+                 "max_depth")]
+
+
+class RespsError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {strerror(code)} ({code})")
+
+
+_lib = None
+
+
+def load() -> ctypes.CDLL:
+    """Loads libresps.so (built in-tree by paper_2601_12212_b200.build); raises if absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: run `python -m paper_2601_12212_b200.build` "
+                          "(there is no fallback path)")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i32, i64, f32 = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_float
+    lib.resps_create.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(RespsShape)]
+    lib.resps_destroy.argtypes = [vp]
+    lib.resps_strerror.argtypes = [i32]
+    lib.resps_strerror.restype = ctypes.c_char_p
+    lib.resps_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int32)]
+    lib.resps_workspace_bytes.argtypes = [vp]
+    lib.resps_workspace_bytes.restype = i64
+    lib.resps_tree_expand.argtypes = [vp, vp, i32, vp, i64, i64, i64, i32, i32, vp,
+                                      vp, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.resps_tree_attention.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp, vp, i64, i64, i64, i64,
+                                         vp, f32, vp]
+    lib.resps_verify_accept.argtypes = [vp, vp, vp, i32, vp, i64, i64, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.resps_kv_compact.argtypes = [vp, vp, i32, vp, vp, vp, vp, i32, i64, i64, i64, vp]
+    for name in EXPORTS:
+        if name not in ("resps_strerror", "resps_workspace_bytes"):
+            getattr(lib, name).restype = i32
+    _lib = lib
+    return lib
+
+
+def strerror(code: int) -> str:
+    return load().resps_strerror(int(code)).decode()
+
+
+def _ptr(t: Optional[torch.Tensor], dtype=None) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError("expected a CUDA tensor")
+    if not t.is_contiguous():
+        raise ValueError("expected a contiguous tensor")
+    if dtype is not None and t.dtype != dtype:
+        raise ValueError(f"expected dtype {dtype}, got {t.dtype}")
+    return t.data_ptr()
+
+
+def _stream(stream: Optional[torch.cuda.Stream]) -> int:
+    return (stream or torch.cuda.current_stream()).cuda_stream
+
+
+def _check(rc: int, where: str) -> None:
+    if rc != RESPS_OK:
+        raise RespsError(rc, where)
+
+
+class Context:
+    """Owns a resps_ctx (the library workspace) for one model shape on the current device."""
+
+    def __init__(self, n_q_heads: int, n_kv_heads: int, head_dim: int, vocab: int,
+                 max_batch: int = 1, max_tt: int = 128, max_k: int = 32, max_depth: int = 8):
+        self.shape = RespsShape(n_q_heads, n_kv_heads, head_dim, vocab, max_batch, max_tt, max_k,
+                                max_depth)
+        self._h = ctypes.c_void_p()
+        _check(load().resps_create(ctypes.byref(self._h), ctypes.byref(self.shape)), "resps_create")
+
+    @property
+    def handle(self):
+        return self._h
+
+    def workspace_bytes(self) -> int:
+        return int(load().resps_workspace_bytes(self._h))
+
+    def status(self, stream=None) -> int:
+        out = ctypes.c_int32()
+        _check(load().resps_status(self._h, _stream(stream), ctypes.byref(out)), "resps_status")
+        return out.value
+
+    def close(self):
+        if self._h:
+            load().resps_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+STEP_DTYPE = torch.int32  # resps_step = 4 x int32 (tt, d, k, prefix_len): tensors of shape [batch, 4]
+
+
+def resps_tree_expand(ctx: Context, steps, batch: int, draft_logits, ld_b: int, ld_level: int,
+                      ld_row: int, n_levels: int, n_slots: int, root_token, tokens, parent, depth,
+                      position_ids, mask, retrieve, n_leaves, n_nodes, stream=None) -> None:
+    i32 = torch.int32
+    _check(load().resps_tree_expand(
+        ctx.handle, _ptr(steps, i32), batch, _ptr(draft_logits, torch.float32), ld_b, ld_level, ld_row,
+        n_levels, n_slots, _ptr(root_token, i32), _ptr(tokens, i32), _ptr(parent, i32),
+        _ptr(depth, i32), _ptr(position_ids, i32), _ptr(mask), _ptr(retrieve, i32),
+        _ptr(n_leaves, i32), _ptr(n_nodes, i32), _stream(stream)), "resps_tree_expand")
+
+
+def resps_tree_attention(ctx: Context, steps, n_nodes, batch: int, q, o, lse, k_cache, v_cache,
+                         kv_stride_seq: int, kv_stride_head: int, kv_stride_tok: int,
+                         kv_capacity: int, mask, softmax_scale: float, stream=None) -> None:
+    i32, bf = torch.int32, torch.bfloat16
+    _check(load().resps_tree_attention(
+        ctx.handle, _ptr(steps, i32), _ptr(n_nodes, i32), batch, _ptr(q, bf), _ptr(o, bf),
+        _ptr(lse, torch.float32), _ptr(k_cache, bf), _ptr(v_cache, bf), kv_stride_seq, kv_stride_head,
+        kv_stride_tok, kv_capacity, _ptr(mask), float(softmax_scale), _stream(stream)),
+        "resps_tree_attention")
+
+
+def resps_verify_accept(ctx: Context, steps, n_nodes, batch: int, target_logits, ld_b: int,
+                        ld_row: int, tokens, parent, target_argmax, accept_path, accept_len,
+                        out_tokens, steps_next=None, stream=None) -> None:
+    i32 = torch.int32
+    _check(load().resps_verify_accept(
+        ctx.handle, _ptr(steps, i32), _ptr(n_nodes, i32), batch, _ptr(target_logits, torch.float32),
+        ld_b, ld_row, _ptr(tokens, i32), _ptr(parent, i32), _ptr(target_argmax, i32),
+        _ptr(accept_path, i32), _ptr(accept_len, i32), _ptr(out_tokens, i32), _ptr(steps_next, i32),
+        _stream(stream)), "resps_verify_accept")
+
+
+def resps_kv_compact(ctx: Context, steps, batch: int, accept_path, accept_len, k_cache_ptrs,
+                     v_cache_ptrs, n_layers: int, kv_stride_seq: int, kv_stride_head: int,
+                     kv_stride_tok: int, stream=None) -> None:
+    """k_cache_ptrs / v_cache_ptrs: int64 CUDA tensors holding n_layers device pointers."""
+    i32 = torch.int32
+    _check(load().resps_kv_compact(
+        ctx.handle, _ptr(steps, i32), batch, _ptr(accept_path, i32), _ptr(accept_len, i32),
+        _ptr(k_cache_ptrs, torch.int64), _ptr(v_cache_ptrs, torch.int64), n_layers, kv_stride_seq,
+        kv_stride_head, kv_stride_tok, _stream(stream)), "resps_kv_compact")
+
+
+def layer_pointer_table(caches: Sequence[torch.Tensor]) -> torch.Tensor:
+    """Device array of the layers' base pointers, as resps_kv_compact expects."""
+    return torch.tensor([c.data_ptr() for c in caches], dtype=torch.int64, device=caches[0].device)

@@ -1,0 +1,146 @@
+// Greedy acceptance walk and in-place KV-cache compaction.
+//
+// accept_walk_kernel (Section 3.2, "Acceptance Criterion" at temperature 0; Algorithm 2,
+// "get accepted tokens"): from the root, follow the child whose token equals the target's
+// argmax at the current node until no child matches.
+//
+// kv_compact_kernel (Appendix D, "input update": rejected tokens are discarded from the
+// KV cache): slot L+j <- slot L+path[j] for j = 0..a, K and V, every KV head and layer.
+#include "common.cuh"
+
+namespace resps {
+namespace {
+
+constexpr unsigned kFull = 0xFFFFFFFFu;
+
+struct AcceptArgs {
+    const resps_step* steps;
+    const int32_t* n_nodes;
+    const int32_t *tokens, *parent, *target_argmax;
+    int max_tt, max_depth;
+    int32_t *accept_path, *accept_len, *out_tokens;
+    resps_step* steps_next;
+};
+
+// One CTA of 128 threads per sequence: thread c owns tree node c.
+__global__ void __launch_bounds__(RESPS_MAX_TT) accept_walk_kernel(const AcceptArgs a) {
+    const int b = blockIdx.x, tid = threadIdx.x;
+    const int n = min(max(a.n_nodes[b], 1), a.max_tt);
+    const int64_t ob = static_cast<int64_t>(b) * a.max_tt;
+    const int cap = a.max_depth + 1;
+    __shared__ int s_tgt[RESPS_MAX_TT];
+    __shared__ int s_next;
+    const int my_tok = (tid < n) ? a.tokens[ob + tid] : -1;
+    const int my_par = (tid < n) ? a.parent[ob + tid] : -2;
+    if (tid < n) s_tgt[tid] = a.target_argmax[ob + tid];
+    if (tid < cap) {
+        a.accept_path[b * cap + tid] = (tid == 0) ? 0 : -1;
+        a.out_tokens[b * cap + tid] = -1;
+    }
+    __syncthreads();
+    int cur = 0, len = 0;
+    for (int hop = 0; hop < a.max_depth; ++hop) {
+        if (tid == 0) s_next = -1;
+        __syncthreads();
+        // children of one node carry distinct tokens, so at most one thread matches
+        if (tid > 0 && tid < n && my_par == cur && my_tok == s_tgt[cur]) s_next = tid;
+        __syncthreads();
+        const int nxt = s_next;
+        __syncthreads();
+        if (nxt < 0) break;
+        cur = nxt;
+        ++len;
+        if (tid == 0) {
+            a.accept_path[b * cap + len] = cur;
+            a.out_tokens[b * cap + len - 1] = a.tokens[ob + cur];
+        }
+    }
+    if (tid == 0) {
+        a.out_tokens[b * cap + len] = s_tgt[cur];
+        a.accept_len[b] = len;
+        if (a.steps_next) {
+            resps_step s = a.steps[b];
+            s.prefix_len += len + 1;
+            a.steps_next[b] = s;
+        }
+    }
+}
+
+struct CompactArgs {
+    const resps_step* steps;
+    const int32_t *accept_path, *accept_len;
+    void* const* k_caches;
+    void* const* v_caches;
+    int64_t stride_seq, stride_head, stride_tok;
+    int n_kv_heads, head_dim, max_depth;
+};
+
+// One CTA per (K-or-V of a KV head, layer, sequence).  All source rows are read into
+// registers before any destination row is written (a destination slot may be the source
+// of an earlier path entry), so the move is safe in place.
+__global__ void __launch_bounds__(128) kv_compact_kernel(const CompactArgs a) {
+    const int b = blockIdx.z, layer = blockIdx.y;
+    const int head = blockIdx.x >> 1, is_v = blockIdx.x & 1;
+    const int cap = a.max_depth + 1;
+    const int len = min(max(a.accept_len[b], 0), a.max_depth);
+    const int L = a.steps[b].prefix_len;
+    __nv_bfloat16* base = static_cast<__nv_bfloat16*>(is_v ? a.v_caches[layer] : a.k_caches[layer]) +
+                          b * a.stride_seq + head * a.stride_head;
+    const int vec_per_row = a.head_dim / 8;  // 16-byte pieces per row
+    const int total = (len + 1) * vec_per_row;
+    constexpr int kMaxPer = (RESPS_MAX_DEPTH + 1) * 16 / 128 + 1;
+    uint4 regs[kMaxPer];
+#pragma unroll
+    for (int i = 0; i < kMaxPer; ++i) {
+        const int idx = threadIdx.x + i * 128;
+        if (idx < total) {
+            const int j = idx / vec_per_row, e = idx % vec_per_row;
+            const int src = a.accept_path[b * cap + j];
+            regs[i] = *reinterpret_cast<const uint4*>(base + static_cast<int64_t>(L + src) * a.stride_tok + e * 8);
+        }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < kMaxPer; ++i) {
+        const int idx = threadIdx.x + i * 128;
+        if (idx < total) {
+            const int j = idx / vec_per_row, e = idx % vec_per_row;
+            *reinterpret_cast<uint4*>(base + static_cast<int64_t>(L + j) * a.stride_tok + e * 8) = regs[i];
+        }
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_accept_walk(const resps_ctx* ctx, const resps_step* d_steps,
+                               const int32_t* d_n_nodes, int batch, const int32_t* tokens,
+                               const int32_t* parent, const int32_t* target_argmax,
+                               int32_t* accept_path, int32_t* accept_len, int32_t* out_tokens,
+                               resps_step* steps_next, cudaStream_t st) {
+    AcceptArgs a;
+    a.steps = d_steps, a.n_nodes = d_n_nodes;
+    a.tokens = tokens, a.parent = parent, a.target_argmax = target_argmax;
+    a.max_tt = ctx->shape.max_tt, a.max_depth = ctx->shape.max_depth;
+    a.accept_path = accept_path, a.accept_len = accept_len, a.out_tokens = out_tokens;
+    a.steps_next = steps_next;
+    accept_walk_kernel<<<batch, RESPS_MAX_TT, 0, st>>>(a);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_kv_compact(const resps_ctx* ctx, const resps_step* d_steps, int batch,
+                              const int32_t* accept_path, const int32_t* accept_len,
+                              void* const* k_caches, void* const* v_caches, int n_layers,
+                              int64_t stride_seq, int64_t stride_head, int64_t stride_tok,
+                              cudaStream_t st) {
+    CompactArgs a;
+    a.steps = d_steps, a.accept_path = accept_path, a.accept_len = accept_len;
+    a.k_caches = k_caches, a.v_caches = v_caches;
+    a.stride_seq = stride_seq, a.stride_head = stride_head, a.stride_tok = stride_tok;
+    a.n_kv_heads = ctx->shape.n_kv_heads, a.head_dim = ctx->shape.head_dim;
+    a.max_depth = ctx->shape.max_depth;
+    dim3 grid(ctx->shape.n_kv_heads * 2, n_layers, batch);
+    kv_compact_kernel<<<grid, 128, 0, st>>>(a);
+    return cudaGetLastError();
+}
+
+}  // namespace resps

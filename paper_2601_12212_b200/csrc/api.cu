@@ -1,0 +1,265 @@
+// C ABI of libresps: argument checks, the context and its workspace, and the
+// sequencing of kernel launches behind each entry point (see include/resps.h).
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "common.cuh"
+
+namespace resps {
+int attention_tile_rows();
+int attention_max_batch();
+}  // namespace resps
+
+namespace {
+
+inline int64_t align_up(int64_t x, int64_t a) { return (x + a - 1) / a * a; }
+
+struct Carver {
+    int64_t off = 0;
+    char* base = nullptr;
+    template <typename T>
+    void take(T*& p, int64_t count) {
+        off = align_up(off, 256);
+        if (base) p = reinterpret_cast<T*>(base + off);
+        off += count * static_cast<int64_t>(sizeof(T));
+    }
+};
+
+void carve(resps_ctx* c, Carver& cv) {
+    const resps_shape& s = c->shape;
+    resps::Workspace& w = c->ws;
+    const int64_t rows = static_cast<int64_t>(s.max_batch) * w.max_rows;
+    const int64_t nodes = static_cast<int64_t>(s.max_batch) * s.max_tt;
+    cv.take(w.status, 64);
+    cv.take(w.row_counter, rows);
+    cv.take(w.amax_counter, nodes);
+    cv.take(w.attn_counter, w.attn_max_groups);
+    const int64_t zero_end = cv.off;  // everything above must start as zero
+    (void)zero_end;
+    cv.take(w.part_key, rows * w.scan_splits * s.max_k);
+    cv.take(w.part_ms, rows * w.scan_splits);
+    cv.take(w.row_val, rows * s.max_k);
+    cv.take(w.row_id, rows * s.max_k);
+    cv.take(w.row_lse, rows);
+    cv.take(w.amax_part, nodes * w.scan_splits);
+    cv.take(w.attn_part_o, static_cast<int64_t>(w.attn_max_items) * resps::attention_tile_rows() * s.head_dim);
+    cv.take(w.attn_part_ml, static_cast<int64_t>(w.attn_max_items) * resps::attention_tile_rows());
+}
+
+#define RESPS_CHECK_PTR(p) \
+    if ((p) == nullptr) return RESPS_ERR_INVALID_ARG
+
+inline bool aligned16(const void* p) { return reinterpret_cast<uintptr_t>(p) % 16 == 0; }
+
+}  // namespace
+
+extern "C" {
+
+const char* resps_strerror(int code) {
+    switch (code) {
+        case RESPS_OK: return "ok";
+        case RESPS_ERR_INVALID_ARG: return "invalid argument";
+        case RESPS_ERR_UNSUPPORTED_SHAPE: return "unsupported shape";
+        case RESPS_ERR_CAPACITY: return "capacity exceeded";
+        case RESPS_ERR_CUDA: return "CUDA error";
+        case RESPS_ERR_NO_DEVICE: return "no usable sm_100 device";
+        default: return "unknown error";
+    }
+}
+
+int resps_create(resps_ctx** out, const resps_shape* shape) {
+    RESPS_CHECK_PTR(out);
+    RESPS_CHECK_PTR(shape);
+    *out = nullptr;
+    const resps_shape& s = *shape;
+    if (s.n_q_heads < 1 || s.n_kv_heads < 1 || s.vocab < 1 || s.max_batch < 1 || s.max_tt < 1 ||
+        s.max_k < 1 || s.max_depth < 1)
+        return RESPS_ERR_INVALID_ARG;
+    if ((s.head_dim != 64 && s.head_dim != 128) || s.n_q_heads % s.n_kv_heads != 0 ||
+        s.max_tt > RESPS_MAX_TT || s.max_k > RESPS_MAX_K || s.max_depth > RESPS_MAX_DEPTH ||
+        s.max_batch > resps::attention_max_batch())
+        return RESPS_ERR_UNSUPPORTED_SHAPE;
+    if (s.max_k + (s.max_depth - 1) * s.max_k * s.max_k > resps::tree_candidate_limit())
+        return RESPS_ERR_UNSUPPORTED_SHAPE;
+
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return RESPS_ERR_NO_DEVICE;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return RESPS_ERR_NO_DEVICE;
+    if (prop.major != 10) return RESPS_ERR_NO_DEVICE;
+
+    resps_ctx* c = new (std::nothrow) resps_ctx();
+    if (!c) return RESPS_ERR_CUDA;
+    c->shape = s;
+    c->device = dev;
+    c->sm_count = prop.multiProcessorCount;
+    resps::Workspace& w = c->ws;
+    int chunk = 8192;
+    if (const char* e = std::getenv("RESPS_SCAN_CHUNK")) chunk = std::max(1024, std::atoi(e) / 1024 * 1024);
+    if ((s.vocab + chunk - 1) / chunk > 64) chunk = static_cast<int>(align_up((s.vocab + 63) / 64, 1024));
+    w.scan_chunk = chunk;
+    w.scan_splits = (s.vocab + chunk - 1) / chunk;
+    w.max_rows = 1 + (s.max_depth - 1) * s.max_k;
+    const int G = s.n_q_heads / s.n_kv_heads;
+    const int tile_rows = resps::attention_tile_rows();
+    w.attn_grid = c->sm_count * 2;
+    w.attn_max_groups = s.max_batch * s.n_kv_heads * ((s.max_tt * G + tile_rows - 1) / tile_rows);
+    w.attn_max_items = w.attn_grid + w.attn_max_groups;
+
+    Carver dry;
+    carve(c, dry);
+    c->arena_bytes = align_up(dry.off, 256);
+    if (cudaMalloc(&c->arena, c->arena_bytes) != cudaSuccess) {
+        delete c;
+        return RESPS_ERR_CUDA;
+    }
+    if (cudaMemset(c->arena, 0, c->arena_bytes) != cudaSuccess) {
+        cudaFree(c->arena);
+        delete c;
+        return RESPS_ERR_CUDA;
+    }
+    Carver real;
+    real.base = static_cast<char*>(c->arena);
+    carve(c, real);
+    if (resps::attention_setup(c) != cudaSuccess || resps::tree_setup(c) != cudaSuccess) {
+        cudaFree(c->arena);
+        delete c;
+        return RESPS_ERR_CUDA;
+    }
+    *out = c;
+    return RESPS_OK;
+}
+
+int resps_destroy(resps_ctx* ctx) {
+    if (!ctx) return RESPS_OK;
+    cudaError_t e = cudaFree(ctx->arena);
+    delete ctx;
+    return e == cudaSuccess ? RESPS_OK : RESPS_ERR_CUDA;
+}
+
+int64_t resps_workspace_bytes(const resps_ctx* ctx) { return ctx ? ctx->arena_bytes : 0; }
+
+int resps_status(resps_ctx* ctx, resps_stream stream, int32_t* status) {
+    RESPS_CHECK_PTR(ctx);
+    RESPS_CHECK_PTR(status);
+    if (cudaMemcpyAsync(status, ctx->ws.status, sizeof(int32_t), cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+        return RESPS_ERR_CUDA;
+    if (cudaMemsetAsync(ctx->ws.status, 0, sizeof(int32_t), stream) != cudaSuccess) return RESPS_ERR_CUDA;
+    if (cudaStreamSynchronize(stream) != cudaSuccess) return RESPS_ERR_CUDA;
+    return RESPS_OK;
+}
+
+int resps_tree_expand(resps_ctx* ctx, const resps_step* d_steps, int batch,
+                      const float* d_draft_logits, int64_t ld_b, int64_t ld_level, int64_t ld_row,
+                      int n_levels, int n_slots, const int32_t* d_root_token,
+                      int32_t* d_tokens, int32_t* d_parent, int32_t* d_depth,
+                      int32_t* d_position_ids, uint64_t* d_mask, int32_t* d_retrieve,
+                      int32_t* d_n_leaves, int32_t* d_n_nodes, resps_stream stream) {
+    RESPS_CHECK_PTR(ctx);
+    RESPS_CHECK_PTR(d_steps);
+    RESPS_CHECK_PTR(d_draft_logits);
+    RESPS_CHECK_PTR(d_root_token);
+    RESPS_CHECK_PTR(d_tokens);
+    RESPS_CHECK_PTR(d_parent);
+    RESPS_CHECK_PTR(d_depth);
+    RESPS_CHECK_PTR(d_position_ids);
+    RESPS_CHECK_PTR(d_mask);
+    RESPS_CHECK_PTR(d_retrieve);
+    RESPS_CHECK_PTR(d_n_leaves);
+    RESPS_CHECK_PTR(d_n_nodes);
+    if (batch < 1 || n_levels < 1 || n_slots < 1 || ld_row < ctx->shape.vocab || ld_level < 0 || ld_b < 0)
+        return RESPS_ERR_INVALID_ARG;
+    if (batch > ctx->shape.max_batch) return RESPS_ERR_CAPACITY;
+    if (n_levels > ctx->shape.max_depth) n_levels = ctx->shape.max_depth;
+    if (n_slots > ctx->shape.max_k) n_slots = ctx->shape.max_k;
+    if (resps::launch_row_scan(ctx, d_steps, batch, d_draft_logits, ld_b, ld_level, ld_row, n_levels,
+                               n_slots, stream) != cudaSuccess)
+        return RESPS_ERR_CUDA;
+    if (resps::launch_tree_build(ctx, d_steps, batch, n_levels, n_slots, d_root_token, d_tokens, d_parent,
+                                 d_depth, d_position_ids, d_mask, d_retrieve, d_n_leaves, d_n_nodes,
+                                 stream) != cudaSuccess)
+        return RESPS_ERR_CUDA;
+    return RESPS_OK;
+}
+
+int resps_tree_attention(resps_ctx* ctx, const resps_step* d_steps, const int32_t* d_n_nodes,
+                         int batch, const void* d_q, void* d_o, float* d_lse,
+                         const void* d_k_cache, const void* d_v_cache, int64_t kv_stride_seq,
+                         int64_t kv_stride_head, int64_t kv_stride_tok, int64_t kv_capacity,
+                         const uint64_t* d_mask, float softmax_scale, resps_stream stream) {
+    RESPS_CHECK_PTR(ctx);
+    RESPS_CHECK_PTR(d_steps);
+    RESPS_CHECK_PTR(d_n_nodes);
+    RESPS_CHECK_PTR(d_q);
+    RESPS_CHECK_PTR(d_o);
+    RESPS_CHECK_PTR(d_k_cache);
+    RESPS_CHECK_PTR(d_v_cache);
+    RESPS_CHECK_PTR(d_mask);
+    if (batch < 1 || kv_capacity < 1 || kv_stride_tok < ctx->shape.head_dim || kv_stride_head < 0 ||
+        kv_stride_seq < 0)
+        return RESPS_ERR_INVALID_ARG;
+    if (!aligned16(d_q) || !aligned16(d_o) || !aligned16(d_k_cache) || !aligned16(d_v_cache) ||
+        kv_stride_seq % 8 || kv_stride_head % 8 || kv_stride_tok % 8)
+        return RESPS_ERR_INVALID_ARG;
+    if (batch > ctx->shape.max_batch || kv_capacity < ctx->shape.max_tt) return RESPS_ERR_CAPACITY;
+    if (resps::launch_tree_attention(ctx, d_steps, d_n_nodes, batch, static_cast<const __nv_bfloat16*>(d_q),
+                                     static_cast<__nv_bfloat16*>(d_o), d_lse,
+                                     static_cast<const __nv_bfloat16*>(d_k_cache),
+                                     static_cast<const __nv_bfloat16*>(d_v_cache), kv_stride_seq,
+                                     kv_stride_head, kv_stride_tok, kv_capacity, d_mask, softmax_scale,
+                                     stream) != cudaSuccess)
+        return RESPS_ERR_CUDA;
+    return RESPS_OK;
+}
+
+int resps_verify_accept(resps_ctx* ctx, const resps_step* d_steps, const int32_t* d_n_nodes,
+                        int batch, const float* d_target_logits, int64_t ld_b, int64_t ld_row,
+                        const int32_t* d_tokens, const int32_t* d_parent,
+                        int32_t* d_target_argmax, int32_t* d_accept_path, int32_t* d_accept_len,
+                        int32_t* d_out_tokens, resps_step* d_steps_next, resps_stream stream) {
+    RESPS_CHECK_PTR(ctx);
+    RESPS_CHECK_PTR(d_steps);
+    RESPS_CHECK_PTR(d_n_nodes);
+    RESPS_CHECK_PTR(d_target_logits);
+    RESPS_CHECK_PTR(d_tokens);
+    RESPS_CHECK_PTR(d_parent);
+    RESPS_CHECK_PTR(d_target_argmax);
+    RESPS_CHECK_PTR(d_accept_path);
+    RESPS_CHECK_PTR(d_accept_len);
+    RESPS_CHECK_PTR(d_out_tokens);
+    if (batch < 1 || ld_row < ctx->shape.vocab || ld_b < 0) return RESPS_ERR_INVALID_ARG;
+    if (batch > ctx->shape.max_batch) return RESPS_ERR_CAPACITY;
+    if (resps::launch_row_argmax(ctx, d_n_nodes, batch, d_target_logits, ld_b, ld_row, d_target_argmax,
+                                 stream) != cudaSuccess)
+        return RESPS_ERR_CUDA;
+    if (resps::launch_accept_walk(ctx, d_steps, d_n_nodes, batch, d_tokens, d_parent, d_target_argmax,
+                                  d_accept_path, d_accept_len, d_out_tokens, d_steps_next,
+                                  stream) != cudaSuccess)
+        return RESPS_ERR_CUDA;
+    return RESPS_OK;
+}
+
+int resps_kv_compact(resps_ctx* ctx, const resps_step* d_steps, int batch,
+                     const int32_t* d_accept_path, const int32_t* d_accept_len,
+                     void* const* d_k_caches, void* const* d_v_caches, int n_layers,
+                     int64_t kv_stride_seq, int64_t kv_stride_head, int64_t kv_stride_tok,
+                     resps_stream stream) {
+    RESPS_CHECK_PTR(ctx);
+    RESPS_CHECK_PTR(d_steps);
+    RESPS_CHECK_PTR(d_accept_path);
+    RESPS_CHECK_PTR(d_accept_len);
+    RESPS_CHECK_PTR(d_k_caches);
+    RESPS_CHECK_PTR(d_v_caches);
+    if (batch < 1 || n_layers < 1 || n_layers > 65535 || kv_stride_tok < ctx->shape.head_dim ||
+        kv_stride_seq % 8 || kv_stride_head % 8 || kv_stride_tok % 8)
+        return RESPS_ERR_INVALID_ARG;
+    if (batch > ctx->shape.max_batch) return RESPS_ERR_CAPACITY;
+    if (resps::launch_kv_compact(ctx, d_steps, batch, d_accept_path, d_accept_len, d_k_caches, d_v_caches,
+                                 n_layers, kv_stride_seq, kv_stride_head, kv_stride_tok,
+                                 stream) != cudaSuccess)
+        return RESPS_ERR_CUDA;
+    return RESPS_OK;
+}
+
+}  // extern "C"

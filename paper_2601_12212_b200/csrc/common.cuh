@@ -1,0 +1,133 @@
+// Shared declarations of the libresps kernels (sm_100a only).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "resps.h"
+
+namespace resps {
+
+constexpr int kScanThreads = 256;
+constexpr int kWarp = 32;
+
+// Host-side description of the context's device workspace.
+struct Workspace {
+    // vocabulary scans
+    int scan_chunk = 0;       // elements of a row handled by one CTA
+    int scan_splits = 0;      // ceil(V / scan_chunk)
+    int max_rows = 0;         // 1 + (max_depth-1)*max_k
+    unsigned long long* part_key = nullptr;  // [max_batch][max_rows][splits][max_k] packed (value,id)
+    float2* part_ms = nullptr;               // [max_batch][max_rows][splits] (max, sum) in log2 domain
+    unsigned int* row_counter = nullptr;     // [max_batch][max_rows]  arrival counters (self-resetting)
+    float* row_val = nullptr;                // [max_batch][max_rows][max_k]
+    int32_t* row_id = nullptr;               // [max_batch][max_rows][max_k]
+    double* row_lse = nullptr;               // [max_batch][max_rows]
+    unsigned long long* amax_part = nullptr; // [max_batch][max_tt][splits]
+    unsigned int* amax_counter = nullptr;    // [max_batch][max_tt]
+    // attention
+    int attn_grid = 0;          // persistent CTAs
+    int attn_max_items = 0;     // partial slots
+    float* attn_part_o = nullptr;   // [items][tile rows][D]
+    float2* attn_part_ml = nullptr; // [items][tile rows]
+    unsigned int* attn_counter = nullptr;  // [groups]
+    int attn_max_groups = 0;
+    // status
+    int32_t* status = nullptr;
+};
+
+}  // namespace resps
+
+struct resps_ctx {
+    resps_shape shape;
+    int device;
+    int sm_count;
+    void* arena;
+    int64_t arena_bytes;
+    resps::Workspace ws;
+};
+
+namespace resps {
+
+// ---- launchers (one per translation unit) ---------------------------------
+cudaError_t launch_row_scan(const resps_ctx* ctx, const resps_step* d_steps, int batch,
+                            const float* logits, int64_t ld_b, int64_t ld_level, int64_t ld_row,
+                            int n_levels, int n_slots, cudaStream_t st);
+cudaError_t launch_tree_build(const resps_ctx* ctx, const resps_step* d_steps, int batch,
+                              int n_levels, int n_slots, const int32_t* root_token,
+                              int32_t* tokens, int32_t* parent, int32_t* depth, int32_t* position_ids,
+                              uint64_t* mask, int32_t* retrieve, int32_t* n_leaves, int32_t* n_nodes,
+                              cudaStream_t st);
+cudaError_t launch_row_argmax(const resps_ctx* ctx, const int32_t* d_n_nodes, int batch,
+                              const float* logits, int64_t ld_b, int64_t ld_row, int32_t* argmax_out,
+                              cudaStream_t st);
+cudaError_t launch_accept_walk(const resps_ctx* ctx, const resps_step* d_steps,
+                               const int32_t* d_n_nodes, int batch, const int32_t* tokens,
+                               const int32_t* parent, const int32_t* target_argmax,
+                               int32_t* accept_path, int32_t* accept_len, int32_t* out_tokens,
+                               resps_step* steps_next, cudaStream_t st);
+cudaError_t launch_kv_compact(const resps_ctx* ctx, const resps_step* d_steps, int batch,
+                              const int32_t* accept_path, const int32_t* accept_len,
+                              void* const* k_caches, void* const* v_caches, int n_layers,
+                              int64_t stride_seq, int64_t stride_head, int64_t stride_tok,
+                              cudaStream_t st);
+cudaError_t launch_tree_attention(const resps_ctx* ctx, const resps_step* d_steps,
+                                  const int32_t* d_n_nodes, int batch, const __nv_bfloat16* q,
+                                  __nv_bfloat16* o, float* lse, const __nv_bfloat16* k_cache,
+                                  const __nv_bfloat16* v_cache, int64_t stride_seq,
+                                  int64_t stride_head, int64_t stride_tok, int64_t capacity,
+                                  const uint64_t* mask, float scale, cudaStream_t st);
+cudaError_t attention_setup(resps_ctx* ctx);  // one-time function attributes
+cudaError_t tree_setup(resps_ctx* ctx);
+int tree_candidate_limit();
+
+// ---- device helpers --------------------------------------------------------
+// Order-preserving map of a finite float onto uint32 (larger float -> larger key);
+// -0 is folded onto +0 first so that equal floats give equal keys.
+__device__ __forceinline__ uint32_t float_to_ordered(float f) {
+    f = f + 0.0f;
+    uint32_t u = __float_as_uint(f);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float ordered_to_float(uint32_t k) {
+    uint32_t u = (k & 0x80000000u) ? (k & 0x7FFFFFFFu) : ~k;
+    return __uint_as_float(u);
+}
+// Packed (value, id): a larger key ranks earlier under (value desc, id asc).
+__device__ __forceinline__ unsigned long long pack_val_id(float v, int id) {
+    return (static_cast<unsigned long long>(float_to_ordered(v)) << 32) |
+           static_cast<unsigned long long>(0xFFFFFFFFu - static_cast<uint32_t>(id));
+}
+__device__ __forceinline__ float key_val(unsigned long long k) {
+    return ordered_to_float(static_cast<uint32_t>(k >> 32));
+}
+__device__ __forceinline__ int key_id(unsigned long long k) {
+    return static_cast<int>(0xFFFFFFFFu - static_cast<uint32_t>(k & 0xFFFFFFFFull));
+}
+
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Step parameters clamped into the extents the caller supplied.
+struct StepDims {
+    int tt, d, k, L;
+    bool clamped;
+};
+__device__ __forceinline__ StepDims clamp_step(const resps_step& s, int n_levels, int n_slots,
+                                                int max_tt, int max_k, int vocab) {
+    StepDims r;
+    r.tt = min(max(s.tt, 1), max_tt);
+    r.d = min(max(s.d, 1), n_levels);
+    int kmax = min(vocab, max_k);
+    if (r.d > 1) kmax = min(kmax, n_slots);  // level 0 has a single row: slots bound k only beyond it
+    r.k = min(max(s.k, 1), kmax);
+    r.L = max(s.prefix_len, 0);
+    r.clamped = (r.tt != s.tt) || (r.d != s.d) || (r.k != s.k) || (r.L != s.prefix_len);
+    return r;
+}
+
+}  // namespace resps
