@@ -283,43 +283,53 @@ __global__ void __launch_bounds__(kAttnThreads, 2) tree_attention_kernel(const A
                 corr[h2] = ex2_approx(row_m[h2] - m_use[h2]);
                 row_m[h2] = m_new;
             }
-            float psum[2] = {0.f, 0.f};
-            uint32_t pf[kBN / 16][4];
-#pragma unroll
-            for (int nt = 0; nt < kBN / 8; ++nt) {
-                const float p0 = ex2_approx(sacc[nt][0] - m_use[0]);
-                const float p1 = ex2_approx(sacc[nt][1] - m_use[0]);
-                const float p2 = ex2_approx(sacc[nt][2] - m_use[1]);
-                const float p3 = ex2_approx(sacc[nt][3] - m_use[1]);
-                psum[0] += p0 + p1;
-                psum[1] += p2 + p3;
-                pf[nt >> 1][(nt & 1) * 2 + 0] = pack_bf16(p0, p1);
-                pf[nt >> 1][(nt & 1) * 2 + 1] = pack_bf16(p2, p3);
-            }
-#pragma unroll
-            for (int h2 = 0; h2 < 2; ++h2) row_l[h2] = row_l[h2] * corr[h2] + psum[h2];
 #pragma unroll
             for (int i = 0; i < D / 8; ++i) {
                 oacc[i][0] *= corr[0], oacc[i][1] *= corr[0];
                 oacc[i][2] *= corr[1], oacc[i][3] *= corr[1];
             }
 
-            // ---- O += P V ------------------------------------------------------------
+            // ---- P = exp2(S - m), O += P V -----------------------------------------------
+            // P is fed to the tensor cores as bf16 hi + bf16 lo (two products per V tile):
+            // a single bf16 rounding of P alone would cost ~0.4 % per weight, which shows up
+            // as ~1 % of a row's rms in the worst element; the split keeps it near fp32.
+            float psum[2] = {0.f, 0.f};
             {
                 const int mi = lane >> 3, r8 = lane & 7;
 #pragma unroll
                 for (int kk = 0; kk < kBN / 16; ++kk) {
+                    uint32_t phi[4], plo[4];
+#pragma unroll
+                    for (int half = 0; half < 2; ++half) {
+                        const int nt = kk * 2 + half;
+                        const float p0 = ex2_approx(sacc[nt][0] - m_use[0]);
+                        const float p1 = ex2_approx(sacc[nt][1] - m_use[0]);
+                        const float p2 = ex2_approx(sacc[nt][2] - m_use[1]);
+                        const float p3 = ex2_approx(sacc[nt][3] - m_use[1]);
+                        psum[0] += p0 + p1;
+                        psum[1] += p2 + p3;
+                        const __nv_bfloat162 h01 = __floats2bfloat162_rn(p0, p1);
+                        const __nv_bfloat162 h23 = __floats2bfloat162_rn(p2, p3);
+                        phi[half * 2 + 0] = *reinterpret_cast<const uint32_t*>(&h01);
+                        phi[half * 2 + 1] = *reinterpret_cast<const uint32_t*>(&h23);
+                        plo[half * 2 + 0] = pack_bf16(p0 - __low2float(h01), p1 - __high2float(h01));
+                        plo[half * 2 + 1] = pack_bf16(p2 - __low2float(h23), p3 - __high2float(h23));
+                    }
 #pragma unroll
                     for (int dp = 0; dp < D / 16; ++dp) {
                         uint32_t bf[4];
                         const int key = kk * 16 + r8 + (mi & 1) * 8;
                         const int chunk = dp * 2 + (mi >> 1);
                         ldsm_x4_t(dv + tile_off<D>(key, chunk), bf);
-                        mma_bf16(oacc[dp * 2], pf[kk], bf[0], bf[1]);
-                        mma_bf16(oacc[dp * 2 + 1], pf[kk], bf[2], bf[3]);
+                        mma_bf16(oacc[dp * 2], phi, bf[0], bf[1]);
+                        mma_bf16(oacc[dp * 2 + 1], phi, bf[2], bf[3]);
+                        mma_bf16(oacc[dp * 2], plo, bf[0], bf[1]);
+                        mma_bf16(oacc[dp * 2 + 1], plo, bf[2], bf[3]);
                     }
                 }
             }
+#pragma unroll
+            for (int h2 = 0; h2 < 2; ++h2) row_l[h2] = row_l[h2] * corr[h2] + psum[h2];
             __syncthreads();  // the stage is free for the load issued next iteration
         }
 

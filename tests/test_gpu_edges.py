@@ -40,8 +40,8 @@ def expand_and_compare(logits, params, roots, max_tt=128, max_k=None, max_d=None
     flat = torch.zeros(offset + B * max_d * max_k * ld_row, dtype=torch.float32, device="cuda")
     view = flat[offset:].view(B, max_d, max_k, ld_row)
     for s, lg in enumerate(logits):
-        d, k, _ = lg.shape
-        view[s, :d, :k, :V].copy_(torch.from_numpy(lg))
+        d, k = min(lg.shape[0], max_d), min(lg.shape[1], max_k)
+        view[s, :d, :k, :V].copy_(torch.from_numpy(np.ascontiguousarray(lg[:d, :k])))
     steps = torch.tensor(params, dtype=torch.int32, device="cuda")
     root = torch.tensor(roots, dtype=torch.int32, device="cuda")
     bufs = Bufs(B, max_tt, max_d + 1)
@@ -181,7 +181,7 @@ def _attention_case(n, Hq, Hkv, D, L, cap, parent=None, poison=False, seed=0, B=
     (17, 6, 2, 128, 2049),
 ])
 def test_attention_shapes_and_boundaries(n, Hq, Hkv, D, L):
-    _attention_case(n, Hq, Hkv, D, L, cap=L + n + 70, poison=True, seed=n)
+    _attention_case(n, Hq, Hkv, D, L, cap=L + 128 + 70, poison=True, seed=n)
 
 
 def test_attention_chain_mask_is_causal():

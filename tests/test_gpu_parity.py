@@ -40,7 +40,7 @@ def test_config2_llama8b_shape():
 
 
 def test_config3_vicuna13b_shape_varying_actions():
-    st = _run(3, 12, 1, 4)
+    st = _run(3, 16, 1, 4)
     assert len(set(st.n_nodes)) > 1          # (TT, d, k) really changes between steps
 
 
