@@ -7,7 +7,7 @@
 #include "common.cuh"
 
 namespace resps {
-int attention_tile_rows();
+int attention_item_rows();
 int attention_max_batch();
 }  // namespace resps
 
@@ -34,7 +34,6 @@ void carve(resps_ctx* c, Carver& cv) {
     cv.take(w.status, 64);
     cv.take(w.row_counter, rows);
     cv.take(w.amax_counter, nodes);
-    cv.take(w.attn_counter, w.attn_max_groups);
     const int64_t zero_end = cv.off;  // everything above must start as zero
     (void)zero_end;
     cv.take(w.part_key, rows * w.scan_splits * s.max_k);
@@ -43,8 +42,8 @@ void carve(resps_ctx* c, Carver& cv) {
     cv.take(w.row_id, rows * s.max_k);
     cv.take(w.row_lse, rows);
     cv.take(w.amax_part, nodes * w.scan_splits);
-    cv.take(w.attn_part_o, static_cast<int64_t>(w.attn_max_items) * resps::attention_tile_rows() * s.head_dim);
-    cv.take(w.attn_part_ml, static_cast<int64_t>(w.attn_max_items) * resps::attention_tile_rows());
+    cv.take(w.attn_part_o, static_cast<int64_t>(w.attn_max_items) * resps::attention_item_rows() * s.head_dim);
+    cv.take(w.attn_part_ml, static_cast<int64_t>(w.attn_max_items) * resps::attention_item_rows());
 }
 
 #define RESPS_CHECK_PTR(p) \
@@ -102,9 +101,12 @@ int resps_create(resps_ctx** out, const resps_shape* shape) {
     w.scan_splits = (s.vocab + chunk - 1) / chunk;
     w.max_rows = 1 + (s.max_depth - 1) * s.max_k;
     const int G = s.n_q_heads / s.n_kv_heads;
-    const int tile_rows = resps::attention_tile_rows();
-    w.attn_grid = c->sm_count * 2;
-    w.attn_max_groups = s.max_batch * s.n_kv_heads * ((s.max_tt * G + tile_rows - 1) / tile_rows);
+    const int item_rows = resps::attention_item_rows();
+    w.attn_grid = c->sm_count;
+    w.attn_combine_grid = c->sm_count * 2;
+    w.attn_min_tiles = 2;
+    if (const char* e = std::getenv("RESPS_ATTN_MIN_TILES")) w.attn_min_tiles = std::max(1, std::atoi(e));
+    w.attn_max_groups = s.max_batch * s.n_kv_heads * ((s.max_tt * G + item_rows - 1) / item_rows);
     w.attn_max_items = w.attn_grid + w.attn_max_groups;
 
     Carver dry;

@@ -1,16 +1,32 @@
 // Tree-masked verification attention (Section 3.2, "Verification Phase": all tree
 // tokens are scored by the target in one pass; Appendix D: the attention mask
-// follows the tree).  Split-KV flash-decode: the query rows of one KV head
-// (tree token x the Hq/Hkv heads sharing it) are packed into 64-row tiles so that
-// QK^T and PV are dense tensor-core contractions; K/V tiles of 64 keys stream
-// through a double-buffered shared-memory pipeline; the ancestor bitmask is applied
-// from registers only on tiles that reach past the prefix.
+// follows the tree).
 //
-// Work list: every (sequence, KV head, row tile, key split) is an item; a persistent
-// grid walks the items.  The list is derived inside the kernel from the device-resident
-// step parameters, so nothing about the launch depends on (TT, d, k, L).  Items of one
-// (sequence, head, row tile) group write un-normalised partials; the group's last
-// arriving CTA combines them.
+// Split-KV flash-decode on the 5th-generation tensor cores.  The query rows of one
+// KV head (tree token x the Hq/Hkv heads sharing it) are packed into 128-row tiles,
+// so that Q K^T and P V are dense contractions: tcgen05.mma with both operands in
+// fp32 accumulators (S and O) in tensor memory.  K/V tiles of 64 keys are staged by
+// TMA (cp.async.bulk.tensor, one elected thread) into 128-byte-swizzled shared memory
+// through a 4-deep mbarrier ring; a second elected thread issues the MMAs; eight
+// warps (one TMEM lane = one query row per thread) do the scaling, the ancestor
+// bitmask (from registers, only on tiles that reach past the prefix) and the online
+// softmax, and write P back into the tensor-memory columns S came from, from where
+// it is the A operand of P V.  P is kept as two bf16 terms (p = hi + lo): one bf16
+// rounding of the weights alone would cost up to 2^-9 per weight, which shows as about
+// 1 % of an output row's rms in the worst element.
+//
+// A CTA works on up to two row tiles (256 rows) of one (sequence, KV head) against a
+// contiguous range of key tiles.  The work list -- every (sequence, KV head, row-tile
+// pair, key split) -- is derived inside the kernel from the device-resident step
+// parameters, so nothing about the launch depends on (TT, d, k, L).  Items whose
+// group has a single split write O directly; the others write un-normalised partials
+// that a second, small kernel combines.
+//
+// Every wait (mbarrier) is bounded: when it runs out the CTA raises
+// RESPS_STATUS_WAIT_TIMEOUT, stops issuing work, drains its copies in flight, frees
+// its tensor memory and returns.
+#include <cuda.h>
+
 #include <cmath>
 
 #include "common.cuh"
@@ -18,10 +34,20 @@
 namespace resps {
 namespace {
 
-constexpr int kAttnThreads = 128;
-constexpr int kBM = 64;  // query rows per item
-constexpr int kBN = 64;  // keys per tile
+constexpr int kBM = 128;           // rows per row tile (one TMEM lane each)
+constexpr int kBN = 64;            // keys per tile
+constexpr int kStages = 4;         // K/V ring depth
+constexpr int kRowTiles = 2;       // row tiles per item
+constexpr int kSoftmaxThreads = 256;
+constexpr int kProducerWarp = 8;
+constexpr int kMmaWarp = 9;
+constexpr int kAttnThreads = 320;
+constexpr int kSyncThreads = 288;  // softmax warps + the MMA warp meet at the end of an item
 constexpr int kMaxBatchSmem = 256;
+constexpr int kTmemCols = 512;
+constexpr int kCombineThreads = 256;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // bounded waits give up after 2 s
+constexpr float kRescaleSlack = 8.0f;  // O is rescaled only when the running max grows by > 2^8
 constexpr unsigned kFull = 0xFFFFFFFFu;
 
 struct AttnArgs {
@@ -31,84 +57,31 @@ struct AttnArgs {
     const __nv_bfloat16* q;
     __nv_bfloat16* o;
     float* lse;
-    const __nv_bfloat16* kc;
-    const __nv_bfloat16* vc;
-    int64_t s_seq, s_head, s_tok, capacity;
+    int64_t capacity;
     const uint64_t* mask;
     float scale_log2;
     int Hq, Hkv, max_tt;
-    float* part_o;
-    float2* part_ml;
-    unsigned int* counter;
+    float4* part_o;   // [items][2 row tiles][D/4][128 rows]
+    float2* part_ml;  // [items][2 row tiles][128 rows]   (running max, running sum)
     int max_items;
+    int sched_grid;   // CTAs of the attention grid (the work list is balanced for it)
+    int min_tiles;    // smallest key-tile count worth a split of its own
     int32_t* status;
 };
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool valid) {
-    const int sz = valid ? 16 : 0;
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(sz));
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() {
-    asm volatile("cp.async.wait_group %0;" ::"n"(N));
-}
-__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t (&r)[4]) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
-                 : "r"(addr));
-}
-__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t (&r)[4]) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
-                 : "r"(addr));
-}
-__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
-        "{%0,%1,%2,%3};"
-        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-    return *reinterpret_cast<uint32_t*>(&v);
-}
-
-// Byte offset of 16-byte piece `chunk` of row `row` in a [rows][D] bf16 tile whose pieces
-// are XOR-swizzled by the row so that 8 consecutive rows hit 8 different bank groups.
-template <int D>
-__device__ __forceinline__ uint32_t tile_off(int row, int chunk) {
-    return static_cast<uint32_t>(row * (D * 2) + ((chunk ^ (row & 7)) << 4));
-}
-
+// ---------------------------------------------------------------------------- work list
 struct Sched {
     int n[kMaxBatchSmem];       // tree nodes (0 = sequence skipped)
     int L[kMaxBatchSmem];
-    int mt[kMaxBatchSmem];      // row tiles
+    int mp[kMaxBatchSmem];      // row-tile pairs
     int kt[kMaxBatchSmem];      // key tiles
     int splits[kMaxBatchSmem];
     int item0[kMaxBatchSmem + 1];
-    int group0[kMaxBatchSmem + 1];
 };
 
-template <int D>
-__global__ void __launch_bounds__(kAttnThreads, 2) tree_attention_kernel(const AttnArgs a) {
-    extern __shared__ __align__(128) unsigned char smem[];
-    __shared__ Sched sc;
-    __shared__ bool s_last;
-    constexpr int kTileBytes = kBN * D * 2;
-    constexpr int kChunks = D / 8;  // 16-byte pieces per row
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+__device__ __forceinline__ void build_sched(const AttnArgs& a, Sched& sc, int tid, int nthreads) {
     const int G = a.Hq / a.Hkv;
-    unsigned char* sK[2] = {smem, smem + kTileBytes};
-    unsigned char* sV[2] = {smem + 2 * kTileBytes, smem + 3 * kTileBytes};
-
-    // ---- work list from the device-resident step parameters ------------------------
-    for (int b = tid; b < a.batch; b += kAttnThreads) {
+    for (int b = tid; b < a.batch; b += nthreads) {
         int n = min(max(a.n_nodes[b], 0), a.max_tt);
         const int L = max(a.steps[b].prefix_len, 0);
         if (static_cast<int64_t>(L) + n > a.capacity) {
@@ -117,312 +90,738 @@ __global__ void __launch_bounds__(kAttnThreads, 2) tree_attention_kernel(const A
         }
         sc.n[b] = n;
         sc.L[b] = L;
-        sc.mt[b] = (n * G + kBM - 1) / kBM;
+        sc.mp[b] = (n * G + kRowTiles * kBM - 1) / (kRowTiles * kBM);
         sc.kt[b] = (n > 0) ? (L + n + kBN - 1) / kBN : 0;
     }
     __syncthreads();
     if (tid == 0) {
-        long long total_tiles = 0;
-        for (int b = 0; b < a.batch; ++b) total_tiles += 1ll * a.Hkv * sc.mt[b] * sc.kt[b];
-        const int tps = max(1, static_cast<int>((total_tiles + gridDim.x - 1) / gridDim.x));
-        int items = 0, groups = 0;
+        long long units = 0;
+        for (int b = 0; b < a.batch; ++b) units += 1ll * a.Hkv * sc.mp[b] * sc.kt[b];
+        int tps = static_cast<int>((units + a.sched_grid - 1) / a.sched_grid);
+        tps = max(tps, max(a.min_tiles, 1));
+        int items = 0;
         for (int b = 0; b < a.batch; ++b) {
             sc.item0[b] = items;
-            sc.group0[b] = groups;
             sc.splits[b] = (sc.kt[b] + tps - 1) / tps;
-            items += a.Hkv * sc.mt[b] * sc.splits[b];
-            groups += a.Hkv * sc.mt[b];
+            items += a.Hkv * sc.mp[b] * sc.splits[b];
         }
         sc.item0[a.batch] = items;
-        sc.group0[a.batch] = groups;
     }
     __syncthreads();
+}
+
+struct Item {
+    int b, g, pair, sp, splits, first_item;
+    int n, L, M, row_base, nmt, t_begin, t_end;
+};
+
+__device__ __forceinline__ Item decode_item(const Sched& sc, int item, int G) {
+    Item it;
+    int b = 0;
+    while (item >= sc.item0[b + 1]) ++b;
+    it.b = b;
+    it.n = sc.n[b], it.L = sc.L[b], it.splits = sc.splits[b];
+    const int local = item - sc.item0[b];
+    it.sp = local % it.splits;
+    const int grp = local / it.splits;  // = g * mp + pair
+    it.pair = grp % sc.mp[b];
+    it.g = grp / sc.mp[b];
+    it.first_item = item - it.sp;
+    it.M = it.n * G;
+    it.row_base = it.pair * kRowTiles * kBM;
+    it.nmt = (it.M - it.row_base > kBM) ? 2 : 1;
+    it.t_begin = static_cast<int>(1ll * sc.kt[b] * it.sp / it.splits);
+    it.t_end = static_cast<int>(1ll * sc.kt[b] * (it.sp + 1) / it.splits);
+    return it;
+}
+
+// ---------------------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ unsigned long long global_timer() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait: false when the CTA has given up (here or elsewhere).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          int32_t* status) {
+    if (mbar_try(bar, parity)) return true;
+    const unsigned long long t0 = global_timer();
+    unsigned spins = 0;
+    for (;;) {
+        if (mbar_try(bar, parity)) return true;
+        if ((++spins & 63u) == 0u) {
+            if (*abort_flag) return false;
+            if (global_timer() - t0 > kWaitLimitNs) {
+                *abort_flag = 1;
+                atomicOr(status, RESPS_STATUS_WAIT_TIMEOUT);
+                return false;
+            }
+        }
+    }
+}
+// Same, with a warp-uniform answer (the callers go on to warp-collective TMEM instructions).
+__device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          int32_t* status) {
+    const bool ok = mbar_wait(bar, parity, abort_flag, status);
+    return __all_sync(0xFFFFFFFFu, ok);
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// TMA: one box of a 4-D tensor (element, slot, head, sequence) into shared memory.
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0,
+                                            int c1, int c2, int c3) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%2, %3, %4, %5}], [%6];" ::"r"(dst),
+        "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar)
+        : "memory");
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle (layout type 2), descriptor version 1.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    uint64_t d = static_cast<uint64_t>((addr & 0x3FFFFu) >> 4);
+    d |= static_cast<uint64_t>(lbo_bytes >> 4) << 16;
+    d |= static_cast<uint64_t>(sbo_bytes >> 4) << 32;
+    d |= 1ull << 46;
+    d |= 2ull << 61;
+    return d;
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, M = 128, A K-major.
+__host__ __device__ constexpr uint32_t instr_desc(int n, bool b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn_major ? (1u << 16) : 0u) |
+           (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(kBM >> 4) << 24);
+}
+__device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                     uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// A operand from tensor memory (lane = row, two bf16 per 32-bit column).
+__device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc,
+                                        uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
+                 : "memory");
+}
+
+#define RESPS_R8(a, o) "%" #a "0" #o
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]),
+          "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]),
+          "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]),
+          "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+#undef RESPS_R8
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};" ::"r"(taddr),
+        "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+        "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]),
+        "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]),
+        "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+        : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// ---------------------------------------------------------------------------- shared memory map
+template <int D>
+struct Smem {
+    static constexpr int kPanels = D / 64;                   // 64-element (128-byte) column panels
+    static constexpr int kQPanel = kBM * 128;                // one panel of a Q row tile
+    static constexpr int kQTile = kPanels * kQPanel;
+    static constexpr int kKVPanel = kBN * 128;
+    static constexpr int kKVTile = kPanels * kKVPanel;
+    static constexpr int kOffQ = 0;
+    static constexpr int kOffK = kOffQ + kRowTiles * kQTile;
+    static constexpr int kOffV = kOffK + kStages * kKVTile;
+    static constexpr int kOffBar = kOffV + kStages * kKVTile;
+    static constexpr int kNumBars = 3 * kStages + 1 + kRowTiles * 4 + 1;
+    static constexpr int kOffMisc = kOffBar + 8 * 32;
+    static constexpr int kUsed = kOffMisc + 64 + 1024;       // + slack to align the base to 1024
+    // Never less than 120 KB, more than half of an SM's shared memory: one CTA per SM, so the
+    // 512-column TMEM allocation can never wait for a neighbour.
+    static constexpr int kBytes = kUsed > 120 * 1024 ? kUsed : 120 * 1024;
+    static_assert(kNumBars <= 32, "barrier area");
+    static_assert(2 * kBytes > 228 * 1024, "two CTAs must not fit on one SM");
+};
+
+// barrier indices
+__device__ __forceinline__ constexpr int bar_kfull(int s) { return s; }
+__device__ __forceinline__ constexpr int bar_vfull(int s) { return kStages + s; }
+__device__ __forceinline__ constexpr int bar_kvempty(int s) { return 2 * kStages + s; }
+__device__ __forceinline__ constexpr int bar_qfull() { return 3 * kStages; }
+__device__ __forceinline__ constexpr int bar_sfull(int m, int buf) { return 3 * kStages + 1 + m * 4 + buf; }
+__device__ __forceinline__ constexpr int bar_pfull(int m) { return 3 * kStages + 1 + m * 4 + 2; }
+__device__ __forceinline__ constexpr int bar_pvdone(int m) { return 3 * kStages + 1 + m * 4 + 3; }
+__device__ __forceinline__ constexpr int bar_item() { return 3 * kStages + 1 + kRowTiles * 4; }
+
+template <int D>
+__global__ void __launch_bounds__(kAttnThreads, 1)
+tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
+                      const __grid_constant__ CUtensorMap map_v) {
+    using S = Smem<D>;
+    extern __shared__ unsigned char smem_raw[];
+    __shared__ Sched sc;
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    unsigned char* base_ptr = smem_raw + (base - smem_u32(smem_raw));
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int G = a.Hq / a.Hkv;
+    const uint32_t bars = base + S::kOffBar;
+    auto bar = [&](int i) { return bars + 8u * i; };
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + S::kOffMisc);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + S::kOffMisc + 8);
+
+    // ---- one-time set-up ---------------------------------------------------------------
+    if (tid == 0) {
+        *abort_flag = 0;
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(bar(bar_kfull(s)), 1);
+            mbar_init(bar(bar_vfull(s)), 1);
+            mbar_init(bar(bar_kvempty(s)), 1);
+        }
+        mbar_init(bar(bar_qfull()), kSoftmaxThreads);
+        for (int m = 0; m < kRowTiles; ++m) {
+            for (int bf = 0; bf < 2; ++bf) {
+                mbar_init(bar(bar_sfull(m, bf)), 1);
+            }
+            mbar_init(bar(bar_pfull(m)), kBM);
+            mbar_init(bar(bar_pvdone(m)), 1);
+        }
+        mbar_init(bar(bar_item()), kSyncThreads);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == kMmaWarp) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                         base + S::kOffMisc),
+                     "r"(kTmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    if (warp == kProducerWarp && lane == 0) {
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_k) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_v) : "memory");
+    }
+    build_sched(a, sc, tid, kAttnThreads);  // ends with __syncthreads()
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
     const int total_items = min(sc.item0[a.batch], a.max_items);
 
-    for (int item = blockIdx.x; item < total_items; item += gridDim.x) {
-        int b = 0;
-        while (item >= sc.item0[b + 1]) ++b;
-        const int n = sc.n[b], L = sc.L[b], splits = sc.splits[b];
-        const int local = item - sc.item0[b];
-        const int sp = local % splits;
-        const int grp_local = local / splits;  // = g * mt + mtile
-        const int mtile = grp_local % sc.mt[b];
-        const int g = grp_local / sc.mt[b];
-        const int group = sc.group0[b] + grp_local;
-        const int kv_len = L + n;
-        const int M = n * G;
-        const int t_begin = static_cast<int>(1ll * sc.kt[b] * sp / splits);
-        const int t_end = static_cast<int>(1ll * sc.kt[b] * (sp + 1) / splits);
-        const int row_base = mtile * kBM;
+    // running use counts of the barrier families (identical in every role: all roles walk
+    // the same items and tiles in the same order)
+    uint32_t kt_run = 0;                 // K/V ring uses
+    uint32_t jj[kRowTiles] = {0, 0};     // tiles processed per row tile (S buffers, P, PV)
+    uint32_t items_run = 0;
+    bool alive = true;
 
-        const __nv_bfloat16* kbase = a.kc + b * a.s_seq + g * a.s_head;
-        const __nv_bfloat16* vbase = a.vc + b * a.s_seq + g * a.s_head;
-        auto issue_tile = [&](int stage, int t) {
-            const int j0 = t * kBN;
-            const uint32_t dk = smem_u32(sK[stage]), dv = smem_u32(sV[stage]);
-            for (int i = tid; i < kBN * kChunks; i += kAttnThreads) {
-                const int r = i / kChunks, c = i % kChunks;
-                const int j = j0 + r;
-                const bool ok = j < kv_len;
-                const int64_t off = static_cast<int64_t>(ok ? j : 0) * a.s_tok + c * 8;
-                cp_async16(dk + tile_off<D>(r, c), kbase + off, ok);
-                cp_async16(dv + tile_off<D>(r, c), vbase + off, ok);
-            }
-        };
-
-        // prologue: first K/V tile into stage 0, the Q tile into the (still free) V stage 1
-        issue_tile(0, t_begin);
-        {
-            const uint32_t dq = smem_u32(sV[1]);
-            for (int i = tid; i < kBM * kChunks; i += kAttnThreads) {
-                const int r = i / kChunks, c = i % kChunks;
-                const int R = row_base + r;
-                const bool ok = R < M;
-                const int t = ok ? R / G : 0, h = g * G + (ok ? R % G : 0);
-                const __nv_bfloat16* src =
-                    a.q + ((static_cast<int64_t>(b) * a.max_tt + t) * a.Hq + h) * D + c * 8;
-                cp_async16(dq + tile_off<D>(r, c), src, ok);
-            }
-        }
-        cp_async_commit();
-        cp_async_wait<0>();
-        __syncthreads();
-        uint32_t qf[D / 16][4];
-        {
-            const uint32_t dq = smem_u32(sV[1]);
-            const int mi = lane >> 3, r8 = lane & 7;
-#pragma unroll
-            for (int ks = 0; ks < D / 16; ++ks) {
-                const int row = warp * 16 + r8 + (mi & 1) * 8;
-                const int chunk = ks * 2 + (mi >> 1);
-                ldsm_x4(dq + tile_off<D>(row, chunk), qf[ks]);
-            }
-        }
-        __syncthreads();
-
-        // rows of this thread: r_lo = warp*16 + lane/4 and r_lo + 8
-        const int r_lo = row_base + warp * 16 + (lane >> 2);
-        unsigned long long mlo[2], mhi[2];
-#pragma unroll
-        for (int h2 = 0; h2 < 2; ++h2) {
-            const int R = r_lo + h2 * 8;
-            const int t = R / G;
-            const bool ok = R < M;
-            mlo[h2] = ok ? a.mask[(static_cast<int64_t>(b) * a.max_tt + t) * 2 + 0] : 0ull;
-            mhi[h2] = ok ? a.mask[(static_cast<int64_t>(b) * a.max_tt + t) * 2 + 1] : 0ull;
-        }
-
-        float oacc[D / 8][4];
-#pragma unroll
-        for (int i = 0; i < D / 8; ++i) oacc[i][0] = oacc[i][1] = oacc[i][2] = oacc[i][3] = 0.f;
-        float row_m[2] = {-INFINITY, -INFINITY}, row_l[2] = {0.f, 0.f};
-
-        for (int t = t_begin; t < t_end; ++t) {
-            const int stage = (t - t_begin) & 1;
-            if (t + 1 < t_end) {
-                issue_tile(stage ^ 1, t + 1);
-                cp_async_commit();
-                cp_async_wait<1>();
-            } else {
-                cp_async_wait<0>();
-            }
-            __syncthreads();
-
-            // ---- S = Q K^T ---------------------------------------------------------
-            float sacc[kBN / 8][4];
-#pragma unroll
-            for (int i = 0; i < kBN / 8; ++i) sacc[i][0] = sacc[i][1] = sacc[i][2] = sacc[i][3] = 0.f;
-            const uint32_t dk = smem_u32(sK[stage]), dv = smem_u32(sV[stage]);
-            {
-                const int mi = lane >> 3, r8 = lane & 7;
-#pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks) {
-#pragma unroll
-                    for (int np = 0; np < kBN / 16; ++np) {
-                        uint32_t bf[4];
-                        const int key = np * 16 + r8 + (mi >> 1) * 8;
-                        const int chunk = ks * 2 + (mi & 1);
-                        ldsm_x4(dk + tile_off<D>(key, chunk), bf);
-                        mma_bf16(sacc[np * 2], qf[ks], bf[0], bf[1]);
-                        mma_bf16(sacc[np * 2 + 1], qf[ks], bf[2], bf[3]);
+    if (warp == kProducerWarp) {
+        // ================================ TMA producer ====================================
+        if (lane == 0) {
+            for (int item = blockIdx.x; item < total_items && alive; item += gridDim.x) {
+                const Item it = decode_item(sc, item, G);
+                for (int t = it.t_begin; t < it.t_end; ++t, ++kt_run) {
+                    const int s = kt_run % kStages;
+                    if (!mbar_wait(bar(bar_kvempty(s)), ((kt_run / kStages) & 1u) ^ 1u, abort_flag, a.status)) {
+                        alive = false;
+                        break;
                     }
+                    const uint32_t dk = base + S::kOffK + s * S::kKVTile;
+                    const uint32_t dv = base + S::kOffV + s * S::kKVTile;
+                    mbar_expect_tx(bar(bar_kfull(s)), S::kKVTile);
+#pragma unroll
+                    for (int p = 0; p < S::kPanels; ++p)
+                        tma_load_4d(dk + p * S::kKVPanel, &map_k, bar(bar_kfull(s)), p * 64, t * kBN, it.g, it.b);
+                    mbar_expect_tx(bar(bar_vfull(s)), S::kKVTile);
+#pragma unroll
+                    for (int p = 0; p < S::kPanels; ++p)
+                        tma_load_4d(dv + p * S::kKVPanel, &map_v, bar(bar_vfull(s)), p * 64, t * kBN, it.g, it.b);
                 }
             }
-
-            // ---- scale, mask, online softmax -----------------------------------------
-            const int j0 = t * kBN;
-            const bool need_mask = (j0 + kBN > L);
-            float tmax[2] = {-INFINITY, -INFINITY};
+            // Drain: every copy this thread issued has landed before the CTA may exit.
+            const uint32_t issued = kt_run;
+            for (uint32_t u = (issued > kStages ? issued - kStages : 0u); u < issued; ++u) {
+                const int s = u % kStages;
+                const uint32_t ph = (u / kStages) & 1u;
+                if (!mbar_wait(bar(bar_kfull(s)), ph, abort_flag, a.status)) break;
+                if (!mbar_wait(bar(bar_vfull(s)), ph, abort_flag, a.status)) break;
+            }
+        }
+    } else if (warp == kMmaWarp) {
+        // ================================ MMA issuer ======================================
+        constexpr uint32_t kIdescQK = instr_desc(kBN, false);
+        constexpr uint32_t kIdescPV = instr_desc(D, true);
+        for (int item = blockIdx.x; item < total_items && alive; item += gridDim.x, ++items_run) {
+            const Item it = decode_item(sc, item, G);
+            if (lane == 0) {
+                alive = mbar_wait(bar(bar_qfull()), items_run & 1u, abort_flag, a.status);
+                tc_fence_after();
+                // PV of a tile is issued after QK of the next one, so the tensor pipe has S(j+1)
+                // to work on while the softmax warps turn S(j) into P(j).  S(j) and P(j) share the
+                // TMEM buffer j & 1; the MMAs of one thread execute in issue order, so QK(j+2) cannot
+                // overwrite it before PV(j) has read it.
+                auto issue_pv = [&](uint32_t kt_use, const uint32_t (&jj_use)[kRowTiles], bool first_tile) {
+                    const int s = kt_use % kStages;
+                    if (!mbar_wait(bar(bar_vfull(s)), (kt_use / kStages) & 1u, abort_flag, a.status)) return false;
+                    for (int m = 0; m < it.nmt; ++m)
+                        if (!mbar_wait(bar(bar_pfull(m)), jj_use[m] & 1u, abort_flag, a.status)) return false;
+                    tc_fence_after();
+                    const uint32_t dv = base + S::kOffV + s * S::kKVTile;
+                    for (int m = 0; m < it.nmt; ++m) {
+                        const uint32_t o_t = tmem + m * 256 + 128;
+                        const uint32_t p_t = tmem + m * 256 + (jj_use[m] & 1u) * kBN;  // hi: +0, lo: +32
 #pragma unroll
-            for (int nt = 0; nt < kBN / 8; ++nt) {
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const int h2 = e >> 1;
-                    float s = sacc[nt][e] * a.scale_log2;
-                    if (need_mask) {
-                        const int j = j0 + nt * 8 + (lane & 3) * 2 + (e & 1);
-                        const int i = j - L;
-                        bool ok = true;
-                        if (i >= 0) {
-                            const unsigned long long w = (i < 64) ? mlo[h2] : mhi[h2];
-                            ok = (i < n) && ((w >> (i & 63)) & 1ull);
+                        for (int kk = 0; kk < kBN / 16; ++kk) {
+                            const uint64_t vdesc = smem_desc(dv + kk * 2048, S::kKVPanel, 1024);
+                            umma_ts(o_t, p_t + kk * 8, vdesc, kIdescPV, (first_tile && kk == 0) ? 0u : 1u);
+                            umma_ts(o_t, p_t + 32 + kk * 8, vdesc, kIdescPV, 1u);
                         }
-                        if (!ok) s = -INFINITY;
+                        umma_commit(bar(bar_pvdone(m)));
                     }
-                    sacc[nt][e] = s;
-                    tmax[h2] = fmaxf(tmax[h2], s);
+                    umma_commit(bar(bar_kvempty(s)));
+                    return true;
+                };
+                uint32_t prev_kt = 0, prev_jj[kRowTiles] = {0, 0};
+                for (int t = it.t_begin; t < it.t_end && alive; ++t) {
+                    const int s = kt_run % kStages;
+                    alive = mbar_wait(bar(bar_kfull(s)), (kt_run / kStages) & 1u, abort_flag, a.status);
+                    if (!alive) break;
+                    tc_fence_after();
+                    const uint32_t dk = base + S::kOffK + s * S::kKVTile;
+                    for (int m = 0; m < it.nmt; ++m) {
+                        const uint32_t s_t = tmem + m * 256 + (jj[m] & 1u) * kBN;
+                        const uint32_t dq = base + S::kOffQ + m * S::kQTile;
+#pragma unroll
+                        for (int ks = 0; ks < D / 16; ++ks)
+                            umma(s_t, smem_desc(dq + (ks >> 2) * S::kQPanel + (ks & 3) * 32, 16, 1024),
+                                 smem_desc(dk + (ks >> 2) * S::kKVPanel + (ks & 3) * 32, 16, 1024), kIdescQK,
+                                 ks > 0 ? 1u : 0u);
+                        umma_commit(bar(bar_sfull(m, jj[m] & 1u)));
+                    }
+                    if (t > it.t_begin) alive = issue_pv(prev_kt, prev_jj, t - 1 == it.t_begin);
+                    prev_kt = kt_run;
+                    prev_jj[0] = jj[0], prev_jj[1] = jj[1];
+                    ++kt_run;
+                    for (int m = 0; m < it.nmt; ++m) ++jj[m];
                 }
+                if (alive && it.t_end > it.t_begin) alive = issue_pv(prev_kt, prev_jj, it.t_end - 1 == it.t_begin);
+                tc_fence_before();
             }
-            float corr[2], m_use[2];
-#pragma unroll
-            for (int h2 = 0; h2 < 2; ++h2) {
-                tmax[h2] = fmaxf(tmax[h2], __shfl_xor_sync(kFull, tmax[h2], 1));
-                tmax[h2] = fmaxf(tmax[h2], __shfl_xor_sync(kFull, tmax[h2], 2));
-                const float m_new = fmaxf(row_m[h2], tmax[h2]);
-                m_use[h2] = (m_new == -INFINITY) ? 0.f : m_new;
-                corr[h2] = ex2_approx(row_m[h2] - m_use[h2]);
-                row_m[h2] = m_new;
-            }
-#pragma unroll
-            for (int i = 0; i < D / 8; ++i) {
-                oacc[i][0] *= corr[0], oacc[i][1] *= corr[0];
-                oacc[i][2] *= corr[1], oacc[i][3] *= corr[1];
-            }
-
-            // ---- P = exp2(S - m), O += P V -----------------------------------------------
-            // P is fed to the tensor cores as bf16 hi + bf16 lo (two products per V tile):
-            // a single bf16 rounding of P alone would cost ~0.4 % per weight, which shows up
-            // as ~1 % of a row's rms in the worst element; the split keeps it near fp32.
-            float psum[2] = {0.f, 0.f};
+            alive = __shfl_sync(kFull, alive ? 1 : 0, 0) != 0;
+            if (!alive) break;
+            // end of item: the softmax warps have read O and S, Q and P may be overwritten
+            mbar_arrive(bar(bar_item()));
+            alive = warp_wait(bar(bar_item()), items_run & 1u, abort_flag, a.status);
+        }
+    } else {
+        // ================================ softmax warps ===================================
+        const int wg = warp >> 2;                      // row tile this warp works on
+        const int r = (warp & 3) * 32 + lane;          // row inside the tile = TMEM lane
+        const uint32_t lane_sel = static_cast<uint32_t>((warp & 3) * 32) << 16;
+        constexpr int kChunks = D / 8;                 // 16-byte pieces of a row
+        for (int item = blockIdx.x; item < total_items && alive; item += gridDim.x, ++items_run) {
+            const Item it = decode_item(sc, item, G);
+            // ---- Q tiles -> shared memory in the swizzled K-major layout ----------------
             {
-                const int mi = lane >> 3, r8 = lane & 7;
+                const int total = it.nmt * kBM * kChunks;
+                for (int i0 = tid; i0 < total; i0 += kSoftmaxThreads * 4) {
+                    uint4 v[4];
 #pragma unroll
-                for (int kk = 0; kk < kBN / 16; ++kk) {
-                    uint32_t phi[4], plo[4];
-#pragma unroll
-                    for (int half = 0; half < 2; ++half) {
-                        const int nt = kk * 2 + half;
-                        const float p0 = ex2_approx(sacc[nt][0] - m_use[0]);
-                        const float p1 = ex2_approx(sacc[nt][1] - m_use[0]);
-                        const float p2 = ex2_approx(sacc[nt][2] - m_use[1]);
-                        const float p3 = ex2_approx(sacc[nt][3] - m_use[1]);
-                        psum[0] += p0 + p1;
-                        psum[1] += p2 + p3;
-                        const __nv_bfloat162 h01 = __floats2bfloat162_rn(p0, p1);
-                        const __nv_bfloat162 h23 = __floats2bfloat162_rn(p2, p3);
-                        phi[half * 2 + 0] = *reinterpret_cast<const uint32_t*>(&h01);
-                        phi[half * 2 + 1] = *reinterpret_cast<const uint32_t*>(&h23);
-                        plo[half * 2 + 0] = pack_bf16(p0 - __low2float(h01), p1 - __high2float(h01));
-                        plo[half * 2 + 1] = pack_bf16(p2 - __low2float(h23), p3 - __high2float(h23));
+                    for (int u = 0; u < 4; ++u) {
+                        const int i = i0 + u * kSoftmaxThreads;
+                        v[u] = make_uint4(0u, 0u, 0u, 0u);
+                        if (i < total) {
+                            const int row = i / kChunks, c = i % kChunks;
+                            const int R = it.row_base + row;
+                            if (R < it.M) {
+                                const int t = R / G, h = it.g * G + R % G;
+                                v[u] = __ldg(reinterpret_cast<const uint4*>(
+                                    a.q + ((static_cast<int64_t>(it.b) * a.max_tt + t) * a.Hq + h) * D + c * 8));
+                            }
+                        }
                     }
 #pragma unroll
-                    for (int dp = 0; dp < D / 16; ++dp) {
-                        uint32_t bf[4];
-                        const int key = kk * 16 + r8 + (mi & 1) * 8;
-                        const int chunk = dp * 2 + (mi >> 1);
-                        ldsm_x4_t(dv + tile_off<D>(key, chunk), bf);
-                        mma_bf16(oacc[dp * 2], phi, bf[0], bf[1]);
-                        mma_bf16(oacc[dp * 2 + 1], phi, bf[2], bf[3]);
-                        mma_bf16(oacc[dp * 2], plo, bf[0], bf[1]);
-                        mma_bf16(oacc[dp * 2 + 1], plo, bf[2], bf[3]);
+                    for (int u = 0; u < 4; ++u) {
+                        const int i = i0 + u * kSoftmaxThreads;
+                        if (i < total) {
+                            const int row = i / kChunks, c = i % kChunks;
+                            const int m = row / kBM, rr = row % kBM;
+                            unsigned char* dst = base_ptr + S::kOffQ + m * S::kQTile + (c >> 3) * S::kQPanel +
+                                                 rr * 128 + (((c & 7) ^ (rr & 7)) << 4);
+                            *reinterpret_cast<uint4*>(dst) = v[u];
+                        }
                     }
                 }
+                fence_proxy_async();
+                mbar_arrive(bar(bar_qfull()));
             }
-#pragma unroll
-            for (int h2 = 0; h2 < 2; ++h2) row_l[h2] = row_l[h2] * corr[h2] + psum[h2];
-            __syncthreads();  // the stage is free for the load issued next iteration
-        }
 
-        // ---- row sums across the 4 lanes of a row --------------------------------------
-#pragma unroll
-        for (int h2 = 0; h2 < 2; ++h2) {
-            row_l[h2] += __shfl_xor_sync(kFull, row_l[h2], 1);
-            row_l[h2] += __shfl_xor_sync(kFull, row_l[h2], 2);
-        }
-
-        if (splits == 1) {
-#pragma unroll
-            for (int h2 = 0; h2 < 2; ++h2) {
-                const int R = r_lo + h2 * 8;
-                if (R >= M) continue;
-                const int t = R / G, h = g * G + R % G;
-                const float inv = 1.f / row_l[h2];
-                __nv_bfloat16* dst = a.o + ((static_cast<int64_t>(b) * a.max_tt + t) * a.Hq + h) * D;
-#pragma unroll
-                for (int i = 0; i < D / 8; ++i) {
-                    const uint32_t v = pack_bf16(oacc[i][h2 * 2] * inv, oacc[i][h2 * 2 + 1] * inv);
-                    *reinterpret_cast<uint32_t*>(dst + i * 8 + (lane & 3) * 2) = v;
+            if (wg < it.nmt) {
+                const int R = it.row_base + wg * kBM + r;
+                const bool row_ok = R < it.M;
+                unsigned long long mlo = 0ull, mhi = 0ull;
+                if (row_ok) {
+                    const int t = R / G;
+                    mlo = a.mask[(static_cast<int64_t>(it.b) * a.max_tt + t) * 2 + 0];
+                    mhi = a.mask[(static_cast<int64_t>(it.b) * a.max_tt + t) * 2 + 1];
+                    // only nodes of this tree can be visible
+                    if (it.n < 64) {
+                        mlo &= (1ull << it.n) - 1ull;
+                        mhi = 0ull;
+                    } else if (it.n < 128) {
+                        mhi &= (1ull << (it.n - 64)) - 1ull;
+                    }
                 }
-                if (a.lse && (lane & 3) == 0)
-                    a.lse[(static_cast<int64_t>(b) * a.max_tt + t) * a.Hq + h] =
-                        (row_m[h2] + log2f(row_l[h2])) * 0.6931471805599453f;
-            }
-            continue;
-        }
+                float m_ref = -INFINITY, l_run = 0.f;
+                const uint32_t o_t = tmem + lane_sel + wg * 256 + 128;
+                const int kv_len = it.L + it.n;
 
-        // ---- partial result, then the group's last CTA combines ------------------------
-        float* po = a.part_o + static_cast<int64_t>(item) * kBM * D;
-        float2* pml = a.part_ml + static_cast<int64_t>(item) * kBM;
+                for (int t = it.t_begin; t < it.t_end; ++t, ++kt_run) {
+                    const uint32_t buf = jj[wg] & 1u;
+                    if (!warp_wait(bar(bar_sfull(wg, buf)), (jj[wg] >> 1) & 1u, abort_flag, a.status)) {
+                        alive = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    uint32_t sr[2][32];
+                    tmem_ld32(tmem + lane_sel + wg * 256 + buf * kBN, sr[0]);
+                    tmem_ld32(tmem + lane_sel + wg * 256 + buf * kBN + 32, sr[1]);
+                    tmem_wait_ld();
+
+                    // ---- scale, ancestor mask, row maximum ---------------------------------
+                    const int j0 = t * kBN;
+                    unsigned long long allowed = ~0ull;
+                    if (j0 + kBN > it.L) {
+                        const int off = j0 - it.L;  // tile start relative to the first tree slot
+                        if (off >= 64)
+                            allowed = mhi >> (off - 64);
+                        else if (off > 0)
+                            allowed = (mlo >> off) | (mhi << (64 - off));
+                        else if (off == 0)
+                            allowed = mlo;
+                        else  // -64 < off < 0: the first -off keys are prefix
+                            allowed = (mlo << (-off)) | ((1ull << (-off)) - 1ull);
+                    }
+                    float tmax = -INFINITY;
 #pragma unroll
-        for (int h2 = 0; h2 < 2; ++h2) {
-            const int r = warp * 16 + (lane >> 2) + h2 * 8;
+                    for (int h = 0; h < 2; ++h)
 #pragma unroll
-            for (int i = 0; i < D / 8; ++i)
-                __stcg(reinterpret_cast<float2*>(po + r * D + i * 8 + (lane & 3) * 2),
-                       make_float2(oacc[i][h2 * 2], oacc[i][h2 * 2 + 1]));
-            if ((lane & 3) == 0) __stcg(pml + r, make_float2(row_m[h2], row_l[h2]));
-        }
-        __threadfence();
-        __syncthreads();
-        if (tid == 0) s_last = (atomicAdd(a.counter + group, 1u) == static_cast<unsigned>(splits - 1));
-        __syncthreads();
-        if (s_last) {
-            __threadfence();
-            const int item_first = item - sp;
-            const int rows_here = min(kBM, M - row_base);
-            // thread -> (row, 4 consecutive columns)
-            for (int idx = tid; idx < rows_here * (D / 4); idx += kAttnThreads) {
-                const int r = idx / (D / 4), c4 = idx % (D / 4);
-                float Mx = -INFINITY;
-                for (int s2 = 0; s2 < splits; ++s2)
-                    Mx = fmaxf(Mx, __ldcg(&a.part_ml[static_cast<int64_t>(item_first + s2) * kBM + r].x));
-                float den = 0.f;
-                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-                for (int s2 = 0; s2 < splits; ++s2) {
-                    const float2 ml = __ldcg(&a.part_ml[static_cast<int64_t>(item_first + s2) * kBM + r]);
-                    const float w = ex2_approx(ml.x - Mx);
-                    den += ml.y * w;
-                    const float4 v = __ldcg(reinterpret_cast<const float4*>(
-                        a.part_o + (static_cast<int64_t>(item_first + s2) * kBM + r) * D + c4 * 4));
-                    acc.x += v.x * w, acc.y += v.y * w, acc.z += v.z * w, acc.w += v.w * w;
+                        for (int c = 0; c < 32; ++c) {
+                            float s = __uint_as_float(sr[h][c]) * a.scale_log2;
+                            if (!((allowed >> (h * 32 + c)) & 1ull)) s = -INFINITY;
+                            sr[h][c] = __float_as_uint(s);
+                            tmax = fmaxf(tmax, s);
+                        }
+                    const bool first = (t == it.t_begin);
+                    const float m_new = fmaxf(m_ref, tmax);
+                    // Lazy rescale: O and l keep the old reference maximum while the true one
+                    // grew by less than 2^kRescaleSlack (fp32 accumulators have the head-room).
+                    const bool need = !first && (m_new > m_ref + kRescaleSlack);
+                    if (first) m_ref = m_new;
+                    bool pv_seen = first;  // every phase of pvdone is observed, so its parity never aliases
+                    if (__any_sync(kFull, need)) {
+                        // O may only be touched once PV of the previous tile has completed
+                        if (!warp_wait(bar(bar_pvdone(wg)), (jj[wg] - 1u) & 1u, abort_flag, a.status)) {
+                            alive = false;
+                            break;
+                        }
+                        pv_seen = true;
+                        const float corr = need ? ex2_approx(m_ref - m_new) : 1.f;
+                        if (need) m_ref = m_new;
+                        l_run *= corr;
+                        tc_fence_after();
+#pragma unroll 1
+                        for (int c0 = 0; c0 < D; c0 += 32) {
+                            uint32_t orr[32];
+                            tmem_ld32(o_t + c0, orr);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int c = 0; c < 32; ++c) orr[c] = __float_as_uint(__uint_as_float(orr[c]) * corr);
+                            tmem_st32(o_t + c0, orr);
+                        }
+                        tmem_wait_st();
+                    }
+                    const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
+
+                    // ---- stale V rows of the sequence's last tile must not reach the MMA --------
+                    if (wg == 0 && j0 + kBN > kv_len) {
+                        const int s = kt_run % kStages;
+                        if (!warp_wait(bar(bar_vfull(s)), (kt_run / kStages) & 1u, abort_flag, a.status)) {
+                            alive = false;
+                            break;
+                        }
+                        const int valid = kv_len - j0;
+                        unsigned char* vt = base_ptr + S::kOffV + s * S::kKVTile;
+                        for (int i = r; i < (kBN - valid) * 8 * S::kPanels; i += kBM) {
+                            const int row = valid + i / (8 * S::kPanels), cc = i % (8 * S::kPanels);
+                            *reinterpret_cast<uint4*>(vt + (cc >> 3) * S::kKVPanel + row * 128 + ((cc & 7) << 4)) =
+                                make_uint4(0u, 0u, 0u, 0u);
+                        }
+                    }
+
+                    // ---- P = exp2(S - m) as bf16 hi + lo, back into the columns S came from ------
+                    float psum = 0.f;
+                    uint32_t plo[32];
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) {
+                        const float p0 = ex2_approx(__uint_as_float(sr[c >> 4][(2 * c) & 31]) - m_use);
+                        const float p1 = ex2_approx(__uint_as_float(sr[c >> 4][(2 * c + 1) & 31]) - m_use);
+                        psum += p0 + p1;
+                        const __nv_bfloat162 hi = __floats2bfloat162_rn(p0, p1);
+                        plo[c] = pack_bf16(p0 - __low2float(hi), p1 - __high2float(hi));
+                        sr[c >> 4][(2 * c) & 31] = *reinterpret_cast<const uint32_t*>(&hi);
+                    }
+                    l_run += psum;
+                    {
+                        // hi words sit at the even positions of sr; gather them into one 32-column store
+                        uint32_t phi[32];
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) phi[c] = sr[c >> 4][(2 * c) & 31];
+                        const uint32_t p_t = tmem + lane_sel + wg * 256 + buf * kBN;
+                        tmem_st32(p_t, phi);
+                        tmem_st32(p_t + 32, plo);
+                        tmem_wait_st();
+                    }
+                    if (wg == 0 && j0 + kBN > kv_len) fence_proxy_async();  // the zeroed V rows
+                    if (!pv_seen && !warp_wait(bar(bar_pvdone(wg)), (jj[wg] - 1u) & 1u, abort_flag, a.status)) {
+                        alive = false;
+                        break;
+                    }
+                    tc_fence_before();
+                    mbar_arrive(bar(bar_pfull(wg)));
+                    ++jj[wg];
                 }
-                const float inv = 1.f / den;
-                const int R = row_base + r;
-                const int t = R / G, h = g * G + R % G;
-                __nv_bfloat16* dst =
-                    a.o + ((static_cast<int64_t>(b) * a.max_tt + t) * a.Hq + h) * D + c4 * 4;
-                uint2 out;
-                out.x = pack_bf16(acc.x * inv, acc.y * inv);
-                out.y = pack_bf16(acc.z * inv, acc.w * inv);
-                *reinterpret_cast<uint2*>(dst) = out;
-                if (a.lse && c4 == 0)
-                    a.lse[(static_cast<int64_t>(b) * a.max_tt + t) * a.Hq + h] =
-                        (Mx + log2f(den)) * 0.6931471805599453f;
+                if (!alive) break;
+
+                // ---- epilogue --------------------------------------------------------------
+                if (it.t_end > it.t_begin) {
+                    if (!warp_wait(bar(bar_pvdone(wg)), (jj[wg] - 1u) & 1u, abort_flag, a.status)) {
+                        alive = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    if (it.splits == 1) {
+                        const float inv = 1.f / l_run;
+                        __nv_bfloat16* dst = nullptr;
+                        if (row_ok) {
+                            const int t = R / G, h = it.g * G + R % G;
+                            dst = a.o + ((static_cast<int64_t>(it.b) * a.max_tt + t) * a.Hq + h) * D;
+                            if (a.lse)
+                                a.lse[(static_cast<int64_t>(it.b) * a.max_tt + t) * a.Hq + h] =
+                                    (m_ref + log2f(l_run)) * 0.6931471805599453f;
+                        }
+#pragma unroll 1
+                        for (int c0 = 0; c0 < D; c0 += 32) {
+                            uint32_t orr[32];
+                            tmem_ld32(o_t + c0, orr);
+                            tmem_wait_ld();
+                            if (row_ok) {
+#pragma unroll
+                                for (int q4 = 0; q4 < 4; ++q4) {
+                                    uint4 v;
+                                    v.x = pack_bf16(__uint_as_float(orr[q4 * 8 + 0]) * inv, __uint_as_float(orr[q4 * 8 + 1]) * inv);
+                                    v.y = pack_bf16(__uint_as_float(orr[q4 * 8 + 2]) * inv, __uint_as_float(orr[q4 * 8 + 3]) * inv);
+                                    v.z = pack_bf16(__uint_as_float(orr[q4 * 8 + 4]) * inv, __uint_as_float(orr[q4 * 8 + 5]) * inv);
+                                    v.w = pack_bf16(__uint_as_float(orr[q4 * 8 + 6]) * inv, __uint_as_float(orr[q4 * 8 + 7]) * inv);
+                                    *reinterpret_cast<uint4*>(dst + c0 + q4 * 8) = v;
+                                }
+                            }
+                        }
+                    } else {
+                        float4* po = a.part_o + (static_cast<int64_t>(item) * kRowTiles + wg) * (D / 4) * kBM + r;
+                        __stcg(a.part_ml + (static_cast<int64_t>(item) * kRowTiles + wg) * kBM + r,
+                               make_float2(m_ref, l_run));
+#pragma unroll 1
+                        for (int c0 = 0; c0 < D; c0 += 32) {
+                            uint32_t orr[32];
+                            tmem_ld32(o_t + c0, orr);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int q4 = 0; q4 < 8; ++q4)
+                                __stcg(po + (c0 / 4 + q4) * kBM,
+                                       make_float4(__uint_as_float(orr[q4 * 4 + 0]), __uint_as_float(orr[q4 * 4 + 1]),
+                                                   __uint_as_float(orr[q4 * 4 + 2]), __uint_as_float(orr[q4 * 4 + 3])));
+                        }
+                    }
+                    tc_fence_before();
+                }
+            } else {
+                // this warp's row tile does not exist in this item: keep the ring counter in step
+                kt_run += static_cast<uint32_t>(it.t_end - it.t_begin);
             }
-            if (tid == 0) a.counter[group] = 0u;
+            mbar_arrive(bar(bar_item()));
+            alive = warp_wait(bar(bar_item()), items_run & 1u, abort_flag, a.status);
         }
-        __syncthreads();
     }
+
+    // ---- tear-down: every role arrives here, whatever happened ------------------------------
+    tc_fence_before();
+    __syncthreads();
+    if (warp == kMmaWarp) {
+        __syncwarp();
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+    }
+}
+
+// Combines the partials of every (sequence, KV head, row-tile pair) group that was split
+// over several items: O = sum_s w_s O_s / sum_s w_s l_s with w_s = 2^(m_s - max m).
+template <int D>
+__global__ void __launch_bounds__(kCombineThreads) attention_combine_kernel(const AttnArgs a) {
+    __shared__ Sched sc;
+    build_sched(a, sc, threadIdx.x, kCombineThreads);
+    const int G = a.Hq / a.Hkv;
+    constexpr int kPerGroup = kRowTiles * kBM * (D / 4);  // (row, 4 columns) work items of a group
+    for (int b = 0; b < a.batch; ++b) {
+        const int splits = sc.splits[b];
+        if (sc.n[b] == 0 || splits <= 1) continue;
+        const int groups = a.Hkv * sc.mp[b];
+        const int M = sc.n[b] * G;
+        const long long total = 1ll * groups * kPerGroup;
+        for (long long idx = 1ll * blockIdx.x * kCombineThreads + threadIdx.x; idx < total;
+             idx += 1ll * gridDim.x * kCombineThreads) {
+            const int grp = static_cast<int>(idx / kPerGroup);
+            const int rem = static_cast<int>(idx % kPerGroup);
+            const int c4 = rem / (kRowTiles * kBM);
+            const int row2 = rem % (kRowTiles * kBM);  // row inside the pair: consecutive threads, consecutive rows
+            const int pair = grp % sc.mp[b], g = grp / sc.mp[b];
+            const int R = pair * kRowTiles * kBM + row2;
+            if (R >= M) continue;
+            const int mt = row2 / kBM, r = row2 % kBM;
+            const int64_t item_first = sc.item0[b] + static_cast<int64_t>(grp) * splits;
+            float Mx = -INFINITY;
+            for (int s = 0; s < splits; ++s)
+                Mx = fmaxf(Mx, __ldcg(&a.part_ml[((item_first + s) * kRowTiles + mt) * kBM + r].x));
+            float den = 0.f;
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 4
+            for (int s = 0; s < splits; ++s) {
+                const float2 ml = __ldcg(&a.part_ml[((item_first + s) * kRowTiles + mt) * kBM + r]);
+                const float4 v = __ldcg(a.part_o + (((item_first + s) * kRowTiles + mt) * (D / 4) + c4) * kBM + r);
+                const float w = (ml.x == -INFINITY) ? 0.f : ex2_approx(ml.x - Mx);
+                den += ml.y * w;
+                acc.x += v.x * w, acc.y += v.y * w, acc.z += v.z * w, acc.w += v.w * w;
+            }
+            const float inv = 1.f / den;
+            const int t = R / G, h = g * G + R % G;
+            __nv_bfloat16* dst = a.o + ((static_cast<int64_t>(b) * a.max_tt + t) * a.Hq + h) * D + c4 * 4;
+            uint2 out;
+            out.x = pack_bf16(acc.x * inv, acc.y * inv);
+            out.y = pack_bf16(acc.z * inv, acc.w * inv);
+            *reinterpret_cast<uint2*>(dst) = out;
+            if (a.lse && c4 == 0)
+                a.lse[(static_cast<int64_t>(b) * a.max_tt + t) * a.Hq + h] = (Mx + log2f(den)) * 0.6931471805599453f;
+        }
+    }
+}
+
+// cuTensorMapEncodeTiled, resolved at run time so that the library has no link-time
+// dependency on the driver (it must load on a machine without one).
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                   CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                   CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            p = nullptr;
+        return reinterpret_cast<EncodeTiledFn>(p);
+    }();
+    return fn;
+}
+
+// (element, slot, head, sequence) view of a bf16 cache; boxes of 64 elements x 64 slots.
+bool make_kv_map(CUtensorMap* map, const void* basep, int D, int64_t capacity, int Hkv, int batch,
+                 int64_t s_tok, int64_t s_head, int64_t s_seq) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    // a dimension of extent 1 never uses its stride; give it a valid one
+    if (s_head <= 0) s_head = capacity * s_tok;
+    if (s_seq <= 0) s_seq = s_head * Hkv;
+    const cuuint64_t dims[4] = {static_cast<cuuint64_t>(D), static_cast<cuuint64_t>(capacity),
+                                static_cast<cuuint64_t>(Hkv), static_cast<cuuint64_t>(batch)};
+    const cuuint64_t strides[3] = {static_cast<cuuint64_t>(s_tok) * 2, static_cast<cuuint64_t>(s_head) * 2,
+                                   static_cast<cuuint64_t>(s_seq) * 2};
+    const cuuint32_t box[4] = {64, static_cast<cuuint32_t>(kBN), 1, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(basep), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int D>
+cudaError_t launch_for_dim(const resps_ctx* ctx, const AttnArgs& a, const CUtensorMap& mk, const CUtensorMap& mv,
+                           cudaStream_t st) {
+    tree_attention_kernel<D><<<ctx->ws.attn_grid, kAttnThreads, Smem<D>::kBytes, st>>>(a, mk, mv);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    attention_combine_kernel<D><<<ctx->ws.attn_combine_grid, kCombineThreads, 0, st>>>(a);
+    return cudaGetLastError();
 }
 
 }  // namespace
 
 cudaError_t attention_setup(resps_ctx*) {
-    cudaError_t e = cudaFuncSetAttribute(tree_attention_kernel<128>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * kBN * 128 * 2);
+    cudaError_t e = cudaFuncSetAttribute(tree_attention_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         Smem<128>::kBytes);
     if (e != cudaSuccess) return e;
     return cudaFuncSetAttribute(tree_attention_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                4 * kBN * 64 * 2);
+                                Smem<64>::kBytes);
 }
 
 cudaError_t launch_tree_attention(const resps_ctx* ctx, const resps_step* d_steps,
@@ -433,23 +832,23 @@ cudaError_t launch_tree_attention(const resps_ctx* ctx, const resps_step* d_step
                                   const uint64_t* mask, float scale, cudaStream_t st) {
     AttnArgs a;
     a.steps = d_steps, a.n_nodes = d_n_nodes, a.batch = batch;
-    a.q = q, a.o = o, a.lse = lse, a.kc = k_cache, a.vc = v_cache;
-    a.s_seq = stride_seq, a.s_head = stride_head, a.s_tok = stride_tok, a.capacity = capacity;
+    a.q = q, a.o = o, a.lse = lse;
+    a.capacity = capacity;
     a.mask = mask;
     a.scale_log2 = scale * 1.4426950408889634f;
     a.Hq = ctx->shape.n_q_heads, a.Hkv = ctx->shape.n_kv_heads, a.max_tt = ctx->shape.max_tt;
-    a.part_o = ctx->ws.attn_part_o, a.part_ml = ctx->ws.attn_part_ml, a.counter = ctx->ws.attn_counter;
-    a.max_items = ctx->ws.attn_max_items, a.status = ctx->ws.status;
+    a.part_o = reinterpret_cast<float4*>(ctx->ws.attn_part_o), a.part_ml = ctx->ws.attn_part_ml;
+    a.max_items = ctx->ws.attn_max_items, a.sched_grid = ctx->ws.attn_grid;
+    a.min_tiles = ctx->ws.attn_min_tiles, a.status = ctx->ws.status;
     const int D = ctx->shape.head_dim;
-    const size_t smem = 4 * kBN * D * 2;
-    if (D == 128)
-        tree_attention_kernel<128><<<ctx->ws.attn_grid, kAttnThreads, smem, st>>>(a);
-    else
-        tree_attention_kernel<64><<<ctx->ws.attn_grid, kAttnThreads, smem, st>>>(a);
-    return cudaGetLastError();
+    CUtensorMap mk, mv;
+    if (!make_kv_map(&mk, k_cache, D, capacity, a.Hkv, batch, stride_tok, stride_head, stride_seq) ||
+        !make_kv_map(&mv, v_cache, D, capacity, a.Hkv, batch, stride_tok, stride_head, stride_seq))
+        return cudaErrorInvalidValue;
+    return D == 128 ? launch_for_dim<128>(ctx, a, mk, mv, st) : launch_for_dim<64>(ctx, a, mk, mv, st);
 }
 
-int attention_tile_rows() { return kBM; }
+int attention_item_rows() { return kRowTiles * kBM; }
 int attention_max_batch() { return kMaxBatchSmem; }
 
 }  // namespace resps

@@ -27,11 +27,12 @@ struct Workspace {
     unsigned long long* amax_part = nullptr; // [max_batch][max_tt][splits]
     unsigned int* amax_counter = nullptr;    // [max_batch][max_tt]
     // attention
-    int attn_grid = 0;          // persistent CTAs
+    int attn_grid = 0;          // persistent CTAs (one per SM)
+    int attn_combine_grid = 0;  // CTAs of the partial-combine kernel
+    int attn_min_tiles = 0;     // smallest key-tile count a split is given
     int attn_max_items = 0;     // partial slots
-    float* attn_part_o = nullptr;   // [items][tile rows][D]
-    float2* attn_part_ml = nullptr; // [items][tile rows]
-    unsigned int* attn_counter = nullptr;  // [groups]
+    float* attn_part_o = nullptr;   // [items][item rows][D]
+    float2* attn_part_ml = nullptr; // [items][item rows]
     int attn_max_groups = 0;
     // status
     int32_t* status = nullptr;
