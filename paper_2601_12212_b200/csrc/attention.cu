@@ -45,8 +45,8 @@ constexpr int kAttnThreads = 320;
 constexpr int kSyncThreads = 288;  // softmax warps + the MMA warp meet at the end of an item
 constexpr int kMaxBatchSmem = 256;
 constexpr int kTmemCols = 512;
-constexpr int kCombineThreads = 256;
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // bounded waits give up after 2 s
+constexpr int kCombineThreads = 128;  // small enough to share an SM with a draining attention CTA
+constexpr long long kWaitLimitCycles = 4000000000ll;  // bounded waits give up after ~2 s of SM clocks
 constexpr float kRescaleSlack = 8.0f;  // O is rescaled only when the running max grows by > 2^8
 constexpr unsigned kFull = 0xFFFFFFFFu;
 
@@ -66,6 +66,7 @@ struct AttnArgs {
     int max_items;
     int sched_grid;   // CTAs of the attention grid (the work list is balanced for it)
     int min_tiles;    // smallest key-tile count worth a split of its own
+    int q_by_tma;     // 1: Q tiles come by TMA (128 % (Hq/Hkv) == 0), 0: by plain loads
     int32_t* status;
 };
 
@@ -130,19 +131,16 @@ __device__ __forceinline__ Item decode_item(const Sched& sc, int item, int G) {
     it.M = it.n * G;
     it.row_base = it.pair * kRowTiles * kBM;
     it.nmt = (it.M - it.row_base > kBM) ? 2 : 1;
-    it.t_begin = static_cast<int>(1ll * sc.kt[b] * it.sp / it.splits);
-    it.t_end = static_cast<int>(1ll * sc.kt[b] * (it.sp + 1) / it.splits);
+    // kt <= 2^15 (cache capacity is checked on the host), so the products fit 32 bits
+    const unsigned kt = static_cast<unsigned>(sc.kt[b]), sp = static_cast<unsigned>(it.sp);
+    it.t_begin = static_cast<int>(kt * sp / static_cast<unsigned>(it.splits));
+    it.t_end = static_cast<int>(kt * (sp + 1u) / static_cast<unsigned>(it.splits));
     return it;
 }
 
 // ---------------------------------------------------------------------------- PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-__device__ __forceinline__ unsigned long long global_timer() {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
 }
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
@@ -168,13 +166,13 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                           int32_t* status) {
     if (mbar_try(bar, parity)) return true;
-    const unsigned long long t0 = global_timer();
+    const long long t0 = clock64();
     unsigned spins = 0;
     for (;;) {
         if (mbar_try(bar, parity)) return true;
         if ((++spins & 63u) == 0u) {
             if (*abort_flag) return false;
-            if (global_timer() - t0 > kWaitLimitNs) {
+            if (clock64() - t0 > kWaitLimitCycles) {
                 *abort_flag = 1;
                 atomicOr(status, RESPS_STATUS_WAIT_TIMEOUT);
                 return false;
@@ -201,6 +199,18 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
         "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar)
         : "memory");
 }
+
+// TMA: one box of the 5-D query view (element, head in group, KV head, token, sequence).
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0,
+                                            int c1, int c2, int c3, int c4) {
+    asm volatile(
+        "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%2, %3, %4, %5, %6}], [%7];" ::"r"(dst),
+        "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 // Shared-memory matrix descriptor, 128-byte swizzle (layout type 2), descriptor version 1.
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
@@ -269,6 +279,36 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
+// Packed fp32 pairs (one instruction for two lanes of arithmetic) and the 3-input maximum.
+__device__ __forceinline__ unsigned long long pack2(float lo, float hi) {
+    unsigned long long r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(unsigned long long v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ unsigned long long fma2(unsigned long long a, unsigned long long b, unsigned long long c) {
+    unsigned long long d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ unsigned long long add2(unsigned long long a, unsigned long long b) {
+    unsigned long long d;
+    asm("add.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ unsigned long long sub2(unsigned long long a, unsigned long long b) {
+    unsigned long long d;
+    asm("sub.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
@@ -286,7 +326,7 @@ struct Smem {
     static constexpr int kOffK = kOffQ + kRowTiles * kQTile;
     static constexpr int kOffV = kOffK + kStages * kKVTile;
     static constexpr int kOffBar = kOffV + kStages * kKVTile;
-    static constexpr int kNumBars = 3 * kStages + 1 + kRowTiles * 4 + 1;
+    static constexpr int kNumBars = 3 * kStages + 1 + kRowTiles * 5 + 2;
     static constexpr int kOffMisc = kOffBar + 8 * 32;
     static constexpr int kUsed = kOffMisc + 64 + 1024;       // + slack to align the base to 1024
     // Never less than 120 KB, more than half of an SM's shared memory: one CTA per SM, so the
@@ -301,15 +341,21 @@ __device__ __forceinline__ constexpr int bar_kfull(int s) { return s; }
 __device__ __forceinline__ constexpr int bar_vfull(int s) { return kStages + s; }
 __device__ __forceinline__ constexpr int bar_kvempty(int s) { return 2 * kStages + s; }
 __device__ __forceinline__ constexpr int bar_qfull() { return 3 * kStages; }
-__device__ __forceinline__ constexpr int bar_sfull(int m, int buf) { return 3 * kStages + 1 + m * 4 + buf; }
-__device__ __forceinline__ constexpr int bar_pfull(int m) { return 3 * kStages + 1 + m * 4 + 2; }
-__device__ __forceinline__ constexpr int bar_pvdone(int m) { return 3 * kStages + 1 + m * 4 + 3; }
-__device__ __forceinline__ constexpr int bar_item() { return 3 * kStages + 1 + kRowTiles * 4; }
+// S and P share a TMEM buffer (tile j uses buffer j & 1) and each buffer has its own pair of
+// barriers: a buffer's next phase cannot complete before the other side has observed the
+// current one (QK(j+2) is issued after PV(j), which is issued after pfull(j) was seen), so a
+// parity wait never falls two phases behind.  One pfull barrier for both buffers would: the
+// softmax warps can finish tile j+1 while the MMA thread still waits for V(j).
+__device__ __forceinline__ constexpr int bar_sfull(int m, int buf) { return 3 * kStages + 1 + m * 5 + buf; }
+__device__ __forceinline__ constexpr int bar_pfull(int m, int buf) { return 3 * kStages + 1 + m * 5 + 2 + buf; }
+__device__ __forceinline__ constexpr int bar_pvdone(int m) { return 3 * kStages + 1 + m * 5 + 4; }
+__device__ __forceinline__ constexpr int bar_item() { return 3 * kStages + 1 + kRowTiles * 5; }
+__device__ __forceinline__ constexpr int bar_qempty() { return 3 * kStages + 2 + kRowTiles * 5; }
 
 template <int D>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
-                      const __grid_constant__ CUtensorMap map_v) {
+                      const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_q) {
     using S = Smem<D>;
     extern __shared__ unsigned char smem_raw[];
     __shared__ Sched sc;
@@ -330,12 +376,13 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
             mbar_init(bar(bar_vfull(s)), 1);
             mbar_init(bar(bar_kvempty(s)), 1);
         }
-        mbar_init(bar(bar_qfull()), kSoftmaxThreads);
+        mbar_init(bar(bar_qfull()), a.q_by_tma ? 1 : kSoftmaxThreads);
+        mbar_init(bar(bar_qempty()), 1);
         for (int m = 0; m < kRowTiles; ++m) {
             for (int bf = 0; bf < 2; ++bf) {
                 mbar_init(bar(bar_sfull(m, bf)), 1);
+                mbar_init(bar(bar_pfull(m, bf)), kBM);
             }
-            mbar_init(bar(bar_pfull(m)), kBM);
             mbar_init(bar(bar_pvdone(m)), 1);
         }
         mbar_init(bar(bar_item()), kSyncThreads);
@@ -351,7 +398,12 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
     if (warp == kProducerWarp && lane == 0) {
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_k) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_v) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_q) : "memory");
     }
+    // Everything above touches no global memory, so under programmatic dependent launch it
+    // overlaps the tail of the preceding kernel.
+    pdl_wait();
+    pdl_launch_dependents();
     build_sched(a, sc, tid, kAttnThreads);  // ends with __syncthreads()
     tc_fence_before();
     __syncthreads();
@@ -371,6 +423,20 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
         if (lane == 0) {
             for (int item = blockIdx.x; item < total_items && alive; item += gridDim.x) {
                 const Item it = decode_item(sc, item, G);
+                if (a.q_by_tma) {
+                    // the Q tiles of the previous item are free once its last QK^T has completed
+                    if (!mbar_wait(bar(bar_qempty()), (items_run & 1u) ^ 1u, abort_flag, a.status)) {
+                        alive = false;
+                        break;
+                    }
+                    mbar_expect_tx(bar(bar_qfull()), it.nmt * S::kQTile);
+                    for (int m = 0; m < it.nmt; ++m)
+#pragma unroll
+                        for (int p = 0; p < S::kPanels; ++p)
+                            tma_load_5d(base + S::kOffQ + m * S::kQTile + p * S::kQPanel, &map_q, bar(bar_qfull()),
+                                        p * 64, 0, it.g, (it.row_base + m * kBM) / G, it.b);
+                    ++items_run;
+                }
                 for (int t = it.t_begin; t < it.t_end; ++t, ++kt_run) {
                     const int s = kt_run % kStages;
                     if (!mbar_wait(bar(bar_kvempty(s)), ((kt_run / kStages) & 1u) ^ 1u, abort_flag, a.status)) {
@@ -390,6 +456,7 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
                 }
             }
             // Drain: every copy this thread issued has landed before the CTA may exit.
+            if (a.q_by_tma && items_run > 0) mbar_wait(bar(bar_qfull()), (items_run - 1u) & 1u, abort_flag, a.status);
             const uint32_t issued = kt_run;
             for (uint32_t u = (issued > kStages ? issued - kStages : 0u); u < issued; ++u) {
                 const int s = u % kStages;
@@ -411,21 +478,26 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
                 // to work on while the softmax warps turn S(j) into P(j).  S(j) and P(j) share the
                 // TMEM buffer j & 1; the MMAs of one thread execute in issue order, so QK(j+2) cannot
                 // overwrite it before PV(j) has read it.
+                // Descriptors differ only in the (16-byte granular) start address, the low 14 bits.
+                const uint64_t qdesc0 = smem_desc(base + S::kOffQ, 16, 1024);
+                const uint64_t kdesc0 = smem_desc(base + S::kOffK, 16, 1024);
+                const uint64_t vdesc0 = smem_desc(base + S::kOffV, S::kKVPanel, 1024);
                 auto issue_pv = [&](uint32_t kt_use, const uint32_t (&jj_use)[kRowTiles], bool first_tile) {
                     const int s = kt_use % kStages;
                     if (!mbar_wait(bar(bar_vfull(s)), (kt_use / kStages) & 1u, abort_flag, a.status)) return false;
                     for (int m = 0; m < it.nmt; ++m)
-                        if (!mbar_wait(bar(bar_pfull(m)), jj_use[m] & 1u, abort_flag, a.status)) return false;
+                        if (!mbar_wait(bar(bar_pfull(m, jj_use[m] & 1u)), (jj_use[m] >> 1) & 1u, abort_flag, a.status))
+                            return false;
                     tc_fence_after();
-                    const uint32_t dv = base + S::kOffV + s * S::kKVTile;
+                    const uint64_t vdesc = vdesc0 + static_cast<uint64_t>(s * (S::kKVTile >> 4));
                     for (int m = 0; m < it.nmt; ++m) {
                         const uint32_t o_t = tmem + m * 256 + 128;
                         const uint32_t p_t = tmem + m * 256 + (jj_use[m] & 1u) * kBN;  // hi: +0, lo: +32
 #pragma unroll
                         for (int kk = 0; kk < kBN / 16; ++kk) {
-                            const uint64_t vdesc = smem_desc(dv + kk * 2048, S::kKVPanel, 1024);
-                            umma_ts(o_t, p_t + kk * 8, vdesc, kIdescPV, (first_tile && kk == 0) ? 0u : 1u);
-                            umma_ts(o_t, p_t + 32 + kk * 8, vdesc, kIdescPV, 1u);
+                            umma_ts(o_t, p_t + kk * 8, vdesc + kk * (2048 >> 4), kIdescPV,
+                                    (first_tile && kk == 0) ? 0u : 1u);
+                            umma_ts(o_t, p_t + 32 + kk * 8, vdesc + kk * (2048 >> 4), kIdescPV, 1u);
                         }
                         umma_commit(bar(bar_pvdone(m)));
                     }
@@ -438,17 +510,17 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
                     alive = mbar_wait(bar(bar_kfull(s)), (kt_run / kStages) & 1u, abort_flag, a.status);
                     if (!alive) break;
                     tc_fence_after();
-                    const uint32_t dk = base + S::kOffK + s * S::kKVTile;
+                    const uint64_t kdesc = kdesc0 + static_cast<uint64_t>(s * (S::kKVTile >> 4));
                     for (int m = 0; m < it.nmt; ++m) {
                         const uint32_t s_t = tmem + m * 256 + (jj[m] & 1u) * kBN;
-                        const uint32_t dq = base + S::kOffQ + m * S::kQTile;
+                        const uint64_t qdesc = qdesc0 + static_cast<uint64_t>(m * (S::kQTile >> 4));
 #pragma unroll
                         for (int ks = 0; ks < D / 16; ++ks)
-                            umma(s_t, smem_desc(dq + (ks >> 2) * S::kQPanel + (ks & 3) * 32, 16, 1024),
-                                 smem_desc(dk + (ks >> 2) * S::kKVPanel + (ks & 3) * 32, 16, 1024), kIdescQK,
-                                 ks > 0 ? 1u : 0u);
+                            umma(s_t, qdesc + ((ks >> 2) * (S::kQPanel >> 4) + (ks & 3) * 2),
+                                 kdesc + ((ks >> 2) * (S::kKVPanel >> 4) + (ks & 3) * 2), kIdescQK, ks > 0 ? 1u : 0u);
                         umma_commit(bar(bar_sfull(m, jj[m] & 1u)));
                     }
+                    if (t + 1 == it.t_end) umma_commit(bar(bar_qempty()));  // Q is free for the next item
                     if (t > it.t_begin) alive = issue_pv(prev_kt, prev_jj, t - 1 == it.t_begin);
                     prev_kt = kt_run;
                     prev_jj[0] = jj[0], prev_jj[1] = jj[1];
@@ -472,35 +544,35 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
         constexpr int kChunks = D / 8;                 // 16-byte pieces of a row
         for (int item = blockIdx.x; item < total_items && alive; item += gridDim.x, ++items_run) {
             const Item it = decode_item(sc, item, G);
-            // ---- Q tiles -> shared memory in the swizzled K-major layout ----------------
-            {
+            // ---- Q tiles -> shared memory in the swizzled K-major layout (only when the group
+            // size does not allow the TMA view) ---------------------------------------------
+            if (!a.q_by_tma) {
                 const int total = it.nmt * kBM * kChunks;
-                for (int i0 = tid; i0 < total; i0 += kSoftmaxThreads * 4) {
-                    uint4 v[4];
+                constexpr int kInFlight = kRowTiles * kBM * kChunks / kSoftmaxThreads;
+                uint4 v[kInFlight];
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const int i = i0 + u * kSoftmaxThreads;
-                        v[u] = make_uint4(0u, 0u, 0u, 0u);
-                        if (i < total) {
-                            const int row = i / kChunks, c = i % kChunks;
-                            const int R = it.row_base + row;
-                            if (R < it.M) {
-                                const int t = R / G, h = it.g * G + R % G;
-                                v[u] = __ldg(reinterpret_cast<const uint4*>(
-                                    a.q + ((static_cast<int64_t>(it.b) * a.max_tt + t) * a.Hq + h) * D + c * 8));
-                            }
+                for (int u = 0; u < kInFlight; ++u) {
+                    const int i = tid + u * kSoftmaxThreads;
+                    v[u] = make_uint4(0u, 0u, 0u, 0u);
+                    if (i < total) {
+                        const int row = i / kChunks, c = i % kChunks;
+                        const int R = it.row_base + row;
+                        if (R < it.M) {
+                            const int t = R / G, h = it.g * G + R % G;
+                            v[u] = __ldg(reinterpret_cast<const uint4*>(
+                                a.q + ((static_cast<int64_t>(it.b) * a.max_tt + t) * a.Hq + h) * D + c * 8));
                         }
                     }
+                }
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const int i = i0 + u * kSoftmaxThreads;
-                        if (i < total) {
-                            const int row = i / kChunks, c = i % kChunks;
-                            const int m = row / kBM, rr = row % kBM;
-                            unsigned char* dst = base_ptr + S::kOffQ + m * S::kQTile + (c >> 3) * S::kQPanel +
-                                                 rr * 128 + (((c & 7) ^ (rr & 7)) << 4);
-                            *reinterpret_cast<uint4*>(dst) = v[u];
-                        }
+                for (int u = 0; u < kInFlight; ++u) {
+                    const int i = tid + u * kSoftmaxThreads;
+                    if (i < total) {
+                        const int row = i / kChunks, c = i % kChunks;
+                        const int m = row / kBM, rr = row % kBM;
+                        unsigned char* dst = base_ptr + S::kOffQ + m * S::kQTile + (c >> 3) * S::kQPanel + rr * 128 +
+                                             (((c & 7) ^ (rr & 7)) << 4);
+                        *reinterpret_cast<uint4*>(dst) = v[u];
                     }
                 }
                 fence_proxy_async();
@@ -525,6 +597,10 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
                 }
                 float m_ref = -INFINITY, l_run = 0.f;
                 const uint32_t o_t = tmem + lane_sel + wg * 256 + 128;
+                // PV completions of this row tile seen so far.  pvdone completes once per tile and a
+                // parity wait must never fall two phases behind, so PV(j-1) is observed before P(j)
+                // is handed over (PV(j) cannot be issued earlier): by then it has usually completed.
+                uint32_t pv_seen = jj[wg];
                 const int kv_len = it.L + it.n;
 
                 for (int t = it.t_begin; t < it.t_end; ++t, ++kt_run) {
@@ -539,11 +615,12 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
                     tmem_ld32(tmem + lane_sel + wg * 256 + buf * kBN + 32, sr[1]);
                     tmem_wait_ld();
 
-                    // ---- scale, ancestor mask, row maximum ---------------------------------
+                    // ---- ancestor mask (tiles that reach past the prefix only), row maximum -------
                     const int j0 = t * kBN;
-                    unsigned long long allowed = ~0ull;
+                    float tmax = -INFINITY;
                     if (j0 + kBN > it.L) {
                         const int off = j0 - it.L;  // tile start relative to the first tree slot
+                        unsigned long long allowed;
                         if (off >= 64)
                             allowed = mhi >> (off - 64);
                         else if (off > 0)
@@ -552,31 +629,36 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
                             allowed = mlo;
                         else  // -64 < off < 0: the first -off keys are prefix
                             allowed = (mlo << (-off)) | ((1ull << (-off)) - 1ull);
+#pragma unroll
+                        for (int h = 0; h < 2; ++h)
+#pragma unroll
+                            for (int c = 0; c < 32; ++c) {
+                                float s = __uint_as_float(sr[h][c]);
+                                if (!((allowed >> (h * 32 + c)) & 1ull)) s = -INFINITY;
+                                sr[h][c] = __float_as_uint(s);
+                                tmax = fmaxf(tmax, s);
+                            }
+                    } else {
+#pragma unroll
+                        for (int h = 0; h < 2; ++h)
+#pragma unroll
+                            for (int c = 0; c < 32; c += 2)
+                                tmax = max3(tmax, __uint_as_float(sr[h][c]), __uint_as_float(sr[h][c + 1]));
                     }
-                    float tmax = -INFINITY;
-#pragma unroll
-                    for (int h = 0; h < 2; ++h)
-#pragma unroll
-                        for (int c = 0; c < 32; ++c) {
-                            float s = __uint_as_float(sr[h][c]) * a.scale_log2;
-                            if (!((allowed >> (h * 32 + c)) & 1ull)) s = -INFINITY;
-                            sr[h][c] = __float_as_uint(s);
-                            tmax = fmaxf(tmax, s);
-                        }
+                    tmax *= a.scale_log2;  // the scale is positive: max(scale * s) = scale * max(s)
                     const bool first = (t == it.t_begin);
                     const float m_new = fmaxf(m_ref, tmax);
                     // Lazy rescale: O and l keep the old reference maximum while the true one
                     // grew by less than 2^kRescaleSlack (fp32 accumulators have the head-room).
                     const bool need = !first && (m_new > m_ref + kRescaleSlack);
                     if (first) m_ref = m_new;
-                    bool pv_seen = first;  // every phase of pvdone is observed, so its parity never aliases
                     if (__any_sync(kFull, need)) {
                         // O may only be touched once PV of the previous tile has completed
-                        if (!warp_wait(bar(bar_pvdone(wg)), (jj[wg] - 1u) & 1u, abort_flag, a.status)) {
-                            alive = false;
-                            break;
+                        while (pv_seen < jj[wg]) {
+                            if (!warp_wait(bar(bar_pvdone(wg)), pv_seen & 1u, abort_flag, a.status)) alive = false;
+                            ++pv_seen;
                         }
-                        pv_seen = true;
+                        if (!alive) break;
                         const float corr = need ? ex2_approx(m_ref - m_new) : 1.f;
                         if (need) m_ref = m_new;
                         l_run *= corr;
@@ -610,88 +692,99 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
                         }
                     }
 
-                    // ---- P = exp2(S - m) as bf16 hi + lo, back into the columns S came from ------
-                    float psum = 0.f;
-                    uint32_t plo[32];
-#pragma unroll
-                    for (int c = 0; c < 32; ++c) {
-                        const float p0 = ex2_approx(__uint_as_float(sr[c >> 4][(2 * c) & 31]) - m_use);
-                        const float p1 = ex2_approx(__uint_as_float(sr[c >> 4][(2 * c + 1) & 31]) - m_use);
-                        psum += p0 + p1;
-                        const __nv_bfloat162 hi = __floats2bfloat162_rn(p0, p1);
-                        plo[c] = pack_bf16(p0 - __low2float(hi), p1 - __high2float(hi));
-                        sr[c >> 4][(2 * c) & 31] = *reinterpret_cast<const uint32_t*>(&hi);
-                    }
-                    l_run += psum;
+                    // ---- P = exp2(scale * S - m) as bf16 hi + lo, back into the columns S came from.
+                    // hi is p truncated to bf16, so p - hi is exact and lo = bf16(p - hi) leaves an
+                    // error of 2^-16 p.  Packed fp32 pairs halve the instruction count.
                     {
-                        // hi words sit at the even positions of sr; gather them into one 32-column store
-                        uint32_t phi[32];
+                        const unsigned long long sc2 = pack2(a.scale_log2, a.scale_log2);
+                        const unsigned long long nm2 = pack2(-m_use, -m_use);
+                        unsigned long long psum2 = pack2(0.f, 0.f);
+                        uint32_t plo[32];
 #pragma unroll
-                        for (int c = 0; c < 32; ++c) phi[c] = sr[c >> 4][(2 * c) & 31];
+                        for (int c = 0; c < 32; ++c) {
+                            const int h = c >> 4, e = (2 * c) & 31;
+                            float x0, x1;
+                            unpack2(fma2(pack2(__uint_as_float(sr[h][e]), __uint_as_float(sr[h][e + 1])), sc2, nm2),
+                                    x0, x1);
+                            const float p0 = ex2_approx(x0), p1 = ex2_approx(x1);
+                            const unsigned long long p2 = pack2(p0, p1);
+                            psum2 = add2(psum2, p2);
+                            const uint32_t b0 = __float_as_uint(p0), b1 = __float_as_uint(p1);
+                            const uint32_t hi = __byte_perm(b0, b1, 0x7632);
+                            float l0, l1;
+                            unpack2(sub2(p2, pack2(__uint_as_float(b0 & 0xFFFF0000u), __uint_as_float(b1 & 0xFFFF0000u))),
+                                    l0, l1);
+                            plo[c] = pack_bf16(l0, l1);
+                            sr[0][c] = hi;  // position c was consumed at iteration c / 2
+                        }
+                        float ps0, ps1;
+                        unpack2(psum2, ps0, ps1);
+                        l_run += ps0 + ps1;
                         const uint32_t p_t = tmem + lane_sel + wg * 256 + buf * kBN;
-                        tmem_st32(p_t, phi);
+                        tmem_st32(p_t, sr[0]);
                         tmem_st32(p_t + 32, plo);
                         tmem_wait_st();
                     }
                     if (wg == 0 && j0 + kBN > kv_len) fence_proxy_async();  // the zeroed V rows
-                    if (!pv_seen && !warp_wait(bar(bar_pvdone(wg)), (jj[wg] - 1u) & 1u, abort_flag, a.status)) {
-                        alive = false;
-                        break;
+                    while (pv_seen < jj[wg]) {
+                        if (!warp_wait(bar(bar_pvdone(wg)), pv_seen & 1u, abort_flag, a.status)) alive = false;
+                        ++pv_seen;
                     }
+                    if (!alive) break;
                     tc_fence_before();
-                    mbar_arrive(bar(bar_pfull(wg)));
+                    mbar_arrive(bar(bar_pfull(wg, buf)));
                     ++jj[wg];
                 }
                 if (!alive) break;
 
                 // ---- epilogue --------------------------------------------------------------
                 if (it.t_end > it.t_begin) {
-                    if (!warp_wait(bar(bar_pvdone(wg)), (jj[wg] - 1u) & 1u, abort_flag, a.status)) {
-                        alive = false;
-                        break;
+                    while (pv_seen < jj[wg]) {
+                        if (!warp_wait(bar(bar_pvdone(wg)), pv_seen & 1u, abort_flag, a.status)) alive = false;
+                        ++pv_seen;
                     }
+                    if (!alive) break;
                     tc_fence_after();
-                    if (it.splits == 1) {
-                        const float inv = 1.f / l_run;
-                        __nv_bfloat16* dst = nullptr;
-                        if (row_ok) {
-                            const int t = R / G, h = it.g * G + R % G;
-                            dst = a.o + ((static_cast<int64_t>(it.b) * a.max_tt + t) * a.Hq + h) * D;
+                    const int t = R / G, h = it.g * G + R % G;
+                    const float inv = 1.f / l_run;
+                    __nv_bfloat16* dst = a.o + ((static_cast<int64_t>(it.b) * a.max_tt + t) * a.Hq + h) * D;
+                    float4* po = a.part_o + (static_cast<int64_t>(item) * kRowTiles + wg) * (D / 4) * kBM + r;
+                    if (row_ok) {
+                        if (it.splits == 1) {
                             if (a.lse)
                                 a.lse[(static_cast<int64_t>(it.b) * a.max_tt + t) * a.Hq + h] =
                                     (m_ref + log2f(l_run)) * 0.6931471805599453f;
+                        } else {
+                            __stcg(a.part_ml + (static_cast<int64_t>(item) * kRowTiles + wg) * kBM + r,
+                                   make_float2(m_ref, l_run));
                         }
+                    }
 #pragma unroll 1
-                        for (int c0 = 0; c0 < D; c0 += 32) {
-                            uint32_t orr[32];
-                            tmem_ld32(o_t + c0, orr);
-                            tmem_wait_ld();
-                            if (row_ok) {
+                    for (int c0 = 0; c0 < D; c0 += 64) {
+                        uint32_t orr[2][32];
+                        tmem_ld32(o_t + c0, orr[0]);
+                        tmem_ld32(o_t + c0 + 32, orr[1]);
+                        tmem_wait_ld();
+                        if (!row_ok) continue;
+                        if (it.splits == 1) {
 #pragma unroll
-                                for (int q4 = 0; q4 < 4; ++q4) {
-                                    uint4 v;
-                                    v.x = pack_bf16(__uint_as_float(orr[q4 * 8 + 0]) * inv, __uint_as_float(orr[q4 * 8 + 1]) * inv);
-                                    v.y = pack_bf16(__uint_as_float(orr[q4 * 8 + 2]) * inv, __uint_as_float(orr[q4 * 8 + 3]) * inv);
-                                    v.z = pack_bf16(__uint_as_float(orr[q4 * 8 + 4]) * inv, __uint_as_float(orr[q4 * 8 + 5]) * inv);
-                                    v.w = pack_bf16(__uint_as_float(orr[q4 * 8 + 6]) * inv, __uint_as_float(orr[q4 * 8 + 7]) * inv);
-                                    *reinterpret_cast<uint4*>(dst + c0 + q4 * 8) = v;
-                                }
+                            for (int q8 = 0; q8 < 8; ++q8) {
+                                const uint32_t* w = &orr[q8 >> 2][(q8 & 3) * 8];
+                                uint4 v;
+                                v.x = pack_bf16(__uint_as_float(w[0]) * inv, __uint_as_float(w[1]) * inv);
+                                v.y = pack_bf16(__uint_as_float(w[2]) * inv, __uint_as_float(w[3]) * inv);
+                                v.z = pack_bf16(__uint_as_float(w[4]) * inv, __uint_as_float(w[5]) * inv);
+                                v.w = pack_bf16(__uint_as_float(w[6]) * inv, __uint_as_float(w[7]) * inv);
+                                *reinterpret_cast<uint4*>(dst + c0 + q8 * 8) = v;
                             }
-                        }
-                    } else {
-                        float4* po = a.part_o + (static_cast<int64_t>(item) * kRowTiles + wg) * (D / 4) * kBM + r;
-                        __stcg(a.part_ml + (static_cast<int64_t>(item) * kRowTiles + wg) * kBM + r,
-                               make_float2(m_ref, l_run));
-#pragma unroll 1
-                        for (int c0 = 0; c0 < D; c0 += 32) {
-                            uint32_t orr[32];
-                            tmem_ld32(o_t + c0, orr);
-                            tmem_wait_ld();
+                        } else {
 #pragma unroll
-                            for (int q4 = 0; q4 < 8; ++q4)
+                            for (int q4 = 0; q4 < 16; ++q4) {
+                                const uint32_t* w = &orr[q4 >> 3][(q4 & 7) * 4];
                                 __stcg(po + (c0 / 4 + q4) * kBM,
-                                       make_float4(__uint_as_float(orr[q4 * 4 + 0]), __uint_as_float(orr[q4 * 4 + 1]),
-                                                   __uint_as_float(orr[q4 * 4 + 2]), __uint_as_float(orr[q4 * 4 + 3])));
+                                       make_float4(__uint_as_float(w[0]), __uint_as_float(w[1]), __uint_as_float(w[2]),
+                                                   __uint_as_float(w[3])));
+                            }
                         }
                     }
                     tc_fence_before();
@@ -720,7 +813,9 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
 template <int D>
 __global__ void __launch_bounds__(kCombineThreads) attention_combine_kernel(const AttnArgs a) {
     __shared__ Sched sc;
-    build_sched(a, sc, threadIdx.x, kCombineThreads);
+    pdl_launch_dependents();
+    build_sched(a, sc, threadIdx.x, kCombineThreads);  // inputs of the attention kernel, complete before it ran
+    pdl_wait();                                        // the attention kernel has finished and its writes are visible
     const int G = a.Hq / a.Hkv;
     constexpr int kPerGroup = kRowTiles * kBM * (D / 4);  // (row, 4 columns) work items of a group
     for (int b = 0; b < a.batch; ++b) {
@@ -740,18 +835,34 @@ __global__ void __launch_bounds__(kCombineThreads) attention_combine_kernel(cons
             if (R >= M) continue;
             const int mt = row2 / kBM, r = row2 % kBM;
             const int64_t item_first = sc.item0[b] + static_cast<int64_t>(grp) * splits;
-            float Mx = -INFINITY;
-            for (int s = 0; s < splits; ++s)
-                Mx = fmaxf(Mx, __ldcg(&a.part_ml[((item_first + s) * kRowTiles + mt) * kBM + r].x));
-            float den = 0.f;
+            // one pass over the splits, eight at a time so that their loads are in flight together
+            constexpr int kBatch = 8;
+            float Mx = -INFINITY, den = 0.f;
             float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll 4
-            for (int s = 0; s < splits; ++s) {
-                const float2 ml = __ldcg(&a.part_ml[((item_first + s) * kRowTiles + mt) * kBM + r]);
-                const float4 v = __ldcg(a.part_o + (((item_first + s) * kRowTiles + mt) * (D / 4) + c4) * kBM + r);
-                const float w = (ml.x == -INFINITY) ? 0.f : ex2_approx(ml.x - Mx);
-                den += ml.y * w;
-                acc.x += v.x * w, acc.y += v.y * w, acc.z += v.z * w, acc.w += v.w * w;
+            for (int s0 = 0; s0 < splits; s0 += kBatch) {
+                float2 ml[kBatch];
+                float4 v[kBatch];
+#pragma unroll
+                for (int u = 0; u < kBatch; ++u) {
+                    const int64_t it2 = item_first + min(s0 + u, splits - 1);
+                    ml[u] = __ldcg(&a.part_ml[(it2 * kRowTiles + mt) * kBM + r]);
+                    v[u] = __ldcg(a.part_o + ((it2 * kRowTiles + mt) * (D / 4) + c4) * kBM + r);
+                }
+                float mx4 = Mx;
+#pragma unroll
+                for (int u = 0; u < kBatch; ++u)
+                    if (s0 + u < splits) mx4 = fmaxf(mx4, ml[u].x);
+                if (mx4 == -INFINITY) continue;
+                const float corr = ex2_approx(Mx - mx4);  // 0 on the first batch
+                den *= corr, acc.x *= corr, acc.y *= corr, acc.z *= corr, acc.w *= corr;
+                Mx = mx4;
+#pragma unroll
+                for (int u = 0; u < kBatch; ++u) {
+                    if (s0 + u >= splits) continue;
+                    const float w = ex2_approx(ml[u].x - Mx);  // 0 for an all-masked split
+                    den += ml[u].y * w;
+                    acc.x += v[u].x * w, acc.y += v[u].y * w, acc.z += v[u].z * w, acc.w += v[u].w * w;
+                }
             }
             const float inv = 1.f / den;
             const int t = R / G, h = g * G + R % G;
@@ -804,14 +915,43 @@ bool make_kv_map(CUtensorMap* map, const void* basep, int D, int64_t capacity, i
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// (element, head in group, KV head, token, sequence) view of Q [batch][max_tt][Hq][D]: a box of
+// 64 elements x G heads x 128/G tokens is one 128-row tile in (token, head) row order.
+bool make_q_map(CUtensorMap* map, const void* basep, int D, int G, int Hkv, int max_tt, int batch) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t Hq = static_cast<cuuint64_t>(G) * Hkv;
+    const cuuint64_t dims[5] = {static_cast<cuuint64_t>(D), static_cast<cuuint64_t>(G), static_cast<cuuint64_t>(Hkv),
+                                static_cast<cuuint64_t>(max_tt), static_cast<cuuint64_t>(batch)};
+    const cuuint64_t strides[4] = {static_cast<cuuint64_t>(D) * 2, static_cast<cuuint64_t>(G) * D * 2, Hq * D * 2,
+                                   static_cast<cuuint64_t>(max_tt) * Hq * D * 2};
+    const cuuint32_t box[5] = {64, static_cast<cuuint32_t>(G), 1, static_cast<cuuint32_t>(kBM / G), 1};
+    const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(basep), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Both kernels are launched with programmatic stream serialization: each starts while its
+// predecessor drains and waits (griddepcontrol.wait) before it touches global memory.
+template <typename Kernel, typename... Args>
+cudaError_t launch_pdl(Kernel kernel, int grid, int block, size_t smem, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid), cfg.blockDim = dim3(block), cfg.dynamicSmemBytes = smem, cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr, cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
 template <int D>
 cudaError_t launch_for_dim(const resps_ctx* ctx, const AttnArgs& a, const CUtensorMap& mk, const CUtensorMap& mv,
-                           cudaStream_t st) {
-    tree_attention_kernel<D><<<ctx->ws.attn_grid, kAttnThreads, Smem<D>::kBytes, st>>>(a, mk, mv);
-    cudaError_t e = cudaGetLastError();
+                           const CUtensorMap& mq, cudaStream_t st) {
+    cudaError_t e = launch_pdl(tree_attention_kernel<D>, ctx->ws.attn_grid, kAttnThreads, Smem<D>::kBytes, st, a, mk,
+                               mv, mq);
     if (e != cudaSuccess) return e;
-    attention_combine_kernel<D><<<ctx->ws.attn_combine_grid, kCombineThreads, 0, st>>>(a);
-    return cudaGetLastError();
+    return launch_pdl(attention_combine_kernel<D>, ctx->ws.attn_combine_grid, kCombineThreads, 0, st, a);
 }
 
 }  // namespace
@@ -841,11 +981,18 @@ cudaError_t launch_tree_attention(const resps_ctx* ctx, const resps_step* d_step
     a.max_items = ctx->ws.attn_max_items, a.sched_grid = ctx->ws.attn_grid;
     a.min_tiles = ctx->ws.attn_min_tiles, a.status = ctx->ws.status;
     const int D = ctx->shape.head_dim;
-    CUtensorMap mk, mv;
+    const int G = a.Hq / a.Hkv;
+    a.q_by_tma = (G <= kBM && kBM % G == 0) ? 1 : 0;
+    CUtensorMap mk, mv, mq;
     if (!make_kv_map(&mk, k_cache, D, capacity, a.Hkv, batch, stride_tok, stride_head, stride_seq) ||
         !make_kv_map(&mv, v_cache, D, capacity, a.Hkv, batch, stride_tok, stride_head, stride_seq))
         return cudaErrorInvalidValue;
-    return D == 128 ? launch_for_dim<128>(ctx, a, mk, mv, st) : launch_for_dim<64>(ctx, a, mk, mv, st);
+    if (a.q_by_tma) {
+        if (!make_q_map(&mq, q, D, G, a.Hkv, a.max_tt, batch)) return cudaErrorInvalidValue;
+    } else {
+        mq = mk;  // unused by the kernel
+    }
+    return D == 128 ? launch_for_dim<128>(ctx, a, mk, mv, mq, st) : launch_for_dim<64>(ctx, a, mk, mv, mq, st);
 }
 
 int attention_item_rows() { return kRowTiles * kBM; }
