@@ -4,27 +4,32 @@
 //
 // Split-KV flash-decode on the 5th-generation tensor cores.  The query rows of one
 // KV head (tree token x the Hq/Hkv heads sharing it) are packed into 128-row tiles,
-// so that Q K^T and P V are dense contractions: tcgen05.mma with both operands in
-// fp32 accumulators (S and O) in tensor memory.  K/V tiles of 64 keys are staged by
-// TMA (cp.async.bulk.tensor, one elected thread) into 128-byte-swizzled shared memory
-// through a 4-deep mbarrier ring; a second elected thread issues the MMAs; eight
-// warps (one TMEM lane = one query row per thread) do the scaling, the ancestor
-// bitmask (from registers, only on tiles that reach past the prefix) and the online
-// softmax, and write P back into the tensor-memory columns S came from, from where
-// it is the A operand of P V.  P is kept as two bf16 terms (p = hi + lo): one bf16
-// rounding of the weights alone would cost up to 2^-9 per weight, which shows as about
-// 1 % of an output row's rms in the worst element.
+// so that Q K^T and P V are dense contractions: tcgen05.mma with the fp32
+// accumulators (S and O) in tensor memory.  K/V tiles of 64 keys are staged by TMA
+// (cp.async.bulk.tensor, one elected thread) into 128-byte-swizzled shared memory
+// through a 4-deep mbarrier ring, Q tiles likewise (prefetched for the next item).
 //
-// A CTA works on up to two row tiles (256 rows) of one (sequence, KV head) against a
-// contiguous range of key tiles.  The work list -- every (sequence, KV head, row-tile
-// pair, key split) -- is derived inside the kernel from the device-resident step
-// parameters, so nothing about the launch depends on (TT, d, k, L).  Items whose
-// group has a single split write O directly; the others write un-normalised partials
-// that a second, small kernel combines.
+// A CTA runs two symmetric lanes.  A lane is an MMA-issuing warp, a softmax warpgroup
+// (one TMEM lane = one query row per thread) and a quarter of tensor memory (two S/P
+// buffers and one O accumulator).  The softmax warpgroup scales, applies the ancestor
+// bitmask (from registers, only on tiles that reach past the prefix), keeps the online
+// softmax state and writes P back into the tensor-memory columns S came from, from
+// where it is the A operand of P V.  P is kept as two bf16 terms (p = hi + lo): one
+// bf16 rounding of the weights alone would cost up to 2^-9 per weight, about 1 % of an
+// output row's rms in the worst element.
+//
+// A work item is (sequence, KV head, pair of row tiles, range of key tiles).  With more
+// than 128 rows left, lane x takes row tile x over all key tiles ("row mode");
+// otherwise both lanes take the one row tile and alternate key tiles ("key mode"),
+// ending with two partial results.  The work list is derived inside the kernel from the
+// device-resident step parameters, so nothing about the launch depends on
+// (TT, d, k, L).  Items whose group has a single split in row mode write O directly;
+// all others write un-normalised partials that a second, small kernel combines.
 //
 // Every wait (mbarrier) is bounded: when it runs out the CTA raises
 // RESPS_STATUS_WAIT_TIMEOUT, stops issuing work, drains its copies in flight, frees
-// its tensor memory and returns.
+// its tensor memory and returns.  Every barrier is used so that a waiter can never
+// fall two phases behind (a parity wait would then never return).
 #include <cuda.h>
 
 #include <cmath>
@@ -40,9 +45,9 @@ constexpr int kStages = 4;         // K/V ring depth
 constexpr int kRowTiles = 2;       // row tiles per item
 constexpr int kSoftmaxThreads = 256;
 constexpr int kProducerWarp = 8;
-constexpr int kMmaWarp = 9;
-constexpr int kAttnThreads = 320;
-constexpr int kSyncThreads = 288;  // softmax warps + the MMA warp meet at the end of an item
+constexpr int kMmaWarp0 = 9;       // lane x is issued by warp kMmaWarp0 + x
+constexpr int kAttnThreads = 352;
+constexpr int kSyncThreads = 320;  // softmax warps + the MMA warps meet at the end of an item
 constexpr int kMaxBatchSmem = 256;
 constexpr int kTmemCols = 512;
 constexpr int kCombineThreads = 128;  // small enough to share an SM with a draining attention CTA
@@ -100,6 +105,16 @@ __device__ __forceinline__ void build_sched(const AttnArgs& a, Sched& sc, int ti
         for (int b = 0; b < a.batch; ++b) units += 1ll * a.Hkv * sc.mp[b] * sc.kt[b];
         int tps = static_cast<int>((units + a.sched_grid - 1) / a.sched_grid);
         tps = max(tps, max(a.min_tiles, 1));
+        // ceil(kt / tps) splits per group can add up to more items than CTAs (a second, nearly
+        // empty round); a slightly larger tile count per split then gives a single round.
+        if (a.batch <= 32) {
+            for (int tries = 0; tries < 8; ++tries) {
+                long long cnt = 0;
+                for (int b = 0; b < a.batch; ++b) cnt += 1ll * a.Hkv * sc.mp[b] * ((sc.kt[b] + tps - 1) / tps);
+                if (cnt <= a.sched_grid) break;
+                ++tps;
+            }
+        }
         int items = 0;
         for (int b = 0; b < a.batch; ++b) {
             sc.item0[b] = items;
@@ -185,6 +200,16 @@ __device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatil
                                           int32_t* status) {
     const bool ok = mbar_wait(bar, parity, abort_flag, status);
     return __all_sync(0xFFFFFFFFu, ok);
+}
+// One lane of a converged warp.
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile(
+        "{\n\t.reg .pred P;\n\t"
+        "elect.sync _|P, 0xFFFFFFFF;\n\t"
+        "selp.u32 %0, 1, 0, P;\n\t}"
+        : "=r"(pred));
+    return pred != 0;
 }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -341,7 +366,7 @@ __device__ __forceinline__ constexpr int bar_kfull(int s) { return s; }
 __device__ __forceinline__ constexpr int bar_vfull(int s) { return kStages + s; }
 __device__ __forceinline__ constexpr int bar_kvempty(int s) { return 2 * kStages + s; }
 __device__ __forceinline__ constexpr int bar_qfull() { return 3 * kStages; }
-// S and P share a TMEM buffer (tile j uses buffer j & 1) and each buffer has its own pair of
+// Lane m's S and P share a TMEM buffer (its j-th tile uses buffer j & 1) and each buffer has its own pair of
 // barriers: a buffer's next phase cannot complete before the other side has observed the
 // current one (QK(j+2) is issued after PV(j), which is issued after pfull(j) was seen), so a
 // parity wait never falls two phases behind.  One pfull barrier for both buffers would: the
@@ -374,10 +399,10 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
         for (int s = 0; s < kStages; ++s) {
             mbar_init(bar(bar_kfull(s)), 1);
             mbar_init(bar(bar_vfull(s)), 1);
-            mbar_init(bar(bar_kvempty(s)), 1);
+            mbar_init(bar(bar_kvempty(s)), 2);  // one arrival per lane
         }
         mbar_init(bar(bar_qfull()), a.q_by_tma ? 1 : kSoftmaxThreads);
-        mbar_init(bar(bar_qempty()), 1);
+        mbar_init(bar(bar_qempty()), 2);
         for (int m = 0; m < kRowTiles; ++m) {
             for (int bf = 0; bf < 2; ++bf) {
                 mbar_init(bar(bar_sfull(m, bf)), 1);
@@ -388,7 +413,7 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
         mbar_init(bar(bar_item()), kSyncThreads);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == kMmaWarp) {
+    if (warp == kMmaWarp0) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
                          base + S::kOffMisc),
                      "r"(kTmemCols)
@@ -411,10 +436,10 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
     const uint32_t tmem = *tmem_slot;
     const int total_items = min(sc.item0[a.batch], a.max_items);
 
-    // running use counts of the barrier families (identical in every role: all roles walk
-    // the same items and tiles in the same order)
-    uint32_t kt_run = 0;                 // K/V ring uses
-    uint32_t jj[kRowTiles] = {0, 0};     // tiles processed per row tile (S buffers, P, PV)
+    // Running use counts of the barrier families.  Every role walks the same items and tiles in
+    // the same order, so each keeps its own copy.
+    uint32_t kt_run = 0;     // K/V ring uses (all tiles of all items)
+    uint32_t jx = 0;         // tiles this lane has taken (S/P buffers, PV completions)
     uint32_t items_run = 0;
     bool alive = true;
 
@@ -465,85 +490,94 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
                 if (!mbar_wait(bar(bar_vfull(s)), ph, abort_flag, a.status)) break;
             }
         }
-    } else if (warp == kMmaWarp) {
-        // ================================ MMA issuer ======================================
+    } else if (warp >= kMmaWarp0) {
+        // ================================ MMA issuer of lane x ============================
+        // The whole warp walks the loop and waits (so that every value stays warp-uniform);
+        // one elected lane issues.  The MMAs of one thread execute in issue order: QK of this
+        // lane's tile j+1 is issued before PV of tile j, so the tensor pipe has S(j+1) to work on
+        // while the softmax warps turn S(j) into P(j), and QK(j+2) cannot overwrite the TMEM
+        // buffer j & 1 before PV(j) has read P(j) from it.
+        const int x = warp - kMmaWarp0;
         constexpr uint32_t kIdescQK = instr_desc(kBN, false);
         constexpr uint32_t kIdescPV = instr_desc(D, true);
+        // Descriptors differ only in the (16-byte granular) start address, the low 14 bits.
+        const uint64_t qdesc0 = smem_desc(base + S::kOffQ, 16, 1024);
+        const uint64_t kdesc0 = smem_desc(base + S::kOffK, 16, 1024);
+        const uint64_t vdesc0 = smem_desc(base + S::kOffV, S::kKVPanel, 1024);
+        const uint32_t o_t = tmem + x * 256 + 128;
         for (int item = blockIdx.x; item < total_items && alive; item += gridDim.x, ++items_run) {
             const Item it = decode_item(sc, item, G);
-            if (lane == 0) {
-                alive = mbar_wait(bar(bar_qfull()), items_run & 1u, abort_flag, a.status);
+            const bool row_mode = it.nmt == 2;
+            const uint64_t qdesc = qdesc0 + static_cast<uint64_t>((row_mode ? x : 0) * (S::kQTile >> 4));
+            alive = warp_wait(bar(bar_qfull()), items_run & 1u, abort_flag, a.status);
+            tc_fence_after();
+            bool have_prev = false, first_pv = true;
+            uint32_t prev_kt = 0, prev_j = 0;
+            auto issue_pv = [&]() {
+                const int s = prev_kt % kStages;
+                if (!warp_wait(bar(bar_vfull(s)), (prev_kt / kStages) & 1u, abort_flag, a.status)) return false;
+                if (!warp_wait(bar(bar_pfull(x, prev_j & 1u)), (prev_j >> 1) & 1u, abort_flag, a.status)) return false;
                 tc_fence_after();
-                // PV of a tile is issued after QK of the next one, so the tensor pipe has S(j+1)
-                // to work on while the softmax warps turn S(j) into P(j).  S(j) and P(j) share the
-                // TMEM buffer j & 1; the MMAs of one thread execute in issue order, so QK(j+2) cannot
-                // overwrite it before PV(j) has read it.
-                // Descriptors differ only in the (16-byte granular) start address, the low 14 bits.
-                const uint64_t qdesc0 = smem_desc(base + S::kOffQ, 16, 1024);
-                const uint64_t kdesc0 = smem_desc(base + S::kOffK, 16, 1024);
-                const uint64_t vdesc0 = smem_desc(base + S::kOffV, S::kKVPanel, 1024);
-                auto issue_pv = [&](uint32_t kt_use, const uint32_t (&jj_use)[kRowTiles], bool first_tile) {
-                    const int s = kt_use % kStages;
-                    if (!mbar_wait(bar(bar_vfull(s)), (kt_use / kStages) & 1u, abort_flag, a.status)) return false;
-                    for (int m = 0; m < it.nmt; ++m)
-                        if (!mbar_wait(bar(bar_pfull(m, jj_use[m] & 1u)), (jj_use[m] >> 1) & 1u, abort_flag, a.status))
-                            return false;
-                    tc_fence_after();
+                if (elect_one()) {
                     const uint64_t vdesc = vdesc0 + static_cast<uint64_t>(s * (S::kKVTile >> 4));
-                    for (int m = 0; m < it.nmt; ++m) {
-                        const uint32_t o_t = tmem + m * 256 + 128;
-                        const uint32_t p_t = tmem + m * 256 + (jj_use[m] & 1u) * kBN;  // hi: +0, lo: +32
+                    const uint32_t p_t = tmem + x * 256 + (prev_j & 1u) * kBN;  // hi: +0, lo: +32
 #pragma unroll
-                        for (int kk = 0; kk < kBN / 16; ++kk) {
-                            umma_ts(o_t, p_t + kk * 8, vdesc + kk * (2048 >> 4), kIdescPV,
-                                    (first_tile && kk == 0) ? 0u : 1u);
-                            umma_ts(o_t, p_t + 32 + kk * 8, vdesc + kk * (2048 >> 4), kIdescPV, 1u);
-                        }
-                        umma_commit(bar(bar_pvdone(m)));
+                    for (int kk = 0; kk < kBN / 16; ++kk) {
+                        umma_ts(o_t, p_t + kk * 8, vdesc + kk * (2048 >> 4), kIdescPV, (first_pv && kk == 0) ? 0u : 1u);
+                        umma_ts(o_t, p_t + 32 + kk * 8, vdesc + kk * (2048 >> 4), kIdescPV, 1u);
                     }
+                    umma_commit(bar(bar_pvdone(x)));
                     umma_commit(bar(bar_kvempty(s)));
-                    return true;
-                };
-                uint32_t prev_kt = 0, prev_jj[kRowTiles] = {0, 0};
-                for (int t = it.t_begin; t < it.t_end && alive; ++t) {
-                    const int s = kt_run % kStages;
-                    alive = mbar_wait(bar(bar_kfull(s)), (kt_run / kStages) & 1u, abort_flag, a.status);
-                    if (!alive) break;
+                }
+                __syncwarp();
+                first_pv = false;
+                return true;
+            };
+            for (int t = it.t_begin; t < it.t_end && alive; ++t, ++kt_run) {
+                const int s = kt_run % kStages;
+                // every tile is waited for, own or not: it paces this lane's arrivals on kvempty
+                alive = warp_wait(bar(bar_kfull(s)), (kt_run / kStages) & 1u, abort_flag, a.status);
+                if (!alive) break;
+                const bool own = row_mode || (((t - it.t_begin) & 1) == x);
+                if (own) {
                     tc_fence_after();
-                    const uint64_t kdesc = kdesc0 + static_cast<uint64_t>(s * (S::kKVTile >> 4));
-                    for (int m = 0; m < it.nmt; ++m) {
-                        const uint32_t s_t = tmem + m * 256 + (jj[m] & 1u) * kBN;
-                        const uint64_t qdesc = qdesc0 + static_cast<uint64_t>(m * (S::kQTile >> 4));
+                    if (elect_one()) {
+                        const uint64_t kdesc = kdesc0 + static_cast<uint64_t>(s * (S::kKVTile >> 4));
+                        const uint32_t s_t = tmem + x * 256 + (jx & 1u) * kBN;
 #pragma unroll
                         for (int ks = 0; ks < D / 16; ++ks)
                             umma(s_t, qdesc + ((ks >> 2) * (S::kQPanel >> 4) + (ks & 3) * 2),
                                  kdesc + ((ks >> 2) * (S::kKVPanel >> 4) + (ks & 3) * 2), kIdescQK, ks > 0 ? 1u : 0u);
-                        umma_commit(bar(bar_sfull(m, jj[m] & 1u)));
+                        umma_commit(bar(bar_sfull(x, jx & 1u)));
                     }
-                    if (t + 1 == it.t_end) umma_commit(bar(bar_qempty()));  // Q is free for the next item
-                    if (t > it.t_begin) alive = issue_pv(prev_kt, prev_jj, t - 1 == it.t_begin);
-                    prev_kt = kt_run;
-                    prev_jj[0] = jj[0], prev_jj[1] = jj[1];
-                    ++kt_run;
-                    for (int m = 0; m < it.nmt; ++m) ++jj[m];
+                    __syncwarp();
+                    if (have_prev) alive = issue_pv();
+                    have_prev = true, prev_kt = kt_run, prev_j = jx;
+                    ++jx;
+                } else if (elect_one()) {
+                    mbar_arrive(bar(bar_kvempty(s)));  // the other lane's tile: nothing of this lane reads it
                 }
-                if (alive && it.t_end > it.t_begin) alive = issue_pv(prev_kt, prev_jj, it.t_end - 1 == it.t_begin);
-                tc_fence_before();
+                // Q is free for the next item once the last QK^T of both lanes has completed
+                if (t + 1 == it.t_end && elect_one()) umma_commit(bar(bar_qempty()));
+                __syncwarp();
             }
-            alive = __shfl_sync(kFull, alive ? 1 : 0, 0) != 0;
+            if (alive && have_prev) alive = issue_pv();
+            tc_fence_before();
             if (!alive) break;
             // end of item: the softmax warps have read O and S, Q and P may be overwritten
             mbar_arrive(bar(bar_item()));
             alive = warp_wait(bar(bar_item()), items_run & 1u, abort_flag, a.status);
         }
     } else {
-        // ================================ softmax warps ===================================
-        const int wg = warp >> 2;                      // row tile this warp works on
+        // ================================ softmax warpgroup of lane x =====================
+        const int x = warp >> 2;
         const int r = (warp & 3) * 32 + lane;          // row inside the tile = TMEM lane
         const uint32_t lane_sel = static_cast<uint32_t>((warp & 3) * 32) << 16;
+        const uint32_t o_t = tmem + lane_sel + x * 256 + 128;
         constexpr int kChunks = D / 8;                 // 16-byte pieces of a row
         for (int item = blockIdx.x; item < total_items && alive; item += gridDim.x, ++items_run) {
             const Item it = decode_item(sc, item, G);
+            const bool row_mode = it.nmt == 2;
             // ---- Q tiles -> shared memory in the swizzled K-major layout (only when the group
             // size does not allow the TMA view) ---------------------------------------------
             if (!a.q_by_tma) {
@@ -579,219 +613,219 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
                 mbar_arrive(bar(bar_qfull()));
             }
 
-            if (wg < it.nmt) {
-                const int R = it.row_base + wg * kBM + r;
-                const bool row_ok = R < it.M;
-                unsigned long long mlo = 0ull, mhi = 0ull;
-                if (row_ok) {
-                    const int t = R / G;
-                    mlo = a.mask[(static_cast<int64_t>(it.b) * a.max_tt + t) * 2 + 0];
-                    mhi = a.mask[(static_cast<int64_t>(it.b) * a.max_tt + t) * 2 + 1];
-                    // only nodes of this tree can be visible
-                    if (it.n < 64) {
-                        mlo &= (1ull << it.n) - 1ull;
-                        mhi = 0ull;
-                    } else if (it.n < 128) {
-                        mhi &= (1ull << (it.n - 64)) - 1ull;
-                    }
+            const int R = it.row_base + (row_mode ? x * kBM : 0) + r;
+            const bool row_ok = R < it.M;
+            unsigned long long mlo = 0ull, mhi = 0ull;
+            if (row_ok) {
+                const int t = R / G;
+                mlo = a.mask[(static_cast<int64_t>(it.b) * a.max_tt + t) * 2 + 0];
+                mhi = a.mask[(static_cast<int64_t>(it.b) * a.max_tt + t) * 2 + 1];
+                // only nodes of this tree can be visible
+                if (it.n < 64) {
+                    mlo &= (1ull << it.n) - 1ull;
+                    mhi = 0ull;
+                } else if (it.n < 128) {
+                    mhi &= (1ull << (it.n - 64)) - 1ull;
                 }
-                float m_ref = -INFINITY, l_run = 0.f;
-                const uint32_t o_t = tmem + lane_sel + wg * 256 + 128;
-                // PV completions of this row tile seen so far.  pvdone completes once per tile and a
-                // parity wait must never fall two phases behind, so PV(j-1) is observed before P(j)
-                // is handed over (PV(j) cannot be issued earlier): by then it has usually completed.
-                uint32_t pv_seen = jj[wg];
-                const int kv_len = it.L + it.n;
+            }
+            float m_ref = -INFINITY, l_run = 0.f;
+            const int kv_len = it.L + it.n;
+            // PV completions of this lane seen so far.  pvdone completes once per tile and a parity
+            // wait must never fall two phases behind, so PV(j-1) is observed before P(j) is handed
+            // over (PV(j) cannot be issued earlier): by then it has usually completed.
+            uint32_t pv_seen = jx;
+            bool first = true;
 
-                for (int t = it.t_begin; t < it.t_end; ++t, ++kt_run) {
-                    const uint32_t buf = jj[wg] & 1u;
-                    if (!warp_wait(bar(bar_sfull(wg, buf)), (jj[wg] >> 1) & 1u, abort_flag, a.status)) {
+            for (int t = it.t_begin; t < it.t_end; ++t, ++kt_run) {
+                if (!(row_mode || (((t - it.t_begin) & 1) == x))) continue;
+                const uint32_t buf = jx & 1u;
+                if (!warp_wait(bar(bar_sfull(x, buf)), (jx >> 1) & 1u, abort_flag, a.status)) {
+                    alive = false;
+                    break;
+                }
+                tc_fence_after();
+                uint32_t sr[2][32];
+                tmem_ld32(tmem + lane_sel + x * 256 + buf * kBN, sr[0]);
+                tmem_ld32(tmem + lane_sel + x * 256 + buf * kBN + 32, sr[1]);
+                tmem_wait_ld();
+
+                // ---- ancestor mask (tiles that reach past the prefix only), row maximum -------
+                const int j0 = t * kBN;
+                float tmax = -INFINITY;
+                if (j0 + kBN > it.L) {
+                    const int off = j0 - it.L;  // tile start relative to the first tree slot
+                    unsigned long long allowed;
+                    if (off >= 64)
+                        allowed = mhi >> (off - 64);
+                    else if (off > 0)
+                        allowed = (mlo >> off) | (mhi << (64 - off));
+                    else if (off == 0)
+                        allowed = mlo;
+                    else  // -64 < off < 0: the first -off keys are prefix
+                        allowed = (mlo << (-off)) | ((1ull << (-off)) - 1ull);
+#pragma unroll
+                    for (int h = 0; h < 2; ++h)
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) {
+                            float s = __uint_as_float(sr[h][c]);
+                            if (!((allowed >> (h * 32 + c)) & 1ull)) s = -INFINITY;
+                            sr[h][c] = __float_as_uint(s);
+                            tmax = fmaxf(tmax, s);
+                        }
+                } else {
+#pragma unroll
+                    for (int h = 0; h < 2; ++h)
+#pragma unroll
+                        for (int c = 0; c < 32; c += 2)
+                            tmax = max3(tmax, __uint_as_float(sr[h][c]), __uint_as_float(sr[h][c + 1]));
+                }
+                tmax *= a.scale_log2;  // the scale is positive: max(scale * s) = scale * max(s)
+                const float m_new = fmaxf(m_ref, tmax);
+                // Lazy rescale: O and l keep the old reference maximum while the true one
+                // grew by less than 2^kRescaleSlack (fp32 accumulators have the head-room).
+                const bool need = !first && (m_new > m_ref + kRescaleSlack);
+                if (first) m_ref = m_new;
+                if (__any_sync(kFull, need)) {
+                    // O may only be touched once PV of the previous tile has completed
+                    while (pv_seen < jx) {
+                        if (!warp_wait(bar(bar_pvdone(x)), pv_seen & 1u, abort_flag, a.status)) alive = false;
+                        ++pv_seen;
+                    }
+                    if (!alive) break;
+                    const float corr = need ? ex2_approx(m_ref - m_new) : 1.f;
+                    if (need) m_ref = m_new;
+                    l_run *= corr;
+                    tc_fence_after();
+#pragma unroll 1
+                    for (int c0 = 0; c0 < D; c0 += 32) {
+                        uint32_t orr[32];
+                        tmem_ld32(o_t + c0, orr);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) orr[c] = __float_as_uint(__uint_as_float(orr[c]) * corr);
+                        tmem_st32(o_t + c0, orr);
+                    }
+                    tmem_wait_st();
+                }
+                const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
+
+                // ---- stale V rows of the sequence's last tile must not reach the MMA (in row mode
+                // both lanes clear them: each lane's PV is ordered behind its own warpgroup only) ----
+                const bool clear_v = j0 + kBN > kv_len;
+                if (clear_v) {
+                    const int s = kt_run % kStages;
+                    if (!warp_wait(bar(bar_vfull(s)), (kt_run / kStages) & 1u, abort_flag, a.status)) {
                         alive = false;
                         break;
                     }
-                    tc_fence_after();
-                    uint32_t sr[2][32];
-                    tmem_ld32(tmem + lane_sel + wg * 256 + buf * kBN, sr[0]);
-                    tmem_ld32(tmem + lane_sel + wg * 256 + buf * kBN + 32, sr[1]);
-                    tmem_wait_ld();
+                    const int valid = kv_len - j0;
+                    unsigned char* vt = base_ptr + S::kOffV + s * S::kKVTile;
+                    for (int i = r; i < (kBN - valid) * 8 * S::kPanels; i += kBM) {
+                        const int row = valid + i / (8 * S::kPanels), cc = i % (8 * S::kPanels);
+                        *reinterpret_cast<uint4*>(vt + (cc >> 3) * S::kKVPanel + row * 128 + ((cc & 7) << 4)) =
+                            make_uint4(0u, 0u, 0u, 0u);
+                    }
+                }
 
-                    // ---- ancestor mask (tiles that reach past the prefix only), row maximum -------
-                    const int j0 = t * kBN;
-                    float tmax = -INFINITY;
-                    if (j0 + kBN > it.L) {
-                        const int off = j0 - it.L;  // tile start relative to the first tree slot
-                        unsigned long long allowed;
-                        if (off >= 64)
-                            allowed = mhi >> (off - 64);
-                        else if (off > 0)
-                            allowed = (mlo >> off) | (mhi << (64 - off));
-                        else if (off == 0)
-                            allowed = mlo;
-                        else  // -64 < off < 0: the first -off keys are prefix
-                            allowed = (mlo << (-off)) | ((1ull << (-off)) - 1ull);
+                // ---- P = exp2(scale * S - m) as bf16 hi + lo, back into the columns S came from.
+                // hi is p truncated to bf16, so p - hi is exact and lo = bf16(p - hi) leaves an
+                // error of 2^-16 p.  Packed fp32 pairs halve the instruction count.
+                {
+                    const unsigned long long sc2 = pack2(a.scale_log2, a.scale_log2);
+                    const unsigned long long nm2 = pack2(-m_use, -m_use);
+                    unsigned long long psum2 = pack2(0.f, 0.f);
+                    uint32_t plo[32];
 #pragma unroll
-                        for (int h = 0; h < 2; ++h)
-#pragma unroll
-                            for (int c = 0; c < 32; ++c) {
-                                float s = __uint_as_float(sr[h][c]);
-                                if (!((allowed >> (h * 32 + c)) & 1ull)) s = -INFINITY;
-                                sr[h][c] = __float_as_uint(s);
-                                tmax = fmaxf(tmax, s);
-                            }
-                    } else {
-#pragma unroll
-                        for (int h = 0; h < 2; ++h)
-#pragma unroll
-                            for (int c = 0; c < 32; c += 2)
-                                tmax = max3(tmax, __uint_as_float(sr[h][c]), __uint_as_float(sr[h][c + 1]));
+                    for (int c = 0; c < 32; ++c) {
+                        const int h = c >> 4, e = (2 * c) & 31;
+                        float x0, x1;
+                        unpack2(fma2(pack2(__uint_as_float(sr[h][e]), __uint_as_float(sr[h][e + 1])), sc2, nm2), x0, x1);
+                        const float p0 = ex2_approx(x0), p1 = ex2_approx(x1);
+                        const unsigned long long p2 = pack2(p0, p1);
+                        psum2 = add2(psum2, p2);
+                        const uint32_t b0 = __float_as_uint(p0), b1 = __float_as_uint(p1);
+                        const uint32_t hi = __byte_perm(b0, b1, 0x7632);
+                        float l0, l1;
+                        unpack2(sub2(p2, pack2(__uint_as_float(b0 & 0xFFFF0000u), __uint_as_float(b1 & 0xFFFF0000u))), l0,
+                                l1);
+                        plo[c] = pack_bf16(l0, l1);
+                        sr[0][c] = hi;  // position c was consumed at iteration c / 2
                     }
-                    tmax *= a.scale_log2;  // the scale is positive: max(scale * s) = scale * max(s)
-                    const bool first = (t == it.t_begin);
-                    const float m_new = fmaxf(m_ref, tmax);
-                    // Lazy rescale: O and l keep the old reference maximum while the true one
-                    // grew by less than 2^kRescaleSlack (fp32 accumulators have the head-room).
-                    const bool need = !first && (m_new > m_ref + kRescaleSlack);
-                    if (first) m_ref = m_new;
-                    if (__any_sync(kFull, need)) {
-                        // O may only be touched once PV of the previous tile has completed
-                        while (pv_seen < jj[wg]) {
-                            if (!warp_wait(bar(bar_pvdone(wg)), pv_seen & 1u, abort_flag, a.status)) alive = false;
-                            ++pv_seen;
-                        }
-                        if (!alive) break;
-                        const float corr = need ? ex2_approx(m_ref - m_new) : 1.f;
-                        if (need) m_ref = m_new;
-                        l_run *= corr;
-                        tc_fence_after();
-#pragma unroll 1
-                        for (int c0 = 0; c0 < D; c0 += 32) {
-                            uint32_t orr[32];
-                            tmem_ld32(o_t + c0, orr);
-                            tmem_wait_ld();
-#pragma unroll
-                            for (int c = 0; c < 32; ++c) orr[c] = __float_as_uint(__uint_as_float(orr[c]) * corr);
-                            tmem_st32(o_t + c0, orr);
-                        }
-                        tmem_wait_st();
-                    }
-                    const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
-
-                    // ---- stale V rows of the sequence's last tile must not reach the MMA --------
-                    if (wg == 0 && j0 + kBN > kv_len) {
-                        const int s = kt_run % kStages;
-                        if (!warp_wait(bar(bar_vfull(s)), (kt_run / kStages) & 1u, abort_flag, a.status)) {
-                            alive = false;
-                            break;
-                        }
-                        const int valid = kv_len - j0;
-                        unsigned char* vt = base_ptr + S::kOffV + s * S::kKVTile;
-                        for (int i = r; i < (kBN - valid) * 8 * S::kPanels; i += kBM) {
-                            const int row = valid + i / (8 * S::kPanels), cc = i % (8 * S::kPanels);
-                            *reinterpret_cast<uint4*>(vt + (cc >> 3) * S::kKVPanel + row * 128 + ((cc & 7) << 4)) =
-                                make_uint4(0u, 0u, 0u, 0u);
-                        }
-                    }
-
-                    // ---- P = exp2(scale * S - m) as bf16 hi + lo, back into the columns S came from.
-                    // hi is p truncated to bf16, so p - hi is exact and lo = bf16(p - hi) leaves an
-                    // error of 2^-16 p.  Packed fp32 pairs halve the instruction count.
-                    {
-                        const unsigned long long sc2 = pack2(a.scale_log2, a.scale_log2);
-                        const unsigned long long nm2 = pack2(-m_use, -m_use);
-                        unsigned long long psum2 = pack2(0.f, 0.f);
-                        uint32_t plo[32];
-#pragma unroll
-                        for (int c = 0; c < 32; ++c) {
-                            const int h = c >> 4, e = (2 * c) & 31;
-                            float x0, x1;
-                            unpack2(fma2(pack2(__uint_as_float(sr[h][e]), __uint_as_float(sr[h][e + 1])), sc2, nm2),
-                                    x0, x1);
-                            const float p0 = ex2_approx(x0), p1 = ex2_approx(x1);
-                            const unsigned long long p2 = pack2(p0, p1);
-                            psum2 = add2(psum2, p2);
-                            const uint32_t b0 = __float_as_uint(p0), b1 = __float_as_uint(p1);
-                            const uint32_t hi = __byte_perm(b0, b1, 0x7632);
-                            float l0, l1;
-                            unpack2(sub2(p2, pack2(__uint_as_float(b0 & 0xFFFF0000u), __uint_as_float(b1 & 0xFFFF0000u))),
-                                    l0, l1);
-                            plo[c] = pack_bf16(l0, l1);
-                            sr[0][c] = hi;  // position c was consumed at iteration c / 2
-                        }
-                        float ps0, ps1;
-                        unpack2(psum2, ps0, ps1);
-                        l_run += ps0 + ps1;
-                        const uint32_t p_t = tmem + lane_sel + wg * 256 + buf * kBN;
-                        tmem_st32(p_t, sr[0]);
-                        tmem_st32(p_t + 32, plo);
-                        tmem_wait_st();
-                    }
-                    if (wg == 0 && j0 + kBN > kv_len) fence_proxy_async();  // the zeroed V rows
-                    while (pv_seen < jj[wg]) {
-                        if (!warp_wait(bar(bar_pvdone(wg)), pv_seen & 1u, abort_flag, a.status)) alive = false;
-                        ++pv_seen;
-                    }
-                    if (!alive) break;
-                    tc_fence_before();
-                    mbar_arrive(bar(bar_pfull(wg, buf)));
-                    ++jj[wg];
+                    float ps0, ps1;
+                    unpack2(psum2, ps0, ps1);
+                    l_run += ps0 + ps1;
+                    const uint32_t p_t = tmem + lane_sel + x * 256 + buf * kBN;
+                    tmem_st32(p_t, sr[0]);
+                    tmem_st32(p_t + 32, plo);
+                    tmem_wait_st();
+                }
+                if (clear_v) fence_proxy_async();
+                while (pv_seen < jx) {
+                    if (!warp_wait(bar(bar_pvdone(x)), pv_seen & 1u, abort_flag, a.status)) alive = false;
+                    ++pv_seen;
                 }
                 if (!alive) break;
+                tc_fence_before();
+                mbar_arrive(bar(bar_pfull(x, buf)));
+                ++jx;
+                first = false;
+            }
+            if (!alive) break;
 
-                // ---- epilogue --------------------------------------------------------------
-                if (it.t_end > it.t_begin) {
-                    while (pv_seen < jj[wg]) {
-                        if (!warp_wait(bar(bar_pvdone(wg)), pv_seen & 1u, abort_flag, a.status)) alive = false;
-                        ++pv_seen;
-                    }
-                    if (!alive) break;
-                    tc_fence_after();
-                    const int t = R / G, h = it.g * G + R % G;
-                    const float inv = 1.f / l_run;
-                    __nv_bfloat16* dst = a.o + ((static_cast<int64_t>(it.b) * a.max_tt + t) * a.Hq + h) * D;
-                    float4* po = a.part_o + (static_cast<int64_t>(item) * kRowTiles + wg) * (D / 4) * kBM + r;
-                    if (row_ok) {
-                        if (it.splits == 1) {
-                            if (a.lse)
-                                a.lse[(static_cast<int64_t>(it.b) * a.max_tt + t) * a.Hq + h] =
-                                    (m_ref + log2f(l_run)) * 0.6931471805599453f;
-                        } else {
-                            __stcg(a.part_ml + (static_cast<int64_t>(item) * kRowTiles + wg) * kBM + r,
-                                   make_float2(m_ref, l_run));
-                        }
-                    }
-#pragma unroll 1
-                    for (int c0 = 0; c0 < D; c0 += 64) {
-                        uint32_t orr[2][32];
-                        tmem_ld32(o_t + c0, orr[0]);
-                        tmem_ld32(o_t + c0 + 32, orr[1]);
-                        tmem_wait_ld();
-                        if (!row_ok) continue;
-                        if (it.splits == 1) {
-#pragma unroll
-                            for (int q8 = 0; q8 < 8; ++q8) {
-                                const uint32_t* w = &orr[q8 >> 2][(q8 & 3) * 8];
-                                uint4 v;
-                                v.x = pack_bf16(__uint_as_float(w[0]) * inv, __uint_as_float(w[1]) * inv);
-                                v.y = pack_bf16(__uint_as_float(w[2]) * inv, __uint_as_float(w[3]) * inv);
-                                v.z = pack_bf16(__uint_as_float(w[4]) * inv, __uint_as_float(w[5]) * inv);
-                                v.w = pack_bf16(__uint_as_float(w[6]) * inv, __uint_as_float(w[7]) * inv);
-                                *reinterpret_cast<uint4*>(dst + c0 + q8 * 8) = v;
-                            }
-                        } else {
-#pragma unroll
-                            for (int q4 = 0; q4 < 16; ++q4) {
-                                const uint32_t* w = &orr[q4 >> 3][(q4 & 7) * 4];
-                                __stcg(po + (c0 / 4 + q4) * kBM,
-                                       make_float4(__uint_as_float(w[0]), __uint_as_float(w[1]), __uint_as_float(w[2]),
-                                                   __uint_as_float(w[3])));
-                            }
-                        }
-                    }
-                    tc_fence_before();
+            // ---- epilogue --------------------------------------------------------------
+            const bool direct = row_mode && it.splits == 1;
+            if (!first) {
+                while (pv_seen < jx) {
+                    if (!warp_wait(bar(bar_pvdone(x)), pv_seen & 1u, abort_flag, a.status)) alive = false;
+                    ++pv_seen;
                 }
-            } else {
-                // this warp's row tile does not exist in this item: keep the ring counter in step
-                kt_run += static_cast<uint32_t>(it.t_end - it.t_begin);
+                if (!alive) break;
+                tc_fence_after();
+                const int t = R / G, h = it.g * G + R % G;
+                const float inv = 1.f / l_run;
+                __nv_bfloat16* dst = a.o + ((static_cast<int64_t>(it.b) * a.max_tt + t) * a.Hq + h) * D;
+                float4* po = a.part_o + (static_cast<int64_t>(item) * kRowTiles + x) * (D / 4) * kBM + r;
+                if (row_ok) {
+                    if (direct) {
+                        if (a.lse)
+                            a.lse[(static_cast<int64_t>(it.b) * a.max_tt + t) * a.Hq + h] =
+                                (m_ref + log2f(l_run)) * 0.6931471805599453f;
+                    } else {
+                        __stcg(a.part_ml + (static_cast<int64_t>(item) * kRowTiles + x) * kBM + r,
+                               make_float2(m_ref, l_run));
+                    }
+                }
+#pragma unroll 1
+                for (int c0 = 0; c0 < D; c0 += 64) {
+                    uint32_t orr[2][32];
+                    tmem_ld32(o_t + c0, orr[0]);
+                    tmem_ld32(o_t + c0 + 32, orr[1]);
+                    tmem_wait_ld();
+                    if (!row_ok) continue;
+                    if (direct) {
+#pragma unroll
+                        for (int q8 = 0; q8 < 8; ++q8) {
+                            const uint32_t* w = &orr[q8 >> 2][(q8 & 3) * 8];
+                            uint4 v;
+                            v.x = pack_bf16(__uint_as_float(w[0]) * inv, __uint_as_float(w[1]) * inv);
+                            v.y = pack_bf16(__uint_as_float(w[2]) * inv, __uint_as_float(w[3]) * inv);
+                            v.z = pack_bf16(__uint_as_float(w[4]) * inv, __uint_as_float(w[5]) * inv);
+                            v.w = pack_bf16(__uint_as_float(w[6]) * inv, __uint_as_float(w[7]) * inv);
+                            *reinterpret_cast<uint4*>(dst + c0 + q8 * 8) = v;
+                        }
+                    } else {
+#pragma unroll
+                        for (int q4 = 0; q4 < 16; ++q4) {
+                            const uint32_t* w = &orr[q4 >> 3][(q4 & 7) * 4];
+                            __stcg(po + (c0 / 4 + q4) * kBM, make_float4(__uint_as_float(w[0]), __uint_as_float(w[1]),
+                                                                       __uint_as_float(w[2]), __uint_as_float(w[3])));
+                        }
+                    }
+                }
+                tc_fence_before();
+            } else if (!row_mode && row_ok) {
+                // key mode and no tile for this lane (a one-tile item): an empty partial
+                __stcg(a.part_ml + (static_cast<int64_t>(item) * kRowTiles + x) * kBM + r, make_float2(-INFINITY, 0.f));
             }
             mbar_arrive(bar(bar_item()));
             alive = warp_wait(bar(bar_item()), items_run & 1u, abort_flag, a.status);
@@ -801,15 +835,17 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
     // ---- tear-down: every role arrives here, whatever happened ------------------------------
     tc_fence_before();
     __syncthreads();
-    if (warp == kMmaWarp) {
+    if (warp == kMmaWarp0) {
         __syncwarp();
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
     }
 }
 
-// Combines the partials of every (sequence, KV head, row-tile pair) group that was split
-// over several items: O = sum_s w_s O_s / sum_s w_s l_s with w_s = 2^(m_s - max m).
+// Combines the partials of every (sequence, KV head, row-tile pair) group that did not write
+// O directly: O = sum_p w_p O_p / sum_p w_p l_p with w_p = 2^(m_p - max m).  A group in row mode
+// has one partial per split and row tile; a group in key mode (at most 128 rows) has two per
+// split, one from each lane.
 template <int D>
 __global__ void __launch_bounds__(kCombineThreads) attention_combine_kernel(const AttnArgs a) {
     __shared__ Sched sc;
@@ -820,9 +856,10 @@ __global__ void __launch_bounds__(kCombineThreads) attention_combine_kernel(cons
     constexpr int kPerGroup = kRowTiles * kBM * (D / 4);  // (row, 4 columns) work items of a group
     for (int b = 0; b < a.batch; ++b) {
         const int splits = sc.splits[b];
-        if (sc.n[b] == 0 || splits <= 1) continue;
+        if (sc.n[b] == 0) continue;
         const int groups = a.Hkv * sc.mp[b];
         const int M = sc.n[b] * G;
+        if (splits <= 1 && M - (sc.mp[b] - 1) * kRowTiles * kBM > kBM) continue;  // every group wrote O directly
         const long long total = 1ll * groups * kPerGroup;
         for (long long idx = 1ll * blockIdx.x * kCombineThreads + threadIdx.x; idx < total;
              idx += 1ll * gridDim.x * kCombineThreads) {
@@ -833,33 +870,38 @@ __global__ void __launch_bounds__(kCombineThreads) attention_combine_kernel(cons
             const int pair = grp % sc.mp[b], g = grp / sc.mp[b];
             const int R = pair * kRowTiles * kBM + row2;
             if (R >= M) continue;
+            const bool key_mode = M - pair * kRowTiles * kBM <= kBM;
+            if (!key_mode && splits <= 1) continue;
             const int mt = row2 / kBM, r = row2 % kBM;
+            const int n_parts = key_mode ? 2 * splits : splits;
             const int64_t item_first = sc.item0[b] + static_cast<int64_t>(grp) * splits;
-            // one pass over the splits, eight at a time so that their loads are in flight together
+            // one pass over the partials, eight at a time so that their loads are in flight together
             constexpr int kBatch = 8;
             float Mx = -INFINITY, den = 0.f;
             float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-            for (int s0 = 0; s0 < splits; s0 += kBatch) {
+            for (int p0 = 0; p0 < n_parts; p0 += kBatch) {
                 float2 ml[kBatch];
                 float4 v[kBatch];
 #pragma unroll
                 for (int u = 0; u < kBatch; ++u) {
-                    const int64_t it2 = item_first + min(s0 + u, splits - 1);
-                    ml[u] = __ldcg(&a.part_ml[(it2 * kRowTiles + mt) * kBM + r]);
-                    v[u] = __ldcg(a.part_o + ((it2 * kRowTiles + mt) * (D / 4) + c4) * kBM + r);
+                    const int p = min(p0 + u, n_parts - 1);
+                    const int64_t slot = key_mode ? (item_first + (p >> 1)) * kRowTiles + (p & 1)
+                                                  : (item_first + p) * kRowTiles + mt;
+                    ml[u] = __ldcg(&a.part_ml[slot * kBM + r]);
+                    v[u] = __ldcg(a.part_o + (slot * (D / 4) + c4) * kBM + r);
                 }
-                float mx4 = Mx;
+                float mx = Mx;
 #pragma unroll
                 for (int u = 0; u < kBatch; ++u)
-                    if (s0 + u < splits) mx4 = fmaxf(mx4, ml[u].x);
-                if (mx4 == -INFINITY) continue;
-                const float corr = ex2_approx(Mx - mx4);  // 0 on the first batch
+                    if (p0 + u < n_parts) mx = fmaxf(mx, ml[u].x);
+                if (mx == -INFINITY) continue;
+                const float corr = ex2_approx(Mx - mx);  // 0 on the first batch
                 den *= corr, acc.x *= corr, acc.y *= corr, acc.z *= corr, acc.w *= corr;
-                Mx = mx4;
+                Mx = mx;
 #pragma unroll
                 for (int u = 0; u < kBatch; ++u) {
-                    if (s0 + u >= splits) continue;
-                    const float w = ex2_approx(ml[u].x - Mx);  // 0 for an all-masked split
+                    if (p0 + u >= n_parts || ml[u].x == -INFINITY) continue;  // an empty partial holds no O
+                    const float w = ex2_approx(ml[u].x - Mx);
                     den += ml[u].y * w;
                     acc.x += v[u].x * w, acc.y += v[u].y * w, acc.z += v[u].z * w, acc.w += v[u].w * w;
                 }
