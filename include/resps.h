@@ -42,6 +42,7 @@ extern "C" {
 #define RESPS_MAX_TT 128
 #define RESPS_MAX_K 32
 #define RESPS_MAX_DEPTH 16
+#define RESPS_STATIC_MAX_ROWS 1024 /* batch * max_tt limit of resps_target_argmax_static */
 
 enum {
     RESPS_OK = 0,
@@ -196,6 +197,40 @@ int resps_kv_compact(resps_ctx* ctx, const resps_step* d_steps, int batch,
                      void* const* d_k_caches, void* const* d_v_caches, int n_layers,
                      int64_t kv_stride_seq, int64_t kv_stride_head, int64_t kv_stride_tok,
                      resps_stream stream);
+
+/*
+ * Per-node target arg-max for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is the arg-max step of resps_verify_accept offered without a context.)
+ *
+ * resps_create() calls cudaMalloc for the workspace its kernels need.  Some callers cannot do
+ * that: a serving process whose device memory was handed over whole to another allocator at
+ * start-up (cudaMalloc then fails or fragments that pool), a plug-in that is only ever called
+ * inside a region where allocation is forbidden, or code that runs after the memory budget of
+ * the GPU has been frozen.  This entry point needs no context and allocates nothing -- no
+ * cudaMalloc, no cudaFree, no allocating library call.  Its scratch (one packed partial result
+ * per 8192-element piece of a row, and one arrival counter per row) lives in a fixed array
+ * inside the library, 516 KB, which every GPU that loads the library holds until the process
+ * exits.
+ *
+ *   d_n_nodes         DEVICE int32 [batch]: rows i < n_nodes[b] of sequence b are reduced
+ *   d_target_logits   DEVICE fp32, element (b, i, v) at b*ld_b + i*ld_row + v
+ *   d_target_argmax   DEVICE int32 [batch][max_tt]: arg-max per node, ties -> lowest id;
+ *                     entries >= n_nodes[b] untouched
+ * Results equal those resps_verify_accept writes to d_target_argmax.
+ *
+ * Limits and rules:
+ *  - batch * max_tt <= RESPS_STATIC_MAX_ROWS (1024) and max_tt <= RESPS_MAX_TT; more returns
+ *    RESPS_ERR_CAPACITY / RESPS_ERR_UNSUPPORTED_SHAPE before anything is enqueued.
+ *  - The first call on each device looks up the array's device address (with that device
+ *    current).  Make that first call outside any stream capture.
+ *  - All calls on a device share the one array, and it keeps what the last call left in it.
+ *    Each call clears its counters on `stream` before the kernel runs, but two calls that can
+ *    overlap on the GPU (different streams without an ordering between them) race on the
+ *    array: order them.
+ */
+int resps_target_argmax_static(const int32_t* d_n_nodes, int batch, int max_tt, int vocab,
+                               const float* d_target_logits, int64_t ld_b, int64_t ld_row,
+                               int32_t* d_target_argmax, resps_stream stream);
 
 #ifdef __cplusplus
 }

@@ -25,7 +25,7 @@ RESPS_STATUS_WAIT_TIMEOUT = 4
 
 EXPORTS = ("resps_create", "resps_destroy", "resps_strerror", "resps_status",
            "resps_workspace_bytes", "resps_tree_expand", "resps_tree_attention",
-           "resps_verify_accept", "resps_kv_compact")
+           "resps_verify_accept", "resps_kv_compact", "resps_target_argmax_static")
 
 
 class RespsShape(ctypes.Structure):
@@ -66,6 +66,7 @@ def load() -> ctypes.CDLL:
                                          vp, f32, vp]
     lib.resps_verify_accept.argtypes = [vp, vp, vp, i32, vp, i64, i64, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.resps_kv_compact.argtypes = [vp, vp, i32, vp, vp, vp, vp, i32, i64, i64, i64, vp]
+    lib.resps_target_argmax_static.argtypes = [vp, i32, i32, i32, vp, i64, i64, vp, vp]
     for name in EXPORTS:
         if name not in ("resps_strerror", "resps_workspace_bytes"):
             getattr(lib, name).restype = i32
@@ -177,6 +178,16 @@ def resps_kv_compact(ctx: Context, steps, batch: int, accept_path, accept_len, k
         ctx.handle, _ptr(steps, i32), batch, _ptr(accept_path, i32), _ptr(accept_len, i32),
         _ptr(k_cache_ptrs, torch.int64), _ptr(v_cache_ptrs, torch.int64), n_layers, kv_stride_seq,
         kv_stride_head, kv_stride_tok, _stream(stream)), "resps_kv_compact")
+
+
+def resps_target_argmax_static(n_nodes, batch: int, max_tt: int, vocab: int, target_logits, ld_b: int,
+                               ld_row: int, target_argmax, stream=None) -> None:
+    """Per-node arg-max with no context and no allocation (scratch is a fixed array inside the
+    library).  For callers that may not call cudaMalloc; batch * max_tt <= 1024."""
+    i32 = torch.int32
+    _check(load().resps_target_argmax_static(
+        _ptr(n_nodes, i32), batch, max_tt, vocab, _ptr(target_logits, torch.float32), ld_b, ld_row,
+        _ptr(target_argmax, i32), _stream(stream)), "resps_target_argmax_static")
 
 
 def layer_pointer_table(caches: Sequence[torch.Tensor]) -> torch.Tensor:

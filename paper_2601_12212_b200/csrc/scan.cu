@@ -8,6 +8,7 @@
 // (atomic arrival counter, self-resetting) merges the partials and writes the
 // row's final result, so no second launch is needed.
 #include <cmath>
+#include <mutex>
 
 #include "common.cuh"
 
@@ -349,4 +350,73 @@ cudaError_t launch_row_argmax(const resps_ctx* ctx, const int32_t* d_n_nodes, in
     return cudaGetLastError();
 }
 
+// ---------------------------------------------------------------------------------------
+// Arg-max without a context and without any allocation (see resps_target_argmax_static in
+// resps.h).  The split partials and arrival counters of row_argmax_kernel live in a
+// file-scope device array instead of a context's cudaMalloc'ed workspace.
+// ---------------------------------------------------------------------------------------
+namespace {
+
+constexpr int kStaticMaxRows = RESPS_STATIC_MAX_ROWS;  // batch * max_tt
+constexpr int kStaticMaxSplits = 64;
+constexpr size_t kStaticPartBytes = sizeof(unsigned long long) * kStaticMaxRows * kStaticMaxSplits;
+constexpr size_t kStaticCounterBytes = sizeof(unsigned int) * kStaticMaxRows;
+
+// [rows][splits] packed (value, id) partials, then [rows] arrival counters: 516 KB per GPU.
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticPartBytes + kStaticCounterBytes];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+unsigned char* g_static_ptr[kMaxDevices] = {};  // device address of g_static_scratch, per device
+
+// In host code the array's name only stands for the symbol; its device address has to be asked
+// for, once per device, with that device current.
+int static_scratch_address(unsigned char** out) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return RESPS_ERR_NO_DEVICE;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_ptr[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return RESPS_ERR_CUDA;
+        g_static_ptr[dev] = static_cast<unsigned char*>(p);
+    }
+    *out = g_static_ptr[dev];
+    return RESPS_OK;
+}
+
+}  // namespace
 }  // namespace resps
+
+extern "C" int resps_target_argmax_static(const int32_t* d_n_nodes, int batch, int max_tt, int vocab,
+                                          const float* d_target_logits, int64_t ld_b, int64_t ld_row,
+                                          int32_t* d_target_argmax, resps_stream stream) {
+    using namespace resps;
+    if (!d_n_nodes || !d_target_logits || !d_target_argmax) return RESPS_ERR_INVALID_ARG;
+    if (batch < 1 || max_tt < 1 || vocab < 1 || ld_row < vocab || ld_b < 0) return RESPS_ERR_INVALID_ARG;
+    if (max_tt > RESPS_MAX_TT) return RESPS_ERR_UNSUPPORTED_SHAPE;
+    if (static_cast<int64_t>(batch) * max_tt > kStaticMaxRows) return RESPS_ERR_CAPACITY;
+    int chunk = 8192;
+    if ((vocab + chunk - 1) / chunk > kStaticMaxSplits)
+        chunk = ((vocab + kStaticMaxSplits - 1) / kStaticMaxSplits + 1023) / 1024 * 1024;
+    const int splits = (vocab + chunk - 1) / chunk;
+    unsigned char* scratch = nullptr;
+    const int rc = static_scratch_address(&scratch);
+    if (rc != RESPS_OK) return rc;
+    ArgmaxArgs a;
+    a.n_nodes = d_n_nodes;
+    a.logits = d_target_logits;
+    a.ld_b = ld_b, a.ld_row = ld_row;
+    a.vocab = vocab, a.max_tt = max_tt, a.chunk = chunk, a.splits = splits;
+    a.part = reinterpret_cast<unsigned long long*>(scratch);
+    a.counter = reinterpret_cast<unsigned int*>(scratch + kStaticPartBytes);
+    a.out = d_target_argmax;
+    // The array keeps whatever the last call left: the counters must start at zero.
+    if (cudaMemsetAsync(a.counter, 0, sizeof(unsigned int) * batch * max_tt, stream) != cudaSuccess)
+        return RESPS_ERR_CUDA;
+    dim3 grid(splits, max_tt, batch);
+    if (vec_ok(d_target_logits, ld_b, ld_row, 0, vocab, chunk))
+        row_argmax_kernel<true><<<grid, kScanThreads, 0, stream>>>(a);
+    else
+        row_argmax_kernel<false><<<grid, kScanThreads, 0, stream>>>(a);
+    return cudaGetLastError() == cudaSuccess ? RESPS_OK : RESPS_ERR_CUDA;
+}
