@@ -144,13 +144,15 @@ int resps_tree_expand(resps_ctx* ctx, const resps_step* d_steps, int batch,
  * The tree tokens' K/V must already be stored at slots L .. L+n-1.  No other slot
  * influences the result.
  *
- * d_q, d_o     DEVICE bf16 [batch][max_tt][Hq][D]; rows >= n are neither read nor written
+ * d_q, d_o     DEVICE bf16 [batch][max_tt][Hq][D]; rows >= n of d_o are never written, rows >= n of
+ *              d_q may be read (whole tiles are fetched) but never influence a result
  * d_lse        DEVICE fp32 [batch][max_tt][Hq] or NULL: natural-log sum of exp of the scaled scores
  * d_k_cache, d_v_cache  DEVICE bf16; element (b, g, slot, e) at
  *              b*kv_stride_seq + g*kv_stride_head + slot*kv_stride_tok + e  (elements);
  *              16-byte aligned, strides multiples of 8 elements
- * kv_capacity  slots per (sequence, head); a sequence with L + n > kv_capacity is skipped
- *              and RESPS_STATUS_KV_OVERFLOW set
+ * kv_capacity  slots per (sequence, head), at most 2^21; a sequence with L + n > kv_capacity is
+ *              skipped and RESPS_STATUS_KV_OVERFLOW set
+ * softmax_scale  must be positive (INVALID_ARG otherwise)
  * d_mask       as written by resps_tree_expand
  * Accumulation is fp32; the result is rounded to bf16 once.
  */

@@ -7,6 +7,7 @@
 #include "common.cuh"
 
 namespace resps {
+int scan_chunk_max();
 int attention_item_rows();
 int attention_max_batch();
 }  // namespace resps
@@ -94,11 +95,16 @@ int resps_create(resps_ctx** out, const resps_shape* shape) {
     c->device = dev;
     c->sm_count = prop.multiProcessorCount;
     resps::Workspace& w = c->ws;
-    int chunk = 8192;
-    if (const char* e = std::getenv("RESPS_SCAN_CHUNK")) chunk = std::max(1024, std::atoi(e) / 1024 * 1024);
-    if ((s.vocab + chunk - 1) / chunk > 64) chunk = static_cast<int>(align_up((s.vocab + 63) / 64, 1024));
+    // a scan CTA keeps its whole chunk in registers; up to 128 chunks per row (vocab <= 2^20)
+    int chunk = resps::scan_chunk_max();
+    if (const char* e = std::getenv("RESPS_SCAN_CHUNK"))
+        chunk = std::min(chunk, std::max(1024, std::atoi(e) / 1024 * 1024));
     w.scan_chunk = chunk;
     w.scan_splits = (s.vocab + chunk - 1) / chunk;
+    if (w.scan_splits > 128) {
+        delete c;
+        return RESPS_ERR_UNSUPPORTED_SHAPE;
+    }
     w.max_rows = 1 + (s.max_depth - 1) * s.max_k;
     const int G = s.n_q_heads / s.n_kv_heads;
     const int item_rows = resps::attention_item_rows();
@@ -199,7 +205,7 @@ int resps_tree_attention(resps_ctx* ctx, const resps_step* d_steps, const int32_
     RESPS_CHECK_PTR(d_v_cache);
     RESPS_CHECK_PTR(d_mask);
     if (batch < 1 || kv_capacity < 1 || kv_stride_tok < ctx->shape.head_dim || kv_stride_head < 0 ||
-        kv_stride_seq < 0)
+        kv_stride_seq < 0 || !(softmax_scale > 0.f) || kv_capacity > (int64_t(1) << 21))
         return RESPS_ERR_INVALID_ARG;
     if (!aligned16(d_q) || !aligned16(d_o) || !aligned16(d_k_cache) || !aligned16(d_v_cache) ||
         kv_stride_seq % 8 || kv_stride_head % 8 || kv_stride_tok % 8)

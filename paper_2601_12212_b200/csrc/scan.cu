@@ -34,63 +34,10 @@ struct ScanArgs {
     int32_t* status;
 };
 
-// Insert `nk` into the warp's descending list (one entry per lane).
-__device__ __forceinline__ void warp_insert(unsigned long long& mine, unsigned long long nk, int lane) {
-    const unsigned ahead = __ballot_sync(kFull, mine > nk);
-    const int pos = __popc(ahead);
-    const unsigned long long up = __shfl_up_sync(kFull, mine, 1);
-    if (lane == pos)
-        mine = nk;
-    else if (lane > pos)
-        mine = up;
-}
-
-struct WarpTopK {
-    unsigned long long mine = 0ull;  // this lane's list entry (0 = empty, ranks last)
-    unsigned long long kth = 0ull;   // entry k-1, warp-uniform
-    float thr = -INFINITY;       // its value: nothing below it can enter the top k
-
-    // Offer up to four consecutive elements per lane; `nvalid` of them exist.
-    __device__ __forceinline__ void offer4(const float (&v)[4], int id0, int nvalid, int k, int lane) {
-        bool hit = false;
-#pragma unroll
-        for (int c = 0; c < 4; ++c) hit |= (c < nvalid) && (v[c] >= thr);
-        if (!__any_sync(kFull, hit)) return;
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            unsigned pending = __ballot_sync(kFull, (c < nvalid) && (v[c] >= thr));
-            const unsigned long long cand = pack_val_id(v[c], id0 + c);
-            while (pending) {
-                const int src = __ffs(pending) - 1;
-                pending &= pending - 1;
-                const unsigned long long nk = __shfl_sync(kFull, cand, src);
-                if (nk > kth) {
-                    warp_insert(mine, nk, lane);
-                    kth = __shfl_sync(kFull, mine, k - 1);
-                    thr = (kth == 0ull) ? -INFINITY : key_val(kth);
-                }
-            }
-        }
-    }
-};
-
 // Running (max, sum) of 2^(y - max) with y = x*log2(e).
 struct LseAcc {
     float m2 = -INFINITY;
     float s = 0.f;
-    __device__ __forceinline__ void add4(const float (&v)[4], int nvalid) {
-        float mx = -INFINITY;
-#pragma unroll
-        for (int c = 0; c < 4; ++c)
-            if (c < nvalid) mx = fmaxf(mx, v[c] * kLog2e);
-        if (mx > m2) {
-            s *= ex2_approx(m2 - mx);
-            m2 = mx;
-        }
-#pragma unroll
-        for (int c = 0; c < 4; ++c)
-            if (c < nvalid) s += ex2_approx(fmaf(v[c], kLog2e, -m2));
-    }
     __device__ __forceinline__ void merge(float om, float os) {
         const float M = fmaxf(m2, om);
         if (M == -INFINITY) return;
@@ -110,8 +57,34 @@ __device__ __forceinline__ void select_top_by_rank(const unsigned long long* key
     }
 }
 
+constexpr int kScanPerThread = 32;                              // logits a thread keeps in registers
+constexpr int kScanChunkMax = kScanThreads * kScanPerThread;    // 8192 per CTA
+constexpr int kQuads = kScanThreads / 4;                        // units of 4 threads = 128 logits
+constexpr int kQuadElems = 4 * kScanPerThread;
+
+__device__ __forceinline__ float max3f(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+
+// One CTA reduces one chunk (<= 8192 logits, all held in registers) of one row.
+//  1. every quad of threads (128 logits) finds its best logit; the k-th best of the 64 quad
+//     maxima, tau, is a lower bound for the chunk's k-th best logit;
+//  2. every logit that ranks at or before tau is a candidate: they belong to the k quads whose
+//     maximum does, so there are between k and 128 k of them (about 2 k for random data);
+//  3. the candidates are ranked by counting and the k best written out.
+// Keys are (ordered value, ~id) pairs, unique, so that "larger key" is exactly the method's order
+// (value descending, token id ascending).  The log-sum-exp partial is a per-thread
+// (max, sum 2^(y - max)) reduced over the CTA.
 template <bool VEC>
 __global__ void __launch_bounds__(kScanThreads, 4) row_scan_kernel(const ScanArgs a) {
+    extern __shared__ unsigned long long s_keys[];  // max(128 max_k, splits max_k) keys
+    __shared__ unsigned long long s_quad[kQuads];
+    __shared__ unsigned long long s_tau;
+    __shared__ int s_count;
+    __shared__ float2 s_ms[kScanThreads / 32];
+    __shared__ bool s_last;
     const int b = blockIdx.z, r = blockIdx.y, sp = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const StepDims sd = clamp_step(a.steps[b], a.n_levels, a.n_slots, a.max_tt, a.max_k, a.vocab);
@@ -125,52 +98,100 @@ __global__ void __launch_bounds__(kScanThreads, 4) row_scan_kernel(const ScanArg
     const int begin = sp * a.chunk;
     const int end = min(a.vocab, begin + a.chunk);
 
-    WarpTopK top;
-    LseAcc acc;
-    constexpr int kUnroll = 4;
-    for (int base = begin; base < end; base += kScanThreads * 4 * kUnroll) {
-        float v[kUnroll][4];
-        int nv[kUnroll];
+    // ---- the chunk into registers: 8 independent 128-bit loads per thread ------------------
+    float v[kScanPerThread];
 #pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
-            const int e0 = base + (u * kScanThreads + tid) * 4;
-            nv[u] = max(0, min(4, end - e0));
-            if (VEC) {
-                if (nv[u] > 0) {  // vocab and chunk are multiples of 4 on this path
-                    const float4 x = __ldcs(reinterpret_cast<const float4*>(row + e0));
-                    v[u][0] = x.x, v[u][1] = x.y, v[u][2] = x.z, v[u][3] = x.w;
-                }
-            } else {
-#pragma unroll
-                for (int c = 0; c < 4; ++c)
-                    if (c < nv[u]) v[u][c] = __ldcs(row + e0 + c);
+    for (int u = 0; u < kScanPerThread / 4; ++u) {
+        const int e0 = begin + (u * kScanThreads + tid) * 4;
+        v[4 * u] = v[4 * u + 1] = v[4 * u + 2] = v[4 * u + 3] = -INFINITY;
+        if (VEC) {
+            if (e0 < end) {  // vocab and chunk are multiples of 4 on this path
+                const float4 x = __ldcs(reinterpret_cast<const float4*>(row + e0));
+                v[4 * u] = x.x, v[4 * u + 1] = x.y, v[4 * u + 2] = x.z, v[4 * u + 3] = x.w;
             }
-        }
+        } else {
 #pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
-            const int e0 = base + (u * kScanThreads + tid) * 4;
-            if (nv[u] > 0) acc.add4(v[u], nv[u]);
-            top.offer4(v[u], e0, nv[u], k, lane);
+            for (int c = 0; c < 4; ++c)
+                if (e0 + c < end) v[4 * u + c] = __ldcs(row + e0 + c);
         }
     }
+    if (tid == 0) s_count = 0;
+    // position i of a thread is logit begin + ((i / 4) * 256 + tid) * 4 + i % 4: ids ascend with i
+    auto elem_id = [&](int i) { return begin + ((i >> 2) * kScanThreads + tid) * 4 + (i & 3); };
 
-    // ---- CTA reduction -------------------------------------------------------
-    __shared__ unsigned long long s_keys[64 * RESPS_MAX_K];  // 8 warp lists, later `splits` partial lists
-    __shared__ float2 s_ms[kScanThreads / 32];
-    __shared__ bool s_last;
+    // ---- thread maximum and its first position ---------------------------------------------
+    float tmax = v[0];
+#pragma unroll
+    for (int i = 1; i + 1 < kScanPerThread; i += 2) tmax = max3f(tmax, v[i], v[i + 1]);
+    tmax = fmaxf(tmax, v[kScanPerThread - 1]);
+    int tpos = 0;
+#pragma unroll
+    for (int i = kScanPerThread - 1; i >= 0; --i)
+        if (v[i] == tmax) tpos = i;
+    const bool has_any = elem_id(0) < end;  // a thread's positions are valid up to some i: 0 is valid or none
+    const unsigned long long my_key = has_any ? pack_val_id(tmax, elem_id(tpos)) : 0ull;
+
+    // ---- log-sum-exp partial (-inf padding adds 2^-inf = 0) ----------------------------------
+    LseAcc acc;
+    if (has_any) {
+        acc.m2 = tmax * kLog2e;
+        float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+        for (int i = 0; i < kScanPerThread; i += 2) {
+            s0 += ex2_approx(fmaf(v[i], kLog2e, -acc.m2));
+            s1 += ex2_approx(fmaf(v[i + 1], kLog2e, -acc.m2));
+        }
+        acc.s = s0 + s1;
+    }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
         const float om = __shfl_xor_sync(kFull, acc.m2, o);
         const float os = __shfl_xor_sync(kFull, acc.s, o);
         acc.merge(om, os);
     }
-    if (lane < k) s_keys[warp * k + lane] = top.mine;
     if (lane == 0) s_ms[warp] = make_float2(acc.m2, acc.s);
+
+    // ---- tau: the k-th best of the 64 quad maxima (0 = fewer than k non-empty quads) -----------
+    unsigned long long quad_key = my_key;
+    {
+        unsigned long long o = __shfl_xor_sync(kFull, quad_key, 1);
+        quad_key = o > quad_key ? o : quad_key;
+        o = __shfl_xor_sync(kFull, quad_key, 2);
+        quad_key = o > quad_key ? o : quad_key;
+    }
+    if ((lane & 3) == 0) s_quad[tid >> 2] = quad_key;
     __syncthreads();
+    if (tid < kQuads) {
+        const unsigned long long mine = s_quad[tid];
+        int rank = 0;
+#pragma unroll 8
+        for (int j = 0; j < kQuads; ++j) {
+            const unsigned long long o = s_quad[j];
+            rank += (o > mine) || (o == mine && j < tid);  // equal keys are both 0 (empty)
+        }
+        if (rank == min(k, kQuads) - 1) s_tau = mine;
+    }
+    __syncthreads();
+    // with k > 64 quads every non-empty quad qualifies; k <= RESPS_MAX_K = 32 keeps this exact
+    const unsigned long long tau = s_tau;
+
+    // ---- candidates: every logit at or before tau ------------------------------------------------
+    if (quad_key >= tau && has_any) {  // only the k quads whose maximum qualifies can hold any
+        const float tau_v = (tau == 0ull) ? -INFINITY : key_val(tau);
+#pragma unroll
+        for (int i = 0; i < kScanPerThread; ++i) {
+            if (v[i] >= tau_v && elem_id(i) < end) {
+                const unsigned long long key = pack_val_id(v[i], elem_id(i));
+                if (key >= tau) s_keys[atomicAdd(&s_count, 1)] = key;
+            }
+        }
+    }
+    __syncthreads();
+    const int n_cand = s_count;  // <= 128 k
     const int64_t prow = static_cast<int64_t>(b) * a.max_rows + r;
     unsigned long long* part = a.part_key + (prow * a.splits + sp) * a.max_k;
-    select_top_by_rank(s_keys, (kScanThreads / 32) * k, k,
-                       [&](int rank, unsigned long long key) { part[rank] = key; });
+    select_top_by_rank(s_keys, n_cand, k, [&](int rank, unsigned long long key) { part[rank] = key; });
+    if (tid >= n_cand && tid < k) part[tid] = 0ull;  // fewer than k logits in the chunk
     if (tid == 0) {
         LseAcc t;
         for (int w = 0; w < kScanThreads / 32; ++w) t.merge(s_ms[w].x, s_ms[w].y);
@@ -187,6 +208,8 @@ __global__ void __launch_bounds__(kScanThreads, 4) row_scan_kernel(const ScanArg
     const unsigned long long* parts = a.part_key + prow * a.splits * a.max_k;
     for (int i = tid; i < a.splits * k; i += kScanThreads)
         s_keys[i] = __ldcg(parts + (i / k) * a.max_k + (i % k));
+    float2 my_ms = make_float2(-INFINITY, 0.f);
+    if (tid < a.splits) my_ms = __ldcg(a.part_ms + prow * a.splits + tid);  // splits <= 128 < threads
     __syncthreads();
     float* oval = a.row_val + prow * a.max_k;
     int32_t* oid = a.row_id + prow * a.max_k;
@@ -194,16 +217,26 @@ __global__ void __launch_bounds__(kScanThreads, 4) row_scan_kernel(const ScanArg
         oval[rank] = key_val(key);
         oid[rank] = key_id(key);
     });
+    if (warp < 4) {  // partial sums: weights in fp32 (relative error 2^-22), accumulation in fp64
+        float M = my_ms.x;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(kFull, M, o));
+        if (lane == 0) s_ms[warp] = make_float2(M, 0.f);
+    }
+    __syncthreads();
+    if (warp < 4) {
+        const float M = fmaxf(fmaxf(s_ms[0].x, s_ms[1].x), fmaxf(s_ms[2].x, s_ms[3].x));
+        double sum = (my_ms.y > 0.f) ? static_cast<double>(my_ms.y) * static_cast<double>(ex2_approx(my_ms.x - M)) : 0.0;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(kFull, sum, o);
+        if (lane == 0) s_quad[warp] = __double_as_longlong(sum);
+    }
+    __syncthreads();
     if (tid == 0) {
-        const float2* ms = a.part_ms + prow * a.splits;
-        double M = -INFINITY;
-        for (int i = 0; i < a.splits; ++i) M = fmax(M, static_cast<double>(__ldcg(&ms[i].x)));
-        double sum = 0.0;
-        for (int i = 0; i < a.splits; ++i) {
-            const float2 p = __ldcg(ms + i);
-            if (p.y > 0.f) sum += static_cast<double>(p.y) * exp2(static_cast<double>(p.x) - M);
-        }
-        a.row_lse[prow] = (M + log2(sum)) * 0.6931471805599453094;
+        const float M = fmaxf(fmaxf(s_ms[0].x, s_ms[1].x), fmaxf(s_ms[2].x, s_ms[3].x));
+        const double sum = __longlong_as_double(s_quad[0]) + __longlong_as_double(s_quad[1]) +
+                           __longlong_as_double(s_quad[2]) + __longlong_as_double(s_quad[3]);
+        a.row_lse[prow] = (static_cast<double>(M) + log2(sum)) * 0.6931471805599453094;
         a.counter[prow] = 0u;
     }
 }
@@ -230,7 +263,7 @@ __global__ void __launch_bounds__(kScanThreads, 4) row_argmax_kernel(const Argma
 
     float best = -INFINITY;
     int best_id = 0x7FFFFFFF;
-    constexpr int kUnroll = 4;
+    constexpr int kUnroll = 8;
     for (int base = begin; base < end; base += kScanThreads * 4 * kUnroll) {
         float v[kUnroll][4];
         int nv[kUnroll];
@@ -308,6 +341,8 @@ inline bool vec_ok(const void* p, int64_t s0, int64_t s1, int64_t s2, int vocab,
 
 }  // namespace
 
+int scan_chunk_max() { return kScanChunkMax; }
+
 cudaError_t launch_row_scan(const resps_ctx* ctx, const resps_step* d_steps, int batch,
                             const float* logits, int64_t ld_b, int64_t ld_level, int64_t ld_row,
                             int n_levels, int n_slots, cudaStream_t st) {
@@ -324,10 +359,11 @@ cudaError_t launch_row_scan(const resps_ctx* ctx, const resps_step* d_steps, int
     const int k_ext = min(n_slots, ctx->shape.max_k);
     const int rows = (n_levels > 1) ? 1 + (n_levels - 1) * k_ext : 1;
     dim3 grid(w.scan_splits, rows, batch);
+    const size_t smem = sizeof(unsigned long long) * ctx->shape.max_k * max(kQuadElems, w.scan_splits);
     if (vec_ok(logits, ld_b, ld_level, ld_row, a.vocab, a.chunk))
-        row_scan_kernel<true><<<grid, kScanThreads, 0, st>>>(a);
+        row_scan_kernel<true><<<grid, kScanThreads, smem, st>>>(a);
     else
-        row_scan_kernel<false><<<grid, kScanThreads, 0, st>>>(a);
+        row_scan_kernel<false><<<grid, kScanThreads, smem, st>>>(a);
     return cudaGetLastError();
 }
 

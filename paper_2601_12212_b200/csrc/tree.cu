@@ -4,11 +4,9 @@
 // best TT-1 kept; Algorithm 2, tree-building loop).  One CTA per sequence; integer
 // and fp64 work on at most k + (d-1)k^2 candidates, all in shared memory.
 //
-// No quadratic loop: the k children of one parent are already sorted (their score
-// is the parent's plus a non-increasing log-probability), so a candidate's rank
-// inside its level is a sum of binary searches over its sibling lists, and its
-// rank in the global rerank is its level rank plus binary searches over the other
-// levels' sorted orders.
+// A candidate's rank inside its level (at most k^2 candidates) is found by counting;
+// its rank in the global rerank is its level rank plus binary searches over the
+// other levels' sorted orders, and only the first TT-1 of a level can be kept at all.
 #include <cmath>
 
 #include "common.cuh"
@@ -113,10 +111,15 @@ __global__ void __launch_bounds__(kTreeThreads, 1) tree_build_kernel(const TreeA
         return frontier[(j - 1) * RESPS_MAX_K + i / k];
     };
 
+    // ---- every candidate's own log-probability, in one round trip to global memory (the rows
+    // a level reads do not depend on the levels before it) -----------------------------------
+    for (int c = tid; c < n_cand; c += kTreeThreads) {
+        const int64_t row = row0 + cand_row(c);
+        const double lp = static_cast<double>(a.row_val[row * a.max_k + cand_rank_in_row(c)]) - a.row_lse[row];
+        score[c] = fmin(lp, 0.0);
+    }
     // ---- level 0 ---------------------------------------------------------------
     if (tid < k) {
-        const double lp = static_cast<double>(a.row_val[row0 * a.max_k + tid]) - a.row_lse[row0];
-        score[tid] = fmin(lp, 0.0);
         sorted[tid] = tid;
         frontier[tid] = tid;
     }
@@ -125,31 +128,17 @@ __global__ void __launch_bounds__(kTreeThreads, 1) tree_build_kernel(const TreeA
     // ---- levels 1..d-1 -----------------------------------------------------------
     for (int j = 1; j < d; ++j) {
         const int base = k + (j - 1) * kk;
-        for (int i = tid; i < kk; i += kTreeThreads) {
-            const int p = i / k, r = i % k;
-            const int64_t row = row0 + 1 + (j - 1) * k + p;
-            const double lp = static_cast<double>(a.row_val[row * a.max_k + r]) - a.row_lse[row];
-            score[base + i] = score[frontier[(j - 1) * RESPS_MAX_K + p]] + fmin(lp, 0.0);
-        }
+        for (int i = tid; i < kk; i += kTreeThreads)
+            score[base + i] += score[frontier[(j - 1) * RESPS_MAX_K + i / k]];
         __syncthreads();
+        // rank inside the level by counting (independent shared-memory reads pipeline; a chain of
+        // dependent binary-search steps does not)
         for (int i = tid; i < kk; i += kTreeThreads) {
-            const int p = i / k, r = i % k, c = base + i;
+            const int c = base + i;
             const double s = score[c];
-            int rank = r;
-            for (int q = 0; q < k; ++q) {
-                if (q == p) continue;
-                // sibling list q is the contiguous run base+q*k .. +k, already in order
-                int lo = 0, hi = k;
-                while (lo < hi) {
-                    const int mid = (lo + hi) >> 1;
-                    const int e = base + q * k + mid;
-                    if (before(score[e], e, s, c))
-                        lo = mid + 1;
-                    else
-                        hi = mid;
-                }
-                rank += lo;
-            }
+            int rank = 0;
+#pragma unroll 4
+            for (int i2 = 0; i2 < kk; ++i2) rank += before(score[base + i2], base + i2, s, c) ? 1 : 0;
             sorted[base + rank] = c;
             if (rank < k) frontier[j * RESPS_MAX_K + rank] = c;
         }
