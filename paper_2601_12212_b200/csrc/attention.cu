@@ -520,11 +520,13 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
                 tc_fence_after();
                 if (elect_one()) {
                     const uint64_t vdesc = vdesc0 + static_cast<uint64_t>(s * (S::kKVTile >> 4));
-                    const uint32_t p_t = tmem + x * 256 + (prev_j & 1u) * kBN;  // hi: +0, lo: +32
+                    // P of keys 32h .. 32h+31: hi in columns 32h .. 32h+15, lo in 32h+16 .. 32h+31
+                    const uint32_t p_t = tmem + x * 256 + (prev_j & 1u) * kBN;
 #pragma unroll
                     for (int kk = 0; kk < kBN / 16; ++kk) {
-                        umma_ts(o_t, p_t + kk * 8, vdesc + kk * (2048 >> 4), kIdescPV, (first_pv && kk == 0) ? 0u : 1u);
-                        umma_ts(o_t, p_t + 32 + kk * 8, vdesc + kk * (2048 >> 4), kIdescPV, 1u);
+                        const uint32_t a_t = p_t + (kk >> 1) * 32 + (kk & 1) * 8;
+                        umma_ts(o_t, a_t, vdesc + kk * (2048 >> 4), kIdescPV, (first_pv && kk == 0) ? 0u : 1u);
+                        umma_ts(o_t, a_t + 16, vdesc + kk * (2048 >> 4), kIdescPV, 1u);
                     }
                     umma_commit(bar(bar_pvdone(x)));
                     umma_commit(bar(bar_kvempty(s)));
@@ -673,11 +675,13 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
                             tmax = fmaxf(tmax, s);
                         }
                 } else {
+                    float t4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};  // four independent chains
 #pragma unroll
                     for (int h = 0; h < 2; ++h)
 #pragma unroll
                         for (int c = 0; c < 32; c += 2)
-                            tmax = max3(tmax, __uint_as_float(sr[h][c]), __uint_as_float(sr[h][c + 1]));
+                            t4[(c >> 1) & 3] = max3(t4[(c >> 1) & 3], __uint_as_float(sr[h][c]), __uint_as_float(sr[h][c + 1]));
+                    tmax = fmaxf(fmaxf(t4[0], t4[1]), fmaxf(t4[2], t4[3]));
                 }
                 tmax *= a.scale_log2;  // the scale is positive: max(scale * s) = scale * max(s)
                 const float m_new = fmaxf(m_ref, tmax);
@@ -729,34 +733,37 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
 
                 // ---- P = exp2(scale * S - m) as bf16 hi + lo, back into the columns S came from.
                 // hi is p truncated to bf16, so p - hi is exact and lo = bf16(p - hi) leaves an
-                // error of 2^-16 p.  Packed fp32 pairs halve the instruction count.
+                // error of 2^-16 p.  Packed fp32 pairs halve the instruction count.  Each half of the
+                // tile (32 keys) becomes 16 columns of hi and 16 of lo in place of its own 32 columns
+                // of S, stored as soon as it is ready so that the store overlaps the other half.
                 {
                     const unsigned long long sc2 = pack2(a.scale_log2, a.scale_log2);
                     const unsigned long long nm2 = pack2(-m_use, -m_use);
                     unsigned long long psum2 = pack2(0.f, 0.f);
-                    uint32_t plo[32];
+                    const uint32_t p_t = tmem + lane_sel + x * 256 + buf * kBN;
 #pragma unroll
-                    for (int c = 0; c < 32; ++c) {
-                        const int h = c >> 4, e = (2 * c) & 31;
-                        float x0, x1;
-                        unpack2(fma2(pack2(__uint_as_float(sr[h][e]), __uint_as_float(sr[h][e + 1])), sc2, nm2), x0, x1);
-                        const float p0 = ex2_approx(x0), p1 = ex2_approx(x1);
-                        const unsigned long long p2 = pack2(p0, p1);
-                        psum2 = add2(psum2, p2);
-                        const uint32_t b0 = __float_as_uint(p0), b1 = __float_as_uint(p1);
-                        const uint32_t hi = __byte_perm(b0, b1, 0x7632);
-                        float l0, l1;
-                        unpack2(sub2(p2, pack2(__uint_as_float(b0 & 0xFFFF0000u), __uint_as_float(b1 & 0xFFFF0000u))), l0,
-                                l1);
-                        plo[c] = pack_bf16(l0, l1);
-                        sr[0][c] = hi;  // position c was consumed at iteration c / 2
+                    for (int h = 0; h < 2; ++h) {
+                        uint32_t w[32];
+#pragma unroll
+                        for (int c = 0; c < 16; ++c) {
+                            float x0, x1;
+                            unpack2(fma2(pack2(__uint_as_float(sr[h][2 * c]), __uint_as_float(sr[h][2 * c + 1])), sc2, nm2),
+                                    x0, x1);
+                            const float p0 = ex2_approx(x0), p1 = ex2_approx(x1);
+                            const unsigned long long p2 = pack2(p0, p1);
+                            psum2 = add2(psum2, p2);
+                            const uint32_t b0 = __float_as_uint(p0), b1 = __float_as_uint(p1);
+                            w[c] = __byte_perm(b0, b1, 0x7632);
+                            float l0, l1;
+                            unpack2(sub2(p2, pack2(__uint_as_float(b0 & 0xFFFF0000u), __uint_as_float(b1 & 0xFFFF0000u))),
+                                    l0, l1);
+                            w[16 + c] = pack_bf16(l0, l1);
+                        }
+                        tmem_st32(p_t + h * 32, w);
                     }
                     float ps0, ps1;
                     unpack2(psum2, ps0, ps1);
                     l_run += ps0 + ps1;
-                    const uint32_t p_t = tmem + lane_sel + x * 256 + buf * kBN;
-                    tmem_st32(p_t, sr[0]);
-                    tmem_st32(p_t + 32, plo);
                     tmem_wait_st();
                 }
                 if (clear_v) fence_proxy_async();
@@ -875,8 +882,8 @@ __global__ void __launch_bounds__(kCombineThreads) attention_combine_kernel(cons
             const int mt = row2 / kBM, r = row2 % kBM;
             const int n_parts = key_mode ? 2 * splits : splits;
             const int64_t item_first = sc.item0[b] + static_cast<int64_t>(grp) * splits;
-            // one pass over the partials, eight at a time so that their loads are in flight together
-            constexpr int kBatch = 8;
+            // one pass over the partials, sixteen at a time so that their loads are in flight together
+            constexpr int kBatch = 16;
             float Mx = -INFINITY, den = 0.f;
             float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
             for (int p0 = 0; p0 < n_parts; p0 += kBatch) {

@@ -131,16 +131,23 @@ __global__ void __launch_bounds__(kTreeThreads, 1) tree_build_kernel(const TreeA
         for (int i = tid; i < kk; i += kTreeThreads)
             score[base + i] += score[frontier[(j - 1) * RESPS_MAX_K + i / k]];
         __syncthreads();
-        // rank inside the level by counting (independent shared-memory reads pipeline; a chain of
-        // dependent binary-search steps does not)
-        for (int i = tid; i < kk; i += kTreeThreads) {
-            const int c = base + i;
+        // rank inside the level by counting, eight threads per candidate (independent shared-memory
+        // reads pipeline; a chain of dependent binary-search steps does not)
+        for (int i0 = 0; i0 < kk; i0 += kTreeThreads / 8) {
+            const int i = i0 + (tid >> 3), sub = tid & 7;
+            const bool live = i < kk;
+            const int c = base + (live ? i : 0);
             const double s = score[c];
             int rank = 0;
-#pragma unroll 4
-            for (int i2 = 0; i2 < kk; ++i2) rank += before(score[base + i2], base + i2, s, c) ? 1 : 0;
-            sorted[base + rank] = c;
-            if (rank < k) frontier[j * RESPS_MAX_K + rank] = c;
+            if (live)
+                for (int i2 = sub; i2 < kk; i2 += 8) rank += before(score[base + i2], base + i2, s, c) ? 1 : 0;
+            rank += __shfl_xor_sync(kFull, rank, 1);
+            rank += __shfl_xor_sync(kFull, rank, 2);
+            rank += __shfl_xor_sync(kFull, rank, 4);
+            if (live && sub == 0) {
+                sorted[base + rank] = c;
+                if (rank < k) frontier[j * RESPS_MAX_K + rank] = c;
+            }
         }
         __syncthreads();
     }
