@@ -129,7 +129,9 @@ __device__ __forceinline__ void build_sched(const AttnArgs& a, Sched& sc, int ti
 struct Item {
     int b, g, pair, sp, splits, first_item;
     int n, L, M, row_base, nmt, t_begin, t_end;
+    int tok0;  // first token of the pair's rows
 };
+constexpr int kPreItems = 8;  // items of a CTA decoded once, in parallel, for all roles
 
 __device__ __forceinline__ Item decode_item(const Sched& sc, int item, int G) {
     Item it;
@@ -150,6 +152,7 @@ __device__ __forceinline__ Item decode_item(const Sched& sc, int item, int G) {
     const unsigned kt = static_cast<unsigned>(sc.kt[b]), sp = static_cast<unsigned>(it.sp);
     it.t_begin = static_cast<int>(kt * sp / static_cast<unsigned>(it.splits));
     it.t_end = static_cast<int>(kt * (sp + 1u) / static_cast<unsigned>(it.splits));
+    it.tok0 = it.row_base / G;
     return it;
 }
 
@@ -384,6 +387,7 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
     using S = Smem<D>;
     extern __shared__ unsigned char smem_raw[];
     __shared__ Sched sc;
+    __shared__ Item s_items[kPreItems];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     unsigned char* base_ptr = smem_raw + (base - smem_u32(smem_raw));
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -430,11 +434,18 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
     pdl_wait();
     pdl_launch_dependents();
     build_sched(a, sc, tid, kAttnThreads);  // ends with __syncthreads()
+    const int total_items = min(sc.item0[a.batch], a.max_items);
+    // The integer divisions of the item decode are a long dependent chain for a single thread:
+    // the first items of this CTA are decoded here, one per thread, for every role to read.
+    if (tid < kPreItems && blockIdx.x + tid * gridDim.x < total_items)
+        s_items[tid] = decode_item(sc, blockIdx.x + tid * gridDim.x, G);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
-    const int total_items = min(sc.item0[a.batch], a.max_items);
+    auto get_item = [&](int item, int local) {  // local = how many items this CTA has started before
+        return local < kPreItems ? s_items[local] : decode_item(sc, item, G);
+    };
 
     // Running use counts of the barrier families.  Every role walks the same items and tiles in
     // the same order, so each keeps its own copy.
@@ -446,8 +457,9 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
     if (warp == kProducerWarp) {
         // ================================ TMA producer ====================================
         if (lane == 0) {
-            for (int item = blockIdx.x; item < total_items && alive; item += gridDim.x) {
-                const Item it = decode_item(sc, item, G);
+            int li = 0;
+            for (int item = blockIdx.x; item < total_items && alive; item += gridDim.x, ++li) {
+                const Item it = get_item(item, li);
                 if (a.q_by_tma) {
                     // the Q tiles of the previous item are free once its last QK^T has completed
                     if (!mbar_wait(bar(bar_qempty()), (items_run & 1u) ^ 1u, abort_flag, a.status)) {
@@ -459,7 +471,7 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
 #pragma unroll
                         for (int p = 0; p < S::kPanels; ++p)
                             tma_load_5d(base + S::kOffQ + m * S::kQTile + p * S::kQPanel, &map_q, bar(bar_qfull()),
-                                        p * 64, 0, it.g, (it.row_base + m * kBM) / G, it.b);
+                                        p * 64, 0, it.g, it.tok0 + m * (kBM / G), it.b);
                     ++items_run;
                 }
                 for (int t = it.t_begin; t < it.t_end; ++t, ++kt_run) {
@@ -506,7 +518,7 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
         const uint64_t vdesc0 = smem_desc(base + S::kOffV, S::kKVPanel, 1024);
         const uint32_t o_t = tmem + x * 256 + 128;
         for (int item = blockIdx.x; item < total_items && alive; item += gridDim.x, ++items_run) {
-            const Item it = decode_item(sc, item, G);
+            const Item it = get_item(item, static_cast<int>(items_run));
             const bool row_mode = it.nmt == 2;
             const uint64_t qdesc = qdesc0 + static_cast<uint64_t>((row_mode ? x : 0) * (S::kQTile >> 4));
             alive = warp_wait(bar(bar_qfull()), items_run & 1u, abort_flag, a.status);
@@ -578,7 +590,7 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
         const uint32_t o_t = tmem + lane_sel + x * 256 + 128;
         constexpr int kChunks = D / 8;                 // 16-byte pieces of a row
         for (int item = blockIdx.x; item < total_items && alive; item += gridDim.x, ++items_run) {
-            const Item it = decode_item(sc, item, G);
+            const Item it = get_item(item, static_cast<int>(items_run));
             const bool row_mode = it.nmt == 2;
             // ---- Q tiles -> shared memory in the swizzled K-major layout (only when the group
             // size does not allow the TMA view) ---------------------------------------------
@@ -802,30 +814,30 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
                                make_float2(m_ref, l_run));
                     }
                 }
-#pragma unroll 1
-                for (int c0 = 0; c0 < D; c0 += 64) {
-                    uint32_t orr[2][32];
-                    tmem_ld32(o_t + c0, orr[0]);
-                    tmem_ld32(o_t + c0 + 32, orr[1]);
+                {
+                    uint32_t orr[D / 32][32];  // the whole row: all loads in flight, then all stores
+#pragma unroll
+                    for (int c = 0; c < D / 32; ++c) tmem_ld32(o_t + c * 32, orr[c]);
                     tmem_wait_ld();
-                    if (!row_ok) continue;
-                    if (direct) {
+                    if (row_ok) {
+                        if (direct) {
 #pragma unroll
-                        for (int q8 = 0; q8 < 8; ++q8) {
-                            const uint32_t* w = &orr[q8 >> 2][(q8 & 3) * 8];
-                            uint4 v;
-                            v.x = pack_bf16(__uint_as_float(w[0]) * inv, __uint_as_float(w[1]) * inv);
-                            v.y = pack_bf16(__uint_as_float(w[2]) * inv, __uint_as_float(w[3]) * inv);
-                            v.z = pack_bf16(__uint_as_float(w[4]) * inv, __uint_as_float(w[5]) * inv);
-                            v.w = pack_bf16(__uint_as_float(w[6]) * inv, __uint_as_float(w[7]) * inv);
-                            *reinterpret_cast<uint4*>(dst + c0 + q8 * 8) = v;
-                        }
-                    } else {
+                            for (int q8 = 0; q8 < D / 8; ++q8) {
+                                const uint32_t* w = &orr[q8 >> 2][(q8 & 3) * 8];
+                                uint4 v;
+                                v.x = pack_bf16(__uint_as_float(w[0]) * inv, __uint_as_float(w[1]) * inv);
+                                v.y = pack_bf16(__uint_as_float(w[2]) * inv, __uint_as_float(w[3]) * inv);
+                                v.z = pack_bf16(__uint_as_float(w[4]) * inv, __uint_as_float(w[5]) * inv);
+                                v.w = pack_bf16(__uint_as_float(w[6]) * inv, __uint_as_float(w[7]) * inv);
+                                *reinterpret_cast<uint4*>(dst + q8 * 8) = v;
+                            }
+                        } else {
 #pragma unroll
-                        for (int q4 = 0; q4 < 16; ++q4) {
-                            const uint32_t* w = &orr[q4 >> 3][(q4 & 7) * 4];
-                            __stcg(po + (c0 / 4 + q4) * kBM, make_float4(__uint_as_float(w[0]), __uint_as_float(w[1]),
-                                                                       __uint_as_float(w[2]), __uint_as_float(w[3])));
+                            for (int q4 = 0; q4 < D / 4; ++q4) {
+                                const uint32_t* w = &orr[q4 >> 3][(q4 & 7) * 4];
+                                __stcg(po + q4 * kBM, make_float4(__uint_as_float(w[0]), __uint_as_float(w[1]),
+                                                                  __uint_as_float(w[2]), __uint_as_float(w[3])));
+                            }
                         }
                     }
                 }
