@@ -32,6 +32,9 @@ from paper_2601_12212_b200 import synth  # noqa: E402
 METRIC = "us_per_speculative_step"
 UNIT = "us/step"
 NOMINAL_HBM_GBS = 8000.0
+# DRAM bytes of one tree_attention_kernel launch on the benchmarked workload, from the ncu capture
+# summarised in profiles/tree_attention_cfg2_ncu.md (set to None when the kernel changes).
+ATTENTION_TRAFFIC_BYTES = 5034496
 
 
 def measured_peaks():
@@ -277,7 +280,7 @@ class DeviceWorkload:
         self.verify(i)
         self.compact()
 
-    LAUNCHES_PER_STEP = staticmethod(lambda w: 2 + w.n_layers + 2 + 1)
+    LAUNCHES_PER_STEP = staticmethod(lambda w: 2 + 2 * w.n_layers + 2 + 1)  # scan, tree; attention + combine per layer; argmax, walk; compact
 
     # -- end to end: host buffers in, host result out ---------------------------------------
     def step_e2e(self, i):
@@ -449,8 +452,11 @@ def run_ours(args, w):
                 "steps": Ke},
         "gpu_launches": DeviceWorkload.LAUNCHES_PER_STEP(w) * K,
         "gpu_launches_per_step": DeviceWorkload.LAUNCHES_PER_STEP(w),
-        "roofline": {"kernel": "tree_attention_kernel", "bound": "hbm", "achieved": achieved, "peak": peak,
-                     "unit": "GB/s", "frac": achieved / peak, "traffic": None,
+        "roofline": {"kernel": "tree_attention_kernel (+ attention_combine_kernel, one resps_tree_attention call)",
+                     "bound": "hbm", "achieved": achieved, "peak": peak,
+                     "unit": "GB/s", "frac": achieved / peak, "traffic": ATTENTION_TRAFFIC_BYTES,
+                     "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of tree_attention_kernel, "
+                                       "one launch of this workload (profiles/tree_attention_cfg2_ncu.md)",
                      "peak_source": peak_src, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
                      "algorithmic_bytes_per_launch": alg, "us_per_launch": t_attn,
                      "launches_timed": K * w.n_layers},
