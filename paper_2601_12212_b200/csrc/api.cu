@@ -100,6 +100,7 @@ int resps_create(resps_ctx** out, const resps_shape* shape) {
     if (const char* e = std::getenv("RESPS_SCAN_CHUNK"))
         chunk = std::min(chunk, std::max(1024, std::atoi(e) / 1024 * 1024));
     w.scan_chunk = chunk;
+    if (const char* e = std::getenv("RESPS_SCAN_SLICES")) w.scan_slices_hint = std::max(0, std::atoi(e));
     w.scan_splits = (s.vocab + chunk - 1) / chunk;
     if (w.scan_splits > 128) {
         delete c;
@@ -130,7 +131,8 @@ int resps_create(resps_ctx** out, const resps_shape* shape) {
     Carver real;
     real.base = static_cast<char*>(c->arena);
     carve(c, real);
-    if (resps::attention_setup(c) != cudaSuccess || resps::tree_setup(c) != cudaSuccess) {
+    if (resps::attention_setup(c) != cudaSuccess || resps::tree_setup(c) != cudaSuccess ||
+        resps::scan_setup(c) != cudaSuccess) {
         cudaFree(c->arena);
         delete c;
         return RESPS_ERR_CUDA;

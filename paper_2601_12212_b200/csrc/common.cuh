@@ -17,6 +17,7 @@ struct Workspace {
     // vocabulary scans
     int scan_chunk = 0;       // elements of a row handled by one CTA
     int scan_splits = 0;      // ceil(V / scan_chunk)
+    int scan_slices_hint = 0; // > 0: slices per row of the streaming scan (tuning aid)
     int max_rows = 0;         // 1 + (max_depth-1)*max_k
     unsigned long long* part_key = nullptr;  // [max_batch][max_rows][splits][max_k] packed (value,id)
     float2* part_ms = nullptr;               // [max_batch][max_rows][splits] (max, sum) in log2 domain
@@ -81,6 +82,7 @@ cudaError_t launch_tree_attention(const resps_ctx* ctx, const resps_step* d_step
                                   const uint64_t* mask, float scale, cudaStream_t st);
 cudaError_t attention_setup(resps_ctx* ctx);  // one-time function attributes
 cudaError_t tree_setup(resps_ctx* ctx);
+cudaError_t scan_setup(resps_ctx* ctx);
 int tree_candidate_limit();
 
 // ---- device helpers --------------------------------------------------------

@@ -25,6 +25,7 @@ struct ScanArgs {
     int n_levels, n_slots;
     int vocab, max_tt, max_k, max_rows;
     int chunk, splits;
+    int slices, cps;  // streaming kernel: slices per row, chunks per slice (partials keep the stride `splits`)
     unsigned long long* part_key;
     float2* part_ms;
     unsigned int* counter;
@@ -49,7 +50,7 @@ struct LseAcc {
 // rank-by-counting selection: the `k` largest of n keys in shared memory, written in order.
 template <typename Out>
 __device__ __forceinline__ void select_top_by_rank(const unsigned long long* keys, int n, int k, Out out) {
-    for (int c = threadIdx.x; c < n; c += blockDim.x) {
+    for (int c = threadIdx.x; c < n; c += kScanThreads) {  // callers run it with kScanThreads threads
         const unsigned long long mine = keys[c];
         int rank = 0;
         for (int j = 0; j < n; ++j) rank += (keys[j] > mine) || (keys[j] == mine && j < c);
@@ -241,6 +242,339 @@ __global__ void __launch_bounds__(kScanThreads, 4) row_scan_kernel(const ScanArg
     }
 }
 
+// ---------------------------------------------------------------------------------------
+// Streaming variant (16-byte aligned rows): a CTA walks a slice of several chunks of one row.
+// One thread issues bulk copies (cp.async.bulk, global -> shared, completion on an mbarrier)
+// three chunks ahead, so the loads of the next chunks run under the arithmetic of the current
+// one.  The first chunk establishes the threshold tau as above; afterwards tau is the k-th best
+// logit seen so far, a chunk contributes only the (few) logits at or above it, and the list is
+// cut back to its k best when it has grown.  The log-sum-exp state stays in registers across
+// chunks.  A chunk whose hits would not fit the list (adversarial order) re-derives a threshold
+// of its own from its quad maxima, which bounds its candidates by 128 k.
+// ---------------------------------------------------------------------------------------
+constexpr int kStreamStages = 3;
+constexpr long long kScanWaitLimitCycles = 4000000000ll;
+
+__device__ __forceinline__ uint32_t scan_smem_u32(const void* p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ bool scan_mbar_try(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded: on expiry the status word is flagged and the caller goes on (its results are then
+// meaningless, but every counter protocol still completes).
+__device__ __forceinline__ void scan_mbar_wait(uint32_t bar, uint32_t parity, int32_t* status) {
+    if (scan_mbar_try(bar, parity)) return;
+    const long long t0 = clock64();
+    unsigned spins = 0;
+    while (!scan_mbar_try(bar, parity)) {
+        if ((++spins & 63u) == 0u && clock64() - t0 > kScanWaitLimitCycles) {
+            atomicOr(status, RESPS_STATUS_WAIT_TIMEOUT);
+            return;
+        }
+    }
+}
+
+constexpr int kStreamThreads = kScanThreads + 32;  // eight consumer warps + the copy-issuing warp
+
+__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+__device__ __forceinline__ bool consumer_any(bool pred) {  // barrier over the consumers, OR of pred
+    uint32_t out;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 q, %1, 0;\n\t"
+        "bar.red.or.pred p, 1, 256, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(out)
+        : "r"(pred ? 1u : 0u)
+        : "memory");
+    return out != 0;
+}
+
+__global__ void __launch_bounds__(kStreamThreads, 2) row_scan_stream_kernel(const ScanArgs a) {
+    extern __shared__ __align__(128) unsigned char s_raw[];
+    float* s_stage = reinterpret_cast<float*>(s_raw);                                    // [3][8192]
+    unsigned long long* s_keys =
+        reinterpret_cast<unsigned long long*>(s_raw + kStreamStages * kScanChunkMax * sizeof(float));  // list
+    __shared__ __align__(8) unsigned long long s_bar[2 * kStreamStages];  // full[3], empty[3]
+    __shared__ unsigned long long s_quad[kQuads];
+    __shared__ unsigned long long s_top[RESPS_MAX_K];
+    __shared__ unsigned long long s_tau;
+    __shared__ int s_count;
+    __shared__ float2 s_ms[kScanThreads / 32];
+    __shared__ bool s_last;
+    const int b = blockIdx.z, r = blockIdx.y, sl = blockIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const StepDims sd = clamp_step(a.steps[b], a.n_levels, a.n_slots, a.max_tt, a.max_k, a.vocab);
+    const int k = sd.k;
+    const int rows = 1 + (sd.d - 1) * k;
+    if (r >= rows) return;
+    if (sd.clamped && r == 0 && sl == 0 && tid == 0) atomicOr(a.status, RESPS_STATUS_STEP_CLAMPED);
+    const int level = (r == 0) ? 0 : 1 + (r - 1) / k;
+    const int slot = (r == 0) ? 0 : (r - 1) % k;
+    const float* row = a.logits + b * a.ld_b + level * a.ld_level + slot * a.ld_row;
+    const int c_begin = sl * a.cps;
+    const int c_end = min(a.splits, c_begin + a.cps);  // chunks [c_begin, c_end) of this row
+    const int list_cap = (kQuadElems + 1) * a.max_k;
+    const uint32_t bar0 = scan_smem_u32(s_bar);
+    auto full_bar = [&](int st) { return bar0 + 8u * st; };
+    auto empty_bar = [&](int st) { return bar0 + 8u * (kStreamStages + st); };
+
+    if (tid == 0) {
+        for (int st = 0; st < kStreamStages; ++st) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(full_bar(st)) : "memory");
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(empty_bar(st)), "r"(kScanThreads) : "memory");
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        s_count = 0;
+        s_tau = 0ull;
+    }
+    __syncthreads();
+
+    if (warp == kScanThreads / 32) {
+        // ---- copy-issuing warp: a stage is refilled as soon as every consumer has read it ----------
+        if (lane == 0) {
+            for (int c = c_begin; c < c_end; ++c) {
+                const int u = c - c_begin, st = u % kStreamStages;
+                scan_mbar_wait(empty_bar(st), ((u / kStreamStages) & 1u) ^ 1u, a.status);
+                const int e0 = c * kScanChunkMax;
+                const uint32_t bytes = static_cast<uint32_t>(min(a.vocab - e0, kScanChunkMax)) * 4u;
+                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(full_bar(st)), "r"(bytes)
+                             : "memory");
+                asm volatile(
+                    "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                        scan_smem_u32(s_stage + st * kScanChunkMax)),
+                    "l"(row + e0), "r"(bytes), "r"(full_bar(st))
+                    : "memory");
+            }
+        }
+        return;  // the consumers wait for every copy that was issued
+    }
+
+    int list_n = 0;                // entries of the candidate list (same in every thread)
+    LseAcc acc;                    // this thread's running (max, sum) over all its logits
+    unsigned long long tau = 0ull; // k-th best so far (0 = none yet: everything qualifies)
+    float tau_v = -INFINITY;
+
+    for (int c = c_begin; c < c_end; ++c) {
+        const int u0 = c - c_begin, st = u0 % kStreamStages;
+        const int begin = c * kScanChunkMax;
+        const int end = min(a.vocab, begin + kScanChunkMax);
+        scan_mbar_wait(full_bar(st), (u0 / kStreamStages) & 1u, a.status);
+        float v[kScanPerThread];
+#pragma unroll
+        for (int u = 0; u < kScanPerThread / 4; ++u) {
+            const int off = (u * kScanThreads + tid) * 4;
+            v[4 * u] = v[4 * u + 1] = v[4 * u + 2] = v[4 * u + 3] = -INFINITY;
+            if (begin + off < end) {  // the vocabulary is a multiple of 4 on this path
+                const float4 x = *reinterpret_cast<const float4*>(s_stage + st * kScanChunkMax + off);
+                v[4 * u] = x.x, v[4 * u + 1] = x.y, v[4 * u + 2] = x.z, v[4 * u + 3] = x.w;
+            }
+        }
+        auto release_stage = [&]() {
+            asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(empty_bar(st)) : "memory");
+        };
+        auto elem_id = [&](int i) { return begin + ((i >> 2) * kScanThreads + tid) * 4 + (i & 3); };
+        const bool has_any = elem_id(0) < end;
+
+        // ---- thread maximum, log-sum-exp update ---------------------------------------------------
+        float tmax = v[0];
+#pragma unroll
+        for (int i = 1; i + 1 < kScanPerThread; i += 2) tmax = max3f(tmax, v[i], v[i + 1]);
+        tmax = fmaxf(tmax, v[kScanPerThread - 1]);
+        if (has_any) {
+            const float m_new = fmaxf(acc.m2, tmax * kLog2e);
+            float s0 = acc.s * ex2_approx(acc.m2 - m_new), s1 = 0.f;  // 0 * 2^-inf = 0 on the first chunk
+#pragma unroll
+            for (int i = 0; i < kScanPerThread; i += 2) {
+                s0 += ex2_approx(fmaf(v[i], kLog2e, -m_new));
+                s1 += ex2_approx(fmaf(v[i + 1], kLog2e, -m_new));
+            }
+            acc.m2 = m_new, acc.s = s0 + s1;
+        }
+        const bool first = (c == c_begin);
+        // One barrier per chunk in the common case: does any thread hold a logit at or above tau?
+        // (branch-free bit mask; the few hits are then re-read from the stage by index)
+        uint32_t hits = 0u;
+        if (!first) {
+#pragma unroll
+            for (int i = 0; i < kScanPerThread; ++i) hits |= (v[i] >= tau_v) ? (1u << i) : 0u;
+            if (!consumer_any(hits != 0u)) {
+                release_stage();
+                continue;
+            }
+        }
+
+        // Threads that hold such logits append them to the list.  Should the list overflow
+        // (adversarial order: every logit beats the threshold), the appended entries are dropped
+        // and the chunk takes the bounded path below.
+        bool slow = first;
+        if (!first) {
+            const float* stage = s_stage + st * kScanChunkMax;
+            while (hits) {
+                const int i = __ffs(hits) - 1;
+                hits &= hits - 1u;
+                const int e = elem_id(i);
+                if (e < end) {
+                    const unsigned long long key = pack_val_id(stage[e - begin], e);
+                    if (key >= tau) {
+                        const int at = atomicAdd(&s_count, 1);
+                        if (at < list_cap) s_keys[at] = key;
+                    }
+                }
+            }
+            consumer_sync();
+            slow = s_count > list_cap;  // fixed until the next barrier
+        }
+        release_stage();
+        if (slow) {
+            // the chunk's own threshold from its quad maxima (see row_scan_kernel); the list is cut
+            // to its k best first so that the chunk's at most 128 k candidates fit behind them
+            if (!first) {  // the first list_n entries are the list as it was before this chunk
+                for (int cidx = tid; cidx < list_n; cidx += kScanThreads) {
+                    const unsigned long long mine = s_keys[cidx];
+                    int rank = 0;
+                    for (int j = 0; j < list_n; ++j) rank += (s_keys[j] > mine) ? 1 : 0;
+                    if (rank < k) s_top[rank] = mine;
+                }
+                consumer_sync();
+                const int nk = min(list_n, k);
+                if (tid < nk) s_keys[tid] = s_top[tid];
+                if (tid == 0) s_count = nk;
+                consumer_sync();
+            }
+            int tpos = 0;
+#pragma unroll
+            for (int i = kScanPerThread - 1; i >= 0; --i)
+                if (v[i] == tmax) tpos = i;
+            const unsigned long long my_key = has_any ? pack_val_id(tmax, elem_id(tpos)) : 0ull;
+            unsigned long long quad_key = my_key;
+            {
+                unsigned long long o = __shfl_xor_sync(kFull, quad_key, 1);
+                quad_key = o > quad_key ? o : quad_key;
+                o = __shfl_xor_sync(kFull, quad_key, 2);
+                quad_key = o > quad_key ? o : quad_key;
+            }
+            if ((lane & 3) == 0) s_quad[tid >> 2] = quad_key;
+            consumer_sync();
+            if (tid < kQuads) {
+                const unsigned long long mine = s_quad[tid];
+                int rank = 0;
+#pragma unroll 8
+                for (int j = 0; j < kQuads; ++j) {
+                    const unsigned long long o = s_quad[j];
+                    rank += (o > mine) || (o == mine && j < tid);
+                }
+                if (rank == min(k, kQuads) - 1) s_tau = mine;
+            }
+            consumer_sync();
+            const unsigned long long tau_c = s_tau > tau ? s_tau : tau;  // never below the running one
+            if (quad_key >= tau_c && has_any) {
+                const float tv = (tau_c == 0ull) ? -INFINITY : key_val(tau_c);
+#pragma unroll
+                for (int i = 0; i < kScanPerThread; ++i)
+                    if (v[i] >= tv && elem_id(i) < end) {
+                        const unsigned long long key = pack_val_id(v[i], elem_id(i));
+                        if (key >= tau_c) s_keys[atomicAdd(&s_count, 1)] = key;
+                    }
+            }
+        }
+        consumer_sync();
+        // ---- tighten: tau = k-th best of the list; cut the list back when it has grown ----------
+        const int n_list = s_count;
+        list_n = n_list;
+        if (slow || n_list > 8 * k) {
+            for (int cidx = tid; cidx < n_list; cidx += kScanThreads) {
+                const unsigned long long mine = s_keys[cidx];
+                int rank = 0;
+                for (int j = 0; j < n_list; ++j) rank += (s_keys[j] > mine) ? 1 : 0;
+                if (rank < k) s_top[rank] = mine;
+            }
+            consumer_sync();
+            const int nk = min(n_list, k);
+            if (tid < nk) s_keys[tid] = s_top[tid];
+            if (tid == 0) {
+                s_count = nk;
+                s_tau = (n_list >= k) ? s_top[k - 1] : 0ull;
+            }
+            consumer_sync();
+            tau = s_tau;
+            tau_v = (tau == 0ull) ? -INFINITY : key_val(tau);
+            list_n = nk;
+        }
+    }
+
+    // ---- the slice's k best and its log-sum-exp partial ------------------------------------------
+    consumer_sync();
+    const int n_cand = s_count;
+    const int64_t prow = static_cast<int64_t>(b) * a.max_rows + r;
+    unsigned long long* part = a.part_key + (prow * a.splits + sl) * a.max_k;
+    select_top_by_rank(s_keys, n_cand, k, [&](int rank, unsigned long long key) { part[rank] = key; });
+    if (tid >= n_cand && tid < k) part[tid] = 0ull;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float om = __shfl_xor_sync(kFull, acc.m2, o);
+        const float os = __shfl_xor_sync(kFull, acc.s, o);
+        acc.merge(om, os);
+    }
+    if (lane == 0) s_ms[warp] = make_float2(acc.m2, acc.s);
+    consumer_sync();
+    if (tid == 0) {
+        LseAcc t;
+        for (int w = 0; w < kScanThreads / 32; ++w) t.merge(s_ms[w].x, s_ms[w].y);
+        a.part_ms[prow * a.splits + sl] = make_float2(t.m2, t.s);
+    }
+    __threadfence();
+    consumer_sync();
+    if (tid == 0) s_last = (atomicAdd(a.counter + prow, 1u) == static_cast<unsigned>(a.slices - 1));
+    consumer_sync();
+    if (!s_last) return;
+
+    // ---- last CTA of the row: merge the slices ---------------------------------------------------
+    __threadfence();
+    const unsigned long long* parts = a.part_key + prow * a.splits * a.max_k;
+    for (int i = tid; i < a.slices * k; i += kScanThreads) s_keys[i] = __ldcg(parts + (i / k) * a.max_k + (i % k));
+    float2 my_ms = make_float2(-INFINITY, 0.f);
+    if (tid < a.slices) my_ms = __ldcg(a.part_ms + prow * a.splits + tid);
+    consumer_sync();
+    float* oval = a.row_val + prow * a.max_k;
+    int32_t* oid = a.row_id + prow * a.max_k;
+    select_top_by_rank(s_keys, a.slices * k, k, [&](int rank, unsigned long long key) {
+        oval[rank] = key_val(key);
+        oid[rank] = key_id(key);
+    });
+    if (warp < 4) {
+        float M = my_ms.x;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(kFull, M, o));
+        if (lane == 0) s_ms[warp] = make_float2(M, 0.f);
+    }
+    consumer_sync();
+    if (warp < 4) {
+        const float M = fmaxf(fmaxf(s_ms[0].x, s_ms[1].x), fmaxf(s_ms[2].x, s_ms[3].x));
+        double sum = (my_ms.y > 0.f) ? static_cast<double>(my_ms.y) * static_cast<double>(ex2_approx(my_ms.x - M)) : 0.0;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(kFull, sum, o);
+        if (lane == 0) s_quad[warp] = __double_as_longlong(sum);
+    }
+    consumer_sync();
+    if (tid == 0) {
+        const float M = fmaxf(fmaxf(s_ms[0].x, s_ms[1].x), fmaxf(s_ms[2].x, s_ms[3].x));
+        const double sum = __longlong_as_double(s_quad[0]) + __longlong_as_double(s_quad[1]) +
+                           __longlong_as_double(s_quad[2]) + __longlong_as_double(s_quad[3]);
+        a.row_lse[prow] = (static_cast<double>(M) + log2(sum)) * 0.6931471805599453094;
+        a.counter[prow] = 0u;
+    }
+}
+
 struct ArgmaxArgs {
     const int32_t* n_nodes;
     const float* logits;
@@ -343,6 +677,16 @@ inline bool vec_ok(const void* p, int64_t s0, int64_t s1, int64_t s2, int vocab,
 
 int scan_chunk_max() { return kScanChunkMax; }
 
+static size_t stream_smem_bytes(int max_k, int slices) {
+    return kStreamStages * kScanChunkMax * sizeof(float) +
+           sizeof(unsigned long long) * max((kQuadElems + 1) * max_k, slices * max_k);
+}
+
+cudaError_t scan_setup(resps_ctx* ctx) {
+    return cudaFuncSetAttribute(row_scan_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                static_cast<int>(stream_smem_bytes(ctx->shape.max_k, 128)));
+}
+
 cudaError_t launch_row_scan(const resps_ctx* ctx, const resps_step* d_steps, int batch,
                             const float* logits, int64_t ld_b, int64_t ld_level, int64_t ld_row,
                             int n_levels, int n_slots, cudaStream_t st) {
@@ -358,12 +702,21 @@ cudaError_t launch_row_scan(const resps_ctx* ctx, const resps_step* d_steps, int
     a.row_val = w.row_val, a.row_id = w.row_id, a.row_lse = w.row_lse, a.status = w.status;
     const int k_ext = min(n_slots, ctx->shape.max_k);
     const int rows = (n_levels > 1) ? 1 + (n_levels - 1) * k_ext : 1;
-    dim3 grid(w.scan_splits, rows, batch);
+    a.slices = w.scan_splits, a.cps = 1;
     const size_t smem = sizeof(unsigned long long) * ctx->shape.max_k * max(kQuadElems, w.scan_splits);
-    if (vec_ok(logits, ld_b, ld_level, ld_row, a.vocab, a.chunk))
-        row_scan_kernel<true><<<grid, kScanThreads, smem, st>>>(a);
-    else
+    if (vec_ok(logits, ld_b, ld_level, ld_row, a.vocab, a.chunk) && w.scan_chunk == kScanChunkMax) {
+        // enough slices for two CTAs per SM over the largest row count, each several chunks long
+        int want = (2 * ctx->sm_count + rows * batch - 1) / (rows * batch);
+        if (w.scan_slices_hint > 0) want = w.scan_slices_hint;
+        const int slices0 = max(1, min(w.scan_splits, want));
+        a.cps = (w.scan_splits + slices0 - 1) / slices0;
+        a.slices = (w.scan_splits + a.cps - 1) / a.cps;
+        dim3 grid(a.slices, rows, batch);
+        row_scan_stream_kernel<<<grid, kStreamThreads, stream_smem_bytes(ctx->shape.max_k, a.slices), st>>>(a);
+    } else {
+        dim3 grid(w.scan_splits, rows, batch);
         row_scan_kernel<false><<<grid, kScanThreads, smem, st>>>(a);
+    }
     return cudaGetLastError();
 }
 
