@@ -103,14 +103,16 @@ __device__ __forceinline__ void build_sched(const AttnArgs& a, Sched& sc, int ti
     if (tid == 0) {
         long long units = 0;
         for (int b = 0; b < a.batch; ++b) units += 1ll * a.Hkv * sc.mp[b] * sc.kt[b];
-        int tps = static_cast<int>((units + a.sched_grid - 1) / a.sched_grid);
+        int tps = (units < (1ll << 30))  // the 64-bit division is a long dependent chain: avoid it when possible
+                      ? (static_cast<int>(units) + a.sched_grid - 1) / a.sched_grid
+                      : static_cast<int>((units + a.sched_grid - 1) / a.sched_grid);
         tps = max(tps, max(a.min_tiles, 1));
         // ceil(kt / tps) splits per group can add up to more items than CTAs (a second, nearly
         // empty round); a slightly larger tile count per split then gives a single round.
         if (a.batch <= 32) {
             for (int tries = 0; tries < 8; ++tries) {
-                long long cnt = 0;
-                for (int b = 0; b < a.batch; ++b) cnt += 1ll * a.Hkv * sc.mp[b] * ((sc.kt[b] + tps - 1) / tps);
+                int cnt = 0;  // batch <= 32 here: no overflow
+                for (int b = 0; b < a.batch; ++b) cnt += a.Hkv * sc.mp[b] * ((sc.kt[b] + tps - 1) / tps);
                 if (cnt <= a.sched_grid) break;
                 ++tps;
             }
@@ -460,20 +462,6 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
             int li = 0;
             for (int item = blockIdx.x; item < total_items && alive; item += gridDim.x, ++li) {
                 const Item it = get_item(item, li);
-                if (a.q_by_tma) {
-                    // the Q tiles of the previous item are free once its last QK^T has completed
-                    if (!mbar_wait(bar(bar_qempty()), (items_run & 1u) ^ 1u, abort_flag, a.status)) {
-                        alive = false;
-                        break;
-                    }
-                    mbar_expect_tx(bar(bar_qfull()), it.nmt * S::kQTile);
-                    for (int m = 0; m < it.nmt; ++m)
-#pragma unroll
-                        for (int p = 0; p < S::kPanels; ++p)
-                            tma_load_5d(base + S::kOffQ + m * S::kQTile + p * S::kQPanel, &map_q, bar(bar_qfull()),
-                                        p * 64, 0, it.g, it.tok0 + m * (kBM / G), it.b);
-                    ++items_run;
-                }
                 for (int t = it.t_begin; t < it.t_end; ++t, ++kt_run) {
                     const int s = kt_run % kStages;
                     if (!mbar_wait(bar(bar_kvempty(s)), ((kt_run / kStages) & 1u) ^ 1u, abort_flag, a.status)) {
@@ -486,6 +474,22 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
 #pragma unroll
                     for (int p = 0; p < S::kPanels; ++p)
                         tma_load_4d(dk + p * S::kKVPanel, &map_k, bar(bar_kfull(s)), p * 64, t * kBN, it.g, it.b);
+                    if (t == it.t_begin && a.q_by_tma) {
+                        // Q goes between the first K and the first V tile: K and Q are what the first
+                        // MMA needs.  The Q tiles of the previous item are free once its last QK^T has
+                        // completed.
+                        if (!mbar_wait(bar(bar_qempty()), (items_run & 1u) ^ 1u, abort_flag, a.status)) {
+                            alive = false;
+                            break;
+                        }
+                        mbar_expect_tx(bar(bar_qfull()), it.nmt * S::kQTile);
+                        for (int m = 0; m < it.nmt; ++m)
+#pragma unroll
+                            for (int p = 0; p < S::kPanels; ++p)
+                                tma_load_5d(base + S::kOffQ + m * S::kQTile + p * S::kQPanel, &map_q,
+                                            bar(bar_qfull()), p * 64, 0, it.g, it.tok0 + m * (kBM / G), it.b);
+                        ++items_run;
+                    }
                     mbar_expect_tx(bar(bar_vfull(s)), S::kKVTile);
 #pragma unroll
                     for (int p = 0; p < S::kPanels; ++p)
@@ -872,23 +876,24 @@ __global__ void __launch_bounds__(kCombineThreads) attention_combine_kernel(cons
     build_sched(a, sc, threadIdx.x, kCombineThreads);  // inputs of the attention kernel, complete before it ran
     pdl_wait();                                        // the attention kernel has finished and its writes are visible
     const int G = a.Hq / a.Hkv;
-    constexpr int kPerGroup = kRowTiles * kBM * (D / 4);  // (row, 4 columns) work items of a group
     for (int b = 0; b < a.batch; ++b) {
         const int splits = sc.splits[b];
         if (sc.n[b] == 0) continue;
-        const int groups = a.Hkv * sc.mp[b];
         const int M = sc.n[b] * G;
-        if (splits <= 1 && M - (sc.mp[b] - 1) * kRowTiles * kBM > kBM) continue;  // every group wrote O directly
-        const long long total = 1ll * groups * kPerGroup;
+        const bool last_is_key_mode = M - (sc.mp[b] - 1) * kRowTiles * kBM <= kBM;
+        if (splits <= 1 && !last_is_key_mode) continue;  // every group wrote O directly
+        // work items: (KV head, 4 columns, row) over the M valid rows; consecutive threads take
+        // consecutive rows
+        const int per_head = M * (D / 4);
+        const long long total = 1ll * a.Hkv * per_head;
         for (long long idx = 1ll * blockIdx.x * kCombineThreads + threadIdx.x; idx < total;
              idx += 1ll * gridDim.x * kCombineThreads) {
-            const int grp = static_cast<int>(idx / kPerGroup);
-            const int rem = static_cast<int>(idx % kPerGroup);
-            const int c4 = rem / (kRowTiles * kBM);
-            const int row2 = rem % (kRowTiles * kBM);  // row inside the pair: consecutive threads, consecutive rows
-            const int pair = grp % sc.mp[b], g = grp / sc.mp[b];
-            const int R = pair * kRowTiles * kBM + row2;
-            if (R >= M) continue;
+            const int g = static_cast<int>(idx / per_head);
+            const int rem = static_cast<int>(idx % per_head);
+            const int c4 = rem / M;
+            const int R = rem % M;
+            const int pair = R / (kRowTiles * kBM), row2 = R % (kRowTiles * kBM);
+            const int grp = g * sc.mp[b] + pair;
             const bool key_mode = M - pair * kRowTiles * kBM <= kBM;
             if (!key_mode && splits <= 1) continue;
             const int mt = row2 / kBM, r = row2 % kBM;
