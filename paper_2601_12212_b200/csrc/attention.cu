@@ -50,7 +50,7 @@ constexpr int kAttnThreads = 352;
 constexpr int kSyncThreads = 320;  // softmax warps + the MMA warps meet at the end of an item
 constexpr int kMaxBatchSmem = 256;
 constexpr int kTmemCols = 512;
-constexpr int kCombineThreads = 128;  // small enough to share an SM with a draining attention CTA
+constexpr int kCombineThreads = 256;
 constexpr long long kWaitLimitCycles = 4000000000ll;  // bounded waits give up after ~2 s of SM clocks
 constexpr float kRescaleSlack = 8.0f;  // O is rescaled only when the running max grows by > 2^8
 constexpr unsigned kFull = 0xFFFFFFFFu;
@@ -872,15 +872,21 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
 template <int D>
 __global__ void __launch_bounds__(kCombineThreads) attention_combine_kernel(const AttnArgs a) {
     __shared__ Sched sc;
+    __shared__ int4 s_sched[kMaxBatchSmem];
     pdl_launch_dependents();
-    build_sched(a, sc, threadIdx.x, kCombineThreads);  // inputs of the attention kernel, complete before it ran
-    pdl_wait();                                        // the attention kernel has finished and its writes are visible
+    // The work list is derived again from the step parameters (inputs of the attention kernel,
+    // complete before it ran): this part runs while the attention kernel drains.
+    build_sched(a, sc, threadIdx.x, kCombineThreads);
+    for (int b = threadIdx.x; b < a.batch; b += kCombineThreads)
+        s_sched[b] = make_int4(sc.n[b], sc.mp[b], sc.splits[b], sc.item0[b]);
+    __syncthreads();
+    pdl_wait();  // the attention kernel has finished and its partials are visible
     const int G = a.Hq / a.Hkv;
     for (int b = 0; b < a.batch; ++b) {
-        const int splits = sc.splits[b];
-        if (sc.n[b] == 0) continue;
-        const int M = sc.n[b] * G;
-        const bool last_is_key_mode = M - (sc.mp[b] - 1) * kRowTiles * kBM <= kBM;
+        const int n_b = s_sched[b].x, mp_b = s_sched[b].y, splits = s_sched[b].z, item0_b = s_sched[b].w;
+        if (n_b == 0) continue;
+        const int M = n_b * G;
+        const bool last_is_key_mode = M - (mp_b - 1) * kRowTiles * kBM <= kBM;
         if (splits <= 1 && !last_is_key_mode) continue;  // every group wrote O directly
         // work items: (KV head, 4 columns, row) over the M valid rows; consecutive threads take
         // consecutive rows
@@ -893,14 +899,14 @@ __global__ void __launch_bounds__(kCombineThreads) attention_combine_kernel(cons
             const int c4 = rem / M;
             const int R = rem % M;
             const int pair = R / (kRowTiles * kBM), row2 = R % (kRowTiles * kBM);
-            const int grp = g * sc.mp[b] + pair;
+            const int grp = g * mp_b + pair;
             const bool key_mode = M - pair * kRowTiles * kBM <= kBM;
             if (!key_mode && splits <= 1) continue;
             const int mt = row2 / kBM, r = row2 % kBM;
             const int n_parts = key_mode ? 2 * splits : splits;
-            const int64_t item_first = sc.item0[b] + static_cast<int64_t>(grp) * splits;
-            // one pass over the partials, sixteen at a time so that their loads are in flight together
-            constexpr int kBatch = 16;
+            const int64_t item_first = item0_b + static_cast<int64_t>(grp) * splits;
+            // one pass over the partials, ten at a time so that their loads are in flight together
+            constexpr int kBatch = 10;
             float Mx = -INFINITY, den = 0.f;
             float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
             for (int p0 = 0; p0 < n_parts; p0 += kBatch) {
