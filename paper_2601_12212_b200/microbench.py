@@ -47,13 +47,24 @@ def attention(name, B, Hq, Hkv, D, Ls, ns, cap, layers, reps=5):
     for l in range(layers):
         call(l)
     torch.cuda.synchronize()
-    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    a.record()
-    for _ in range(reps):
-        for l in range(layers):
-            call(l)
-    b.record()
-    torch.cuda.synchronize()
+    # one CUDA graph of all layers, replayed: launch overhead of the host does not enter the timing
+    stream = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        call(0)
+        torch.cuda.synchronize()
+        with torch.cuda.graph(graph, stream=stream):
+            for l in range(layers):
+                binding.resps_tree_attention(ctx, steps, nn, B, q, o, None, ks[l], vs[l], Hkv * cap * D, cap * D,
+                                             D, cap, mask, scale, stream=stream)
+        graph.replay()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(reps):
+            graph.replay()
+        b.record(stream)
+        torch.cuda.synchronize()
     us = a.elapsed_time(b) * 1e3 / (reps * layers)
     byts = sum(2 * (Ls[s] + ns[s]) * Hkv * D * 2 + 2 * ns[s] * Hq * D * 2 for s in range(B))
     flops = sum(4 * ns[s] * Hq * (Ls[s] + ns[s]) * D for s in range(B))
