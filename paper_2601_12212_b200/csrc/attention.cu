@@ -31,6 +31,7 @@
 // its tensor memory and returns.  Every barrier is used so that a waiter can never
 // fall two phases behind (a parity wait would then never return).
 #include <cuda.h>
+#include <cuda_fp16.h>
 
 #include <cmath>
 
@@ -66,8 +67,12 @@ struct AttnArgs {
     const uint64_t* mask;
     float scale_log2;
     int Hq, Hkv, max_tt;
-    float4* part_o;   // [items][2 row tiles][D/4][128 rows]
-    float2* part_ml;  // [items][2 row tiles][128 rows]   (running max, running sum)
+    // Partials of split groups.  O is stored normalised (O / l, a convex combination of V rows) as
+    // fp16 times a per-row power of two that only differs from 1 when a value would leave the fp16
+    // range: half the bytes of fp32, and 11 significant bits per element (2^-11, against the 2^-9
+    // of the final bf16 rounding).
+    uint4* part_o;    // [items][2 row tiles][D/8][128 rows]  eight fp16 each
+    float4* part_ml;  // [items][2 row tiles][128 rows]   (running max m, running sum l, l * row scale, -)
     int max_items;
     int sched_grid;   // CTAs of the attention grid (the work list is balanced for it)
     int min_tiles;    // smallest key-tile count worth a split of its own
@@ -807,17 +812,10 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
                 const int t = R / G, h = it.g * G + R % G;
                 const float inv = 1.f / l_run;
                 __nv_bfloat16* dst = a.o + ((static_cast<int64_t>(it.b) * a.max_tt + t) * a.Hq + h) * D;
-                float4* po = a.part_o + (static_cast<int64_t>(item) * kRowTiles + x) * (D / 4) * kBM + r;
-                if (row_ok) {
-                    if (direct) {
-                        if (a.lse)
-                            a.lse[(static_cast<int64_t>(it.b) * a.max_tt + t) * a.Hq + h] =
-                                (m_ref + log2f(l_run)) * 0.6931471805599453f;
-                    } else {
-                        __stcg(a.part_ml + (static_cast<int64_t>(item) * kRowTiles + x) * kBM + r,
-                               make_float2(m_ref, l_run));
-                    }
-                }
+                uint4* po = a.part_o + (static_cast<int64_t>(item) * kRowTiles + x) * (D / 8) * kBM + r;
+                if (row_ok && direct && a.lse)
+                    a.lse[(static_cast<int64_t>(it.b) * a.max_tt + t) * a.Hq + h] =
+                        (m_ref + log2f(l_run)) * 0.6931471805599453f;
                 {
                     uint32_t orr[D / 32][32];  // the whole row: all loads in flight, then all stores
 #pragma unroll
@@ -836,11 +834,32 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
                                 *reinterpret_cast<uint4*>(dst + q8 * 8) = v;
                             }
                         } else {
+                            // row scale: 1 unless |O / l| would exceed 2^14 (fp16 holds up to 65504)
+                            float amax = 0.f;
 #pragma unroll
-                            for (int q4 = 0; q4 < D / 4; ++q4) {
-                                const uint32_t* w = &orr[q4 >> 3][(q4 & 7) * 4];
-                                __stcg(po + q4 * kBM, make_float4(__uint_as_float(w[0]), __uint_as_float(w[1]),
-                                                                  __uint_as_float(w[2]), __uint_as_float(w[3])));
+                            for (int c = 0; c < D; c += 2)
+                                amax = max3(amax, fabsf(__uint_as_float(orr[c >> 5][c & 31])),
+                                            fabsf(__uint_as_float(orr[c >> 5][(c & 31) + 1])));
+                            float scale = 1.f;  // O = Ohat * l * scale
+                            const float nmax = amax * inv;
+                            if (nmax > 16384.f) scale = exp2f(ceilf(log2f(nmax)) - 14.f);
+                            const float mul = (l_run > 0.f) ? inv / scale : 0.f;
+                            __stcg(a.part_ml + (static_cast<int64_t>(item) * kRowTiles + x) * kBM + r,
+                                   make_float4(l_run > 0.f ? m_ref : -INFINITY, l_run, l_run * scale, 0.f));
+#pragma unroll
+                            for (int q8 = 0; q8 < D / 8; ++q8) {
+                                const uint32_t* w = &orr[q8 >> 2][(q8 & 3) * 8];
+                                uint4 v;
+                                __half2 h2;
+                                h2 = __floats2half2_rn(__uint_as_float(w[0]) * mul, __uint_as_float(w[1]) * mul);
+                                v.x = *reinterpret_cast<uint32_t*>(&h2);
+                                h2 = __floats2half2_rn(__uint_as_float(w[2]) * mul, __uint_as_float(w[3]) * mul);
+                                v.y = *reinterpret_cast<uint32_t*>(&h2);
+                                h2 = __floats2half2_rn(__uint_as_float(w[4]) * mul, __uint_as_float(w[5]) * mul);
+                                v.z = *reinterpret_cast<uint32_t*>(&h2);
+                                h2 = __floats2half2_rn(__uint_as_float(w[6]) * mul, __uint_as_float(w[7]) * mul);
+                                v.w = *reinterpret_cast<uint32_t*>(&h2);
+                                __stcg(po + q8 * kBM, v);
                             }
                         }
                     }
@@ -848,7 +867,8 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
                 tc_fence_before();
             } else if (!row_mode && row_ok) {
                 // key mode and no tile for this lane (a one-tile item): an empty partial
-                __stcg(a.part_ml + (static_cast<int64_t>(item) * kRowTiles + x) * kBM + r, make_float2(-INFINITY, 0.f));
+                __stcg(a.part_ml + (static_cast<int64_t>(item) * kRowTiles + x) * kBM + r,
+                       make_float4(-INFINITY, 0.f, 0.f, 0.f));
             }
             mbar_arrive(bar(bar_item()));
             alive = warp_wait(bar(bar_item()), items_run & 1u, abort_flag, a.status);
@@ -888,15 +908,15 @@ __global__ void __launch_bounds__(kCombineThreads) attention_combine_kernel(cons
         const int M = n_b * G;
         const bool last_is_key_mode = M - (mp_b - 1) * kRowTiles * kBM <= kBM;
         if (splits <= 1 && !last_is_key_mode) continue;  // every group wrote O directly
-        // work items: (KV head, 4 columns, row) over the M valid rows; consecutive threads take
+        // work items: (KV head, 8 columns, row) over the M valid rows; consecutive threads take
         // consecutive rows
-        const int per_head = M * (D / 4);
+        const int per_head = M * (D / 8);
         const long long total = 1ll * a.Hkv * per_head;
         for (long long idx = 1ll * blockIdx.x * kCombineThreads + threadIdx.x; idx < total;
              idx += 1ll * gridDim.x * kCombineThreads) {
             const int g = static_cast<int>(idx / per_head);
             const int rem = static_cast<int>(idx % per_head);
-            const int c4 = rem / M;
+            const int c8 = rem / M;
             const int R = rem % M;
             const int pair = R / (kRowTiles * kBM), row2 = R % (kRowTiles * kBM);
             const int grp = g * mp_b + pair;
@@ -908,17 +928,17 @@ __global__ void __launch_bounds__(kCombineThreads) attention_combine_kernel(cons
             // one pass over the partials, ten at a time so that their loads are in flight together
             constexpr int kBatch = 10;
             float Mx = -INFINITY, den = 0.f;
-            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
             for (int p0 = 0; p0 < n_parts; p0 += kBatch) {
-                float2 ml[kBatch];
-                float4 v[kBatch];
+                float4 ml[kBatch];
+                uint4 v[kBatch];
 #pragma unroll
                 for (int u = 0; u < kBatch; ++u) {
                     const int p = min(p0 + u, n_parts - 1);
                     const int64_t slot = key_mode ? (item_first + (p >> 1)) * kRowTiles + (p & 1)
                                                   : (item_first + p) * kRowTiles + mt;
                     ml[u] = __ldcg(&a.part_ml[slot * kBM + r]);
-                    v[u] = __ldcg(a.part_o + (slot * (D / 4) + c4) * kBM + r);
+                    v[u] = __ldcg(a.part_o + (slot * (D / 8) + c8) * kBM + r);
                 }
                 float mx = Mx;
 #pragma unroll
@@ -926,24 +946,34 @@ __global__ void __launch_bounds__(kCombineThreads) attention_combine_kernel(cons
                     if (p0 + u < n_parts) mx = fmaxf(mx, ml[u].x);
                 if (mx == -INFINITY) continue;
                 const float corr = ex2_approx(Mx - mx);  // 0 on the first batch
-                den *= corr, acc.x *= corr, acc.y *= corr, acc.z *= corr, acc.w *= corr;
+                den *= corr;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc[e] *= corr;
                 Mx = mx;
 #pragma unroll
                 for (int u = 0; u < kBatch; ++u) {
                     if (p0 + u >= n_parts || ml[u].x == -INFINITY) continue;  // an empty partial holds no O
                     const float w = ex2_approx(ml[u].x - Mx);
                     den += ml[u].y * w;
-                    acc.x += v[u].x * w, acc.y += v[u].y * w, acc.z += v[u].z * w, acc.w += v[u].w * w;
+                    const float wo = ml[u].z * w;  // O_p = Ohat * l * row scale
+                    const uint32_t hw[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&hw[e]));
+                        acc[2 * e] += f.x * wo, acc[2 * e + 1] += f.y * wo;
+                    }
                 }
             }
             const float inv = 1.f / den;
             const int t = R / G, h = g * G + R % G;
-            __nv_bfloat16* dst = a.o + ((static_cast<int64_t>(b) * a.max_tt + t) * a.Hq + h) * D + c4 * 4;
-            uint2 out;
-            out.x = pack_bf16(acc.x * inv, acc.y * inv);
-            out.y = pack_bf16(acc.z * inv, acc.w * inv);
-            *reinterpret_cast<uint2*>(dst) = out;
-            if (a.lse && c4 == 0)
+            __nv_bfloat16* dst = a.o + ((static_cast<int64_t>(b) * a.max_tt + t) * a.Hq + h) * D + c8 * 8;
+            uint4 out;
+            out.x = pack_bf16(acc[0] * inv, acc[1] * inv);
+            out.y = pack_bf16(acc[2] * inv, acc[3] * inv);
+            out.z = pack_bf16(acc[4] * inv, acc[5] * inv);
+            out.w = pack_bf16(acc[6] * inv, acc[7] * inv);
+            *reinterpret_cast<uint4*>(dst) = out;
+            if (a.lse && c8 == 0)
                 a.lse[(static_cast<int64_t>(b) * a.max_tt + t) * a.Hq + h] = (Mx + log2f(den)) * 0.6931471805599453f;
         }
     }
@@ -1049,7 +1079,7 @@ cudaError_t launch_tree_attention(const resps_ctx* ctx, const resps_step* d_step
     a.mask = mask;
     a.scale_log2 = scale * 1.4426950408889634f;
     a.Hq = ctx->shape.n_q_heads, a.Hkv = ctx->shape.n_kv_heads, a.max_tt = ctx->shape.max_tt;
-    a.part_o = reinterpret_cast<float4*>(ctx->ws.attn_part_o), a.part_ml = ctx->ws.attn_part_ml;
+    a.part_o = reinterpret_cast<uint4*>(ctx->ws.attn_part_o), a.part_ml = ctx->ws.attn_part_ml;
     a.max_items = ctx->ws.attn_max_items, a.sched_grid = ctx->ws.attn_grid;
     a.min_tiles = ctx->ws.attn_min_tiles, a.status = ctx->ws.status;
     const int D = ctx->shape.head_dim;

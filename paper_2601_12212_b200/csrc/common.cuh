@@ -2,6 +2,7 @@
 #pragma once
 
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -32,8 +33,8 @@ struct Workspace {
     int attn_combine_grid = 0;  // CTAs of the partial-combine kernel
     int attn_min_tiles = 0;     // smallest key-tile count a split is given
     int attn_max_items = 0;     // partial slots
-    float* attn_part_o = nullptr;   // [items][item rows][D]
-    float2* attn_part_ml = nullptr; // [items][item rows]
+    __half* attn_part_o = nullptr;  // [items][item rows][D] fp16
+    float4* attn_part_ml = nullptr; // [items][item rows]
     int attn_max_groups = 0;
     // status
     int32_t* status = nullptr;
