@@ -45,9 +45,12 @@ constexpr int kBN = 64;            // keys per tile
 constexpr int kStages = 4;         // K/V ring depth
 constexpr int kRowTiles = 2;       // row tiles per item
 constexpr int kSoftmaxThreads = 256;
-constexpr int kProducerWarp = 8;
+constexpr int kProducerWarp = 8;   // K and Q tiles
 constexpr int kMmaWarp0 = 9;       // lane x is issued by warp kMmaWarp0 + x
-constexpr int kAttnThreads = 352;
+constexpr int kVProducerWarp = 11; // V tiles
+constexpr int kAttnThreads = 384;
+constexpr int kRegsSoftmax = 216;  // setmaxnreg: 256 x 216 + 128 x 72 = 384 x 168 <= 64 K registers
+constexpr int kRegsIssue = 72;
 constexpr int kSyncThreads = 320;  // softmax warps + the MMA warps meet at the end of an item
 constexpr int kMaxBatchSmem = 256;
 constexpr int kTmemCols = 512;
@@ -92,6 +95,51 @@ struct Sched {
 
 __device__ __forceinline__ void build_sched(const AttnArgs& a, Sched& sc, int tid, int nthreads) {
     const int G = a.Hq / a.Hkv;
+    if (a.batch <= 32) {
+        // One warp, one lane per sequence: the loads, the divisions and the sums run side by side
+        // and the block meets once.  (Every count below fits 32 bits: at most 32 sequences of at
+        // most 2^15 key tiles, and the row-tile pairs of all KV heads are bounded by the context.)
+        if (tid < 32) {
+            const int b = tid;
+            int n = 0, L = 0, mp = 0, kt = 0;
+            if (b < a.batch) {
+                n = min(max(a.n_nodes[b], 0), a.max_tt);
+                L = max(a.steps[b].prefix_len, 0);
+                if (static_cast<int64_t>(L) + n > a.capacity) {
+                    atomicOr(a.status, RESPS_STATUS_KV_OVERFLOW);
+                    n = 0;
+                }
+                mp = (n * G + kRowTiles * kBM - 1) / (kRowTiles * kBM);
+                kt = (n > 0) ? (L + n + kBN - 1) / kBN : 0;
+            }
+            const unsigned grp = static_cast<unsigned>(a.Hkv * mp);
+            const unsigned units = __reduce_add_sync(0xFFFFFFFFu, grp * static_cast<unsigned>(kt));
+            unsigned tps = (units + a.sched_grid - 1) / a.sched_grid;
+            tps = max(tps, static_cast<unsigned>(max(a.min_tiles, 1)));
+            // ceil(kt / tps) splits per group can add up to more items than CTAs (a second, nearly
+            // empty round); a slightly larger tile count per split then gives a single round.
+            for (int tries = 0; tries < 8; ++tries) {
+                const unsigned cnt = __reduce_add_sync(0xFFFFFFFFu, grp * ((kt + tps - 1) / tps));
+                if (cnt <= static_cast<unsigned>(a.sched_grid)) break;
+                ++tps;
+            }
+            const int splits = (kt + tps - 1) / tps;
+            const int mine = static_cast<int>(grp) * splits;
+            int incl = mine;  // inclusive prefix sum over the lanes
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const int v = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+                if (b >= d) incl += v;
+            }
+            if (b < a.batch) {
+                sc.n[b] = n, sc.L[b] = L, sc.mp[b] = mp, sc.kt[b] = kt, sc.splits[b] = splits;
+                sc.item0[b] = incl - mine;
+                if (b == a.batch - 1) sc.item0[a.batch] = incl;
+            }
+        }
+        __syncthreads();
+        return;
+    }
     for (int b = tid; b < a.batch; b += nthreads) {
         int n = min(max(a.n_nodes[b], 0), a.max_tt);
         const int L = max(a.steps[b].prefix_len, 0);
@@ -112,16 +160,6 @@ __device__ __forceinline__ void build_sched(const AttnArgs& a, Sched& sc, int ti
                       ? (static_cast<int>(units) + a.sched_grid - 1) / a.sched_grid
                       : static_cast<int>((units + a.sched_grid - 1) / a.sched_grid);
         tps = max(tps, max(a.min_tiles, 1));
-        // ceil(kt / tps) splits per group can add up to more items than CTAs (a second, nearly
-        // empty round); a slightly larger tile count per split then gives a single round.
-        if (a.batch <= 32) {
-            for (int tries = 0; tries < 8; ++tries) {
-                int cnt = 0;  // batch <= 32 here: no overflow
-                for (int b = 0; b < a.batch; ++b) cnt += a.Hkv * sc.mp[b] * ((sc.kt[b] + tps - 1) / tps);
-                if (cnt <= a.sched_grid) break;
-                ++tps;
-            }
-        }
         int items = 0;
         for (int b = 0; b < a.batch; ++b) {
             sc.item0[b] = items;
@@ -225,17 +263,9 @@ __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-// TMA: one box of a 4-D tensor (element, slot, head, sequence) into shared memory.
-__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0,
-                                            int c1, int c2, int c3) {
-    asm volatile(
-        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes"
-        " [%0], [%1, {%2, %3, %4, %5}], [%6];" ::"r"(dst),
-        "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar)
-        : "memory");
-}
-
-// TMA: one box of the 5-D query view (element, head in group, KV head, token, sequence).
+// TMA: one box of a 5-D view into shared memory.  The last dimension of every view is the
+// 64-element column panel, so that one copy brings all panels of a tile, each in its own
+// 128-byte-swizzled block (the innermost coordinate is always 0).
 __device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0,
                                             int c1, int c2, int c3, int c4) {
     asm volatile(
@@ -361,7 +391,7 @@ struct Smem {
     static constexpr int kOffK = kOffQ + kRowTiles * kQTile;
     static constexpr int kOffV = kOffK + kStages * kKVTile;
     static constexpr int kOffBar = kOffV + kStages * kKVTile;
-    static constexpr int kNumBars = 3 * kStages + 1 + kRowTiles * 5 + 2;
+    static constexpr int kNumBars = 4 * kStages + 1 + kRowTiles * 5 + 2;
     static constexpr int kOffMisc = kOffBar + 8 * 32;
     static constexpr int kUsed = kOffMisc + 64 + 1024;       // + slack to align the base to 1024
     // Never less than 120 KB, more than half of an SM's shared memory: one CTA per SM, so the
@@ -374,18 +404,22 @@ struct Smem {
 // barrier indices
 __device__ __forceinline__ constexpr int bar_kfull(int s) { return s; }
 __device__ __forceinline__ constexpr int bar_vfull(int s) { return kStages + s; }
-__device__ __forceinline__ constexpr int bar_kvempty(int s) { return 2 * kStages + s; }
-__device__ __forceinline__ constexpr int bar_qfull() { return 3 * kStages; }
+// K and V stages are released separately: a K tile is dead once its Q K^T has completed, long
+// before the P V of the same tile, and the next K can be on its way meanwhile.
+__device__ __forceinline__ constexpr int bar_kempty(int s) { return 2 * kStages + s; }
+__device__ __forceinline__ constexpr int bar_vempty(int s) { return 3 * kStages + s; }
+constexpr int kBar0 = 4 * kStages;  // first barrier after the ring's
+__device__ __forceinline__ constexpr int bar_qfull() { return kBar0; }
 // Lane m's S and P share a TMEM buffer (its j-th tile uses buffer j & 1) and each buffer has its own pair of
 // barriers: a buffer's next phase cannot complete before the other side has observed the
 // current one (QK(j+2) is issued after PV(j), which is issued after pfull(j) was seen), so a
 // parity wait never falls two phases behind.  One pfull barrier for both buffers would: the
 // softmax warps can finish tile j+1 while the MMA thread still waits for V(j).
-__device__ __forceinline__ constexpr int bar_sfull(int m, int buf) { return 3 * kStages + 1 + m * 5 + buf; }
-__device__ __forceinline__ constexpr int bar_pfull(int m, int buf) { return 3 * kStages + 1 + m * 5 + 2 + buf; }
-__device__ __forceinline__ constexpr int bar_pvdone(int m) { return 3 * kStages + 1 + m * 5 + 4; }
-__device__ __forceinline__ constexpr int bar_item() { return 3 * kStages + 1 + kRowTiles * 5; }
-__device__ __forceinline__ constexpr int bar_qempty() { return 3 * kStages + 2 + kRowTiles * 5; }
+__device__ __forceinline__ constexpr int bar_sfull(int m, int buf) { return kBar0 + 1 + m * 5 + buf; }
+__device__ __forceinline__ constexpr int bar_pfull(int m, int buf) { return kBar0 + 1 + m * 5 + 2 + buf; }
+__device__ __forceinline__ constexpr int bar_pvdone(int m) { return kBar0 + 1 + m * 5 + 4; }
+__device__ __forceinline__ constexpr int bar_item() { return kBar0 + 1 + kRowTiles * 5; }
+__device__ __forceinline__ constexpr int bar_qempty() { return kBar0 + 2 + kRowTiles * 5; }
 
 template <int D>
 __global__ void __launch_bounds__(kAttnThreads, 1)
@@ -410,7 +444,8 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
         for (int s = 0; s < kStages; ++s) {
             mbar_init(bar(bar_kfull(s)), 1);
             mbar_init(bar(bar_vfull(s)), 1);
-            mbar_init(bar(bar_kvempty(s)), 2);  // one arrival per lane
+            mbar_init(bar(bar_kempty(s)), 2);  // one arrival per lane (two from the owner in key mode)
+            mbar_init(bar(bar_vempty(s)), 2);
         }
         mbar_init(bar(bar_qfull()), a.q_by_tma ? 1 : kSoftmaxThreads);
         mbar_init(bar(bar_qempty()), 2);
@@ -442,6 +477,27 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
     pdl_launch_dependents();
     build_sched(a, sc, tid, kAttnThreads);  // ends with __syncthreads()
     const int total_items = min(sc.item0[a.batch], a.max_items);
+    // The producers issue the first copies of the CTA's first item at once, each from its own
+    // decode of that item: the rest of the set-up (item list, tensor memory address, register
+    // hand-over) runs while the data is on its way.
+    const bool early = (warp == kProducerWarp || warp == kVProducerWarp) && lane == 0 &&
+                       static_cast<int>(blockIdx.x) < total_items;
+    if (early) {
+        const Item it = decode_item(sc, blockIdx.x, G);
+        if (warp == kProducerWarp) {
+            mbar_expect_tx(bar(bar_kfull(0)), S::kKVTile);
+            tma_load_5d(base + S::kOffK, &map_k, bar(bar_kfull(0)), 0, it.t_begin * kBN, it.g, it.b, 0);
+            if (a.q_by_tma) {
+                mbar_expect_tx(bar(bar_qfull()), it.nmt * S::kQTile);
+                for (int m = 0; m < it.nmt; ++m)
+                    tma_load_5d(base + S::kOffQ + m * S::kQTile, &map_q, bar(bar_qfull()), 0, 0, it.g,
+                                it.b * a.max_tt + it.tok0 + m * (kBM / G), 0);
+            }
+        } else {
+            mbar_expect_tx(bar(bar_vfull(0)), S::kKVTile);
+            tma_load_5d(base + S::kOffV, &map_v, bar(bar_vfull(0)), 0, it.t_begin * kBN, it.g, it.b, 0);
+        }
+    }
     // The integer divisions of the item decode are a long dependent chain for a single thread:
     // the first items of this CTA are decoded here, one per thread, for every role to read.
     if (tid < kPreItems && blockIdx.x + tid * gridDim.x < total_items)
@@ -456,62 +512,81 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
 
     // Running use counts of the barrier families.  Every role walks the same items and tiles in
     // the same order, so each keeps its own copy.
+    // Registers follow the roles: the softmax warpgroups hold a tile of S, a tile of P and a row of
+    // O; the warpgroup of the producers and MMA issuers needs few (384 x 168 at launch).
     uint32_t kt_run = 0;     // K/V ring uses (all tiles of all items)
     uint32_t jx = 0;         // tiles this lane has taken (S/P buffers, PV completions)
     uint32_t items_run = 0;
     bool alive = true;
 
+    if (warp >= kProducerWarp) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsIssue));
     if (warp == kProducerWarp) {
-        // ================================ TMA producer ====================================
+        // ================================ TMA producer: K tiles and Q =======================
         if (lane == 0) {
             int li = 0;
             for (int item = blockIdx.x; item < total_items && alive; item += gridDim.x, ++li) {
                 const Item it = get_item(item, li);
                 for (int t = it.t_begin; t < it.t_end; ++t, ++kt_run) {
                     const int s = kt_run % kStages;
-                    if (!mbar_wait(bar(bar_kvempty(s)), ((kt_run / kStages) & 1u) ^ 1u, abort_flag, a.status)) {
-                        alive = false;
-                        break;
-                    }
-                    const uint32_t dk = base + S::kOffK + s * S::kKVTile;
-                    const uint32_t dv = base + S::kOffV + s * S::kKVTile;
-                    mbar_expect_tx(bar(bar_kfull(s)), S::kKVTile);
-#pragma unroll
-                    for (int p = 0; p < S::kPanels; ++p)
-                        tma_load_4d(dk + p * S::kKVPanel, &map_k, bar(bar_kfull(s)), p * 64, t * kBN, it.g, it.b);
-                    if (t == it.t_begin && a.q_by_tma) {
-                        // Q goes between the first K and the first V tile: K and Q are what the first
-                        // MMA needs.  The Q tiles of the previous item are free once its last QK^T has
-                        // completed.
-                        if (!mbar_wait(bar(bar_qempty()), (items_run & 1u) ^ 1u, abort_flag, a.status)) {
+                    if (kt_run > 0) {  // the CTA's very first tile went out during the set-up
+                        // the first use of a stage finds it free
+                        if (kt_run >= kStages &&
+                            !mbar_wait(bar(bar_kempty(s)), ((kt_run / kStages) & 1u) ^ 1u, abort_flag, a.status)) {
                             alive = false;
                             break;
                         }
-                        mbar_expect_tx(bar(bar_qfull()), it.nmt * S::kQTile);
-                        for (int m = 0; m < it.nmt; ++m)
-#pragma unroll
-                            for (int p = 0; p < S::kPanels; ++p)
-                                tma_load_5d(base + S::kOffQ + m * S::kQTile + p * S::kQPanel, &map_q,
-                                            bar(bar_qfull()), p * 64, 0, it.g, it.tok0 + m * (kBM / G), it.b);
+                        mbar_expect_tx(bar(bar_kfull(s)), S::kKVTile);
+                        tma_load_5d(base + S::kOffK + s * S::kKVTile, &map_k, bar(bar_kfull(s)), 0, t * kBN, it.g,
+                                    it.b, 0);
+                    }
+                    if (t == it.t_begin && a.q_by_tma) {
+                        // Q follows the first K tile: K and Q are what the first MMA needs.  The Q
+                        // tiles of the previous item are free once its last QK^T has completed.
+                        if (items_run > 0) {
+                            if (!mbar_wait(bar(bar_qempty()), (items_run & 1u) ^ 1u, abort_flag, a.status)) {
+                                alive = false;
+                                break;
+                            }
+                            mbar_expect_tx(bar(bar_qfull()), it.nmt * S::kQTile);
+                            for (int m = 0; m < it.nmt; ++m)
+                                tma_load_5d(base + S::kOffQ + m * S::kQTile, &map_q, bar(bar_qfull()), 0, 0, it.g,
+                                            it.b * a.max_tt + it.tok0 + m * (kBM / G), 0);
+                        }
                         ++items_run;
                     }
-                    mbar_expect_tx(bar(bar_vfull(s)), S::kKVTile);
-#pragma unroll
-                    for (int p = 0; p < S::kPanels; ++p)
-                        tma_load_4d(dv + p * S::kKVPanel, &map_v, bar(bar_vfull(s)), p * 64, t * kBN, it.g, it.b);
                 }
             }
             // Drain: every copy this thread issued has landed before the CTA may exit.
             if (a.q_by_tma && items_run > 0) mbar_wait(bar(bar_qfull()), (items_run - 1u) & 1u, abort_flag, a.status);
             const uint32_t issued = kt_run;
-            for (uint32_t u = (issued > kStages ? issued - kStages : 0u); u < issued; ++u) {
-                const int s = u % kStages;
-                const uint32_t ph = (u / kStages) & 1u;
-                if (!mbar_wait(bar(bar_kfull(s)), ph, abort_flag, a.status)) break;
-                if (!mbar_wait(bar(bar_vfull(s)), ph, abort_flag, a.status)) break;
-            }
+            for (uint32_t u = (issued > kStages ? issued - kStages : 0u); u < issued; ++u)
+                if (!mbar_wait(bar(bar_kfull(u % kStages)), (u / kStages) & 1u, abort_flag, a.status)) break;
         }
-    } else if (warp >= kMmaWarp0) {
+    } else if (warp == kVProducerWarp) {
+        // ================================ TMA producer: V tiles =============================
+        if (lane == 0) {
+            int li = 0;
+            for (int item = blockIdx.x; item < total_items && alive; item += gridDim.x, ++li) {
+                const Item it = get_item(item, li);
+                for (int t = it.t_begin; t < it.t_end; ++t, ++kt_run) {
+                    const int s = kt_run % kStages;
+                    if (kt_run == 0) continue;  // went out during the set-up
+                    if (kt_run >= kStages &&
+                        !mbar_wait(bar(bar_vempty(s)), ((kt_run / kStages) & 1u) ^ 1u, abort_flag, a.status)) {
+                        alive = false;
+                        break;
+                    }
+                    mbar_expect_tx(bar(bar_vfull(s)), S::kKVTile);
+                    tma_load_5d(base + S::kOffV + s * S::kKVTile, &map_v, bar(bar_vfull(s)), 0, t * kBN, it.g, it.b,
+                                0);
+                }
+            }
+            const uint32_t issued = kt_run;
+            for (uint32_t u = (issued > kStages ? issued - kStages : 0u); u < issued; ++u)
+                if (!mbar_wait(bar(bar_vfull(u % kStages)), (u / kStages) & 1u, abort_flag, a.status)) break;
+        }
+    } else if (warp == kMmaWarp0 || warp == kMmaWarp0 + 1) {
         // ================================ MMA issuer of lane x ============================
         // The whole warp walks the loop and waits (so that every value stays warp-uniform);
         // one elected lane issues.  The MMAs of one thread execute in issue order: QK of this
@@ -526,6 +601,7 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
         const uint64_t kdesc0 = smem_desc(base + S::kOffK, 16, 1024);
         const uint64_t vdesc0 = smem_desc(base + S::kOffV, S::kKVPanel, 1024);
         const uint32_t o_t = tmem + x * 256 + 128;
+        uint32_t k_seen = 0xFFFFFFFFu;  // ring use whose K tile this warp has already seen arrive
         for (int item = blockIdx.x; item < total_items && alive; item += gridDim.x, ++items_run) {
             const Item it = get_item(item, static_cast<int>(items_run));
             const bool row_mode = it.nmt == 2;
@@ -534,9 +610,17 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
             tc_fence_after();
             bool have_prev = false, first_pv = true;
             uint32_t prev_kt = 0, prev_j = 0;
-            auto issue_pv = [&]() {
+            // In key mode a tile belongs to one lane alone: its owner releases the stage for both.
+            const int releases = row_mode ? 1 : 2;
+            // P V of this lane's previous tile.  While it waits for P it looks (without blocking) at
+            // the K tile of the lane's next Q K^T, whose wait would otherwise sit between P V and the
+            // next Q K^T: the chain that decides when the softmax warps get their next S.
+            auto issue_pv = [&](uint32_t next_use) {
                 const int s = prev_kt % kStages;
                 if (!warp_wait(bar(bar_vfull(s)), (prev_kt / kStages) & 1u, abort_flag, a.status)) return false;
+                if (next_use != 0xFFFFFFFFu &&
+                    __all_sync(kFull, mbar_try(bar(bar_kfull(next_use % kStages)), (next_use / kStages) & 1u)))
+                    k_seen = next_use;
                 if (!warp_wait(bar(bar_pfull(x, prev_j & 1u)), (prev_j >> 1) & 1u, abort_flag, a.status)) return false;
                 tc_fence_after();
                 if (elect_one()) {
@@ -550,19 +634,20 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
                         umma_ts(o_t, a_t + 16, vdesc + kk * (2048 >> 4), kIdescPV, 1u);
                     }
                     umma_commit(bar(bar_pvdone(x)));
-                    umma_commit(bar(bar_kvempty(s)));
+                    for (int rls = 0; rls < releases; ++rls) umma_commit(bar(bar_vempty(s)));
                 }
                 __syncwarp();
                 first_pv = false;
                 return true;
             };
+            const int t_step = row_mode ? 1 : 2;  // distance to this lane's next tile
             for (int t = it.t_begin; t < it.t_end && alive; ++t, ++kt_run) {
                 const int s = kt_run % kStages;
-                // every tile is waited for, own or not: it paces this lane's arrivals on kvempty
-                alive = warp_wait(bar(bar_kfull(s)), (kt_run / kStages) & 1u, abort_flag, a.status);
-                if (!alive) break;
                 const bool own = row_mode || (((t - it.t_begin) & 1) == x);
                 if (own) {
+                    if (k_seen != kt_run)
+                        alive = warp_wait(bar(bar_kfull(s)), (kt_run / kStages) & 1u, abort_flag, a.status);
+                    if (!alive) break;
                     tc_fence_after();
                     if (elect_one()) {
                         const uint64_t kdesc = kdesc0 + static_cast<uint64_t>(s * (S::kKVTile >> 4));
@@ -572,27 +657,29 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
                             umma(s_t, qdesc + ((ks >> 2) * (S::kQPanel >> 4) + (ks & 3) * 2),
                                  kdesc + ((ks >> 2) * (S::kKVPanel >> 4) + (ks & 3) * 2), kIdescQK, ks > 0 ? 1u : 0u);
                         umma_commit(bar(bar_sfull(x, jx & 1u)));
+                        for (int rls = 0; rls < releases; ++rls) umma_commit(bar(bar_kempty(s)));
                     }
                     __syncwarp();
-                    if (have_prev) alive = issue_pv();
+                    if (have_prev)
+                        alive = issue_pv(t + t_step < it.t_end ? kt_run + static_cast<uint32_t>(t_step) : 0xFFFFFFFFu);
                     have_prev = true, prev_kt = kt_run, prev_j = jx;
                     ++jx;
-                } else if (elect_one()) {
-                    mbar_arrive(bar(bar_kvempty(s)));  // the other lane's tile: nothing of this lane reads it
                 }
                 // Q is free for the next item once the last QK^T of both lanes has completed
                 if (t + 1 == it.t_end && elect_one()) umma_commit(bar(bar_qempty()));
                 __syncwarp();
             }
-            if (alive && have_prev) alive = issue_pv();
+            if (alive && have_prev) alive = issue_pv(0xFFFFFFFFu);
             tc_fence_before();
             if (!alive) break;
             // end of item: the softmax warps have read O and S, Q and P may be overwritten
             mbar_arrive(bar(bar_item()));
             alive = warp_wait(bar(bar_item()), items_run & 1u, abort_flag, a.status);
         }
+    }
     } else {
         // ================================ softmax warpgroup of lane x =====================
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
         const int x = warp >> 2;
         const int r = (warp & 3) * 32 + lane;          // row inside the tile = TMEM lane
         const uint32_t lane_sel = static_cast<uint32_t>((warp & 3) * 32) << 16;
@@ -658,18 +745,27 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
             // over (PV(j) cannot be issued earlier): by then it has usually completed.
             uint32_t pv_seen = jx;
             bool first = true;
+            // A wait on a barrier costs a few hundred cycles even when its phase completed long ago,
+            // and this loop is the longest dependent chain of the kernel.  So the two things a tile
+            // has to wait for are looked at early, without blocking, and the answers are used later:
+            // PV(j-1) before the exponentials, S(j+1) between their halves.  When S(j+1) is there its
+            // load is issued before P(j) is handed over, and the next round starts with the data.
+            uint32_t sr[2][32];
+            bool s_loaded = false;
+            const int t_step = row_mode ? 1 : 2;  // distance to this lane's next tile
 
             for (int t = it.t_begin; t < it.t_end; ++t, ++kt_run) {
                 if (!(row_mode || (((t - it.t_begin) & 1) == x))) continue;
                 const uint32_t buf = jx & 1u;
-                if (!warp_wait(bar(bar_sfull(x, buf)), (jx >> 1) & 1u, abort_flag, a.status)) {
-                    alive = false;
-                    break;
+                if (!s_loaded) {
+                    if (!warp_wait(bar(bar_sfull(x, buf)), (jx >> 1) & 1u, abort_flag, a.status)) {
+                        alive = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    tmem_ld32(tmem + lane_sel + x * 256 + buf * kBN, sr[0]);
+                    tmem_ld32(tmem + lane_sel + x * 256 + buf * kBN + 32, sr[1]);
                 }
-                tc_fence_after();
-                uint32_t sr[2][32];
-                tmem_ld32(tmem + lane_sel + x * 256 + buf * kBN, sr[0]);
-                tmem_ld32(tmem + lane_sel + x * 256 + buf * kBN + 32, sr[1]);
                 tmem_wait_ld();
 
                 // ---- ancestor mask (tiles that reach past the prefix only), row maximum -------
@@ -733,6 +829,10 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
                     tmem_wait_st();
                 }
                 const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
+                // PV(j-1): asked now, answered after the exponentials (pv_seen is jx or jx - 1 here)
+                const bool pv_probe = (pv_seen == jx) || mbar_try(bar(bar_pvdone(x)), pv_seen & 1u);
+                const bool has_next = t + t_step < it.t_end;
+                bool s_probe = false;
 
                 // ---- stale V rows of the sequence's last tile must not reach the MMA (in row mode
                 // both lanes clear them: each lane's PV is ordered behind its own warpgroup only) ----
@@ -764,6 +864,8 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
                     const uint32_t p_t = tmem + lane_sel + x * 256 + buf * kBN;
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
+                        if (h == 1 && has_next)
+                            s_probe = mbar_try(bar(bar_sfull(x, buf ^ 1u)), ((jx + 1u) >> 1) & 1u);
                         uint32_t w[32];
 #pragma unroll
                         for (int c = 0; c < 16; ++c) {
@@ -785,11 +887,25 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
                     float ps0, ps1;
                     unpack2(psum2, ps0, ps1);
                     l_run += ps0 + ps1;
-                    tmem_wait_st();
                 }
+                // S of this lane's next tile, if it has arrived (sr is free now)
+                s_loaded = false;
+                if (has_next) {
+                    if (!__all_sync(kFull, s_probe))
+                        s_probe = mbar_try(bar(bar_sfull(x, buf ^ 1u)), ((jx + 1u) >> 1) & 1u);
+                    if (__all_sync(kFull, s_probe)) {
+                        tc_fence_after();
+                        tmem_ld32(tmem + lane_sel + x * 256 + (buf ^ 1u) * kBN, sr[0]);
+                        tmem_ld32(tmem + lane_sel + x * 256 + (buf ^ 1u) * kBN + 32, sr[1]);
+                        s_loaded = true;
+                    }
+                }
+                tmem_wait_st();
                 if (clear_v) fence_proxy_async();
-                while (pv_seen < jx) {
-                    if (!warp_wait(bar(bar_pvdone(x)), pv_seen & 1u, abort_flag, a.status)) alive = false;
+                if (pv_seen < jx) {
+                    if (!__all_sync(kFull, pv_probe) &&
+                        !warp_wait(bar(bar_pvdone(x)), pv_seen & 1u, abort_flag, a.status))
+                        alive = false;
                     ++pv_seen;
                 }
                 if (!alive) break;
@@ -998,7 +1114,7 @@ EncodeTiledFn encode_tiled_fn() {
     return fn;
 }
 
-// (element, slot, head, sequence) view of a bf16 cache; boxes of 64 elements x 64 slots.
+// (element, slot, head, sequence, panel) view of a bf16 cache; a box is 64 slots of all panels.
 bool make_kv_map(CUtensorMap* map, const void* basep, int D, int64_t capacity, int Hkv, int batch,
                  int64_t s_tok, int64_t s_head, int64_t s_seq) {
     EncodeTiledFn fn = encode_tiled_fn();
@@ -1006,28 +1122,31 @@ bool make_kv_map(CUtensorMap* map, const void* basep, int D, int64_t capacity, i
     // a dimension of extent 1 never uses its stride; give it a valid one
     if (s_head <= 0) s_head = capacity * s_tok;
     if (s_seq <= 0) s_seq = s_head * Hkv;
-    const cuuint64_t dims[4] = {static_cast<cuuint64_t>(D), static_cast<cuuint64_t>(capacity),
-                                static_cast<cuuint64_t>(Hkv), static_cast<cuuint64_t>(batch)};
-    const cuuint64_t strides[3] = {static_cast<cuuint64_t>(s_tok) * 2, static_cast<cuuint64_t>(s_head) * 2,
-                                   static_cast<cuuint64_t>(s_seq) * 2};
-    const cuuint32_t box[4] = {64, static_cast<cuuint32_t>(kBN), 1, 1};
-    const cuuint32_t estr[4] = {1, 1, 1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(basep), dims, strides, box, estr,
+    const cuuint32_t panels = static_cast<cuuint32_t>(D / 64);
+    const cuuint64_t dims[5] = {64, static_cast<cuuint64_t>(capacity), static_cast<cuuint64_t>(Hkv),
+                                static_cast<cuuint64_t>(batch), panels};
+    const cuuint64_t strides[4] = {static_cast<cuuint64_t>(s_tok) * 2, static_cast<cuuint64_t>(s_head) * 2,
+                                   static_cast<cuuint64_t>(s_seq) * 2, 128};
+    const cuuint32_t box[5] = {64, static_cast<cuuint32_t>(kBN), 1, 1, panels};
+    const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(basep), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// (element, head in group, KV head, token, sequence) view of Q [batch][max_tt][Hq][D]: a box of
-// 64 elements x G heads x 128/G tokens is one 128-row tile in (token, head) row order.
+// (element, head in group, KV head, token of any sequence, panel) view of Q [batch][max_tt][Hq][D]:
+// a box of 64 elements x G heads x 128/G tokens x all panels is one 128-row tile in (token, head)
+// row order.  The sequences are folded into the token dimension (they are contiguous), so rows
+// past a sequence's max_tt read the next sequence's; such rows are never valid.
 bool make_q_map(CUtensorMap* map, const void* basep, int D, int G, int Hkv, int max_tt, int batch) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
     const cuuint64_t Hq = static_cast<cuuint64_t>(G) * Hkv;
-    const cuuint64_t dims[5] = {static_cast<cuuint64_t>(D), static_cast<cuuint64_t>(G), static_cast<cuuint64_t>(Hkv),
-                                static_cast<cuuint64_t>(max_tt), static_cast<cuuint64_t>(batch)};
-    const cuuint64_t strides[4] = {static_cast<cuuint64_t>(D) * 2, static_cast<cuuint64_t>(G) * D * 2, Hq * D * 2,
-                                   static_cast<cuuint64_t>(max_tt) * Hq * D * 2};
-    const cuuint32_t box[5] = {64, static_cast<cuuint32_t>(G), 1, static_cast<cuuint32_t>(kBM / G), 1};
+    const cuuint32_t panels = static_cast<cuuint32_t>(D / 64);
+    const cuuint64_t dims[5] = {64, static_cast<cuuint64_t>(G), static_cast<cuuint64_t>(Hkv),
+                                static_cast<cuuint64_t>(max_tt) * batch, panels};
+    const cuuint64_t strides[4] = {static_cast<cuuint64_t>(D) * 2, static_cast<cuuint64_t>(G) * D * 2, Hq * D * 2, 128};
+    const cuuint32_t box[5] = {64, static_cast<cuuint32_t>(G), 1, static_cast<cuuint32_t>(kBM / G), panels};
     const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(basep), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
