@@ -176,7 +176,6 @@ struct Item {
     int n, L, M, row_base, nmt, t_begin, t_end;
     int tok0;  // first token of the pair's rows
 };
-constexpr int kPreItems = 8;  // items of a CTA decoded once, in parallel, for all roles
 
 __device__ __forceinline__ Item decode_item(const Sched& sc, int item, int G) {
     Item it;
@@ -185,10 +184,11 @@ __device__ __forceinline__ Item decode_item(const Sched& sc, int item, int G) {
     it.b = b;
     it.n = sc.n[b], it.L = sc.L[b], it.splits = sc.splits[b];
     const int local = item - sc.item0[b];
-    it.sp = local % it.splits;
     const int grp = local / it.splits;  // = g * mp + pair
-    it.pair = grp % sc.mp[b];
-    it.g = grp / sc.mp[b];
+    it.sp = local - grp * it.splits;
+    const int mp = sc.mp[b];
+    it.g = (mp == 1) ? grp : grp / mp;
+    it.pair = grp - it.g * mp;
     it.first_item = item - it.sp;
     it.M = it.n * G;
     it.row_base = it.pair * kRowTiles * kBM;
@@ -197,7 +197,7 @@ __device__ __forceinline__ Item decode_item(const Sched& sc, int item, int G) {
     const unsigned kt = static_cast<unsigned>(sc.kt[b]), sp = static_cast<unsigned>(it.sp);
     it.t_begin = static_cast<int>(kt * sp / static_cast<unsigned>(it.splits));
     it.t_end = static_cast<int>(kt * (sp + 1u) / static_cast<unsigned>(it.splits));
-    it.tok0 = it.row_base / G;
+    it.tok0 = (it.row_base == 0) ? 0 : it.row_base / G;
     return it;
 }
 
@@ -378,6 +378,10 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
 }
+__device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
+    __half2 v = __floats2half2_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
 
 // ---------------------------------------------------------------------------- shared memory map
 template <int D>
@@ -428,7 +432,6 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
     using S = Smem<D>;
     extern __shared__ unsigned char smem_raw[];
     __shared__ Sched sc;
-    __shared__ Item s_items[kPreItems];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     unsigned char* base_ptr = smem_raw + (base - smem_u32(smem_raw));
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -475,15 +478,20 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
     // overlaps the tail of the preceding kernel.
     pdl_wait();
     pdl_launch_dependents();
-    build_sched(a, sc, tid, kAttnThreads);  // ends with __syncthreads()
+    tc_fence_before();
+    build_sched(a, sc, tid, kAttnThreads);  // ends with __syncthreads(): barriers, TMEM address and schedule are visible
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
     const int total_items = min(sc.item0[a.batch], a.max_items);
-    // The producers issue the first copies of the CTA's first item at once, each from its own
-    // decode of that item: the rest of the set-up (item list, tensor memory address, register
-    // hand-over) runs while the data is on its way.
+    // Every thread decodes the CTA's first item for itself (a CTA rarely has a second one): no
+    // role waits for another before it starts.
+    Item first_it = {};
+    if (static_cast<int>(blockIdx.x) < total_items) first_it = decode_item(sc, blockIdx.x, G);
+    // The producers issue the first copies of the CTA's first item at once.
     const bool early = (warp == kProducerWarp || warp == kVProducerWarp) && lane == 0 &&
                        static_cast<int>(blockIdx.x) < total_items;
     if (early) {
-        const Item it = decode_item(sc, blockIdx.x, G);
+        const Item& it = first_it;
         if (warp == kProducerWarp) {
             mbar_expect_tx(bar(bar_kfull(0)), S::kKVTile);
             tma_load_5d(base + S::kOffK, &map_k, bar(bar_kfull(0)), 0, it.t_begin * kBN, it.g, it.b, 0);
@@ -498,27 +506,19 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
             tma_load_5d(base + S::kOffV, &map_v, bar(bar_vfull(0)), 0, it.t_begin * kBN, it.g, it.b, 0);
         }
     }
-    // The integer divisions of the item decode are a long dependent chain for a single thread:
-    // the first items of this CTA are decoded here, one per thread, for every role to read.
-    if (tid < kPreItems && blockIdx.x + tid * gridDim.x < total_items)
-        s_items[tid] = decode_item(sc, blockIdx.x + tid * gridDim.x, G);
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem = *tmem_slot;
     auto get_item = [&](int item, int local) {  // local = how many items this CTA has started before
-        return local < kPreItems ? s_items[local] : decode_item(sc, item, G);
+        return local == 0 ? first_it : decode_item(sc, item, G);
     };
 
     // Running use counts of the barrier families.  Every role walks the same items and tiles in
     // the same order, so each keeps its own copy.
-    // Registers follow the roles: the softmax warpgroups hold a tile of S, a tile of P and a row of
-    // O; the warpgroup of the producers and MMA issuers needs few (384 x 168 at launch).
     uint32_t kt_run = 0;     // K/V ring uses (all tiles of all items)
     uint32_t jx = 0;         // tiles this lane has taken (S/P buffers, PV completions)
     uint32_t items_run = 0;
     bool alive = true;
 
+    // Registers follow the roles: the softmax warpgroups hold a tile of S, a tile of P and a row of
+    // O; the warpgroup of the producers and MMA issuers needs few (384 x 168 at launch).
     if (warp >= kProducerWarp) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsIssue));
     if (warp == kProducerWarp) {
@@ -919,66 +919,87 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
             // ---- epilogue --------------------------------------------------------------
             const bool direct = row_mode && it.splits == 1;
             if (!first) {
+                const int t = R / G, h = it.g * G + R % G;
+                const float inv = 1.f / l_run;
+                __nv_bfloat16* dst = a.o + ((static_cast<int64_t>(it.b) * a.max_tt + t) * a.Hq + h) * D;
+                uint4* po = a.part_o + (static_cast<int64_t>(item) * kRowTiles + x) * (D / 8) * kBM + r;
                 while (pv_seen < jx) {
                     if (!warp_wait(bar(bar_pvdone(x)), pv_seen & 1u, abort_flag, a.status)) alive = false;
                     ++pv_seen;
                 }
                 if (!alive) break;
                 tc_fence_after();
-                const int t = R / G, h = it.g * G + R % G;
-                const float inv = 1.f / l_run;
-                __nv_bfloat16* dst = a.o + ((static_cast<int64_t>(it.b) * a.max_tt + t) * a.Hq + h) * D;
-                uint4* po = a.part_o + (static_cast<int64_t>(item) * kRowTiles + x) * (D / 8) * kBM + r;
                 if (row_ok && direct && a.lse)
                     a.lse[(static_cast<int64_t>(it.b) * a.max_tt + t) * a.Hq + h] =
                         (m_ref + log2f(l_run)) * 0.6931471805599453f;
                 {
-                    uint32_t orr[D / 32][32];  // the whole row: all loads in flight, then all stores
+                    // One pass over the row in 32-column pieces: the next piece is on its way from
+                    // tensor memory while this one is converted and stored.  Partials assume a row
+                    // scale of 1 and keep the row's largest magnitude; the rare row that would leave
+                    // the fp16 range is written again with its scale.
+                    const float mul1 = direct ? inv : ((l_run > 0.f) ? inv : 0.f);
+                    float am[4] = {0.f, 0.f, 0.f, 0.f};
+                    uint32_t orr[2][32];
+                    tmem_ld32(o_t, orr[0]);
 #pragma unroll
-                    for (int c = 0; c < D / 32; ++c) tmem_ld32(o_t + c * 32, orr[c]);
-                    tmem_wait_ld();
-                    if (row_ok) {
-                        if (direct) {
+                    for (int c = 0; c < D / 32; ++c) {
+                        tmem_wait_ld();
+                        if (c + 1 < D / 32) tmem_ld32(o_t + (c + 1) * 32, orr[(c + 1) & 1]);
+                        const uint32_t* w = orr[c & 1];
+                        if (row_ok) {
 #pragma unroll
-                            for (int q8 = 0; q8 < D / 8; ++q8) {
-                                const uint32_t* w = &orr[q8 >> 2][(q8 & 3) * 8];
+                            for (int q4 = 0; q4 < 4; ++q4) {
+                                float f[8];
+#pragma unroll
+                                for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(w[q4 * 8 + e]);
                                 uint4 v;
-                                v.x = pack_bf16(__uint_as_float(w[0]) * inv, __uint_as_float(w[1]) * inv);
-                                v.y = pack_bf16(__uint_as_float(w[2]) * inv, __uint_as_float(w[3]) * inv);
-                                v.z = pack_bf16(__uint_as_float(w[4]) * inv, __uint_as_float(w[5]) * inv);
-                                v.w = pack_bf16(__uint_as_float(w[6]) * inv, __uint_as_float(w[7]) * inv);
-                                *reinterpret_cast<uint4*>(dst + q8 * 8) = v;
-                            }
-                        } else {
-                            // row scale: 1 unless |O / l| would exceed 2^14 (fp16 holds up to 65504)
-                            float amax = 0.f;
-#pragma unroll
-                            for (int c = 0; c < D; c += 2)
-                                amax = max3(amax, fabsf(__uint_as_float(orr[c >> 5][c & 31])),
-                                            fabsf(__uint_as_float(orr[c >> 5][(c & 31) + 1])));
-                            float scale = 1.f;  // O = Ohat * l * scale
-                            const float nmax = amax * inv;
-                            if (nmax > 16384.f) scale = exp2f(ceilf(log2f(nmax)) - 14.f);
-                            const float mul = (l_run > 0.f) ? inv / scale : 0.f;
-                            __stcg(a.part_ml + (static_cast<int64_t>(item) * kRowTiles + x) * kBM + r,
-                                   make_float4(l_run > 0.f ? m_ref : -INFINITY, l_run, l_run * scale, 0.f));
-#pragma unroll
-                            for (int q8 = 0; q8 < D / 8; ++q8) {
-                                const uint32_t* w = &orr[q8 >> 2][(q8 & 3) * 8];
-                                uint4 v;
-                                __half2 h2;
-                                h2 = __floats2half2_rn(__uint_as_float(w[0]) * mul, __uint_as_float(w[1]) * mul);
-                                v.x = *reinterpret_cast<uint32_t*>(&h2);
-                                h2 = __floats2half2_rn(__uint_as_float(w[2]) * mul, __uint_as_float(w[3]) * mul);
-                                v.y = *reinterpret_cast<uint32_t*>(&h2);
-                                h2 = __floats2half2_rn(__uint_as_float(w[4]) * mul, __uint_as_float(w[5]) * mul);
-                                v.z = *reinterpret_cast<uint32_t*>(&h2);
-                                h2 = __floats2half2_rn(__uint_as_float(w[6]) * mul, __uint_as_float(w[7]) * mul);
-                                v.w = *reinterpret_cast<uint32_t*>(&h2);
-                                __stcg(po + q8 * kBM, v);
+                                if (direct) {
+                                    v.x = pack_bf16(f[0] * mul1, f[1] * mul1), v.y = pack_bf16(f[2] * mul1, f[3] * mul1);
+                                    v.z = pack_bf16(f[4] * mul1, f[5] * mul1), v.w = pack_bf16(f[6] * mul1, f[7] * mul1);
+                                    *reinterpret_cast<uint4*>(dst + (c * 4 + q4) * 8) = v;
+                                } else {
+                                    am[q4] = max3(am[q4], fabsf(f[0]), fabsf(f[1]));
+                                    am[q4] = max3(am[q4], fabsf(f[2]), fabsf(f[3]));
+                                    am[q4] = max3(am[q4], fabsf(f[4]), fabsf(f[5]));
+                                    am[q4] = max3(am[q4], fabsf(f[6]), fabsf(f[7]));
+                                    v.x = pack_half2(f[0] * mul1, f[1] * mul1), v.y = pack_half2(f[2] * mul1, f[3] * mul1);
+                                    v.z = pack_half2(f[4] * mul1, f[5] * mul1), v.w = pack_half2(f[6] * mul1, f[7] * mul1);
+                                    __stcg(po + (c * 4 + q4) * kBM, v);
+                                }
                             }
                         }
                     }
+                    // row scale: 1 unless |O / l| would exceed 2^14 (fp16 holds up to 65504)
+                    float scale = 1.f;  // O = Ohat * l * scale
+                    if (row_ok && !direct) {
+                        const float nmax = fmaxf(fmaxf(am[0], am[1]), fmaxf(am[2], am[3])) * inv;
+                        if (nmax > 16384.f && l_run > 0.f) scale = exp2f(ceilf(log2f(nmax)) - 14.f);
+                    }
+                    // the loads from tensor memory are warp-wide: the whole warp goes through them
+                    // when one of its rows needs its scale
+                    if (__any_sync(kFull, scale != 1.f)) {
+                        const float mul = inv / scale;
+#pragma unroll 1
+                        for (int c = 0; c < D / 32; ++c) {
+                            tmem_ld32(o_t + c * 32, orr[0]);
+                            tmem_wait_ld();
+                            if (scale != 1.f) {
+#pragma unroll
+                                for (int q4 = 0; q4 < 4; ++q4) {
+                                    const uint32_t* w = &orr[0][q4 * 8];
+                                    uint4 v;
+                                    v.x = pack_half2(__uint_as_float(w[0]) * mul, __uint_as_float(w[1]) * mul);
+                                    v.y = pack_half2(__uint_as_float(w[2]) * mul, __uint_as_float(w[3]) * mul);
+                                    v.z = pack_half2(__uint_as_float(w[4]) * mul, __uint_as_float(w[5]) * mul);
+                                    v.w = pack_half2(__uint_as_float(w[6]) * mul, __uint_as_float(w[7]) * mul);
+                                    __stcg(po + (c * 4 + q4) * kBM, v);
+                                }
+                            }
+                        }
+                    }
+                    if (row_ok && !direct)
+                        __stcg(a.part_ml + (static_cast<int64_t>(item) * kRowTiles + x) * kBM + r,
+                               make_float4(l_run > 0.f ? m_ref : -INFINITY, l_run, l_run * scale, 0.f));
                 }
                 tc_fence_before();
             } else if (!row_mode && row_ok) {

@@ -124,7 +124,7 @@ def test_ragged_batch_and_clamping_sets_status():
 
 
 # ------------------------------------------------------------------------ attention
-def _attention_case(n, Hq, Hkv, D, L, cap, parent=None, poison=False, seed=0, B=1, max_tt=128):
+def _attention_case(n, Hq, Hkv, D, L, cap, parent=None, poison=False, seed=0, B=1, max_tt=128, v_scale=1.0):
     oracle, binding, synth = _imports()
     from harness import check_attention, u16_to_bf16_cuda, bf16_to_f64
     rng = np.random.default_rng(seed)
@@ -133,7 +133,7 @@ def _attention_case(n, Hq, Hkv, D, L, cap, parent=None, poison=False, seed=0, B=
     Ls = [L] * B if isinstance(L, int) else L
     q = synth.to_bf16_bits(rng.normal(size=(B, max_tt, Hq, D)).astype(np.float32).ravel()).reshape(B, max_tt, Hq, D)
     kc = synth.to_bf16_bits(rng.normal(size=(B, Hkv, cap, D)).astype(np.float32).ravel()).reshape(B, Hkv, cap, D)
-    vc = synth.to_bf16_bits(rng.normal(size=(B, Hkv, cap, D)).astype(np.float32).ravel()).reshape(B, Hkv, cap, D)
+    vc = synth.to_bf16_bits((rng.normal(size=(B, Hkv, cap, D)) * v_scale).astype(np.float32).ravel()).reshape(B, Hkv, cap, D)
     masks = np.zeros((B, max_tt, 2), np.uint64)
     for s in range(B):
         par = parent if parent is not None else [-1] + [int(rng.integers(max(0, i - 9), i)) for i in range(1, ns[s])]
@@ -165,7 +165,10 @@ def _attention_case(n, Hq, Hkv, D, L, cap, parent=None, poison=False, seed=0, B=
         g = bf16_to_f64(do)
         for s in range(B):
             ref = oracle.tree_attention(q[s, :ns[s]], kc[s], vc[s], Ls[s], masks[s, :ns[s]], scale)
-            check_attention(g[s, :ns[s]], ref)
+            if v_scale == 1.0:
+                check_attention(g[s, :ns[s]], ref)
+            else:  # the absolute gate is stated for values of order one: scale it with the values
+                check_attention(g[s, :ns[s]] / v_scale, ref / v_scale)
             assert np.isnan(g[s, ns[s]:]).all()
     ctx.close()
     return masks
@@ -182,6 +185,13 @@ def _attention_case(n, Hq, Hkv, D, L, cap, parent=None, poison=False, seed=0, B=
 ])
 def test_attention_shapes_and_boundaries(n, Hq, Hkv, D, L):
     _attention_case(n, Hq, Hkv, D, L, cap=L + 128 + 70, poison=True, seed=n)
+
+
+@pytest.mark.parametrize("n,Hq,Hkv", [(20, 8, 2), (70, 16, 4)])
+def test_attention_large_values_survive_the_split_partials(n, Hq, Hkv):
+    """V far beyond the fp16 range, on a prefix long enough to be split: the partial results carry a
+    per-row scale."""
+    _attention_case(n, Hq, Hkv, 128, 5000, cap=5200, seed=11, v_scale=3.0e5)
 
 
 def test_attention_chain_mask_is_causal():
