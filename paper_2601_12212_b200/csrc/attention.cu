@@ -55,7 +55,7 @@ constexpr int kSyncThreads = 320;  // softmax warps + the MMA warps meet at the 
 constexpr int kMaxBatchSmem = 256;
 constexpr int kTmemCols = 512;
 constexpr int kCombineThreads = 256;
-constexpr long long kWaitLimitCycles = 4000000000ll;  // bounded waits give up after ~2 s of SM clocks
+constexpr uint32_t kWaitLimitCycles = 0x70000000u;  // bounded waits give up after ~1 s of SM clocks
 constexpr float kRescaleSlack = 8.0f;  // O is rescaled only when the running max grows by > 2^8
 constexpr unsigned kFull = 0xFFFFFFFFu;
 
@@ -84,89 +84,95 @@ struct AttnArgs {
 };
 
 // ---------------------------------------------------------------------------- work list
+// A group is (sequence, KV head, pair of row tiles).  A pair with more than 128 rows runs in row
+// mode and costs two units per key tile; the last pair of a head may have at most 128 rows, runs
+// in key mode and costs one.  Every group is cut into splits of at most T units, with the smallest
+// T for which the items fit one round of the grid (found by a short search; steps of 1/16), so
+// that the CTAs finish together whatever the mix of tree sizes and prefix lengths.
 struct Sched {
     int n[kMaxBatchSmem];       // tree nodes (0 = sequence skipped)
     int L[kMaxBatchSmem];
     int mp[kMaxBatchSmem];      // row-tile pairs
+    int nfull[kMaxBatchSmem];   // pairs in row mode (mp or mp - 1)
     int kt[kMaxBatchSmem];      // key tiles
-    int splits[kMaxBatchSmem];
+    int s_row[kMaxBatchSmem];   // splits of a row-mode group
+    int s_key[kMaxBatchSmem];   // splits of the key-mode group
     int item0[kMaxBatchSmem + 1];
 };
 
-__device__ __forceinline__ void build_sched(const AttnArgs& a, Sched& sc, int tid, int nthreads) {
-    const int G = a.Hq / a.Hkv;
-    if (a.batch <= 32) {
-        // One warp, one lane per sequence: the loads, the divisions and the sums run side by side
-        // and the block meets once.  (Every count below fits 32 bits: at most 32 sequences of at
-        // most 2^15 key tiles, and the row-tile pairs of all KV heads are bounded by the context.)
-        if (tid < 32) {
-            const int b = tid;
-            int n = 0, L = 0, mp = 0, kt = 0;
+__device__ __forceinline__ int ceil_div(int a, int b) {  // a >= 0, b > 0: the unsigned division is the shorter one
+    return static_cast<int>((static_cast<unsigned>(a) + static_cast<unsigned>(b) - 1u) / static_cast<unsigned>(b));
+}
+
+// Runs in the first warp (one lane per sequence, eight rounds for the largest batch); the block
+// meets once at the end.  This sits at the head of the kernel's critical path (nothing can be
+// fetched before the CTA knows its item), hence the care for the length of the dependent chain.
+__device__ __forceinline__ void build_sched(const AttnArgs& a, Sched& sc, int tid) {
+    if (tid < 32) {
+        const int G = a.Hq / a.Hkv;
+        const int nblk = (a.batch + 31) >> 5;
+        const int mt = max(a.min_tiles, 1);
+        // round 0 of the lane stays in registers (the only round up to 32 sequences)
+        int kt0 = 0, nfull0 = 0, nkey0 = 0;
+        unsigned cost = 0;  // saturates: it only seeds the search below
+#pragma unroll 1
+        for (int i = 0; i < nblk; ++i) {
+            const int b = i * 32 + tid;
             if (b < a.batch) {
-                n = min(max(a.n_nodes[b], 0), a.max_tt);
-                L = max(a.steps[b].prefix_len, 0);
+                int n = min(max(a.n_nodes[b], 0), a.max_tt);
+                const int L = max(a.steps[b].prefix_len, 0);
                 if (static_cast<int64_t>(L) + n > a.capacity) {
                     atomicOr(a.status, RESPS_STATUS_KV_OVERFLOW);
                     n = 0;
                 }
-                mp = (n * G + kRowTiles * kBM - 1) / (kRowTiles * kBM);
-                kt = (n > 0) ? (L + n + kBN - 1) / kBN : 0;
+                const int M = n * G;
+                const int mp = (M + kRowTiles * kBM - 1) / (kRowTiles * kBM);
+                const int nfull = (mp > 0 && M - (mp - 1) * kRowTiles * kBM <= kBM) ? mp - 1 : mp;
+                const int kt = (n > 0) ? (L + n + kBN - 1) / kBN : 0;
+                sc.n[b] = n, sc.L[b] = L, sc.mp[b] = mp, sc.nfull[b] = nfull, sc.kt[b] = kt;
+                if (i == 0) kt0 = kt, nfull0 = nfull, nkey0 = mp - nfull;
+                cost += min(static_cast<unsigned>(a.Hkv * (nfull + mp)) * static_cast<unsigned>(kt), 1u << 23);
             }
-            const unsigned grp = static_cast<unsigned>(a.Hkv * mp);
-            const unsigned units = __reduce_add_sync(0xFFFFFFFFu, grp * static_cast<unsigned>(kt));
-            unsigned tps = (units + a.sched_grid - 1) / a.sched_grid;
-            tps = max(tps, static_cast<unsigned>(max(a.min_tiles, 1)));
-            // ceil(kt / tps) splits per group can add up to more items than CTAs (a second, nearly
-            // empty round); a slightly larger tile count per split then gives a single round.
-            for (int tries = 0; tries < 8; ++tries) {
-                const unsigned cnt = __reduce_add_sync(0xFFFFFFFFu, grp * ((kt + tps - 1) / tps));
-                if (cnt <= static_cast<unsigned>(a.sched_grid)) break;
-                ++tps;
+        }
+        cost = __reduce_add_sync(0xFFFFFFFFu, min(cost, 1u << 26));
+        int T = max(ceil_div(static_cast<int>(cost), a.sched_grid), 1);
+        int s_row0 = 0, s_key0 = 0;
+#pragma unroll 1
+        for (int tries = 0; tries < 24; ++tries) {
+            const int t_row = max((T + 1) >> 1, mt), t_key = max(T, mt);
+            s_row0 = ceil_div(kt0, t_row), s_key0 = ceil_div(kt0, t_key);
+            unsigned cnt = a.Hkv * (nfull0 * s_row0 + nkey0 * s_key0);
+#pragma unroll 1
+            for (int i = 1; i < nblk; ++i) {
+                const int b = i * 32 + tid;
+                if (b < a.batch)
+                    cnt += a.Hkv * (sc.nfull[b] * ceil_div(sc.kt[b], t_row) +
+                                    (sc.mp[b] - sc.nfull[b]) * ceil_div(sc.kt[b], t_key));
             }
-            const int splits = (kt + tps - 1) / tps;
-            const int mine = static_cast<int>(grp) * splits;
+            cnt = __reduce_add_sync(0xFFFFFFFFu, min(cnt, 1u << 20));
+            if (cnt <= static_cast<unsigned>(a.sched_grid)) break;
+            T += max(1, T >> 4);
+        }
+        const int t_row = max((T + 1) >> 1, mt), t_key = max(T, mt);
+        int base = 0;
+#pragma unroll 1
+        for (int i = 0; i < nblk; ++i) {
+            const int b = i * 32 + tid;
+            int mine = 0, s_row = s_row0, s_key = s_key0;
+            if (i > 0 && b < a.batch) s_row = ceil_div(sc.kt[b], t_row), s_key = ceil_div(sc.kt[b], t_key);
+            if (b < a.batch) mine = a.Hkv * (sc.nfull[b] * s_row + (sc.mp[b] - sc.nfull[b]) * s_key);
             int incl = mine;  // inclusive prefix sum over the lanes
+            if (a.batch > 1) {
 #pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                const int v = __shfl_up_sync(0xFFFFFFFFu, incl, d);
-                if (b >= d) incl += v;
+                for (int d = 1; d < 32; d <<= 1) {
+                    const int v = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+                    if (tid >= d) incl += v;
+                }
             }
-            if (b < a.batch) {
-                sc.n[b] = n, sc.L[b] = L, sc.mp[b] = mp, sc.kt[b] = kt, sc.splits[b] = splits;
-                sc.item0[b] = incl - mine;
-                if (b == a.batch - 1) sc.item0[a.batch] = incl;
-            }
+            if (b < a.batch) sc.s_row[b] = s_row, sc.s_key[b] = s_key, sc.item0[b] = base + incl - mine;
+            base += __shfl_sync(0xFFFFFFFFu, incl, a.batch > 1 ? 31 : 0);
         }
-        __syncthreads();
-        return;
-    }
-    for (int b = tid; b < a.batch; b += nthreads) {
-        int n = min(max(a.n_nodes[b], 0), a.max_tt);
-        const int L = max(a.steps[b].prefix_len, 0);
-        if (static_cast<int64_t>(L) + n > a.capacity) {
-            atomicOr(a.status, RESPS_STATUS_KV_OVERFLOW);
-            n = 0;
-        }
-        sc.n[b] = n;
-        sc.L[b] = L;
-        sc.mp[b] = (n * G + kRowTiles * kBM - 1) / (kRowTiles * kBM);
-        sc.kt[b] = (n > 0) ? (L + n + kBN - 1) / kBN : 0;
-    }
-    __syncthreads();
-    if (tid == 0) {
-        long long units = 0;
-        for (int b = 0; b < a.batch; ++b) units += 1ll * a.Hkv * sc.mp[b] * sc.kt[b];
-        int tps = (units < (1ll << 30))  // the 64-bit division is a long dependent chain: avoid it when possible
-                      ? (static_cast<int>(units) + a.sched_grid - 1) / a.sched_grid
-                      : static_cast<int>((units + a.sched_grid - 1) / a.sched_grid);
-        tps = max(tps, max(a.min_tiles, 1));
-        int items = 0;
-        for (int b = 0; b < a.batch; ++b) {
-            sc.item0[b] = items;
-            sc.splits[b] = (sc.kt[b] + tps - 1) / tps;
-            items += a.Hkv * sc.mp[b] * sc.splits[b];
-        }
-        sc.item0[a.batch] = items;
+        if (tid == 0) sc.item0[a.batch] = base;
     }
     __syncthreads();
 }
@@ -182,13 +188,22 @@ __device__ __forceinline__ Item decode_item(const Sched& sc, int item, int G) {
     int b = 0;
     while (item >= sc.item0[b + 1]) ++b;
     it.b = b;
-    it.n = sc.n[b], it.L = sc.L[b], it.splits = sc.splits[b];
+    it.n = sc.n[b], it.L = sc.L[b];
+    const int nfull = sc.nfull[b], s_row = sc.s_row[b], s_key = sc.s_key[b];
+    const int row_items = nfull * s_row;
+    const int per_head = row_items + (sc.mp[b] - nfull) * s_key;
     const int local = item - sc.item0[b];
-    const int grp = local / it.splits;  // = g * mp + pair
-    it.sp = local - grp * it.splits;
-    const int mp = sc.mp[b];
-    it.g = (mp == 1) ? grp : grp / mp;
-    it.pair = grp - it.g * mp;
+    it.g = static_cast<int>(static_cast<unsigned>(local) / static_cast<unsigned>(per_head));
+    const int rem = local - it.g * per_head;
+    if (rem < row_items) {
+        it.pair = (nfull == 1) ? 0 : static_cast<int>(static_cast<unsigned>(rem) / static_cast<unsigned>(s_row));
+        it.sp = rem - it.pair * s_row;
+        it.splits = s_row;
+    } else {
+        it.pair = nfull;
+        it.sp = rem - row_items;
+        it.splits = s_key;
+    }
     it.first_item = item - it.sp;
     it.M = it.n * G;
     it.row_base = it.pair * kRowTiles * kBM;
@@ -225,28 +240,23 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// Bounded wait: false when the CTA has given up (here or elsewhere).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                          int32_t* status) {
-    if (mbar_try(bar, parity)) return true;
-    const long long t0 = clock64();
-    unsigned spins = 0;
-    for (;;) {
-        if (mbar_try(bar, parity)) return true;
-        if ((++spins & 63u) == 0u) {
-            if (*abort_flag) return false;
-            if (clock64() - t0 > kWaitLimitCycles) {
-                *abort_flag = 1;
-                atomicOr(status, RESPS_STATUS_WAIT_TIMEOUT);
-                return false;
-            }
-        }
+// Bounded wait: false when this wait ran out (about a second of SM clocks) or another thread of
+// the CTA has given up.  Kept to a few instructions, because it is inlined at every wait and the
+// kernel's code has to stay small (see the note on code size at the kernel); the caller records
+// the failure in its `alive` flag, and the status word is written once, at the end of the kernel.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    const uint32_t t0 = static_cast<uint32_t>(clock());
+    uint32_t spins = 0;
+    while (!mbar_try(bar, parity)) {
+        // the 32-bit cycle counter wraps after two seconds; it is read far more often than that
+        if ((++spins & 255u) == 0u && (*abort_flag || static_cast<uint32_t>(clock()) - t0 > kWaitLimitCycles))
+            return false;
     }
+    return true;
 }
 // Same, with a warp-uniform answer (the callers go on to warp-collective TMEM instructions).
-__device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                          int32_t* status) {
-    const bool ok = mbar_wait(bar, parity, abort_flag, status);
+__device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    const bool ok = mbar_wait(bar, parity, abort_flag);
     return __all_sync(0xFFFFFFFFu, ok);
 }
 // One lane of a converged warp.
@@ -479,7 +489,7 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
     pdl_wait();
     pdl_launch_dependents();
     tc_fence_before();
-    build_sched(a, sc, tid, kAttnThreads);  // ends with __syncthreads(): barriers, TMEM address and schedule are visible
+    build_sched(a, sc, tid);  // ends with __syncthreads(): barriers, TMEM address and schedule are visible
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
     const int total_items = min(sc.item0[a.batch], a.max_items);
@@ -532,7 +542,7 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
                     if (kt_run > 0) {  // the CTA's very first tile went out during the set-up
                         // the first use of a stage finds it free
                         if (kt_run >= kStages &&
-                            !mbar_wait(bar(bar_kempty(s)), ((kt_run / kStages) & 1u) ^ 1u, abort_flag, a.status)) {
+                            !mbar_wait(bar(bar_kempty(s)), ((kt_run / kStages) & 1u) ^ 1u, abort_flag)) {
                             alive = false;
                             break;
                         }
@@ -544,7 +554,7 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
                         // Q follows the first K tile: K and Q are what the first MMA needs.  The Q
                         // tiles of the previous item are free once its last QK^T has completed.
                         if (items_run > 0) {
-                            if (!mbar_wait(bar(bar_qempty()), (items_run & 1u) ^ 1u, abort_flag, a.status)) {
+                            if (!mbar_wait(bar(bar_qempty()), (items_run & 1u) ^ 1u, abort_flag)) {
                                 alive = false;
                                 break;
                             }
@@ -558,10 +568,11 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
                 }
             }
             // Drain: every copy this thread issued has landed before the CTA may exit.
-            if (a.q_by_tma && items_run > 0) mbar_wait(bar(bar_qfull()), (items_run - 1u) & 1u, abort_flag, a.status);
+            bool landed = !(a.q_by_tma && items_run > 0) || mbar_wait(bar(bar_qfull()), (items_run - 1u) & 1u, abort_flag);
             const uint32_t issued = kt_run;
-            for (uint32_t u = (issued > kStages ? issued - kStages : 0u); u < issued; ++u)
-                if (!mbar_wait(bar(bar_kfull(u % kStages)), (u / kStages) & 1u, abort_flag, a.status)) break;
+            for (uint32_t u = (issued > kStages ? issued - kStages : 0u); u < issued && landed; ++u)
+                landed = mbar_wait(bar(bar_kfull(u % kStages)), (u / kStages) & 1u, abort_flag);
+            alive = alive && landed;
         }
     } else if (warp == kVProducerWarp) {
         // ================================ TMA producer: V tiles =============================
@@ -573,7 +584,7 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
                     const int s = kt_run % kStages;
                     if (kt_run == 0) continue;  // went out during the set-up
                     if (kt_run >= kStages &&
-                        !mbar_wait(bar(bar_vempty(s)), ((kt_run / kStages) & 1u) ^ 1u, abort_flag, a.status)) {
+                        !mbar_wait(bar(bar_vempty(s)), ((kt_run / kStages) & 1u) ^ 1u, abort_flag)) {
                         alive = false;
                         break;
                     }
@@ -583,8 +594,10 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
                 }
             }
             const uint32_t issued = kt_run;
-            for (uint32_t u = (issued > kStages ? issued - kStages : 0u); u < issued; ++u)
-                if (!mbar_wait(bar(bar_vfull(u % kStages)), (u / kStages) & 1u, abort_flag, a.status)) break;
+            bool landed = true;
+            for (uint32_t u = (issued > kStages ? issued - kStages : 0u); u < issued && landed; ++u)
+                landed = mbar_wait(bar(bar_vfull(u % kStages)), (u / kStages) & 1u, abort_flag);
+            alive = alive && landed;
         }
     } else if (warp == kMmaWarp0 || warp == kMmaWarp0 + 1) {
         // ================================ MMA issuer of lane x ============================
@@ -606,7 +619,7 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
             const Item it = get_item(item, static_cast<int>(items_run));
             const bool row_mode = it.nmt == 2;
             const uint64_t qdesc = qdesc0 + static_cast<uint64_t>((row_mode ? x : 0) * (S::kQTile >> 4));
-            alive = warp_wait(bar(bar_qfull()), items_run & 1u, abort_flag, a.status);
+            alive = warp_wait(bar(bar_qfull()), items_run & 1u, abort_flag);
             tc_fence_after();
             bool have_prev = false, first_pv = true;
             uint32_t prev_kt = 0, prev_j = 0;
@@ -617,11 +630,11 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
             // next Q K^T: the chain that decides when the softmax warps get their next S.
             auto issue_pv = [&](uint32_t next_use) {
                 const int s = prev_kt % kStages;
-                if (!warp_wait(bar(bar_vfull(s)), (prev_kt / kStages) & 1u, abort_flag, a.status)) return false;
+                if (!warp_wait(bar(bar_vfull(s)), (prev_kt / kStages) & 1u, abort_flag)) return false;
                 if (next_use != 0xFFFFFFFFu &&
                     __all_sync(kFull, mbar_try(bar(bar_kfull(next_use % kStages)), (next_use / kStages) & 1u)))
                     k_seen = next_use;
-                if (!warp_wait(bar(bar_pfull(x, prev_j & 1u)), (prev_j >> 1) & 1u, abort_flag, a.status)) return false;
+                if (!warp_wait(bar(bar_pfull(x, prev_j & 1u)), (prev_j >> 1) & 1u, abort_flag)) return false;
                 tc_fence_after();
                 if (elect_one()) {
                     const uint64_t vdesc = vdesc0 + static_cast<uint64_t>(s * (S::kKVTile >> 4));
@@ -646,7 +659,7 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
                 const bool own = row_mode || (((t - it.t_begin) & 1) == x);
                 if (own) {
                     if (k_seen != kt_run)
-                        alive = warp_wait(bar(bar_kfull(s)), (kt_run / kStages) & 1u, abort_flag, a.status);
+                        alive = warp_wait(bar(bar_kfull(s)), (kt_run / kStages) & 1u, abort_flag);
                     if (!alive) break;
                     tc_fence_after();
                     if (elect_one()) {
@@ -674,7 +687,7 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
             if (!alive) break;
             // end of item: the softmax warps have read O and S, Q and P may be overwritten
             mbar_arrive(bar(bar_item()));
-            alive = warp_wait(bar(bar_item()), items_run & 1u, abort_flag, a.status);
+            alive = warp_wait(bar(bar_item()), items_run & 1u, abort_flag);
         }
     }
     } else {
@@ -691,33 +704,23 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
             // ---- Q tiles -> shared memory in the swizzled K-major layout (only when the group
             // size does not allow the TMA view) ---------------------------------------------
             if (!a.q_by_tma) {
+                // (a plain loop: this path serves group sizes that do not divide 128 and is not
+                // worth its unrolled form's code size)
                 const int total = it.nmt * kBM * kChunks;
-                constexpr int kInFlight = kRowTiles * kBM * kChunks / kSoftmaxThreads;
-                uint4 v[kInFlight];
-#pragma unroll
-                for (int u = 0; u < kInFlight; ++u) {
-                    const int i = tid + u * kSoftmaxThreads;
-                    v[u] = make_uint4(0u, 0u, 0u, 0u);
-                    if (i < total) {
-                        const int row = i / kChunks, c = i % kChunks;
-                        const int R = it.row_base + row;
-                        if (R < it.M) {
-                            const int t = R / G, h = it.g * G + R % G;
-                            v[u] = __ldg(reinterpret_cast<const uint4*>(
-                                a.q + ((static_cast<int64_t>(it.b) * a.max_tt + t) * a.Hq + h) * D + c * 8));
-                        }
+#pragma unroll 1
+                for (int i = tid; i < total; i += kSoftmaxThreads) {
+                    const int row = i / kChunks, c = i % kChunks;
+                    const int Rq = it.row_base + row;
+                    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                    if (Rq < it.M) {
+                        const int t = Rq / G, h = it.g * G + Rq % G;
+                        v = __ldg(reinterpret_cast<const uint4*>(
+                            a.q + ((static_cast<int64_t>(it.b) * a.max_tt + t) * a.Hq + h) * D + c * 8));
                     }
-                }
-#pragma unroll
-                for (int u = 0; u < kInFlight; ++u) {
-                    const int i = tid + u * kSoftmaxThreads;
-                    if (i < total) {
-                        const int row = i / kChunks, c = i % kChunks;
-                        const int m = row / kBM, rr = row % kBM;
-                        unsigned char* dst = base_ptr + S::kOffQ + m * S::kQTile + (c >> 3) * S::kQPanel + rr * 128 +
-                                             (((c & 7) ^ (rr & 7)) << 4);
-                        *reinterpret_cast<uint4*>(dst) = v[u];
-                    }
+                    const int m = row / kBM, rr = row % kBM;
+                    unsigned char* dst = base_ptr + S::kOffQ + m * S::kQTile + (c >> 3) * S::kQPanel + rr * 128 +
+                                         (((c & 7) ^ (rr & 7)) << 4);
+                    *reinterpret_cast<uint4*>(dst) = v;
                 }
                 fence_proxy_async();
                 mbar_arrive(bar(bar_qfull()));
@@ -758,7 +761,7 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
                 if (!(row_mode || (((t - it.t_begin) & 1) == x))) continue;
                 const uint32_t buf = jx & 1u;
                 if (!s_loaded) {
-                    if (!warp_wait(bar(bar_sfull(x, buf)), (jx >> 1) & 1u, abort_flag, a.status)) {
+                    if (!warp_wait(bar(bar_sfull(x, buf)), (jx >> 1) & 1u, abort_flag)) {
                         alive = false;
                         break;
                     }
@@ -809,7 +812,7 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
                 if (__any_sync(kFull, need)) {
                     // O may only be touched once PV of the previous tile has completed
                     while (pv_seen < jx) {
-                        if (!warp_wait(bar(bar_pvdone(x)), pv_seen & 1u, abort_flag, a.status)) alive = false;
+                        if (!warp_wait(bar(bar_pvdone(x)), pv_seen & 1u, abort_flag)) alive = false;
                         ++pv_seen;
                     }
                     if (!alive) break;
@@ -839,7 +842,7 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
                 const bool clear_v = j0 + kBN > kv_len;
                 if (clear_v) {
                     const int s = kt_run % kStages;
-                    if (!warp_wait(bar(bar_vfull(s)), (kt_run / kStages) & 1u, abort_flag, a.status)) {
+                    if (!warp_wait(bar(bar_vfull(s)), (kt_run / kStages) & 1u, abort_flag)) {
                         alive = false;
                         break;
                     }
@@ -904,7 +907,7 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
                 if (clear_v) fence_proxy_async();
                 if (pv_seen < jx) {
                     if (!__all_sync(kFull, pv_probe) &&
-                        !warp_wait(bar(bar_pvdone(x)), pv_seen & 1u, abort_flag, a.status))
+                        !warp_wait(bar(bar_pvdone(x)), pv_seen & 1u, abort_flag))
                         alive = false;
                     ++pv_seen;
                 }
@@ -924,7 +927,7 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
                 __nv_bfloat16* dst = a.o + ((static_cast<int64_t>(it.b) * a.max_tt + t) * a.Hq + h) * D;
                 uint4* po = a.part_o + (static_cast<int64_t>(item) * kRowTiles + x) * (D / 8) * kBM + r;
                 while (pv_seen < jx) {
-                    if (!warp_wait(bar(bar_pvdone(x)), pv_seen & 1u, abort_flag, a.status)) alive = false;
+                    if (!warp_wait(bar(bar_pvdone(x)), pv_seen & 1u, abort_flag)) alive = false;
                     ++pv_seen;
                 }
                 if (!alive) break;
@@ -933,69 +936,53 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
                     a.lse[(static_cast<int64_t>(it.b) * a.max_tt + t) * a.Hq + h] =
                         (m_ref + log2f(l_run)) * 0.6931471805599453f;
                 {
-                    // One pass over the row in 32-column pieces: the next piece is on its way from
-                    // tensor memory while this one is converted and stored.  Partials assume a row
-                    // scale of 1 and keep the row's largest magnitude; the rare row that would leave
-                    // the fp16 range is written again with its scale.
-                    const float mul1 = direct ? inv : ((l_run > 0.f) ? inv : 0.f);
+                    // The row leaves tensor memory in 32-column pieces (plain loops: the stores, not
+                    // the loads, bound this part, and it runs once per item, so small code wins).
+                    // Partials assume a row scale of 1 and keep the row's largest magnitude; when a
+                    // row of the warp would leave the fp16 range, a second pass writes such rows
+                    // again with their scale.
                     float am[4] = {0.f, 0.f, 0.f, 0.f};
-                    uint32_t orr[2][32];
-                    tmem_ld32(o_t, orr[0]);
-#pragma unroll
-                    for (int c = 0; c < D / 32; ++c) {
-                        tmem_wait_ld();
-                        if (c + 1 < D / 32) tmem_ld32(o_t + (c + 1) * 32, orr[(c + 1) & 1]);
-                        const uint32_t* w = orr[c & 1];
-                        if (row_ok) {
-#pragma unroll
-                            for (int q4 = 0; q4 < 4; ++q4) {
-                                float f[8];
-#pragma unroll
-                                for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(w[q4 * 8 + e]);
-                                uint4 v;
-                                if (direct) {
-                                    v.x = pack_bf16(f[0] * mul1, f[1] * mul1), v.y = pack_bf16(f[2] * mul1, f[3] * mul1);
-                                    v.z = pack_bf16(f[4] * mul1, f[5] * mul1), v.w = pack_bf16(f[6] * mul1, f[7] * mul1);
-                                    *reinterpret_cast<uint4*>(dst + (c * 4 + q4) * 8) = v;
-                                } else {
-                                    am[q4] = max3(am[q4], fabsf(f[0]), fabsf(f[1]));
-                                    am[q4] = max3(am[q4], fabsf(f[2]), fabsf(f[3]));
-                                    am[q4] = max3(am[q4], fabsf(f[4]), fabsf(f[5]));
-                                    am[q4] = max3(am[q4], fabsf(f[6]), fabsf(f[7]));
-                                    v.x = pack_half2(f[0] * mul1, f[1] * mul1), v.y = pack_half2(f[2] * mul1, f[3] * mul1);
-                                    v.z = pack_half2(f[4] * mul1, f[5] * mul1), v.w = pack_half2(f[6] * mul1, f[7] * mul1);
-                                    __stcg(po + (c * 4 + q4) * kBM, v);
-                                }
-                            }
-                        }
-                    }
-                    // row scale: 1 unless |O / l| would exceed 2^14 (fp16 holds up to 65504)
                     float scale = 1.f;  // O = Ohat * l * scale
-                    if (row_ok && !direct) {
-                        const float nmax = fmaxf(fmaxf(am[0], am[1]), fmaxf(am[2], am[3])) * inv;
-                        if (nmax > 16384.f && l_run > 0.f) scale = exp2f(ceilf(log2f(nmax)) - 14.f);
-                    }
-                    // the loads from tensor memory are warp-wide: the whole warp goes through them
-                    // when one of its rows needs its scale
-                    if (__any_sync(kFull, scale != 1.f)) {
-                        const float mul = inv / scale;
+                    uint32_t orr[32];
+#pragma unroll 1
+                    for (int pass = 0; pass < 2; ++pass) {
+                        const float mul = (pass == 0) ? ((direct || l_run > 0.f) ? inv : 0.f) : inv / scale;
+                        const bool store = row_ok && (pass == 0 || scale != 1.f);
 #pragma unroll 1
                         for (int c = 0; c < D / 32; ++c) {
-                            tmem_ld32(o_t + c * 32, orr[0]);
+                            tmem_ld32(o_t + c * 32, orr);
                             tmem_wait_ld();
-                            if (scale != 1.f) {
+                            if (store) {
 #pragma unroll
                                 for (int q4 = 0; q4 < 4; ++q4) {
-                                    const uint32_t* w = &orr[0][q4 * 8];
+                                    float f[8];
+#pragma unroll
+                                    for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(orr[q4 * 8 + e]);
                                     uint4 v;
-                                    v.x = pack_half2(__uint_as_float(w[0]) * mul, __uint_as_float(w[1]) * mul);
-                                    v.y = pack_half2(__uint_as_float(w[2]) * mul, __uint_as_float(w[3]) * mul);
-                                    v.z = pack_half2(__uint_as_float(w[4]) * mul, __uint_as_float(w[5]) * mul);
-                                    v.w = pack_half2(__uint_as_float(w[6]) * mul, __uint_as_float(w[7]) * mul);
-                                    __stcg(po + (c * 4 + q4) * kBM, v);
+                                    if (direct) {
+                                        v.x = pack_bf16(f[0] * mul, f[1] * mul), v.y = pack_bf16(f[2] * mul, f[3] * mul);
+                                        v.z = pack_bf16(f[4] * mul, f[5] * mul), v.w = pack_bf16(f[6] * mul, f[7] * mul);
+                                        *reinterpret_cast<uint4*>(dst + (c * 4 + q4) * 8) = v;
+                                    } else {
+                                        am[q4] = max3(am[q4], fabsf(f[0]), fabsf(f[1]));
+                                        am[q4] = max3(am[q4], fabsf(f[2]), fabsf(f[3]));
+                                        am[q4] = max3(am[q4], fabsf(f[4]), fabsf(f[5]));
+                                        am[q4] = max3(am[q4], fabsf(f[6]), fabsf(f[7]));
+                                        v.x = pack_half2(f[0] * mul, f[1] * mul), v.y = pack_half2(f[2] * mul, f[3] * mul);
+                                        v.z = pack_half2(f[4] * mul, f[5] * mul), v.w = pack_half2(f[6] * mul, f[7] * mul);
+                                        __stcg(po + (c * 4 + q4) * kBM, v);
+                                    }
                                 }
                             }
                         }
+                        if (direct || pass == 1) break;
+                        // row scale: 1 unless |O / l| would exceed 2^14 (fp16 holds up to 65504)
+                        if (row_ok) {
+                            const float nmax = fmaxf(fmaxf(am[0], am[1]), fmaxf(am[2], am[3])) * inv;
+                            if (nmax > 16384.f && l_run > 0.f) scale = exp2f(ceilf(log2f(nmax)) - 14.f);
+                        }
+                        // (the loads from tensor memory are warp-wide: the whole warp goes round again)
+                        if (!__any_sync(kFull, scale != 1.f)) break;
                     }
                     if (row_ok && !direct)
                         __stcg(a.part_ml + (static_cast<int64_t>(item) * kRowTiles + x) * kBM + r,
@@ -1008,11 +995,15 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
                        make_float4(-INFINITY, 0.f, 0.f, 0.f));
             }
             mbar_arrive(bar(bar_item()));
-            alive = warp_wait(bar(bar_item()), items_run & 1u, abort_flag, a.status);
+            alive = warp_wait(bar(bar_item()), items_run & 1u, abort_flag);
         }
     }
 
     // ---- tear-down: every role arrives here, whatever happened ------------------------------
+    if (!alive) {
+        *abort_flag = 1;
+        atomicOr(a.status, RESPS_STATUS_WAIT_TIMEOUT);
+    }
     tc_fence_before();
     __syncthreads();
     if (warp == kMmaWarp0) {
@@ -1029,22 +1020,20 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
 template <int D>
 __global__ void __launch_bounds__(kCombineThreads) attention_combine_kernel(const AttnArgs a) {
     __shared__ Sched sc;
-    __shared__ int4 s_sched[kMaxBatchSmem];
     pdl_launch_dependents();
     // The work list is derived again from the step parameters (inputs of the attention kernel,
     // complete before it ran): this part runs while the attention kernel drains.
-    build_sched(a, sc, threadIdx.x, kCombineThreads);
-    for (int b = threadIdx.x; b < a.batch; b += kCombineThreads)
-        s_sched[b] = make_int4(sc.n[b], sc.mp[b], sc.splits[b], sc.item0[b]);
-    __syncthreads();
+    build_sched(a, sc, threadIdx.x);  // ends with __syncthreads()
     pdl_wait();  // the attention kernel has finished and its partials are visible
     const int G = a.Hq / a.Hkv;
     for (int b = 0; b < a.batch; ++b) {
-        const int n_b = s_sched[b].x, mp_b = s_sched[b].y, splits = s_sched[b].z, item0_b = s_sched[b].w;
+        const int n_b = sc.n[b], mp_b = sc.mp[b], nfull = sc.nfull[b], s_row = sc.s_row[b], s_key = sc.s_key[b];
+        const int item0_b = sc.item0[b];
         if (n_b == 0) continue;
         const int M = n_b * G;
-        const bool last_is_key_mode = M - (mp_b - 1) * kRowTiles * kBM <= kBM;
-        if (splits <= 1 && !last_is_key_mode) continue;  // every group wrote O directly
+        if (s_row <= 1 && nfull == mp_b) continue;  // every group wrote O directly
+        const int row_items = nfull * s_row;
+        const int per_head_items = row_items + (mp_b - nfull) * s_key;
         // work items: (KV head, 8 columns, row) over the M valid rows; consecutive threads take
         // consecutive rows
         const int per_head = M * (D / 8);
@@ -1056,12 +1045,13 @@ __global__ void __launch_bounds__(kCombineThreads) attention_combine_kernel(cons
             const int c8 = rem / M;
             const int R = rem % M;
             const int pair = R / (kRowTiles * kBM), row2 = R % (kRowTiles * kBM);
-            const int grp = g * mp_b + pair;
-            const bool key_mode = M - pair * kRowTiles * kBM <= kBM;
+            const bool key_mode = pair >= nfull;
+            const int splits = key_mode ? s_key : s_row;
             if (!key_mode && splits <= 1) continue;
             const int mt = row2 / kBM, r = row2 % kBM;
             const int n_parts = key_mode ? 2 * splits : splits;
-            const int64_t item_first = item0_b + static_cast<int64_t>(grp) * splits;
+            const int64_t item_first = item0_b + static_cast<int64_t>(g) * per_head_items +
+                                       (key_mode ? row_items : pair * s_row);
             // one pass over the partials, ten at a time so that their loads are in flight together
             constexpr int kBatch = 10;
             float Mx = -INFINITY, den = 0.f;
