@@ -33,6 +33,7 @@
 #include <cuda.h>
 #include <cuda_fp16.h>
 
+#include <algorithm>
 #include <cmath>
 
 #include "common.cuh"
@@ -1021,88 +1022,118 @@ template <int D>
 __global__ void __launch_bounds__(kCombineThreads) attention_combine_kernel(const AttnArgs a) {
     __shared__ Sched sc;
     pdl_launch_dependents();
+    // A CTA past the last row of the largest tree has nothing to do.  It learns that from one
+    // load and leaves: it may have started only after the attention kernel ended, and whatever it
+    // does until it exits delays the next kernel in the stream.
+    {
+        const int b = threadIdx.x;  // the batch is at most the CTA's thread count
+        const bool mine = b < a.batch && static_cast<long long>(blockIdx.x) * kCombineThreads <
+                                             1ll * min(max(a.n_nodes[b], 0), a.max_tt) * a.Hq * (D / 8);
+        if (!__syncthreads_or(mine)) return;
+    }
     // The work list is derived again from the step parameters (inputs of the attention kernel,
-    // complete before it ran): this part runs while the attention kernel drains.
+    // complete before it ran), and the thread's first piece of work is located, before the wait
+    // for the attention kernel: all of this runs while that kernel drains.
     build_sched(a, sc, threadIdx.x);  // ends with __syncthreads()
-    pdl_wait();  // the attention kernel has finished and its partials are visible
-    const int G = a.Hq / a.Hkv;
-    for (int b = 0; b < a.batch; ++b) {
-        const int n_b = sc.n[b], mp_b = sc.mp[b], nfull = sc.nfull[b], s_row = sc.s_row[b], s_key = sc.s_key[b];
-        const int item0_b = sc.item0[b];
-        if (n_b == 0) continue;
-        const int M = n_b * G;
-        if (s_row <= 1 && nfull == mp_b) continue;  // every group wrote O directly
-        const int row_items = nfull * s_row;
-        const int per_head_items = row_items + (mp_b - nfull) * s_key;
-        // work items: (KV head, 8 columns, row) over the M valid rows; consecutive threads take
-        // consecutive rows
-        const int per_head = M * (D / 8);
-        const long long total = 1ll * a.Hkv * per_head;
-        for (long long idx = 1ll * blockIdx.x * kCombineThreads + threadIdx.x; idx < total;
-             idx += 1ll * gridDim.x * kCombineThreads) {
-            const int g = static_cast<int>(idx / per_head);
-            const int rem = static_cast<int>(idx % per_head);
-            const int c8 = rem / M;
-            const int R = rem % M;
-            const int pair = R / (kRowTiles * kBM), row2 = R % (kRowTiles * kBM);
-            const bool key_mode = pair >= nfull;
-            const int splits = key_mode ? s_key : s_row;
-            if (!key_mode && splits <= 1) continue;
-            const int mt = row2 / kBM, r = row2 % kBM;
-            const int n_parts = key_mode ? 2 * splits : splits;
-            const int64_t item_first = item0_b + static_cast<int64_t>(g) * per_head_items +
-                                       (key_mode ? row_items : pair * s_row);
-            // one pass over the partials, ten at a time so that their loads are in flight together
-            constexpr int kBatch = 10;
-            float Mx = -INFINITY, den = 0.f;
-            float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-            for (int p0 = 0; p0 < n_parts; p0 += kBatch) {
-                float4 ml[kBatch];
-                uint4 v[kBatch];
+    const unsigned G = static_cast<unsigned>(a.Hq / a.Hkv);
+    const unsigned stride = gridDim.x * kCombineThreads;
+    // Work: (sequence, KV head, 8 columns, row) over the valid rows of groups that wrote partials;
+    // consecutive threads take consecutive rows.  Every count fits 32 bits (at most 2^11 rows per
+    // KV head, 2^4 column pieces, 2^7 heads).
+    int b = 0;
+    unsigned idx = blockIdx.x * kCombineThreads + threadIdx.x;
+    bool waited = false;
+    for (;;) {
+        // ---- the next piece of work of this thread ------------------------------------------
+        bool have = false;
+        unsigned g = 0, c8 = 0, R = 0, M = 0;
+        int splits = 0, n_parts = 0;
+        bool key_mode = false;
+        int64_t item_first = 0;
+        for (; b < a.batch; ++b, idx = blockIdx.x * kCombineThreads + threadIdx.x) {
+            const int nfull = sc.nfull[b], mp_b = sc.mp[b], s_row = sc.s_row[b];
+            if (sc.n[b] == 0 || (s_row <= 1 && nfull == mp_b)) continue;  // every group wrote O directly
+            M = static_cast<unsigned>(sc.n[b]) * G;
+            const unsigned per_head = M * (D / 8);
+            for (; idx < a.Hkv * per_head; idx += stride) {
+                g = idx / per_head;
+                const unsigned rem = idx - g * per_head;
+                c8 = rem / M;
+                R = rem - c8 * M;
+                const int pair = static_cast<int>(R / (kRowTiles * kBM));
+                key_mode = pair >= nfull;
+                splits = key_mode ? sc.s_key[b] : s_row;
+                if (!key_mode && splits <= 1) continue;
+                const int row_items = nfull * s_row;
+                item_first = sc.item0[b] + static_cast<int64_t>(g) * (row_items + (mp_b - nfull) * sc.s_key[b]) +
+                             (key_mode ? row_items : pair * s_row);
+                n_parts = key_mode ? 2 * splits : splits;
+                have = true;
+                break;
+            }
+            if (have) break;
+        }
+        if (!waited) {
+            pdl_wait();  // the attention kernel has finished and its partials are visible
+            waited = true;
+        }
+        if (!have) break;
+
+        // ---- O = sum_p w_p O_p / sum_p w_p l_p, w_p = 2^(m_p - max m): one pass over the partials,
+        // ten at a time so that their loads are in flight together ---------------------------------
+        const unsigned row2 = R % (kRowTiles * kBM);
+        const unsigned mt = row2 / kBM, r = row2 % kBM;
+        constexpr int kBatch = 10;
+        float Mx = -INFINITY, den = 0.f;
+        float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll 1
+        for (int p0 = 0; p0 < n_parts; p0 += kBatch) {
+            float4 ml[kBatch];
+            uint4 v[kBatch];
 #pragma unroll
-                for (int u = 0; u < kBatch; ++u) {
-                    const int p = min(p0 + u, n_parts - 1);
-                    const int64_t slot = key_mode ? (item_first + (p >> 1)) * kRowTiles + (p & 1)
-                                                  : (item_first + p) * kRowTiles + mt;
-                    ml[u] = __ldcg(&a.part_ml[slot * kBM + r]);
-                    v[u] = __ldcg(a.part_o + (slot * (D / 8) + c8) * kBM + r);
-                }
-                float mx = Mx;
+            for (int u = 0; u < kBatch; ++u) {
+                const int p = min(p0 + u, n_parts - 1);
+                const int64_t slot = key_mode ? (item_first + (p >> 1)) * kRowTiles + (p & 1)
+                                              : (item_first + p) * kRowTiles + mt;
+                ml[u] = __ldcg(&a.part_ml[slot * kBM + r]);
+                v[u] = __ldcg(a.part_o + (slot * (D / 8) + c8) * kBM + r);
+            }
+            float mx = Mx;
 #pragma unroll
-                for (int u = 0; u < kBatch; ++u)
-                    if (p0 + u < n_parts) mx = fmaxf(mx, ml[u].x);
-                if (mx == -INFINITY) continue;
-                const float corr = ex2_approx(Mx - mx);  // 0 on the first batch
-                den *= corr;
+            for (int u = 0; u < kBatch; ++u)
+                if (p0 + u < n_parts) mx = fmaxf(mx, ml[u].x);
+            if (mx == -INFINITY) continue;
+            const float corr = ex2_approx(Mx - mx);  // 0 on the first batch
+            den *= corr;
 #pragma unroll
-                for (int e = 0; e < 8; ++e) acc[e] *= corr;
-                Mx = mx;
+            for (int e = 0; e < 8; ++e) acc[e] *= corr;
+            Mx = mx;
 #pragma unroll
-                for (int u = 0; u < kBatch; ++u) {
-                    if (p0 + u >= n_parts || ml[u].x == -INFINITY) continue;  // an empty partial holds no O
-                    const float w = ex2_approx(ml[u].x - Mx);
-                    den += ml[u].y * w;
-                    const float wo = ml[u].z * w;  // O_p = Ohat * l * row scale
-                    const uint32_t hw[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+            for (int u = 0; u < kBatch; ++u) {
+                if (p0 + u >= n_parts || ml[u].x == -INFINITY) continue;  // an empty partial holds no O
+                const float w = ex2_approx(ml[u].x - Mx);
+                den += ml[u].y * w;
+                const float wo = ml[u].z * w;  // O_p = Ohat * l * row scale
+                const uint32_t hw[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&hw[e]));
-                        acc[2 * e] += f.x * wo, acc[2 * e + 1] += f.y * wo;
-                    }
+                for (int e = 0; e < 4; ++e) {
+                    const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&hw[e]));
+                    acc[2 * e] += f.x * wo, acc[2 * e + 1] += f.y * wo;
                 }
             }
-            const float inv = 1.f / den;
-            const int t = R / G, h = g * G + R % G;
-            __nv_bfloat16* dst = a.o + ((static_cast<int64_t>(b) * a.max_tt + t) * a.Hq + h) * D + c8 * 8;
-            uint4 out;
-            out.x = pack_bf16(acc[0] * inv, acc[1] * inv);
-            out.y = pack_bf16(acc[2] * inv, acc[3] * inv);
-            out.z = pack_bf16(acc[4] * inv, acc[5] * inv);
-            out.w = pack_bf16(acc[6] * inv, acc[7] * inv);
-            *reinterpret_cast<uint4*>(dst) = out;
-            if (a.lse && c8 == 0)
-                a.lse[(static_cast<int64_t>(b) * a.max_tt + t) * a.Hq + h] = (Mx + log2f(den)) * 0.6931471805599453f;
         }
+        const float inv = 1.f / den;
+        const unsigned t = R / G, h = g * G + (R - t * G);
+        __nv_bfloat16* dst = a.o + ((static_cast<int64_t>(b) * a.max_tt + t) * a.Hq + h) * D + c8 * 8;
+        uint4 out;
+        out.x = pack_bf16(acc[0] * inv, acc[1] * inv);
+        out.y = pack_bf16(acc[2] * inv, acc[3] * inv);
+        out.z = pack_bf16(acc[4] * inv, acc[5] * inv);
+        out.w = pack_bf16(acc[6] * inv, acc[7] * inv);
+        *reinterpret_cast<uint4*>(dst) = out;
+        if (a.lse && c8 == 0)
+            a.lse[(static_cast<int64_t>(b) * a.max_tt + t) * a.Hq + h] = (Mx + log2f(den)) * 0.6931471805599453f;
+        idx += stride;
     }
 }
 
@@ -1183,17 +1214,29 @@ cudaError_t launch_for_dim(const resps_ctx* ctx, const AttnArgs& a, const CUtens
     cudaError_t e = launch_pdl(tree_attention_kernel<D>, ctx->ws.attn_grid, kAttnThreads, Smem<D>::kBytes, st, a, mk,
                                mv, mq);
     if (e != cudaSuccess) return e;
-    return launch_pdl(attention_combine_kernel<D>, ctx->ws.attn_combine_grid, kCombineThreads, 0, st, a);
+    // one resident round of CTAs at most, and no more than the largest trees could use
+    const long long most = (1ll * a.batch * a.max_tt * a.Hq * (D / 8) + kCombineThreads - 1) / kCombineThreads;
+    const int grid = static_cast<int>(std::min<long long>(ctx->ws.attn_combine_grid, std::max<long long>(most, 1)));
+    return launch_pdl(attention_combine_kernel<D>, grid, kCombineThreads, 0, st, a);
 }
 
 }  // namespace
 
-cudaError_t attention_setup(resps_ctx*) {
+cudaError_t attention_setup(resps_ctx* ctx) {
     cudaError_t e = cudaFuncSetAttribute(tree_attention_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          Smem<128>::kBytes);
     if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(tree_attention_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                Smem<64>::kBytes);
+    e = cudaFuncSetAttribute(tree_attention_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<64>::kBytes);
+    if (e != cudaSuccess) return e;
+    // The combine kernel runs as one resident round: a CTA that has to wait for a free SM pays
+    // its set-up after the attention kernel has ended instead of under its tail.
+    int per_sm = 0;
+    e = (ctx->shape.head_dim == 128)
+            ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, attention_combine_kernel<128>, kCombineThreads, 0)
+            : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, attention_combine_kernel<64>, kCombineThreads, 0);
+    if (e != cudaSuccess) return e;
+    ctx->ws.attn_combine_grid = ctx->sm_count * std::max(per_sm, 1);
+    return cudaSuccess;
 }
 
 cudaError_t launch_tree_attention(const resps_ctx* ctx, const resps_step* d_steps,
