@@ -246,6 +246,7 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
 // kernel's code has to stay small (see the note on code size at the kernel); the caller records
 // the failure in its `alive` flag, and the status word is written once, at the end of the kernel.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    if (mbar_try(bar, parity)) return true;  // the common case does not even read the clock
     const uint32_t t0 = static_cast<uint32_t>(clock());
     uint32_t spins = 0;
     while (!mbar_try(bar, parity)) {
