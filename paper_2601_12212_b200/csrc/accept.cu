@@ -24,6 +24,8 @@ struct AcceptArgs {
 
 // One CTA of 128 threads per sequence: thread c owns tree node c.
 __global__ void __launch_bounds__(RESPS_MAX_TT) accept_walk_kernel(const AcceptArgs a) {
+    pdl_wait();  // the kernel before this one in the stream has completed
+    pdl_launch_dependents();
     const int b = blockIdx.x, tid = threadIdx.x;
     const int n = min(max(a.n_nodes[b], 1), a.max_tt);
     const int64_t ob = static_cast<int64_t>(b) * a.max_tt;
@@ -79,6 +81,8 @@ struct CompactArgs {
 // registers before any destination row is written (a destination slot may be the source
 // of an earlier path entry), so the move is safe in place.
 __global__ void __launch_bounds__(128) kv_compact_kernel(const CompactArgs a) {
+    pdl_wait();  // the kernel before this one in the stream has completed
+    pdl_launch_dependents();
     const int b = blockIdx.z, layer = blockIdx.y;
     const int head = blockIdx.x >> 1, is_v = blockIdx.x & 1;
     const int cap = a.max_depth + 1;
@@ -123,8 +127,7 @@ cudaError_t launch_accept_walk(const resps_ctx* ctx, const resps_step* d_steps,
     a.max_tt = ctx->shape.max_tt, a.max_depth = ctx->shape.max_depth;
     a.accept_path = accept_path, a.accept_len = accept_len, a.out_tokens = out_tokens;
     a.steps_next = steps_next;
-    accept_walk_kernel<<<batch, RESPS_MAX_TT, 0, st>>>(a);
-    return cudaGetLastError();
+    return launch_pdl(accept_walk_kernel, dim3(batch), dim3(RESPS_MAX_TT), 0, st, a);
 }
 
 cudaError_t launch_kv_compact(const resps_ctx* ctx, const resps_step* d_steps, int batch,
@@ -139,8 +142,7 @@ cudaError_t launch_kv_compact(const resps_ctx* ctx, const resps_step* d_steps, i
     a.n_kv_heads = ctx->shape.n_kv_heads, a.head_dim = ctx->shape.head_dim;
     a.max_depth = ctx->shape.max_depth;
     dim3 grid(ctx->shape.n_kv_heads * 2, n_layers, batch);
-    kv_compact_kernel<<<grid, 128, 0, st>>>(a);
-    return cudaGetLastError();
+    return launch_pdl(kv_compact_kernel, grid, dim3(128), 0, st, a);
 }
 
 }  // namespace resps

@@ -286,8 +286,6 @@ __device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map
         "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(bar)
         : "memory");
 }
-__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 // Shared-memory matrix descriptor, 128-byte swizzle (layout type 2), descriptor version 1.
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
@@ -1138,6 +1136,194 @@ __global__ void __launch_bounds__(kCombineThreads) attention_combine_kernel(cons
     }
 }
 
+// The same for batches of several sequences.  The kernel is a chain of two dependent memory round
+// trips (partials in, O out) behind a
+// dependency wait, so it is laid out for latency: one flat index space over all sequences (no
+// pass per sequence), a piece of work = (row, 8 columns, one of 1, 2 or 4 shares of the partials)
+// so that a thread has at most four partials (eight loads) to fetch and they are all in flight
+// at once, the shares merged by shuffles, and few enough registers for four CTAs per SM, so
+// that even the largest trees are one resident round.
+constexpr int kCombineBatch = 4;  // partials a thread fetches at once
+
+template <int D>
+__global__ void __launch_bounds__(kCombineThreads, 4) attention_combine_flat_kernel(const AttnArgs a) {
+    __shared__ Sched sc;
+    __shared__ unsigned s_work0[kMaxBatchSmem + 1];  // first flat index of a sequence
+    __shared__ unsigned char s_shares[kMaxBatchSmem];
+    pdl_launch_dependents();
+    // A CTA past the last piece of work that the trees at hand could need has nothing to do.  It
+    // learns that from one load and leaves: it may have started only after the attention kernel
+    // ended, and whatever it does until it exits delays the next kernel in the stream.
+    {
+        const int b = threadIdx.x;  // the batch is at most the CTA's thread count
+        unsigned long long bound = 0;
+        if (b < a.batch) bound = 4ull * min(max(a.n_nodes[b], 0), a.max_tt) * a.Hq * (D / 8) + 4;
+        // (sum over the CTA's threads: every sequence's bound, four shares each)
+        __shared__ unsigned long long s_bound;
+        if (threadIdx.x == 0) s_bound = 0;
+        __syncthreads();
+        if (bound) atomicAdd(&s_bound, bound);
+        __syncthreads();
+        if (static_cast<unsigned long long>(blockIdx.x) * kCombineThreads >= s_bound) return;
+    }
+    // The work list is derived again from the step parameters (inputs of the attention kernel,
+    // complete before it ran), and the thread's first piece of work is located, before the wait
+    // for the attention kernel: all of this runs while that kernel drains.
+    build_sched(a, sc, threadIdx.x);  // ends with __syncthreads()
+    const unsigned G = static_cast<unsigned>(a.Hq / a.Hkv);
+    if (threadIdx.x < 32) {
+        // shares per piece of work and flat offsets (every sequence's range is a multiple of 4,
+        // so that the shares of a piece sit in adjacent, aligned lanes)
+        unsigned base = 0;
+        for (int b0 = 0; b0 < a.batch; b0 += 32) {
+            const int b = b0 + threadIdx.x;
+            unsigned mine = 0;
+            if (b < a.batch && sc.n[b] > 0) {
+                const int nfull = sc.nfull[b], nkey = sc.mp[b] - nfull;
+                const int parts = max(nfull > 0 && sc.s_row[b] > 1 ? sc.s_row[b] : 0, nkey > 0 ? 2 * sc.s_key[b] : 0);
+                const unsigned shares = parts <= kCombineBatch ? 1u : parts <= 2 * kCombineBatch ? 2u : 4u;
+                s_shares[b] = static_cast<unsigned char>(shares);
+                if (parts > 0) mine = (static_cast<unsigned>(sc.n[b]) * a.Hq * (D / 8) * shares + 3u) & ~3u;
+            }
+            unsigned incl = mine;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const unsigned v = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+                if (threadIdx.x >= d) incl += v;
+            }
+            if (b < a.batch) s_work0[b] = base + incl - mine;
+            base += __shfl_sync(0xFFFFFFFFu, incl, 31);
+        }
+        if (threadIdx.x == 0) s_work0[a.batch] = base;
+    }
+    __syncthreads();
+    const unsigned total = s_work0[a.batch];
+    const unsigned stride = gridDim.x * kCombineThreads;
+    bool waited = false;
+    // every lane of a warp goes round the same number of times (the merge is by shuffles)
+    for (unsigned w0 = blockIdx.x * kCombineThreads + (threadIdx.x & ~31u); w0 < total || !waited; w0 += stride) {
+        const unsigned w = w0 + (threadIdx.x & 31u);
+        // ---- this thread's piece of work ------------------------------------------------------
+        bool have = false;
+        int b = 0, n_parts = 0, splits = 0;
+        unsigned g = 0, c8 = 0, R = 0, share = 0, shares = 1;
+        bool key_mode = false;
+        int64_t item_first = 0;
+        if (w < total) {
+            int lo = 0, hi = a.batch;  // last sequence whose range starts at or before w
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (s_work0[mid] <= w) lo = mid; else hi = mid;
+            }
+            b = lo;
+            shares = s_shares[b];
+            const unsigned local = w - s_work0[b];
+            const unsigned piece = local / shares;
+            share = local - piece * shares;
+            const unsigned M = static_cast<unsigned>(sc.n[b]) * G;
+            const unsigned per_head = M * (D / 8);
+            if (piece < a.Hkv * per_head) {  // (the range is padded to a multiple of 4)
+                g = piece / per_head;
+                const unsigned rem = piece - g * per_head;
+                c8 = rem / M;
+                R = rem - c8 * M;
+                const int nfull = sc.nfull[b], s_row = sc.s_row[b];
+                const int pair = static_cast<int>(R / (kRowTiles * kBM));
+                key_mode = pair >= nfull;
+                splits = key_mode ? sc.s_key[b] : s_row;
+                if (key_mode || splits > 1) {  // otherwise the group wrote O directly
+                    const int row_items = nfull * s_row;
+                    item_first = sc.item0[b] + static_cast<int64_t>(g) * (row_items + (sc.mp[b] - nfull) * sc.s_key[b]) +
+                                 (key_mode ? row_items : pair * s_row);
+                    n_parts = key_mode ? 2 * splits : splits;
+                    have = true;
+                }
+            }
+        }
+        if (!waited) {
+            pdl_wait();  // the attention kernel has finished and its partials are visible
+            waited = true;
+        }
+        if (!__any_sync(0xFFFFFFFFu, have)) continue;
+
+        // ---- this share's partials: p = share, share + shares, ... ------------------------------
+        const unsigned row2 = R % (kRowTiles * kBM);
+        const unsigned mt = row2 / kBM, r = row2 % kBM;
+        float Mx = -INFINITY, den = 0.f;
+        float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        if (have) {
+#pragma unroll 1
+            for (int p0 = static_cast<int>(share); p0 < n_parts; p0 += kCombineBatch * static_cast<int>(shares)) {
+                float4 ml[kCombineBatch];
+                uint4 v[kCombineBatch];
+#pragma unroll
+                for (int u = 0; u < kCombineBatch; ++u) {
+                    const int p = min(p0 + u * static_cast<int>(shares), n_parts - 1);
+                    const int64_t slot = key_mode ? (item_first + (p >> 1)) * kRowTiles + (p & 1)
+                                                  : (item_first + p) * kRowTiles + mt;
+                    ml[u] = __ldcg(&a.part_ml[slot * kBM + r]);
+                    v[u] = __ldcg(a.part_o + (slot * (D / 8) + c8) * kBM + r);
+                }
+                float mx = Mx;
+#pragma unroll
+                for (int u = 0; u < kCombineBatch; ++u)
+                    if (p0 + u * static_cast<int>(shares) < n_parts) mx = fmaxf(mx, ml[u].x);
+                if (mx == -INFINITY) continue;
+                const float corr = ex2_approx(Mx - mx);  // 0 on the first batch
+                den *= corr;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc[e] *= corr;
+                Mx = mx;
+#pragma unroll
+                for (int u = 0; u < kCombineBatch; ++u) {
+                    if (p0 + u * static_cast<int>(shares) >= n_parts || ml[u].x == -INFINITY) continue;  // an empty partial holds no O
+                    const float wgt = ex2_approx(ml[u].x - Mx);
+                    den += ml[u].y * wgt;
+                    const float wo = ml[u].z * wgt;  // O_p = Ohat * l * row scale
+                    const uint32_t hw[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&hw[e]));
+                        acc[2 * e] += f.x * wo, acc[2 * e + 1] += f.y * wo;
+                    }
+                }
+            }
+        }
+        // ---- the shares of a piece sit in adjacent lanes: merge them (every lane takes part) ----
+#pragma unroll
+        for (unsigned d = 1; d < 4; d <<= 1) {
+            const float Mo = __shfl_xor_sync(0xFFFFFFFFu, Mx, d);
+            const float Mn = fmaxf(Mx, Mo);
+            const float sc_self = (Mx == -INFINITY) ? 0.f : ex2_approx(Mx - Mn);
+            const bool on = d < shares;
+            float dn = den * sc_self;
+            float ac[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) ac[e] = acc[e] * sc_self;
+            const float dno = __shfl_xor_sync(0xFFFFFFFFu, dn, d);
+            if (on) den = dn + dno, Mx = Mn;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const float o = __shfl_xor_sync(0xFFFFFFFFu, ac[e], d);
+                if (on) acc[e] = ac[e] + o;
+            }
+        }
+        if (have && share == 0) {
+            const float inv = 1.f / den;
+            const unsigned t = R / G, h = g * G + (R - t * G);
+            __nv_bfloat16* dst = a.o + ((static_cast<int64_t>(b) * a.max_tt + t) * a.Hq + h) * D + c8 * 8;
+            uint4 out;
+            out.x = pack_bf16(acc[0] * inv, acc[1] * inv);
+            out.y = pack_bf16(acc[2] * inv, acc[3] * inv);
+            out.z = pack_bf16(acc[4] * inv, acc[5] * inv);
+            out.w = pack_bf16(acc[6] * inv, acc[7] * inv);
+            *reinterpret_cast<uint4*>(dst) = out;
+            if (a.lse && c8 == 0)
+                a.lse[(static_cast<int64_t>(b) * a.max_tt + t) * a.Hq + h] = (Mx + log2f(den)) * 0.6931471805599453f;
+        }
+    }
+}
+
 // cuTensorMapEncodeTiled, resolved at run time so that the library has no link-time
 // dependency on the driver (it must load on a machine without one).
 using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -1196,29 +1382,24 @@ bool make_q_map(CUtensorMap* map, const void* basep, int D, int G, int Hkv, int 
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// Both kernels are launched with programmatic stream serialization: each starts while its
-// predecessor drains and waits (griddepcontrol.wait) before it touches global memory.
-template <typename Kernel, typename... Args>
-cudaError_t launch_pdl(Kernel kernel, int grid, int block, size_t smem, cudaStream_t st, Args... args) {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(grid), cfg.blockDim = dim3(block), cfg.dynamicSmemBytes = smem, cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr, cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, kernel, args...);
-}
-
 template <int D>
 cudaError_t launch_for_dim(const resps_ctx* ctx, const AttnArgs& a, const CUtensorMap& mk, const CUtensorMap& mv,
                            const CUtensorMap& mq, cudaStream_t st) {
-    cudaError_t e = launch_pdl(tree_attention_kernel<D>, ctx->ws.attn_grid, kAttnThreads, Smem<D>::kBytes, st, a, mk,
+    cudaError_t e = launch_pdl(tree_attention_kernel<D>, dim3(ctx->ws.attn_grid), dim3(kAttnThreads), Smem<D>::kBytes, st, a, mk,
                                mv, mq);
     if (e != cudaSuccess) return e;
-    // one resident round of CTAs at most, and no more than the largest trees could use
-    const long long most = (1ll * a.batch * a.max_tt * a.Hq * (D / 8) + kCombineThreads - 1) / kCombineThreads;
+    // One resident round of CTAs at most, and no more than the largest trees could use.  A single
+    // sequence (or two) is served best by few, register-heavy threads that all start under the
+    // attention kernel's tail; a batch by the flat index space and four CTAs per SM.
+    const long long pieces = 1ll * a.max_tt * a.Hq * (D / 8);
+    if (a.batch > 2) {
+        const long long most = (4ll * a.batch * (pieces + 1) + kCombineThreads - 1) / kCombineThreads;
+        const int grid = static_cast<int>(std::min<long long>(ctx->ws.attn_combine_flat_grid, std::max<long long>(most, 1)));
+        return launch_pdl(attention_combine_flat_kernel<D>, dim3(grid), dim3(kCombineThreads), 0, st, a);
+    }
+    const long long most = (a.batch * pieces + kCombineThreads - 1) / kCombineThreads;
     const int grid = static_cast<int>(std::min<long long>(ctx->ws.attn_combine_grid, std::max<long long>(most, 1)));
-    return launch_pdl(attention_combine_kernel<D>, grid, kCombineThreads, 0, st, a);
+    return launch_pdl(attention_combine_kernel<D>, dim3(grid), dim3(kCombineThreads), 0, st, a);
 }
 
 }  // namespace
@@ -1237,6 +1418,11 @@ cudaError_t attention_setup(resps_ctx* ctx) {
             : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, attention_combine_kernel<64>, kCombineThreads, 0);
     if (e != cudaSuccess) return e;
     ctx->ws.attn_combine_grid = ctx->sm_count * std::max(per_sm, 1);
+    e = (ctx->shape.head_dim == 128)
+            ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, attention_combine_flat_kernel<128>, kCombineThreads, 0)
+            : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, attention_combine_flat_kernel<64>, kCombineThreads, 0);
+    if (e != cudaSuccess) return e;
+    ctx->ws.attn_combine_flat_grid = ctx->sm_count * std::max(per_sm, 1);
     return cudaSuccess;
 }
 

@@ -31,6 +31,7 @@ struct Workspace {
     // attention
     int attn_grid = 0;          // persistent CTAs (one per SM)
     int attn_combine_grid = 0;  // CTAs of the partial-combine kernel
+    int attn_combine_flat_grid = 0;  // ... of its variant for batches
     int attn_min_tiles = 0;     // smallest key-tile count a split is given
     int attn_max_items = 0;     // partial slots
     __half* attn_part_o = nullptr;  // [items][item rows][D] fp16
@@ -82,6 +83,18 @@ cudaError_t launch_tree_attention(const resps_ctx* ctx, const resps_step* d_step
                                   int64_t stride_head, int64_t stride_tok, int64_t capacity,
                                   const uint64_t* mask, float scale, cudaStream_t st);
 cudaError_t attention_setup(resps_ctx* ctx);  // one-time function attributes
+
+// Launch with programmatic stream serialization (see pdl_wait above).
+template <typename Kernel, typename... Args>
+cudaError_t launch_pdl(Kernel kernel, dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid, cfg.blockDim = block, cfg.dynamicSmemBytes = smem, cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr, cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
 cudaError_t tree_setup(resps_ctx* ctx);
 cudaError_t scan_setup(resps_ctx* ctx);
 int tree_candidate_limit();
@@ -109,6 +122,13 @@ __device__ __forceinline__ float key_val(unsigned long long k) {
 __device__ __forceinline__ int key_id(unsigned long long k) {
     return static_cast<int>(0xFFFFFFFFu - static_cast<uint32_t>(k & 0xFFFFFFFFull));
 }
+
+// Programmatic dependent launch.  Every kernel of the library is launched so that it may start
+// while its predecessor in the stream drains; it waits here before its first access to global
+// memory and lets its own successor start right away (the successor waits in the same way, and
+// the wait returns only when this grid has completed and flushed its writes).
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 __device__ __forceinline__ float ex2_approx(float x) {
     float y;

@@ -80,6 +80,8 @@ __device__ __forceinline__ float max3f(float a, float b, float c) {
 // (max, sum 2^(y - max)) reduced over the CTA.
 template <bool VEC>
 __global__ void __launch_bounds__(kScanThreads, 4) row_scan_kernel(const ScanArgs a) {
+    pdl_wait();  // the kernel before this one in the stream has completed
+    pdl_launch_dependents();
     extern __shared__ unsigned long long s_keys[];  // max(128 max_k, splits max_k) keys
     __shared__ unsigned long long s_quad[kQuads];
     __shared__ unsigned long long s_tau;
@@ -300,6 +302,8 @@ __device__ __forceinline__ bool consumer_any(bool pred) {  // barrier over the c
 }
 
 __global__ void __launch_bounds__(kStreamThreads, 2) row_scan_stream_kernel(const ScanArgs a) {
+    pdl_wait();  // the kernel before this one in the stream has completed
+    pdl_launch_dependents();
     extern __shared__ __align__(128) unsigned char s_raw[];
     float* s_stage = reinterpret_cast<float*>(s_raw);                                    // [3][8192]
     unsigned long long* s_keys =
@@ -587,6 +591,8 @@ struct ArgmaxArgs {
 
 template <bool VEC>
 __global__ void __launch_bounds__(kScanThreads, 4) row_argmax_kernel(const ArgmaxArgs a) {
+    pdl_wait();  // the kernel before this one in the stream has completed
+    pdl_launch_dependents();
     const int b = blockIdx.z, r = blockIdx.y, sp = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int n = min(max(a.n_nodes[b], 0), a.max_tt);
@@ -712,10 +718,10 @@ cudaError_t launch_row_scan(const resps_ctx* ctx, const resps_step* d_steps, int
         a.cps = (w.scan_splits + slices0 - 1) / slices0;
         a.slices = (w.scan_splits + a.cps - 1) / a.cps;
         dim3 grid(a.slices, rows, batch);
-        row_scan_stream_kernel<<<grid, kStreamThreads, stream_smem_bytes(ctx->shape.max_k, a.slices), st>>>(a);
+        return launch_pdl(row_scan_stream_kernel, grid, dim3(kStreamThreads), stream_smem_bytes(ctx->shape.max_k, a.slices), st, a);
     } else {
         dim3 grid(w.scan_splits, rows, batch);
-        row_scan_kernel<false><<<grid, kScanThreads, smem, st>>>(a);
+        return launch_pdl(row_scan_kernel<false>, grid, dim3(kScanThreads), smem, st, a);
     }
     return cudaGetLastError();
 }
@@ -733,9 +739,9 @@ cudaError_t launch_row_argmax(const resps_ctx* ctx, const int32_t* d_n_nodes, in
     a.part = w.amax_part, a.counter = w.amax_counter, a.out = argmax_out;
     dim3 grid(w.scan_splits, ctx->shape.max_tt, batch);
     if (vec_ok(logits, ld_b, ld_row, 0, a.vocab, a.chunk))
-        row_argmax_kernel<true><<<grid, kScanThreads, 0, st>>>(a);
+        return launch_pdl(row_argmax_kernel<true>, grid, dim3(kScanThreads), 0, st, a);
     else
-        row_argmax_kernel<false><<<grid, kScanThreads, 0, st>>>(a);
+        return launch_pdl(row_argmax_kernel<false>, grid, dim3(kScanThreads), 0, st, a);
     return cudaGetLastError();
 }
 

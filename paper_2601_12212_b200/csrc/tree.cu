@@ -81,6 +81,8 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* s_warp, int& tot
 }
 
 __global__ void __launch_bounds__(kTreeThreads, 1) tree_build_kernel(const TreeArgs a) {
+    pdl_wait();  // the kernel before this one in the stream has completed
+    pdl_launch_dependents();
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int b = blockIdx.x, tid = threadIdx.x;
     const StepDims sd = clamp_step(a.steps[b], a.n_levels, a.n_slots, a.max_tt, a.max_k, a.vocab);
@@ -284,8 +286,7 @@ cudaError_t launch_tree_build(const resps_ctx* ctx, const resps_step* d_steps, i
     a.status = ctx->ws.status;
     a.cand_cap = s.max_k + (s.max_depth - 1) * s.max_k * s.max_k;
     const size_t smem = tree_smem_bytes(a.cand_cap);
-    tree_build_kernel<<<batch, kTreeThreads, smem, st>>>(a);
-    return cudaGetLastError();
+    return launch_pdl(tree_build_kernel, dim3(batch), dim3(kTreeThreads), smem, st, a);
 }
 
 // Largest k + (d-1)k^2 the shared-memory arrays can hold.
