@@ -315,6 +315,22 @@ def attention_algorithmic_bytes(w, L, n):
     return 2 * (L + n) * w.n_kv_heads * w.head_dim * 2 + 2 * n * w.n_q_heads * w.head_dim * 2
 
 
+def max_over_ranks(values, world, device):
+    """Device times of a multi-GPU run are reported as the maximum over the ranks (replicas run
+    side by side, the job is as slow as its slowest rank); a single rank keeps its own."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(values, dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t.cpu()]
+
+
+def whole_job_value(t_step_us, world):
+    """us per speculative step of the whole job: `world` replicas finish one step each in t_step_us."""
+    return t_step_us / world
+
+
 def run_ours(args, w):
     import torch
     import torch.distributed as dist
@@ -406,10 +422,7 @@ def run_ours(args, w):
             torch.cuda.synchronize()
             phases[name + "_us"] = a.elapsed_time(b) * 1e3 / reps
 
-    times = torch.tensor([t_step, t_attn, t_e2e], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    t_step, t_attn, t_e2e = [float(x) for x in times.cpu()]
+    t_step, t_attn, t_e2e = max_over_ranks([t_step, t_attn, t_e2e], world, "cuda")
     status = dw.ctx.status()
     if rank != 0:
         if world > 1:
@@ -439,7 +452,7 @@ def run_ours(args, w):
                          "verify": parts["verify"] * 1e6, "compact_per_layer": parts["compact_per_layer"] * 1e6}}
 
     line = {
-        "metric": METRIC, "value": t_step / world, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+        "metric": METRIC, "value": whole_job_value(t_step, world), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": t_step / 1e3, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16 attention (fp32 accumulate), fp32 logits", "data": "synthetic (seeded)",
         "config": workload_config(w, {
