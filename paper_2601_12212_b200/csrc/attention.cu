@@ -1094,7 +1094,7 @@ __global__ void __launch_bounds__(kCombineThreads) attention_combine_kernel(cons
                 const int p = min(p0 + u, n_parts - 1);
                 const int64_t slot = key_mode ? (item_first + (p >> 1)) * kRowTiles + (p & 1)
                                               : (item_first + p) * kRowTiles + mt;
-                ml[u] = __ldcg(&a.part_ml[slot * kBM + r]);
+                ml[u] = a.part_ml[slot * kBM + r];  // shared by the 16 column pieces of a row: through L1
                 v[u] = __ldcg(a.part_o + (slot * (D / 8) + c8) * kBM + r);
             }
             float mx = Mx;
@@ -1261,7 +1261,7 @@ __global__ void __launch_bounds__(kCombineThreads, 4) attention_combine_flat_ker
                     const int p = min(p0 + u * static_cast<int>(shares), n_parts - 1);
                     const int64_t slot = key_mode ? (item_first + (p >> 1)) * kRowTiles + (p & 1)
                                                   : (item_first + p) * kRowTiles + mt;
-                    ml[u] = __ldcg(&a.part_ml[slot * kBM + r]);
+                    ml[u] = a.part_ml[slot * kBM + r];  // shared by the 16 column pieces of a row: through L1
                     v[u] = __ldcg(a.part_o + (slot * (D / 8) + c8) * kBM + r);
                 }
                 float mx = Mx;
