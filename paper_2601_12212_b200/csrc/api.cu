@@ -9,6 +9,7 @@
 namespace resps {
 int scan_chunk_max();
 int attention_item_rows();
+int attention_max_rounds();
 int attention_max_batch();
 }  // namespace resps
 
@@ -113,8 +114,9 @@ int resps_create(resps_ctx** out, const resps_shape* shape) {
     w.attn_combine_grid = c->sm_count * 4;
     w.attn_min_tiles = 2;
     if (const char* e = std::getenv("RESPS_ATTN_MIN_TILES")) w.attn_min_tiles = std::max(1, std::atoi(e));
+    if (const char* e = std::getenv("RESPS_ATTN_ROUNDS")) w.attn_rounds = std::max(0, std::atoi(e));
     w.attn_max_groups = s.max_batch * s.n_kv_heads * ((s.max_tt * G + item_rows - 1) / item_rows);
-    w.attn_max_items = w.attn_grid + w.attn_max_groups;
+    w.attn_max_items = resps::attention_max_rounds() * w.attn_grid + w.attn_max_groups;
 
     Carver dry;
     carve(c, dry);

@@ -56,6 +56,7 @@ constexpr int kSyncThreads = 320;  // softmax warps + the MMA warps meet at the 
 constexpr int kMaxBatchSmem = 256;
 constexpr int kTmemCols = 512;
 constexpr int kCombineThreads = 256;
+constexpr int kMaxRounds = 4;      // rounds of items the work list may plan for (long sequences only)
 constexpr uint32_t kWaitLimitCycles = 0x70000000u;  // bounded waits give up after ~1 s of SM clocks
 constexpr float kRescaleSlack = 8.0f;  // O is rescaled only when the running max grows by > 2^8
 constexpr unsigned kFull = 0xFFFFFFFFu;
@@ -80,6 +81,7 @@ struct AttnArgs {
     int max_items;
     int sched_grid;   // CTAs of the attention grid (the work list is balanced for it)
     int min_tiles;    // smallest key-tile count worth a split of its own
+    int rounds;       // 0: the work list chooses its number of rounds; 1..kMaxRounds: as told (tests)
     int q_by_tma;     // 1: Q tiles come by TMA (128 % (Hq/Hkv) == 0), 0: by plain loads
     int32_t* status;
 };
@@ -136,24 +138,37 @@ __device__ __forceinline__ void build_sched(const AttnArgs& a, Sched& sc, int ti
             }
         }
         cost = __reduce_add_sync(0xFFFFFFFFu, min(cost, 1u << 26));
-        int T = max(ceil_div(static_cast<int>(cost), a.sched_grid), 1);
-        int s_row0 = 0, s_key0 = 0;
+        // Smallest T (in steps of T/16) for which the items fit `rounds` rounds of the grid.  One round
+        // is the rule.  With long sequences and few groups it can leave CTAs idle (40 groups of 3 splits
+        // are 120 items for 148 CTAs); two to four rounds of shorter items then fill the grid better.
+        // An item more costs a CTA about kItemUnits units (its epilogue and the start of the next), so
+        // more rounds are only looked at when items are long, where the time of this search does not
+        // matter either.
+        constexpr int kItemUnits = 8;
+        const int forced = min(a.rounds, kMaxRounds);
+        int T = 1, best = 0x7FFFFFFF;
 #pragma unroll 1
-        for (int tries = 0; tries < 24; ++tries) {
-            const int t_row = max((T + 1) >> 1, mt), t_key = max(T, mt);
-            s_row0 = ceil_div(kt0, t_row), s_key0 = ceil_div(kt0, t_key);
-            unsigned cnt = a.Hkv * (nfull0 * s_row0 + nkey0 * s_key0);
+        for (int rounds = max(forced, 1); rounds <= (forced > 0 ? forced : kMaxRounds); ++rounds) {
+            int Tr = max(ceil_div(static_cast<int>(cost), rounds * a.sched_grid), 1);
 #pragma unroll 1
-            for (int i = 1; i < nblk; ++i) {
-                const int b = i * 32 + tid;
-                if (b < a.batch)
-                    cnt += a.Hkv * (sc.nfull[b] * ceil_div(sc.kt[b], t_row) +
-                                    (sc.mp[b] - sc.nfull[b]) * ceil_div(sc.kt[b], t_key));
+            for (int tries = 0; tries < 24; ++tries) {
+                const int t_row = max((Tr + 1) >> 1, mt), t_key = max(Tr, mt);
+                unsigned cnt = a.Hkv * (nfull0 * ceil_div(kt0, t_row) + nkey0 * ceil_div(kt0, t_key));
+#pragma unroll 1
+                for (int i = 1; i < nblk; ++i) {
+                    const int b = i * 32 + tid;
+                    if (b < a.batch)
+                        cnt += a.Hkv * (sc.nfull[b] * ceil_div(sc.kt[b], t_row) +
+                                        (sc.mp[b] - sc.nfull[b]) * ceil_div(sc.kt[b], t_key));
+                }
+                cnt = __reduce_add_sync(0xFFFFFFFFu, min(cnt, 1u << 20));
+                if (cnt <= static_cast<unsigned>(rounds * a.sched_grid)) break;
+                Tr += max(1, Tr >> 4);
             }
-            cnt = __reduce_add_sync(0xFFFFFFFFu, min(cnt, 1u << 20));
-            if (cnt <= static_cast<unsigned>(a.sched_grid)) break;
-            T += max(1, T >> 4);
+            if (rounds * (Tr + kItemUnits) < best) best = rounds * (Tr + kItemUnits), T = Tr;
+            if (forced == 0 && Tr < 8 * kItemUnits) break;  // short items: no further rounds
         }
+        const int s_row0 = ceil_div(kt0, max((T + 1) >> 1, mt)), s_key0 = ceil_div(kt0, max(T, mt));
         const int t_row = max((T + 1) >> 1, mt), t_key = max(T, mt);
         int base = 0;
 #pragma unroll 1
@@ -1442,6 +1457,7 @@ cudaError_t launch_tree_attention(const resps_ctx* ctx, const resps_step* d_step
     a.part_o = reinterpret_cast<uint4*>(ctx->ws.attn_part_o), a.part_ml = ctx->ws.attn_part_ml;
     a.max_items = ctx->ws.attn_max_items, a.sched_grid = ctx->ws.attn_grid;
     a.min_tiles = ctx->ws.attn_min_tiles, a.status = ctx->ws.status;
+    a.rounds = ctx->ws.attn_rounds;
     const int D = ctx->shape.head_dim;
     const int G = a.Hq / a.Hkv;
     a.q_by_tma = (G <= kBM && kBM % G == 0) ? 1 : 0;
@@ -1458,6 +1474,7 @@ cudaError_t launch_tree_attention(const resps_ctx* ctx, const resps_step* d_step
 }
 
 int attention_item_rows() { return kRowTiles * kBM; }
+int attention_max_rounds() { return kMaxRounds; }
 int attention_max_batch() { return kMaxBatchSmem; }
 
 }  // namespace resps

@@ -194,6 +194,15 @@ def test_attention_large_values_survive_the_split_partials(n, Hq, Hkv):
     _attention_case(n, Hq, Hkv, 128, 5000, cap=5200, seed=11, v_scale=3.0e5)
 
 
+@pytest.mark.parametrize("rounds", [2, 3, 4])
+def test_attention_work_list_of_several_rounds(rounds, monkeypatch):
+    """Long sequences may be cut into more items than CTAs (a CTA then takes several, one after the
+    other); the environment variable forces that on a problem small enough for the oracle."""
+    monkeypatch.setenv("RESPS_ATTN_ROUNDS", str(rounds))
+    _attention_case(40, 16, 4, 128, 9000, cap=9300, seed=rounds)
+    _attention_case([9, 70, 33], 8, 8, 128, [5000, 2500, 7777], cap=8192, seed=rounds, B=3)
+
+
 def test_attention_chain_mask_is_causal():
     n = 100
     _attention_case(n, 8, 2, 128, 50, cap=300, parent=list(range(-1, n - 1)), poison=True)
