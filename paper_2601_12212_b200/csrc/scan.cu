@@ -711,8 +711,10 @@ cudaError_t launch_row_scan(const resps_ctx* ctx, const resps_step* d_steps, int
     a.slices = w.scan_splits, a.cps = 1;
     const size_t smem = sizeof(unsigned long long) * ctx->shape.max_k * max(kQuadElems, w.scan_splits);
     if (vec_ok(logits, ld_b, ld_level, ld_row, a.vocab, a.chunk) && w.scan_chunk == kScanChunkMax) {
-        // enough slices for two CTAs per SM over the largest row count, each several chunks long
-        int want = (2 * ctx->sm_count + rows * batch - 1) / (rows * batch);
+        // Slices per row: two CTAs fit an SM, and a slice's first chunk costs about three later ones (the
+        // threshold has to be found), so a row is cut only as far as all CTAs still run at once; with
+        // more rows than that, one slice per row (measured at 712 rows: 108 us in one slice, 119 in two).
+        int want = max(1, 2 * ctx->sm_count / max(rows * batch, 1));
         if (w.scan_slices_hint > 0) want = w.scan_slices_hint;
         const int slices0 = max(1, min(w.scan_splits, want));
         a.cps = (w.scan_splits + slices0 - 1) / slices0;
