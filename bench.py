@@ -488,7 +488,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--config", type=int, default=2, help="1-based index into BASELINE.json configs")
+    ap.add_argument("--config", type=int, default=2, help="1-based index of the synthetic workload (synth.WORKLOADS)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     args = ap.parse_args()
     w = synth.WORKLOADS[args.config]

@@ -21,7 +21,7 @@
 //   compaction     : gather definition, identity path is a no-op
 //   whole step     : greedy speculative decoding over a tiny random transformer
 //                    reproduces greedy autoregressive decoding token for token
-// Parity unpinned (conventions of this build that no external value fixes):
+// Parity unpinned (conventions of this implementation that no external value fixes):
 //   the tie-break orders (equal logits -> lower token id, equal scores -> lower
 //   candidate index), the node order (ascending candidate index), the retrieve
 //   row order, and reading "depth d" as d draft levels.

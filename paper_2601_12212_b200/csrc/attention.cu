@@ -115,7 +115,7 @@ __device__ __forceinline__ void build_sched(const AttnArgs& a, Sched& sc, int ti
         const int G = a.Hq / a.Hkv;
         const int nblk = (a.batch + 31) >> 5;
         const int mt = max(a.min_tiles, 1);
-        // round 0 of the lane stays in registers (the only round up to 32 sequences)
+        // the lane's first sequence stays in registers (its only one up to 32 sequences)
         int kt0 = 0, nfull0 = 0, nkey0 = 0;
         unsigned cost = 0;  // saturates: it only seeds the search below
 #pragma unroll 1

@@ -3,7 +3,7 @@
     python -m paper_2601_12212_b200.microbench attention [2 3 4 5 long]
     python -m paper_2601_12212_b200.microbench vocab     [2 3 4 5]
 
-The numbers name the BASELINE workload whose shape is used.  `attention` times
+The numbers name the synthetic workload (synth.WORKLOADS) whose shape is used.  `attention` times
 resps_tree_attention over distinct KV-cache layers; `vocab` times resps_tree_expand (row scan +
 tree build) and resps_verify_accept (arg-max + accept walk) over a pool of distinct logit sets.
 Values are random (timing only); parity is the business of tests/.
@@ -126,7 +126,7 @@ def main(argv):
             Ls = [random.randint(1024, 8192) for _ in range(8)]
             ns = [random.choice([16, 32, 37, 48, 53, 60, 69, 80]) for _ in range(8)]
             attention("cfg5 ragged x8 32q/8kv", 8, 32, 8, 128, Ls, ns, 12288, 4)
-        if "long" in which:  # not a BASELINE workload: the HBM-bound shape of workload 3 at a long context
+        if "long" in which:  # not one of the workloads: the HBM-bound shape of workload 3 at a long context
             attention("MHA 40 heads L=32768 n=48", 1, 40, 40, 128, [32768], [48], 32768 + 128, 2)
             attention("32q/8kv L=65536 n=28", 1, 32, 8, 128, [65536], [28], 65536 + 128, 2)
     elif what == "vocab":
