@@ -115,6 +115,7 @@ int resps_create(resps_ctx** out, const resps_shape* shape) {
     w.attn_min_tiles = 2;
     if (const char* e = std::getenv("RESPS_ATTN_MIN_TILES")) w.attn_min_tiles = std::max(1, std::atoi(e));
     if (const char* e = std::getenv("RESPS_ATTN_ROUNDS")) w.attn_rounds = std::max(0, std::atoi(e));
+    if (const char* e = std::getenv("RESPS_ATTN_STAGGER")) w.attn_stagger = std::min(100000, std::max(0, std::atoi(e)));
     w.attn_max_groups = s.max_batch * s.n_kv_heads * ((s.max_tt * G + item_rows - 1) / item_rows);
     w.attn_max_items = resps::attention_max_rounds() * w.attn_grid + w.attn_max_groups;
 

@@ -82,6 +82,7 @@ struct AttnArgs {
     int sched_grid;   // CTAs of the attention grid (the work list is balanced for it)
     int min_tiles;    // smallest key-tile count worth a split of its own
     int rounds;       // 0: the work list chooses its number of rounds; 1..kMaxRounds: as told (tests)
+    int stagger;      // cycles lane 1 starts behind lane 0 in row mode
     int q_by_tma;     // 1: Q tiles come by TMA (128 % (Hq/Hkv) == 0), 0: by plain loads
     int32_t* status;
 };
@@ -636,6 +637,13 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
             const uint64_t qdesc = qdesc0 + static_cast<uint64_t>((row_mode ? x : 0) * (S::kQTile >> 4));
             alive = warp_wait(bar(bar_qfull()), items_run & 1u, abort_flag);
             tc_fence_after();
+            if (row_mode && x == 1) {
+                // Lane 1 starts half a tile period behind lane 0: the lanes' bursts of MMAs (P V of one
+                // tile, Q K^T of the tile after next) then take turns on the tensor pipe instead of
+                // queueing behind each other, which is what decides when a lane gets its next S.
+                const long long t_go = clock64() + a.stagger;
+                while (clock64() < t_go) {}
+            }
             bool have_prev = false, first_pv = true;
             uint32_t prev_kt = 0, prev_j = 0;
             // In key mode a tile belongs to one lane alone: its owner releases the stage for both.
@@ -1458,6 +1466,7 @@ cudaError_t launch_tree_attention(const resps_ctx* ctx, const resps_step* d_step
     a.max_items = ctx->ws.attn_max_items, a.sched_grid = ctx->ws.attn_grid;
     a.min_tiles = ctx->ws.attn_min_tiles, a.status = ctx->ws.status;
     a.rounds = ctx->ws.attn_rounds;
+    a.stagger = ctx->ws.attn_stagger;
     const int D = ctx->shape.head_dim;
     const int G = a.Hq / a.Hkv;
     a.q_by_tma = (G <= kBM && kBM % G == 0) ? 1 : 0;

@@ -33,6 +33,7 @@ struct Workspace {
     int attn_combine_grid = 0;  // CTAs of the partial-combine kernel
     int attn_combine_flat_grid = 0;  // ... of its variant for batches
     int attn_min_tiles = 0;     // smallest key-tile count a split is given
+    int attn_stagger = 1000;    // cycles lane 1 starts behind lane 0 (RESPS_ATTN_STAGGER)
     int attn_rounds = 0;        // 0: chosen by the work list; else forced (RESPS_ATTN_ROUNDS, for tests)
     int attn_max_items = 0;     // partial slots
     __half* attn_part_o = nullptr;  // [items][item rows][D] fp16
