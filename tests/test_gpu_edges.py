@@ -257,6 +257,17 @@ def test_attention_ragged_batch():
     _attention_case([5, 128, 33, 1], 16, 4, 128, [900, 10, 4000, 123], cap=4200, B=4, poison=True)
 
 
+def test_attention_batch_of_more_than_a_warp_of_sequences():
+    """The work list is built by one warp, a lane per sequence, in rounds of 32: 70 sequences of mixed
+    sizes go through three rounds and through the flat combine."""
+    rng = np.random.default_rng(3)
+    B = 70
+    ns = [int(x) for x in rng.choice([1, 2, 7, 20, 33], size=B)]
+    ns[0], ns[31], ns[32], ns[69] = 20, 33, 7, 1
+    Ls = [int(x) for x in rng.integers(0, 700, size=B)]
+    _attention_case(ns, 8, 2, 64, Ls, cap=800, B=B, max_tt=40, seed=9)
+
+
 def test_attention_overflowing_sequence_is_skipped_and_flagged():
     oracle, binding, synth = _imports()
     ctx = binding.Context(4, 1, 64, 100, max_batch=2, max_tt=16, max_k=4, max_depth=4)
