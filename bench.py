@@ -34,7 +34,7 @@ UNIT = "us/step"
 NOMINAL_HBM_GBS = 8000.0
 # DRAM bytes of one tree_attention_kernel launch on the benchmarked workload, from the ncu capture
 # summarised in profiles/tree_attention_cfg2_ncu.md (set to None when the kernel changes).
-ATTENTION_TRAFFIC_BYTES = 5017856
+ATTENTION_TRAFFIC_BYTES = 5018624
 
 
 def measured_peaks():
