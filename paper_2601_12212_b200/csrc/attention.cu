@@ -7,7 +7,7 @@
 // so that Q K^T and P V are dense contractions: tcgen05.mma with the fp32
 // accumulators (S and O) in tensor memory.  K/V tiles of 64 keys are staged by TMA
 // (cp.async.bulk.tensor, one elected thread) into 128-byte-swizzled shared memory
-// through a 4-deep mbarrier ring, Q tiles likewise (prefetched for the next item).
+// through mbarrier rings (four K stages, five V stages), Q tiles likewise (prefetched for the next item).
 //
 // A CTA runs two symmetric lanes.  A lane is an MMA-issuing warp, a softmax warpgroup
 // (one TMEM lane = one query row per thread) and a quarter of tensor memory (two S/P
@@ -43,7 +43,8 @@ namespace {
 
 constexpr int kBM = 128;           // rows per row tile (one TMEM lane each)
 constexpr int kBN = 64;            // keys per tile
-constexpr int kStages = 4;         // K/V ring depth
+constexpr int kStagesK = 4;        // K ring depth
+constexpr int kStagesV = 5;        // V ring depth (a V tile is held until its P V, a K tile only until its Q K^T)
 constexpr int kRowTiles = 2;       // row tiles per item
 constexpr int kSoftmaxThreads = 256;
 constexpr int kProducerWarp = 8;   // K and Q tiles
@@ -419,9 +420,9 @@ struct Smem {
     static constexpr int kKVTile = kPanels * kKVPanel;
     static constexpr int kOffQ = 0;
     static constexpr int kOffK = kOffQ + kRowTiles * kQTile;
-    static constexpr int kOffV = kOffK + kStages * kKVTile;
-    static constexpr int kOffBar = kOffV + kStages * kKVTile;
-    static constexpr int kNumBars = 4 * kStages + 1 + kRowTiles * 5 + 2;
+    static constexpr int kOffV = kOffK + kStagesK * kKVTile;
+    static constexpr int kOffBar = kOffV + kStagesV * kKVTile;
+    static constexpr int kNumBars = 2 * (kStagesK + kStagesV) + 1 + kRowTiles * 5 + 2;
     static constexpr int kOffMisc = kOffBar + 8 * 32;
     static constexpr int kUsed = kOffMisc + 64 + 1024;       // + slack to align the base to 1024
     // Never less than 120 KB, more than half of an SM's shared memory: one CTA per SM, so the
@@ -433,12 +434,12 @@ struct Smem {
 
 // barrier indices
 __device__ __forceinline__ constexpr int bar_kfull(int s) { return s; }
-__device__ __forceinline__ constexpr int bar_vfull(int s) { return kStages + s; }
+__device__ __forceinline__ constexpr int bar_vfull(int s) { return kStagesK + s; }
 // K and V stages are released separately: a K tile is dead once its Q K^T has completed, long
 // before the P V of the same tile, and the next K can be on its way meanwhile.
-__device__ __forceinline__ constexpr int bar_kempty(int s) { return 2 * kStages + s; }
-__device__ __forceinline__ constexpr int bar_vempty(int s) { return 3 * kStages + s; }
-constexpr int kBar0 = 4 * kStages;  // first barrier after the ring's
+__device__ __forceinline__ constexpr int bar_kempty(int s) { return kStagesK + kStagesV + s; }
+__device__ __forceinline__ constexpr int bar_vempty(int s) { return 2 * kStagesK + kStagesV + s; }
+constexpr int kBar0 = 2 * (kStagesK + kStagesV);  // first barrier after the ring's
 __device__ __forceinline__ constexpr int bar_qfull() { return kBar0; }
 // Lane m's S and P share a TMEM buffer (its j-th tile uses buffer j & 1) and each buffer has its own pair of
 // barriers: a buffer's next phase cannot complete before the other side has observed the
@@ -470,10 +471,12 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
     // ---- one-time set-up ---------------------------------------------------------------
     if (tid == 0) {
         *abort_flag = 0;
-        for (int s = 0; s < kStages; ++s) {
+        for (int s = 0; s < kStagesK; ++s) {
             mbar_init(bar(bar_kfull(s)), 1);
-            mbar_init(bar(bar_vfull(s)), 1);
             mbar_init(bar(bar_kempty(s)), 2);  // one arrival per lane (two from the owner in key mode)
+        }
+        for (int s = 0; s < kStagesV; ++s) {
+            mbar_init(bar(bar_vfull(s)), 1);
             mbar_init(bar(bar_vempty(s)), 2);
         }
         mbar_init(bar(bar_qfull()), a.q_by_tma ? 1 : kSoftmaxThreads);
@@ -554,11 +557,11 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
             for (int item = blockIdx.x; item < total_items && alive; item += gridDim.x, ++li) {
                 const Item it = get_item(item, li);
                 for (int t = it.t_begin; t < it.t_end; ++t, ++kt_run) {
-                    const int s = kt_run % kStages;
+                    const int s = kt_run % kStagesK;
                     if (kt_run > 0) {  // the CTA's very first tile went out during the set-up
                         // the first use of a stage finds it free
-                        if (kt_run >= kStages &&
-                            !mbar_wait(bar(bar_kempty(s)), ((kt_run / kStages) & 1u) ^ 1u, abort_flag)) {
+                        if (kt_run >= kStagesK &&
+                            !mbar_wait(bar(bar_kempty(s)), ((kt_run / kStagesK) & 1u) ^ 1u, abort_flag)) {
                             alive = false;
                             break;
                         }
@@ -586,8 +589,8 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
             // Drain: every copy this thread issued has landed before the CTA may exit.
             bool landed = !(a.q_by_tma && items_run > 0) || mbar_wait(bar(bar_qfull()), (items_run - 1u) & 1u, abort_flag);
             const uint32_t issued = kt_run;
-            for (uint32_t u = (issued > kStages ? issued - kStages : 0u); u < issued && landed; ++u)
-                landed = mbar_wait(bar(bar_kfull(u % kStages)), (u / kStages) & 1u, abort_flag);
+            for (uint32_t u = (issued > kStagesK ? issued - kStagesK : 0u); u < issued && landed; ++u)
+                landed = mbar_wait(bar(bar_kfull(u % kStagesK)), (u / kStagesK) & 1u, abort_flag);
             alive = alive && landed;
         }
     } else if (warp == kVProducerWarp) {
@@ -597,10 +600,10 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
             for (int item = blockIdx.x; item < total_items && alive; item += gridDim.x, ++li) {
                 const Item it = get_item(item, li);
                 for (int t = it.t_begin; t < it.t_end; ++t, ++kt_run) {
-                    const int s = kt_run % kStages;
+                    const int s = kt_run % kStagesV;
                     if (kt_run == 0) continue;  // went out during the set-up
-                    if (kt_run >= kStages &&
-                        !mbar_wait(bar(bar_vempty(s)), ((kt_run / kStages) & 1u) ^ 1u, abort_flag)) {
+                    if (kt_run >= kStagesV &&
+                        !mbar_wait(bar(bar_vempty(s)), ((kt_run / kStagesV) & 1u) ^ 1u, abort_flag)) {
                         alive = false;
                         break;
                     }
@@ -611,8 +614,8 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
             }
             const uint32_t issued = kt_run;
             bool landed = true;
-            for (uint32_t u = (issued > kStages ? issued - kStages : 0u); u < issued && landed; ++u)
-                landed = mbar_wait(bar(bar_vfull(u % kStages)), (u / kStages) & 1u, abort_flag);
+            for (uint32_t u = (issued > kStagesV ? issued - kStagesV : 0u); u < issued && landed; ++u)
+                landed = mbar_wait(bar(bar_vfull(u % kStagesV)), (u / kStagesV) & 1u, abort_flag);
             alive = alive && landed;
         }
     } else if (warp == kMmaWarp0 || warp == kMmaWarp0 + 1) {
@@ -652,10 +655,10 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
             // the K tile of the lane's next Q K^T, whose wait would otherwise sit between P V and the
             // next Q K^T: the chain that decides when the softmax warps get their next S.
             auto issue_pv = [&](uint32_t next_use) {
-                const int s = prev_kt % kStages;
-                if (!warp_wait(bar(bar_vfull(s)), (prev_kt / kStages) & 1u, abort_flag)) return false;
+                const int s = prev_kt % kStagesV;
+                if (!warp_wait(bar(bar_vfull(s)), (prev_kt / kStagesV) & 1u, abort_flag)) return false;
                 if (next_use != 0xFFFFFFFFu &&
-                    __all_sync(kFull, mbar_try(bar(bar_kfull(next_use % kStages)), (next_use / kStages) & 1u)))
+                    __all_sync(kFull, mbar_try(bar(bar_kfull(next_use % kStagesK)), (next_use / kStagesK) & 1u)))
                     k_seen = next_use;
                 if (!warp_wait(bar(bar_pfull(x, prev_j & 1u)), (prev_j >> 1) & 1u, abort_flag)) return false;
                 tc_fence_after();
@@ -678,11 +681,11 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
             };
             const int t_step = row_mode ? 1 : 2;  // distance to this lane's next tile
             for (int t = it.t_begin; t < it.t_end && alive; ++t, ++kt_run) {
-                const int s = kt_run % kStages;
+                const int s = kt_run % kStagesK;
                 const bool own = row_mode || (((t - it.t_begin) & 1) == x);
                 if (own) {
                     if (k_seen != kt_run)
-                        alive = warp_wait(bar(bar_kfull(s)), (kt_run / kStages) & 1u, abort_flag);
+                        alive = warp_wait(bar(bar_kfull(s)), (kt_run / kStagesK) & 1u, abort_flag);
                     if (!alive) break;
                     tc_fence_after();
                     if (elect_one()) {
@@ -864,8 +867,8 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
                 // both lanes clear them: each lane's PV is ordered behind its own warpgroup only) ----
                 const bool clear_v = j0 + kBN > kv_len;
                 if (clear_v) {
-                    const int s = kt_run % kStages;
-                    if (!warp_wait(bar(bar_vfull(s)), (kt_run / kStages) & 1u, abort_flag)) {
+                    const int s = kt_run % kStagesV;
+                    if (!warp_wait(bar(bar_vfull(s)), (kt_run / kStagesV) & 1u, abort_flag)) {
                         alive = false;
                         break;
                     }
