@@ -7,7 +7,7 @@
 // so that Q K^T and P V are dense contractions: tcgen05.mma with the fp32
 // accumulators (S and O) in tensor memory.  K/V tiles of 64 keys are staged by TMA
 // (cp.async.bulk.tensor, one elected thread) into 128-byte-swizzled shared memory
-// through mbarrier rings (four K stages, five V stages), Q tiles likewise (prefetched for the next item).
+// through mbarrier rings (four stages each for K and V), Q tiles likewise (prefetched for the next item).
 //
 // A CTA runs two symmetric lanes.  A lane is an MMA-issuing warp, a softmax warpgroup
 // (one TMEM lane = one query row per thread) and a quarter of tensor memory (two S/P
@@ -43,8 +43,13 @@ namespace {
 
 constexpr int kBM = 128;           // rows per row tile (one TMEM lane each)
 constexpr int kBN = 64;            // keys per tile
-constexpr int kStagesK = 4;        // K ring depth
-constexpr int kStagesV = 5;        // V ring depth (a V tile is held until its P V, a K tile only until its Q K^T)
+// Ring depths.  Both must be even: in key mode the lanes take alternate tiles and a lane waits for
+// (and looks ahead at) the "full" barriers of its own tiles only, so the previous use of a stage
+// must have been its own too -- with an odd depth it would be the other lane's, which this lane has
+// not seen complete, and a parity wait cannot tell "not yet" from "one phase on".
+constexpr int kStagesK = 4;
+constexpr int kStagesV = 4;
+static_assert(kStagesK % 2 == 0 && kStagesV % 2 == 0, "ring depths must be even (key mode)");
 constexpr int kRowTiles = 2;       // row tiles per item
 constexpr int kSoftmaxThreads = 256;
 constexpr int kProducerWarp = 8;   // K and Q tiles
