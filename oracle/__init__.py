@@ -72,11 +72,15 @@ class Tree:
     cand_parent: np.ndarray   # int32 [n_cand], -1 = root
     frontier: np.ndarray      # int32 [d, k]: candidates expanded after each level
     min_gap: float
+    near_pairs: np.ndarray    # int32 [n_near, 2]: boundary pairs (before, after) with a gap below tau
 
 
 def tree_expand(root_token: int, logits: np.ndarray, TT: int, d: int, k: int, L: int,
-                max_tt: int = 128, ret_stride: int | None = None) -> Tree:
-    """Draft-tree construction. ``logits`` is fp32 [>=d][>=k][V]; level 0 uses slot 0."""
+                max_tt: int = 128, ret_stride: int | None = None, tau: float = 0.0,
+                order_bias: np.ndarray | None = None) -> Tree:
+    """Draft-tree construction. ``logits`` is fp32 [>=d][>=k][V]; level 0 uses slot 0.
+    ``tau``: boundary pairs with a smaller score gap are listed in ``near_pairs``.
+    ``order_bias`` (fp64 [n_cand]) is added where candidates are ordered (see the C++ header)."""
     logits = _c(logits, np.float32)
     assert logits.ndim == 3 and logits.shape[0] >= d and (d == 1 or logits.shape[1] >= k)
     V = logits.shape[2]
@@ -98,16 +102,44 @@ def tree_expand(root_token: int, logits: np.ndarray, TT: int, d: int, k: int, L:
     cpar = np.zeros(n_cand, np.int32)
     frontier = np.zeros((d, k), np.int32)
     gap = ctypes.c_double()
+    max_near = 64
+    near = np.zeros((max_near, 2), np.int32)
+    n_near = ctypes.c_int32()
+    if order_bias is not None:
+        order_bias = _c(order_bias, np.float64)
+        assert order_bias.shape == (n_cand,)
     rc = _load().oracle_tree_expand(
         ctypes.c_int32(int(root_token)), _p(logits), ctypes.c_int64(ld_level), ctypes.c_int64(ld_row),
         V, TT, d, k, L, max_tt, ret_stride, _p(tokens), _p(parent), _p(depth), _p(pos), _p(mask),
         _p(retrieve), ctypes.byref(n_leaves), ctypes.byref(n_nodes), _p(cand), _p(ctok), _p(cpar),
-        _p(frontier), ctypes.byref(gap))
+        _p(frontier), ctypes.byref(gap), _p(order_bias) if order_bias is not None else None,
+        ctypes.c_double(tau), _p(near), max_near, ctypes.byref(n_near))
     if rc != 0:
         raise ValueError(f"oracle_tree_expand rc={rc}")
     n = n_nodes.value
     return Tree(tokens[:n], parent[:n], depth[:n], pos[:n], mask[:n], retrieve[:n_leaves.value],
-                n, n_leaves.value, cand, ctok, cpar, frontier, gap.value)
+                n, n_leaves.value, cand, ctok, cpar, frontier, gap.value, near[:n_near.value].copy())
+
+
+def tree_expand_swapped(root_token: int, logits: np.ndarray, TT: int, d: int, k: int, L: int,
+                        tau: float, max_tt: int = 128, ret_stride: int | None = None):
+    """The trees that differ from ``tree_expand``'s only by swaps among candidates whose scores
+    lie within ``tau`` of each other at a selection boundary: for every non-empty subset of the
+    near pairs, the tree built with the pair's second candidate ordered just before its first.
+    Yields (flipped pairs, Tree).  At most 6 near pairs (63 variants) are explored."""
+    base = tree_expand(root_token, logits, TT, d, k, L, max_tt, ret_stride, tau=tau)
+    pairs = [tuple(int(x) for x in p) for p in base.near_pairs][:6]
+    for subset in range(1, 1 << len(pairs)):
+        bias = np.zeros(base.cand_score.shape[0], np.float64)
+        flipped = []
+        for i, (before, after) in enumerate(pairs):
+            if subset >> i & 1:
+                # lift `after` just above `before` (1e-9 is far above fp64 rounding of a score
+                # and far below any tau worth the name)
+                bias[after] += base.cand_score[before] - base.cand_score[after] + 1e-9
+                flipped.append((before, after))
+        yield flipped, tree_expand(root_token, logits, TT, d, k, L, max_tt, ret_stride, tau=tau,
+                                   order_bias=bias)
 
 
 def tree_attention(q: np.ndarray, k_cache: np.ndarray, v_cache: np.ndarray, L: int,

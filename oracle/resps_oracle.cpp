@@ -129,21 +129,47 @@ int oracle_topk_lse(const float* row, int V, int k, float* out_val, int32_t* out
 //   expanded child, candidate c = k + (j-1)k^2 + p*k + r for level j >= 1,
 //   frontier[d][k] (optional): the candidates chosen for expansion after each
 //   level (row j = the frontier whose draft rows are logits[j+1][.]),
-//   min_gap (optional): smallest fp64 score gap across any selection boundary
-//   (k-th vs (k+1)-th of a level, m-th vs (m+1)-th of the rerank); +inf if none.
+//   min_gap (optional): smallest fp64 score gap across any selection boundary; +inf if
+//   none.  The boundaries are the pairs of neighbours in score order whose order
+//   decides the result: among the k+1 best of a level that is expanded further
+//   (levels 1..d-2: the rank inside the frontier is the slot whose draft row the
+//   node is given, the (k+1)-th is the first one left out; level 0 is ordered by
+//   the raw logits of one row, which is exact), and the m-th vs the (m+1)-th of
+//   the rerank.
+//
+// Near ties (test support for implementations whose log-sum-exp is summed in another
+// order and may therefore resolve a gap below `tau` the other way):
+//   near_pairs (optional, capacity max_near pairs): every boundary pair (before,
+//   after) as above whose gap is below tau; n_near = their number.
+//   order_bias (optional, [n_cand]): added to a candidate's score where candidates
+//   are *ordered* (frontier choice and rerank), never to the score its children
+//   inherit.  A bias that lifts `after` just above `before` yields the tree of the
+//   swapped order, i.e. the result "up to a swap among candidates within tau".
 // ---------------------------------------------------------------------------
 int oracle_tree_expand(int32_t root_token, const float* logits, int64_t ld_level, int64_t ld_row,
                        int V, int TT, int d, int k, int L, int max_tt, int ret_stride,
                        int32_t* tokens, int32_t* parent, int32_t* depth, int32_t* position_ids,
                        uint64_t* mask, int32_t* retrieve, int32_t* n_leaves, int32_t* n_nodes,
                        double* cand_score, int32_t* cand_token, int32_t* cand_parent,
-                       int32_t* frontier_out, double* min_gap) {
+                       int32_t* frontier_out, double* min_gap, const double* order_bias, double tau,
+                       int32_t* near_pairs, int max_near, int32_t* n_near) {
     if (V < 1 || k < 1 || k > V || d < 1 || TT < 1 || TT > max_tt || max_tt > 128) return -1;
     if (ret_stride < d + 1) return -1;
     const int n_cand = k + (d - 1) * k * k;
     std::vector<int32_t> c_tok(n_cand), c_par(n_cand), c_dep(n_cand);
     std::vector<double> c_score(n_cand);
     double gap = std::numeric_limits<double>::infinity();
+    int near = 0;
+    auto boundary = [&](const ScoreIdx& before, const ScoreIdx& after) {
+        const double g = before.s - after.s;
+        gap = std::min(gap, g);
+        if (g < tau && near_pairs && near < max_near) {
+            near_pairs[2 * near + 0] = before.c;
+            near_pairs[2 * near + 1] = after.c;
+            ++near;
+        }
+    };
+    auto ordering_score = [&](double s, int c) { return order_bias ? s + order_bias[c] : s; };
     std::vector<ValId> top(k);
     double lse;
 
@@ -176,20 +202,21 @@ int oracle_tree_expand(int32_t root_token, const float* logits, int64_t ld_level
             }
         }
         std::vector<ScoreIdx> layer(k * k);
-        for (int i = 0; i < k * k; ++i) layer[i] = ScoreIdx{c_score[base + i], base + i};
+        for (int i = 0; i < k * k; ++i) layer[i] = ScoreIdx{ordering_score(c_score[base + i], base + i), base + i};
         std::sort(layer.begin(), layer.end(), score_before);
         for (int r = 0; r < k; ++r) frontier[r] = layer[r].c;
         if (frontier_out)
             for (int r = 0; r < k; ++r) frontier_out[j * k + r] = frontier[r];
-        if (k * k > k) gap = std::min(gap, layer[k - 1].s - layer[k].s);
+        if (j + 1 < d)  // this frontier is expanded: its members and their order matter
+            for (int r = 0; r < k && r + 1 < k * k; ++r) boundary(layer[r], layer[r + 1]);
     }
 
     // Rerank every candidate; keep the best m, in candidate order.
     const int m = std::min(TT - 1, n_cand);
     std::vector<ScoreIdx> all(n_cand);
-    for (int c = 0; c < n_cand; ++c) all[c] = ScoreIdx{c_score[c], c};
+    for (int c = 0; c < n_cand; ++c) all[c] = ScoreIdx{ordering_score(c_score[c], c), c};
     std::sort(all.begin(), all.end(), score_before);
-    if (m >= 1 && m < n_cand) gap = std::min(gap, all[m - 1].s - all[m].s);
+    if (m >= 1 && m < n_cand) boundary(all[m - 1], all[m]);
     std::vector<int32_t> kept(m);
     for (int i = 0; i < m; ++i) kept[i] = all[i].c;
     std::sort(kept.begin(), kept.end());
@@ -241,6 +268,7 @@ int oracle_tree_expand(int32_t root_token, const float* logits, int64_t ld_level
         if (cand_parent) cand_parent[c] = c_par[c];
     }
     if (min_gap) *min_gap = gap;
+    if (n_near) *n_near = near;
     return 0;
 }
 

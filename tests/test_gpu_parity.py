@@ -1,6 +1,13 @@
 """Parity of the CUDA path against the CPU oracle on the five workloads, called through the
 C-ABI: tree indices, masks, retrieve rows, argmax, accepted path/tokens and the compacted
-cache must be bit-exact; attention within max-abs 2e-2 / max-rel 1e-2."""
+cache must be bit-exact; attention within max-abs 2e-2 / max-rel 1e-2.
+
+Two lengths.  The default run takes a few steps of every workload (seconds to a minute each).
+With RESPS_PARITY_FULL=1 every workload runs ALL its steps (200 / 500 / 200 / 300): every integer
+output of every step is compared, the cache on the slots each step moved (and in full on the first
+and the last step), attention on the first 3 steps and then on 1 step in 25.  A summary line per
+workload is appended to $RESPS_PARITY_LOG when that is set."""
+import json
 import os
 
 import numpy as np
@@ -8,24 +15,50 @@ import pytest
 
 pytestmark = pytest.mark.gpu
 
+FULL = os.environ.get("RESPS_PARITY_FULL", "0") == "1"
 SCALE = float(os.environ.get("RESPS_TEST_STEPS_SCALE", "1"))
+ONLY = os.environ.get("RESPS_PARITY_ONLY")  # e.g. "3,5": restrict the full run to these workloads
 
 
-def _run(index, n_steps, n_layers, attn_every, attn_seqs=None, cap=None):
+def _run(index, n_steps, n_layers, attn_every, attn_seqs=None, cap=None, all_seqs_on_step0=False):
     from harness import Runner
     from paper_2601_12212_b200 import synth
     w = synth.WORKLOADS[index]
+    if FULL:
+        if ONLY and str(index) not in ONLY.split(","):
+            pytest.skip("not in RESPS_PARITY_ONLY")
+        n_steps, n_layers = w.steps, 1
+    else:
+        n_steps = max(1, int(n_steps * SCALE))
     r = Runner(w, n_layers=n_layers, kv_capacity=cap)
-    n_steps = max(1, int(n_steps * SCALE))
     for step in range(n_steps):
-        layers = range(n_layers) if step % attn_every == 0 else ()
-        r.step(step, attn_layers=layers, attn_seqs=attn_seqs)
+        if FULL:
+            sampled = step < 3 or step % 25 == 0
+            layers = range(n_layers) if sampled else ()
+            seqs = None if step == 0 else attn_seqs
+            r.step(step, attn_layers=layers, attn_seqs=seqs,
+                   check_compaction="full" if step in (0, n_steps - 1) else "touched")
+        else:
+            layers = range(n_layers) if step % attn_every == 0 else ()
+            seqs = None if (all_seqs_on_step0 and step == 0) else attn_seqs
+            r.step(step, attn_layers=layers, attn_seqs=seqs)
     st = r.stats
+    final_prefix = list(r.L)
     r.close()
-    print(f"\n[cfg{index}] steps={st.steps} near_tie={st.near_tie_steps} (mismatch {st.near_tie_mismatch}) "
-          f"attn_checks={st.attn_checks} max_abs={st.attn_max_abs:.2e} max_rel={st.attn_max_rel:.2e} "
-          f"mean_accept={np.mean(st.accept_lens):.2f} mean_n={np.mean(st.n_nodes):.1f}")
-    assert st.near_tie_mismatch <= max(1, st.steps // 50)
+    summary = {"workload": index, "steps": st.steps, "near_tie_steps": st.near_tie_steps,
+               "near_tie_swaps": [[a, b, [list(p) for p in f]] for a, b, f in st.near_tie_swaps],
+               "attn_checks": st.attn_checks, "attn_max_abs": st.attn_max_abs, "attn_max_rel": st.attn_max_rel,
+               "mean_accept": float(np.mean(st.accept_lens)), "mean_n": float(np.mean(st.n_nodes)),
+               "final_prefix": final_prefix}
+    print("\n[parity] " + json.dumps(summary))
+    if os.environ.get("RESPS_PARITY_LOG"):
+        with open(os.environ["RESPS_PARITY_LOG"], "a") as f:
+            f.write(json.dumps(summary) + "\n")
+    # A tree that differs from the oracle's passes only as a swap among candidates within TAU of a
+    # selection boundary (harness.Runner.step fails on anything else).  The seeded workloads have
+    # none in their first steps; the full-length runs list whatever they meet.
+    if not FULL:
+        assert st.near_tie_swaps == []
     return st
 
 
@@ -50,5 +83,6 @@ def test_config4_llama70b_shape():
 
 
 def test_config5_ragged_batch():
-    st = _run(5, 5, 1, 4, attn_seqs=(0, 5))
+    # attention of all 8 sequences on the first step, of two of them afterwards
+    st = _run(5, 5, 1, 4, attn_seqs=(0, 5), all_seqs_on_step0=True)
     assert len(set(st.n_nodes)) > 2

@@ -154,3 +154,32 @@ def test_gqa_head_to_kv_head_mapping():
     out = oracle.tree_attention(q, kc, vc, L, chain_mask(n), 0.25)
     for h in range(Hq):
         np.testing.assert_allclose(out[:, h], h // 2 + 1, atol=1e-12)
+
+
+def test_lse_matches_library_logsumexp_and_the_closed_form():
+    """The optional log-sum-exp output: against scipy's and torch's logsumexp over score rows
+    built by one matrix product per KV head (not the oracle's per-key loop), and against the
+    closed form log(#allowed keys) when every score is zero."""
+    from scipy.special import logsumexp
+    rng = np.random.default_rng(11)
+    n, Hq, Hkv, D, L = 70, 6, 2, 64, 23
+    q, kc, vc = make(rng, n, Hq, Hkv, D, L)
+    parent, mask = random_tree_mask(rng, n)
+    scale = 0.37
+    _, lse = oracle.tree_attention(q, kc, vc, L, mask, scale, want_lse=True)
+    G = Hq // Hkv
+    Q, K = f64(q), f64(kc)
+    allow = np.zeros((n, L + n), bool)
+    allow[:, :L] = True
+    for t in range(n):
+        for j in range(n):
+            allow[t, L + j] = (int(mask[t, j >> 6]) >> (j & 63)) & 1
+    for g in range(Hkv):
+        scores = np.einsum("thd,jd->thj", Q[:, g * G:(g + 1) * G], K[g, : L + n]) * scale   # [n][G][L+n]
+        masked = np.where(allow[:, None, :], scores, -np.inf)
+        np.testing.assert_allclose(lse[:, g * G:(g + 1) * G], logsumexp(masked, axis=-1), atol=1e-11)
+        np.testing.assert_allclose(lse[:, g * G:(g + 1) * G],
+                                   torch.logsumexp(torch.from_numpy(masked), dim=-1).numpy(), atol=1e-11)
+    _, lse0 = oracle.tree_attention(q, np.zeros_like(kc), vc, L, mask, scale, want_lse=True)
+    depth = np.array([bin((int(mask[t, 1]) << 64) | int(mask[t, 0])).count("1") for t in range(n)])
+    np.testing.assert_allclose(lse0, np.log(L + depth)[:, None].repeat(Hq, 1), atol=1e-12)

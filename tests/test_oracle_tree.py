@@ -42,6 +42,51 @@ def test_hand_worked_example():
             assert t.min_gap == pytest.approx(math.log(0.275 / 0.27), abs=1e-6)
 
 
+def test_near_pairs_and_swapped_trees_by_hand():
+    """Near-tie support of the oracle, on values worked by hand from Section 3.2's V_i (product of
+    the draft confidences along the root path).  k = 2, d = 3, V = 4.
+      level 0, p = [.5, .4, .06, .04]:  c0 = tok 0 (V .5), c1 = tok 1 (V .4)
+      level 1, after c0 p = [.6, .2, .15, .05]: c2 = tok 0 (.30), c3 = tok 1 (.10)
+               after c1 p = [.05, .7499, .1501, .05]: c4 = tok 1 (.29996), c5 = tok 2 (.06004)
+        frontier = [c2, c4], third is c3: the pair (c2, c4) is log(.30/.29996) = 1.3e-4 apart
+      level 2, slot 0 p = [.1, .2, .3, .4]: c6 = tok 3, c7 = tok 2 under frontier[0]
+               slot 1 p = [.9, .05, .03, .02]: c8 = tok 0, c9 = tok 1 under frontier[1]
+    TT = 7 keeps the six best: c0, c1, c2, c4, c8 (.269964), c6 (.12); next is c3 (.10).
+    With the pair swapped the slots change hands: c6 hangs under c4 and c8 under c2; the kept set
+    stays (c8 = .27, c6 = .119984)."""
+    logits = np.zeros((3, 2, 4), np.float32)
+    logits[0, 0] = np.log([.5, .4, .06, .04])
+    logits[1, 0] = np.log([.6, .2, .15, .05])
+    logits[1, 1] = np.log([.05, .7499, .1501, .05])
+    logits[2, 0] = np.log([.1, .2, .3, .4])
+    logits[2, 1] = np.log([.9, .05, .03, .02])
+    t = oracle.tree_expand(9, logits, 7, 3, 2, 0, tau=1e-3)
+    assert t.tokens.tolist() == [9, 0, 1, 0, 1, 3, 0]
+    assert t.parent.tolist() == [-1, 0, 0, 1, 2, 3, 4]
+    assert t.min_gap == pytest.approx(math.log(.30 / .29996), abs=1e-6)
+    assert t.near_pairs.tolist() == [[2, 4]]
+    # a tau below the gap lists nothing, and then there is no swapped tree either
+    assert oracle.tree_expand(9, logits, 7, 3, 2, 0, tau=1e-4).near_pairs.shape[0] == 0
+    assert list(oracle.tree_expand_swapped(9, logits, 7, 3, 2, 0, tau=1e-4)) == []
+    variants = list(oracle.tree_expand_swapped(9, logits, 7, 3, 2, 0, tau=1e-3))
+    assert len(variants) == 1
+    flipped, tv = variants[0]
+    assert flipped == [(2, 4)]
+    assert tv.tokens.tolist() == [9, 0, 1, 0, 1, 3, 0]
+    assert tv.parent.tolist() == [-1, 0, 0, 1, 2, 4, 3]
+    assert tv.frontier[1].tolist() == [4, 2]
+    np.testing.assert_allclose(np.exp(tv.cand_score[[6, 8]]), [.119984, .27], rtol=1e-6)
+    check_invariants(tv, logits, 9, 7, 3, 2, 0)
+    # the last level's frontier is expanded by nobody: its order is no boundary (d = 2 here)
+    t2 = oracle.tree_expand(9, logits, 100, 2, 2, 0, tau=1e-3)
+    assert t2.near_pairs.shape[0] == 0 and t2.min_gap == float("inf")
+    # the rerank boundary is one: TT = 4 keeps c0, c1, c2 and drops c4 by the same 1.3e-4
+    t3 = oracle.tree_expand(9, logits, 4, 2, 2, 0, tau=1e-3)
+    assert t3.near_pairs.tolist() == [[2, 4]] and t3.tokens.tolist() == [9, 0, 1, 0]
+    (fl, tv3), = oracle.tree_expand_swapped(9, logits, 4, 2, 2, 0, tau=1e-3)
+    assert tv3.tokens.tolist() == [9, 0, 1, 1] and tv3.parent.tolist() == [-1, 0, 0, 2]
+
+
 # ---------------------------------------------------------------------- invariants
 def check_invariants(t, logits, root, TT, d, k, L):
     n = t.n_nodes

@@ -2,7 +2,10 @@
 (a process whose GPU memory was handed to another allocator at start-up, or code that only runs
 where cudaMalloc is forbidden).  It needs no context; its scratch is a fixed array inside the
 library.  Checked here through the C-ABI against what resps_verify_accept writes, bit for bit,
-on two calls in a row (the second call finds the array as the first one left it).
+on two calls in a row (the second call finds the array as the first one left it), and -- since
+both entry points run the same kernel -- against the CPU oracle's arg-max of the same rows.
+The shapes cover one piece per row, many pieces per row, rows of odd length on the scalar path
+with several pieces, and a vocabulary so large that the pieces are made longer than 8192.
 
 Collected last on purpose: a run that stops at the first failure has then run every other test."""
 import ctypes
@@ -31,9 +34,10 @@ def _reference_argmax(binding, torch, logits, n_nodes, T, V):
     return out.cpu().numpy()
 
 
-@pytest.mark.parametrize("B,T,V", [(2, 60, 128256), (3, 17, 1001)])
+@pytest.mark.parametrize("B,T,V", [(2, 60, 128256), (3, 17, 1001), (2, 5, 20001), (1, 2, 600001)])
 def test_static_argmax_matches_verify_accept_twice_in_a_row(B, T, V):
     import torch
+    import oracle
     from paper_2601_12212_b200 import binding
     g = torch.Generator(device="cuda")
     g.manual_seed(B * 1000 + T)
@@ -41,15 +45,20 @@ def test_static_argmax_matches_verify_accept_twice_in_a_row(B, T, V):
     for call in range(2):
         logits = torch.randn(B, T, V, generator=g, device="cuda")
         logits[:, :, V // 3] = logits[:, :, 7]            # ties: the lower id must win
+        logits[:, ::2, 7] = 50.0                          # ... also where the tied value is the maximum,
+        logits[:, ::2, V // 3] = 50.0                     # in different pieces of the row
         want = _reference_argmax(binding, torch, logits, n_nodes, T, V)
         got = torch.full((B, T), -7, dtype=torch.int32, device="cuda")
         binding.resps_target_argmax_static(n_nodes, B, T, V, logits, T * V, V, got)
         torch.cuda.synchronize()
         got = got.cpu().numpy()
+        host = logits.cpu().numpy()
         for b in range(B):
             n = int(n_nodes[b])
             assert np.array_equal(got[b, :n], want[b, :n]), f"call {call}, sequence {b}"
             assert (got[b, n:] == -7).all(), "entries past n_nodes must stay untouched"
+            ref = oracle.verify_accept(host[b, :n], np.zeros(n, np.int32), np.full(n, -1, np.int32)).target_argmax
+            assert np.array_equal(got[b, :n], ref), f"call {call}, sequence {b}: differs from the oracle"
 
 
 def test_static_argmax_rejects_sizes_beyond_its_array():
