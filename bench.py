@@ -271,7 +271,7 @@ class DeviceWorkload:
 
     def compact(self):
         self.binding.resps_kv_compact(self.ctx, self.d_steps, self.B, self.path, self.alen, self.k_ptrs,
-                                      self.v_ptrs, self.w.n_layers, *self.kv_strides)
+                                      self.v_ptrs, self.w.n_layers, *self.kv_strides, self.cap)
 
     def step(self, i):
         self.expand(i)

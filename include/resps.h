@@ -58,7 +58,9 @@ enum {
     RESPS_STATUS_STEP_CLAMPED = 1,   /* a step's tt/d/k was outside the supplied extents       */
     RESPS_STATUS_KV_OVERFLOW = 2,    /* prefix_len + n exceeds kv_capacity (the KV-cache       */
                                      /* overflow the paper's results section warns of); skipped */
-    RESPS_STATUS_WAIT_TIMEOUT = 4    /* a bounded device-side wait gave up                     */
+    RESPS_STATUS_WAIT_TIMEOUT = 4,   /* a bounded device-side wait gave up                     */
+    RESPS_STATUS_STALE_PLAN = 8      /* resps_tree_attention ran on a work list made for other  */
+                                     /* step parameters (see resps_attention_replan)            */
 };
 
 typedef struct resps_ctx resps_ctx;      /* opaque */
@@ -96,6 +98,19 @@ const char* resps_strerror(int code);
 int resps_status(resps_ctx* ctx, resps_stream stream, int32_t* status);
 /* Bytes of device workspace held by the context. */
 int64_t resps_workspace_bytes(const resps_ctx* ctx);
+
+/*
+ * Test and tuning aid, NOT part of the path: overrides one scheduling choice the library
+ * otherwise makes by itself.  Results never depend on these values, only how the work is cut.
+ * Returns INVALID_ARG for an unknown key.  (The paper has no counterpart.)
+ */
+enum {
+    RESPS_DEBUG_ATTN_ROUNDS = 1,    /* rounds of work items the attention work list plans: 0 = its own choice */
+    RESPS_DEBUG_ATTN_MIN_TILES = 2, /* fewest 64-key tiles a split of the keys is given (default 2)           */
+    RESPS_DEBUG_ATTN_STAGGER = 3,   /* SM cycles the second half of a CTA starts behind the first (default 1000) */
+    RESPS_DEBUG_SCAN_SLICES = 4     /* slices a logits row is cut into by the streaming scan: 0 = its own choice */
+};
+int resps_debug_set(resps_ctx* ctx, int key, int value);
 
 /*
  * Draft-tree construction (Section 3.2, "Draft Tree Expansion" and "Confidence-Based
@@ -155,12 +170,23 @@ int resps_tree_expand(resps_ctx* ctx, const resps_step* d_steps, int batch,
  * softmax_scale  must be positive (INVALID_ARG otherwise)
  * d_mask       as written by resps_tree_expand
  * Accumulation is fp32; the result is rounded to bf16 once.
+ *
+ * How the work is cut over the GPU depends only on (d_steps, d_n_nodes), which are the same for
+ * every layer of a step: the first call after resps_tree_expand (or after a resps_verify_accept
+ * that advanced these d_steps, or resps_attention_replan) derives that work list on the device,
+ * later calls with the same d_steps, d_n_nodes, batch, kv_capacity and stream reuse it.  A caller
+ * that changes the contents of d_steps or d_n_nodes by other means between two calls must call
+ * resps_attention_replan() in between; a call that finds its list out of date sets
+ * RESPS_STATUS_STALE_PLAN (its results are then undefined).
  */
 int resps_tree_attention(resps_ctx* ctx, const resps_step* d_steps, const int32_t* d_n_nodes,
                          int batch, const void* d_q, void* d_o, float* d_lse,
                          const void* d_k_cache, const void* d_v_cache, int64_t kv_stride_seq,
                          int64_t kv_stride_head, int64_t kv_stride_tok, int64_t kv_capacity,
                          const uint64_t* d_mask, float softmax_scale, resps_stream stream);
+
+/* Host-only: the next resps_tree_attention call derives its work list anew (see there). */
+int resps_attention_replan(resps_ctx* ctx);
 
 /*
  * Greedy verification and acceptance (Section 3.1: greedy decoding; Section 3.2,
@@ -176,8 +202,10 @@ int resps_tree_attention(resps_ctx* ctx, const resps_step* d_steps, const int32_
  *   d_accept_len    int32 [batch]           a = accepted draft tokens
  *   d_out_tokens    int32 [batch][max_depth+1]  the a accepted tokens then the bonus token
  *                                           (target argmax at the last accepted node), unused -1
- *   d_steps_next    resps_step [batch] or NULL: copy of d_steps with prefix_len += a+1
- *                   (may alias d_steps)
+ *   d_steps_next    resps_step [batch] or NULL: copy of d_steps with prefix_len += a+1.
+ *                   It may alias d_steps (the step loop then advances on the device with no host
+ *                   write); resps_kv_compact must in that case be told that the prefix lengths it
+ *                   is given are the advanced ones (steps_advanced = 1).
  */
 int resps_verify_accept(resps_ctx* ctx, const resps_step* d_steps, const int32_t* d_n_nodes,
                         int batch, const float* d_target_logits, int64_t ld_b, int64_t ld_row,
@@ -188,17 +216,26 @@ int resps_verify_accept(resps_ctx* ctx, const resps_step* d_steps, const int32_t
 /*
  * In-place KV-cache compaction (Appendix D, "input update": rejected tokens are discarded
  * from the cache).  For every bound layer, KV head and j = 0..a:
- *   slot L+j  <-  slot L+path[j]     (K and V),   L = d_steps[b].prefix_len (before the step).
+ *   slot L+j  <-  slot L+path[j]     (K and V),   L = the prefix length before the step.
  * Slots beyond L+a are left as they are.
  *
+ * d_steps         DEVICE resps_step [batch].  steps_advanced = 0: prefix_len is the step's own L.
+ *                 steps_advanced = 1: the array was already advanced by resps_verify_accept
+ *                 (d_steps_next aliased d_steps), i.e. prefix_len = L + a + 1, and L is recovered
+ *                 from it and d_accept_len.
  * d_k_caches, d_v_caches  DEVICE arrays of n_layers DEVICE pointers (bf16 caches laid out as
  *                         in resps_tree_attention)
+ * kv_capacity     slots per (sequence, head).  A sequence whose path would touch a slot outside
+ *                 [0, kv_capacity) -- the sequence resps_tree_attention skipped for the same
+ *                 reason -- or whose path holds an entry outside [0, max_tt) is left untouched and
+ *                 RESPS_STATUS_KV_OVERFLOW set (the KV-cache overflow the paper's results section
+ *                 warns of).
  */
-int resps_kv_compact(resps_ctx* ctx, const resps_step* d_steps, int batch,
+int resps_kv_compact(resps_ctx* ctx, const resps_step* d_steps, int steps_advanced, int batch,
                      const int32_t* d_accept_path, const int32_t* d_accept_len,
                      void* const* d_k_caches, void* const* d_v_caches, int n_layers,
                      int64_t kv_stride_seq, int64_t kv_stride_head, int64_t kv_stride_tok,
-                     resps_stream stream);
+                     int64_t kv_capacity, resps_stream stream);
 
 /*
  * Per-node target arg-max for callers that cannot allocate device memory.  (The paper has no

@@ -22,9 +22,14 @@ RESPS_ERR_NO_DEVICE = -5
 RESPS_STATUS_STEP_CLAMPED = 1
 RESPS_STATUS_KV_OVERFLOW = 2
 RESPS_STATUS_WAIT_TIMEOUT = 4
+RESPS_STATUS_STALE_PLAN = 8
+RESPS_DEBUG_ATTN_ROUNDS = 1
+RESPS_DEBUG_ATTN_MIN_TILES = 2
+RESPS_DEBUG_ATTN_STAGGER = 3
+RESPS_DEBUG_SCAN_SLICES = 4
 
 EXPORTS = ("resps_create", "resps_destroy", "resps_strerror", "resps_status",
-           "resps_workspace_bytes", "resps_tree_expand", "resps_tree_attention",
+           "resps_workspace_bytes", "resps_debug_set", "resps_attention_replan", "resps_tree_expand", "resps_tree_attention",
            "resps_verify_accept", "resps_kv_compact", "resps_target_argmax_static")
 
 
@@ -65,7 +70,9 @@ def load() -> ctypes.CDLL:
     lib.resps_tree_attention.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp, vp, i64, i64, i64, i64,
                                          vp, f32, vp]
     lib.resps_verify_accept.argtypes = [vp, vp, vp, i32, vp, i64, i64, vp, vp, vp, vp, vp, vp, vp, vp]
-    lib.resps_kv_compact.argtypes = [vp, vp, i32, vp, vp, vp, vp, i32, i64, i64, i64, vp]
+    lib.resps_kv_compact.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp, i32, i64, i64, i64, i64, vp]
+    lib.resps_debug_set.argtypes = [vp, i32, i32]
+    lib.resps_attention_replan.argtypes = [vp]
     lib.resps_target_argmax_static.argtypes = [vp, i32, i32, i32, vp, i64, i64, vp, vp]
     for name in EXPORTS:
         if name not in ("resps_strerror", "resps_workspace_bytes"):
@@ -121,6 +128,15 @@ class Context:
         _check(load().resps_status(self._h, _stream(stream), ctypes.byref(out)), "resps_status")
         return out.value
 
+    def debug_set(self, key: int, value: int) -> None:
+        """Test and tuning aid (see resps_debug_set in resps.h); never changes a result."""
+        _check(load().resps_debug_set(self._h, int(key), int(value)), "resps_debug_set")
+
+    def attention_replan(self) -> None:
+        """The step parameters or node counts were changed behind the library's back: the next
+        resps_tree_attention call derives its work list anew."""
+        _check(load().resps_attention_replan(self._h), "resps_attention_replan")
+
     def close(self):
         if self._h:
             load().resps_destroy(self._h)
@@ -171,13 +187,15 @@ def resps_verify_accept(ctx: Context, steps, n_nodes, batch: int, target_logits,
 
 def resps_kv_compact(ctx: Context, steps, batch: int, accept_path, accept_len, k_cache_ptrs,
                      v_cache_ptrs, n_layers: int, kv_stride_seq: int, kv_stride_head: int,
-                     kv_stride_tok: int, stream=None) -> None:
-    """k_cache_ptrs / v_cache_ptrs: int64 CUDA tensors holding n_layers device pointers."""
+                     kv_stride_tok: int, kv_capacity: int, steps_advanced: bool = False,
+                     stream=None) -> None:
+    """k_cache_ptrs / v_cache_ptrs: int64 CUDA tensors holding n_layers device pointers.
+    steps_advanced: `steps` was already advanced by resps_verify_accept (steps_next aliased it)."""
     i32 = torch.int32
     _check(load().resps_kv_compact(
-        ctx.handle, _ptr(steps, i32), batch, _ptr(accept_path, i32), _ptr(accept_len, i32),
-        _ptr(k_cache_ptrs, torch.int64), _ptr(v_cache_ptrs, torch.int64), n_layers, kv_stride_seq,
-        kv_stride_head, kv_stride_tok, _stream(stream)), "resps_kv_compact")
+        ctx.handle, _ptr(steps, i32), int(bool(steps_advanced)), batch, _ptr(accept_path, i32),
+        _ptr(accept_len, i32), _ptr(k_cache_ptrs, torch.int64), _ptr(v_cache_ptrs, torch.int64), n_layers,
+        kv_stride_seq, kv_stride_head, kv_stride_tok, kv_capacity, _stream(stream)), "resps_kv_compact")
 
 
 def resps_target_argmax_static(n_nodes, batch: int, max_tt: int, vocab: int, target_logits, ld_b: int,

@@ -70,11 +70,13 @@ __global__ void __launch_bounds__(RESPS_MAX_TT) accept_walk_kernel(const AcceptA
 
 struct CompactArgs {
     const resps_step* steps;
+    int steps_advanced;  // 1: steps[b].prefix_len already holds L + a + 1
     const int32_t *accept_path, *accept_len;
     void* const* k_caches;
     void* const* v_caches;
-    int64_t stride_seq, stride_head, stride_tok;
-    int n_kv_heads, head_dim, max_depth;
+    int64_t stride_seq, stride_head, stride_tok, capacity;
+    int n_kv_heads, head_dim, max_depth, max_tt;
+    int32_t* status;
 };
 
 // One CTA per (K-or-V of a KV head, layer, sequence).  All source rows are read into
@@ -87,7 +89,20 @@ __global__ void __launch_bounds__(128) kv_compact_kernel(const CompactArgs a) {
     const int head = blockIdx.x >> 1, is_v = blockIdx.x & 1;
     const int cap = a.max_depth + 1;
     const int len = min(max(a.accept_len[b], 0), a.max_depth);
-    const int L = a.steps[b].prefix_len;
+    const int L = max(a.steps[b].prefix_len - (a.steps_advanced ? len + 1 : 0), 0);
+    // Every slot the move reads or writes must lie inside the cache, every path entry inside a tree.
+    {
+        int bad = 0;
+        if (threadIdx.x <= len) {
+            const int src = a.accept_path[b * cap + threadIdx.x];
+            bad = (src < 0 || src >= a.max_tt || static_cast<int64_t>(L) + src >= a.capacity ||
+                   static_cast<int64_t>(L) + threadIdx.x >= a.capacity);
+        }
+        if (__syncthreads_or(bad)) {
+            if (threadIdx.x == 0 && blockIdx.x == 0 && layer == 0) atomicOr(a.status, RESPS_STATUS_KV_OVERFLOW);
+            return;
+        }
+    }
     __nv_bfloat16* base = static_cast<__nv_bfloat16*>(is_v ? a.v_caches[layer] : a.k_caches[layer]) +
                           b * a.stride_seq + head * a.stride_head;
     const int vec_per_row = a.head_dim / 8;  // 16-byte pieces per row
@@ -130,17 +145,20 @@ cudaError_t launch_accept_walk(const resps_ctx* ctx, const resps_step* d_steps,
     return launch_pdl(accept_walk_kernel, dim3(batch), dim3(RESPS_MAX_TT), 0, st, a);
 }
 
-cudaError_t launch_kv_compact(const resps_ctx* ctx, const resps_step* d_steps, int batch,
+cudaError_t launch_kv_compact(const resps_ctx* ctx, const resps_step* d_steps, int steps_advanced, int batch,
                               const int32_t* accept_path, const int32_t* accept_len,
                               void* const* k_caches, void* const* v_caches, int n_layers,
                               int64_t stride_seq, int64_t stride_head, int64_t stride_tok,
-                              cudaStream_t st) {
+                              int64_t capacity, cudaStream_t st) {
     CompactArgs a;
-    a.steps = d_steps, a.accept_path = accept_path, a.accept_len = accept_len;
+    a.steps = d_steps, a.steps_advanced = steps_advanced;
+    a.accept_path = accept_path, a.accept_len = accept_len;
     a.k_caches = k_caches, a.v_caches = v_caches;
     a.stride_seq = stride_seq, a.stride_head = stride_head, a.stride_tok = stride_tok;
+    a.capacity = capacity;
     a.n_kv_heads = ctx->shape.n_kv_heads, a.head_dim = ctx->shape.head_dim;
-    a.max_depth = ctx->shape.max_depth;
+    a.max_depth = ctx->shape.max_depth, a.max_tt = ctx->shape.max_tt;
+    a.status = ctx->ws.status;
     dim3 grid(ctx->shape.n_kv_heads * 2, n_layers, batch);
     return launch_pdl(kv_compact_kernel, grid, dim3(128), 0, st, a);
 }

@@ -1,6 +1,6 @@
 // C ABI of libresps: argument checks, the context and its workspace, and the
 // sequencing of kernel launches behind each entry point (see include/resps.h).
-#include <cstdlib>
+#include <algorithm>
 #include <cstring>
 #include <new>
 
@@ -44,6 +44,7 @@ void carve(resps_ctx* c, Carver& cv) {
     cv.take(w.row_id, rows * s.max_k);
     cv.take(w.row_lse, rows);
     cv.take(w.amax_part, nodes * w.scan_splits);
+    cv.take(w.attn_plan, static_cast<int64_t>(resps::attention_plan_bytes(s.max_batch, w.attn_max_items)));
     cv.take(w.attn_part_o, static_cast<int64_t>(w.attn_max_items) * resps::attention_item_rows() * s.head_dim);
     cv.take(w.attn_part_ml, static_cast<int64_t>(w.attn_max_items) * resps::attention_item_rows());
 }
@@ -92,16 +93,14 @@ int resps_create(resps_ctx** out, const resps_shape* shape) {
 
     resps_ctx* c = new (std::nothrow) resps_ctx();
     if (!c) return RESPS_ERR_CUDA;
+    c->attn_host = nullptr;
     c->shape = s;
     c->device = dev;
     c->sm_count = prop.multiProcessorCount;
     resps::Workspace& w = c->ws;
     // a scan CTA keeps its whole chunk in registers; up to 128 chunks per row (vocab <= 2^20)
-    int chunk = resps::scan_chunk_max();
-    if (const char* e = std::getenv("RESPS_SCAN_CHUNK"))
-        chunk = std::min(chunk, std::max(1024, std::atoi(e) / 1024 * 1024));
+    const int chunk = resps::scan_chunk_max();
     w.scan_chunk = chunk;
-    if (const char* e = std::getenv("RESPS_SCAN_SLICES")) w.scan_slices_hint = std::max(0, std::atoi(e));
     w.scan_splits = (s.vocab + chunk - 1) / chunk;
     if (w.scan_splits > 128) {
         delete c;
@@ -113,10 +112,7 @@ int resps_create(resps_ctx** out, const resps_shape* shape) {
     w.attn_grid = c->sm_count;
     w.attn_combine_grid = c->sm_count * 4;
     w.attn_min_tiles = 2;
-    if (const char* e = std::getenv("RESPS_ATTN_MIN_TILES")) w.attn_min_tiles = std::max(1, std::atoi(e));
-    if (const char* e = std::getenv("RESPS_ATTN_ROUNDS")) w.attn_rounds = std::max(0, std::atoi(e));
-    if (const char* e = std::getenv("RESPS_ATTN_STAGGER")) w.attn_stagger = std::min(100000, std::max(0, std::atoi(e)));
-    w.attn_max_groups = s.max_batch * s.n_kv_heads * ((s.max_tt * G + item_rows - 1) / item_rows);
+    w.attn_max_groups = s.max_batch * s.n_kv_heads * ((s.max_tt * G + item_rows / 2 - 1) / (item_rows / 2));  // single row tiles
     w.attn_max_items = resps::attention_max_rounds() * w.attn_grid + w.attn_max_groups;
 
     Carver dry;
@@ -137,6 +133,7 @@ int resps_create(resps_ctx** out, const resps_shape* shape) {
     if (resps::attention_setup(c) != cudaSuccess || resps::tree_setup(c) != cudaSuccess ||
         resps::scan_setup(c) != cudaSuccess) {
         cudaFree(c->arena);
+        resps::attention_teardown(c);
         delete c;
         return RESPS_ERR_CUDA;
     }
@@ -147,8 +144,29 @@ int resps_create(resps_ctx** out, const resps_shape* shape) {
 int resps_destroy(resps_ctx* ctx) {
     if (!ctx) return RESPS_OK;
     cudaError_t e = cudaFree(ctx->arena);
+    resps::attention_teardown(ctx);
     delete ctx;
     return e == cudaSuccess ? RESPS_OK : RESPS_ERR_CUDA;
+}
+
+int resps_attention_replan(resps_ctx* ctx) {
+    RESPS_CHECK_PTR(ctx);
+    resps::attention_plan_invalidate(ctx);
+    return RESPS_OK;
+}
+
+int resps_debug_set(resps_ctx* ctx, int key, int value) {
+    RESPS_CHECK_PTR(ctx);
+    resps::Workspace& w = ctx->ws;
+    switch (key) {
+        case RESPS_DEBUG_ATTN_ROUNDS: w.attn_rounds = std::max(0, value); break;
+        case RESPS_DEBUG_ATTN_MIN_TILES: w.attn_min_tiles = std::max(1, value); break;
+        case RESPS_DEBUG_ATTN_STAGGER: w.attn_stagger = std::min(100000, std::max(0, value)); break;
+        case RESPS_DEBUG_SCAN_SLICES: w.scan_slices_hint = std::max(0, value); break;
+        default: return RESPS_ERR_INVALID_ARG;
+    }
+    resps::attention_plan_invalidate(ctx);
+    return RESPS_OK;
 }
 
 int64_t resps_workspace_bytes(const resps_ctx* ctx) { return ctx ? ctx->arena_bytes : 0; }
@@ -186,6 +204,7 @@ int resps_tree_expand(resps_ctx* ctx, const resps_step* d_steps, int batch,
     if (batch > ctx->shape.max_batch) return RESPS_ERR_CAPACITY;
     if (n_levels > ctx->shape.max_depth) n_levels = ctx->shape.max_depth;
     if (n_slots > ctx->shape.max_k) n_slots = ctx->shape.max_k;
+    resps::attention_plan_invalidate(ctx);  // a new tree: new node counts, possibly new step parameters
     if (resps::launch_row_scan(ctx, d_steps, batch, d_draft_logits, ld_b, ld_level, ld_row, n_levels,
                                n_slots, stream) != cudaSuccess)
         return RESPS_ERR_CUDA;
@@ -243,6 +262,7 @@ int resps_verify_accept(resps_ctx* ctx, const resps_step* d_steps, const int32_t
     RESPS_CHECK_PTR(d_out_tokens);
     if (batch < 1 || ld_row < ctx->shape.vocab || ld_b < 0) return RESPS_ERR_INVALID_ARG;
     if (batch > ctx->shape.max_batch) return RESPS_ERR_CAPACITY;
+    if (d_steps_next) resps::attention_plan_invalidate(ctx, d_steps_next);  // prefix lengths move on
     if (resps::launch_row_argmax(ctx, d_n_nodes, batch, d_target_logits, ld_b, ld_row, d_target_argmax,
                                  stream) != cudaSuccess)
         return RESPS_ERR_CUDA;
@@ -253,11 +273,11 @@ int resps_verify_accept(resps_ctx* ctx, const resps_step* d_steps, const int32_t
     return RESPS_OK;
 }
 
-int resps_kv_compact(resps_ctx* ctx, const resps_step* d_steps, int batch,
+int resps_kv_compact(resps_ctx* ctx, const resps_step* d_steps, int steps_advanced, int batch,
                      const int32_t* d_accept_path, const int32_t* d_accept_len,
                      void* const* d_k_caches, void* const* d_v_caches, int n_layers,
                      int64_t kv_stride_seq, int64_t kv_stride_head, int64_t kv_stride_tok,
-                     resps_stream stream) {
+                     int64_t kv_capacity, resps_stream stream) {
     RESPS_CHECK_PTR(ctx);
     RESPS_CHECK_PTR(d_steps);
     RESPS_CHECK_PTR(d_accept_path);
@@ -265,11 +285,12 @@ int resps_kv_compact(resps_ctx* ctx, const resps_step* d_steps, int batch,
     RESPS_CHECK_PTR(d_k_caches);
     RESPS_CHECK_PTR(d_v_caches);
     if (batch < 1 || n_layers < 1 || n_layers > 65535 || kv_stride_tok < ctx->shape.head_dim ||
-        kv_stride_seq % 8 || kv_stride_head % 8 || kv_stride_tok % 8)
+        kv_stride_seq % 8 || kv_stride_head % 8 || kv_stride_tok % 8 || kv_capacity < 1 ||
+        (steps_advanced != 0 && steps_advanced != 1))
         return RESPS_ERR_INVALID_ARG;
     if (batch > ctx->shape.max_batch) return RESPS_ERR_CAPACITY;
-    if (resps::launch_kv_compact(ctx, d_steps, batch, d_accept_path, d_accept_len, d_k_caches, d_v_caches,
-                                 n_layers, kv_stride_seq, kv_stride_head, kv_stride_tok,
+    if (resps::launch_kv_compact(ctx, d_steps, steps_advanced, batch, d_accept_path, d_accept_len, d_k_caches,
+                                 d_v_caches, n_layers, kv_stride_seq, kv_stride_head, kv_stride_tok, kv_capacity,
                                  stream) != cudaSuccess)
         return RESPS_ERR_CUDA;
     return RESPS_OK;

@@ -18,13 +18,16 @@
 // bf16 rounding of the weights alone would cost up to 2^-9 per weight, about 1 % of an
 // output row's rms in the worst element.
 //
-// A work item is (sequence, KV head, pair of row tiles, range of key tiles).  With more
-// than 128 rows left, lane x takes row tile x over all key tiles ("row mode");
-// otherwise both lanes take the one row tile and alternate key tiles ("key mode"),
-// ending with two partial results.  The work list is derived inside the kernel from the
-// device-resident step parameters, so nothing about the launch depends on
-// (TT, d, k, L).  Items whose group has a single split in row mode write O directly;
-// all others write un-normalised partials that a second, small kernel combines.
+// A work item is (sequence, KV head, group of row tiles, range of key tiles).  With more
+// than 128 rows in the group, lane x takes row tile x over all key tiles ("row mode");
+// otherwise both lanes take the one row tile and alternate key tiles ("key mode") and
+// merge their two results inside the CTA (a lane reads the other's accumulator straight
+// from tensor memory).  The work list depends only on the step parameters, which are the
+// same for every layer of a step: a one-CTA kernel derives it once from the
+// device-resident parameters and leaves it in the workspace as a table (one 32-byte
+// descriptor per item), so nothing about a launch depends on (TT, d, k, L) and a CTA
+// learns its work from one load.  Items whose group has a single split write O directly;
+// all others write normalised partials that a second, small kernel combines.
 //
 // Every wait (mbarrier) is bounded: when it runs out the CTA raises
 // RESPS_STATUS_WAIT_TIMEOUT, stops issuing work, drains its copies in flight, frees
@@ -35,6 +38,9 @@
 
 #include <algorithm>
 #include <cmath>
+#include <mutex>
+#include <new>
+#include <unordered_map>
 
 #include "common.cuh"
 
@@ -67,6 +73,19 @@ constexpr uint32_t kWaitLimitCycles = 0x70000000u;  // bounded waits give up aft
 constexpr float kRescaleSlack = 8.0f;  // O is rescaled only when the running max grows by > 2^8
 constexpr unsigned kFull = 0xFFFFFFFFu;
 
+// What the work list keeps per sequence (the combine kernels walk rows, not items) ...
+struct PlanSeq {
+    int n, L, mp, nfull, kt, s_row, s_key, item0;
+};
+// ... and per item: everything a CTA needs to start.
+struct PlanItem {
+    int b_g;          // sequence | KV head << 16
+    int pair_splits;  // group index within the head | splits of the group << 16
+    int sp, first_item, t_begin, t_end;
+    int n, L;         // the sequence's tree size and prefix length
+};
+static_assert(sizeof(PlanSeq) == 32 && sizeof(PlanItem) == 32, "two 16-byte loads each");
+
 struct AttnArgs {
     const resps_step* steps;
     const int32_t* n_nodes;
@@ -90,7 +109,12 @@ struct AttnArgs {
     int rounds;       // 0: the work list chooses its number of rounds; 1..kMaxRounds: as told (tests)
     int stagger;      // cycles lane 1 starts behind lane 0 in row mode
     int q_by_tma;     // 1: Q tiles come by TMA (128 % (Hq/Hkv) == 0), 0: by plain loads
+    int plan_after_wait;  // 1: the work list was written by the kernel just before this one
     int32_t* status;
+    // The work list, written by attention_plan_kernel.
+    int4* plan_head;             // (items, rows per group, -, -)
+    PlanSeq* plan_seq;       // [batch + 1]; entry [batch].item0 = items
+    PlanItem* plan_item;  // [max_items]
 };
 
 // ---------------------------------------------------------------------------- work list
@@ -99,7 +123,11 @@ struct AttnArgs {
 // in key mode and costs one.  Every group is cut into splits of at most T units, with the smallest
 // T for which the items fit one round of the grid (found by a short search; steps of 1/16), so
 // that the CTAs finish together whatever the mix of tree sizes and prefix lengths.
+// When even the shortest row-mode items would leave half of the grid idle (a single short
+// sequence), groups are single row tiles instead, all in key mode: twice the items, each with
+// half the key tiles per lane, for the price of reading K and V through L2 once more.
 struct Sched {
+    int group_rows;             // rows of a group: 256 (pairs of row tiles) or 128 (single tiles)
     int n[kMaxBatchSmem];       // tree nodes (0 = sequence skipped)
     int L[kMaxBatchSmem];
     int mp[kMaxBatchSmem];      // row-tile pairs
@@ -122,8 +150,8 @@ __device__ __forceinline__ void build_sched(const AttnArgs& a, Sched& sc, int ti
         const int G = a.Hq / a.Hkv;
         const int nblk = (a.batch + 31) >> 5;
         const int mt = max(a.min_tiles, 1);
-        // the lane's first sequence stays in registers (its only one up to 32 sequences)
-        int kt0 = 0, nfull0 = 0, nkey0 = 0;
+        // ---- pass 1: sizes, and the cost in row-tile x key-tile units (the same for both groupings:
+        // a row-mode pair costs two units per key tile, a single tile one) ----------------------------
         unsigned cost = 0;  // saturates: it only seeds the search below
 #pragma unroll 1
         for (int i = 0; i < nblk; ++i) {
@@ -135,16 +163,31 @@ __device__ __forceinline__ void build_sched(const AttnArgs& a, Sched& sc, int ti
                     atomicOr(a.status, RESPS_STATUS_KV_OVERFLOW);
                     n = 0;
                 }
-                const int M = n * G;
-                const int mp = (M + kRowTiles * kBM - 1) / (kRowTiles * kBM);
-                const int nfull = (mp > 0 && M - (mp - 1) * kRowTiles * kBM <= kBM) ? mp - 1 : mp;
+                const int tiles = (n * G + kBM - 1) / kBM;
                 const int kt = (n > 0) ? (L + n + kBN - 1) / kBN : 0;
-                sc.n[b] = n, sc.L[b] = L, sc.mp[b] = mp, sc.nfull[b] = nfull, sc.kt[b] = kt;
-                if (i == 0) kt0 = kt, nfull0 = nfull, nkey0 = mp - nfull;
-                cost += min(static_cast<unsigned>(a.Hkv * (nfull + mp)) * static_cast<unsigned>(kt), 1u << 23);
+                sc.n[b] = n, sc.L[b] = L, sc.kt[b] = kt;
+                cost += min(static_cast<unsigned>(a.Hkv * tiles) * static_cast<unsigned>(kt), 1u << 23);
             }
         }
         cost = __reduce_add_sync(0xFFFFFFFFu, min(cost, 1u << 26));
+        // Row-mode items of mt key tiles cost 2 mt units each: if the whole call is worth no more than
+        // half a grid of those, single tiles in key mode fill the grid better.
+        const bool single = cost <= static_cast<unsigned>(mt * a.sched_grid);
+        const int group_rows = single ? kBM : kRowTiles * kBM;
+        if (tid == 0) sc.group_rows = group_rows;
+#pragma unroll 1
+        for (int i = 0; i < nblk; ++i) {
+            const int b = i * 32 + tid;
+            if (b < a.batch) {
+                const int M = sc.n[b] * G;
+                const int mp = (M + group_rows - 1) / group_rows;
+                sc.mp[b] = mp;
+                sc.nfull[b] = single ? 0 : ((mp > 0 && M - (mp - 1) * group_rows <= kBM) ? mp - 1 : mp);
+            }
+        }
+        // the lane's first sequence stays in registers (its only one up to 32 sequences)
+        int kt0 = 0, nfull0 = 0, nkey0 = 0;
+        if (tid < a.batch) kt0 = sc.kt[tid], nfull0 = sc.nfull[tid], nkey0 = sc.mp[tid] - nfull0;
         // Smallest T (in steps of T/16) for which the items fit `rounds` rounds of the grid.  One round
         // is the rule.  With long sequences and few groups it can leave CTAs idle (40 groups of 3 splits
         // are 120 items for 148 CTAs); two to four rounds of shorter items then fill the grid better.
@@ -203,38 +246,72 @@ __device__ __forceinline__ void build_sched(const AttnArgs& a, Sched& sc, int ti
 struct Item {
     int b, g, pair, sp, splits, first_item;
     int n, L, M, row_base, nmt, t_begin, t_end;
-    int tok0;  // first token of the pair's rows
+    int tok0;  // first token of the group's rows
 };
 
-__device__ __forceinline__ Item decode_item(const Sched& sc, int item, int G) {
-    Item it;
+__device__ __forceinline__ PlanItem plan_entry(const Sched& sc, int item) {
+    PlanItem p;
     int b = 0;
     while (item >= sc.item0[b + 1]) ++b;
-    it.b = b;
-    it.n = sc.n[b], it.L = sc.L[b];
     const int nfull = sc.nfull[b], s_row = sc.s_row[b], s_key = sc.s_key[b];
     const int row_items = nfull * s_row;
     const int per_head = row_items + (sc.mp[b] - nfull) * s_key;
     const int local = item - sc.item0[b];
-    it.g = static_cast<int>(static_cast<unsigned>(local) / static_cast<unsigned>(per_head));
-    const int rem = local - it.g * per_head;
+    const int g = static_cast<int>(static_cast<unsigned>(local) / static_cast<unsigned>(per_head));
+    const int rem = local - g * per_head;
+    int pair, splits;
     if (rem < row_items) {
-        it.pair = (nfull == 1) ? 0 : static_cast<int>(static_cast<unsigned>(rem) / static_cast<unsigned>(s_row));
-        it.sp = rem - it.pair * s_row;
-        it.splits = s_row;
+        pair = static_cast<int>(static_cast<unsigned>(rem) / static_cast<unsigned>(s_row));
+        p.sp = rem - pair * s_row;
+        splits = s_row;
     } else {
-        it.pair = nfull;
-        it.sp = rem - row_items;
-        it.splits = s_key;
+        pair = nfull + static_cast<int>(static_cast<unsigned>(rem - row_items) / static_cast<unsigned>(s_key));
+        p.sp = rem - row_items - (pair - nfull) * s_key;
+        splits = s_key;
     }
-    it.first_item = item - it.sp;
-    it.M = it.n * G;
-    it.row_base = it.pair * kRowTiles * kBM;
-    it.nmt = (it.M - it.row_base > kBM) ? 2 : 1;
+    p.b_g = static_cast<int>(static_cast<unsigned>(b) | (static_cast<unsigned>(g) << 16));
+    p.pair_splits = static_cast<int>(static_cast<unsigned>(pair) | (static_cast<unsigned>(splits) << 16));
+    p.first_item = item - p.sp;
     // kt <= 2^15 (cache capacity is checked on the host), so the products fit 32 bits
-    const unsigned kt = static_cast<unsigned>(sc.kt[b]), sp = static_cast<unsigned>(it.sp);
-    it.t_begin = static_cast<int>(kt * sp / static_cast<unsigned>(it.splits));
-    it.t_end = static_cast<int>(kt * (sp + 1u) / static_cast<unsigned>(it.splits));
+    const unsigned kt = static_cast<unsigned>(sc.kt[b]), sp = static_cast<unsigned>(p.sp);
+    p.t_begin = static_cast<int>(kt * sp / static_cast<unsigned>(splits));
+    p.t_end = static_cast<int>(kt * (sp + 1u) / static_cast<unsigned>(splits));
+    p.n = sc.n[b], p.L = sc.L[b];
+    return p;
+}
+
+// The work list of one call: the per-sequence figures and one descriptor per item, written to the
+// workspace.  One CTA; it runs once per step (the list is the same for every layer).
+__global__ void __launch_bounds__(256) attention_plan_kernel(const AttnArgs a) {
+    __shared__ Sched sc;
+    pdl_wait();  // the step parameters and node counts are complete
+    pdl_launch_dependents();
+    build_sched(a, sc, threadIdx.x);  // ends with __syncthreads()
+    const int total = min(sc.item0[a.batch], a.max_items);
+    if (threadIdx.x == 0) *a.plan_head = make_int4(total, sc.group_rows, 0, 0);
+    for (int b = threadIdx.x; b <= a.batch; b += blockDim.x) {
+        PlanSeq q = {};
+        q.item0 = sc.item0[b];
+        if (b < a.batch)
+            q.n = sc.n[b], q.L = sc.L[b], q.mp = sc.mp[b], q.nfull = sc.nfull[b], q.kt = sc.kt[b],
+            q.s_row = sc.s_row[b], q.s_key = sc.s_key[b];
+        a.plan_seq[b] = q;
+    }
+    for (int item = threadIdx.x; item < total; item += blockDim.x) a.plan_item[item] = plan_entry(sc, item);
+}
+
+// A CTA's view of one entry of the work list.
+__device__ __forceinline__ Item load_item(const AttnArgs& a, int item, int group_rows, int G) {
+    const int4* src = reinterpret_cast<const int4*>(a.plan_item + item);
+    const int4 lo = __ldcg(src), hi = __ldcg(src + 1);
+    Item it;
+    it.b = lo.x & 0xFFFF, it.g = static_cast<int>(static_cast<unsigned>(lo.x) >> 16);
+    it.pair = lo.y & 0xFFFF, it.splits = static_cast<int>(static_cast<unsigned>(lo.y) >> 16);
+    it.sp = lo.z, it.first_item = lo.w;
+    it.t_begin = hi.x, it.t_end = hi.y, it.n = hi.z, it.L = hi.w;
+    it.M = it.n * G;
+    it.row_base = it.pair * group_rows;
+    it.nmt = (group_rows > kBM && it.M - it.row_base > kBM) ? 2 : 1;
     it.tok0 = (it.row_base == 0) ? 0 : it.row_base / G;
     return it;
 }
@@ -427,9 +504,10 @@ struct Smem {
     static constexpr int kOffK = kOffQ + kRowTiles * kQTile;
     static constexpr int kOffV = kOffK + kStagesK * kKVTile;
     static constexpr int kOffBar = kOffV + kStagesV * kKVTile;
-    static constexpr int kNumBars = 2 * (kStagesK + kStagesV) + 1 + kRowTiles * 5 + 2;
+    static constexpr int kNumBars = 2 * (kStagesK + kStagesV) + 1 + kRowTiles * 5 + 3;
     static constexpr int kOffMisc = kOffBar + 8 * 32;
-    static constexpr int kUsed = kOffMisc + 64 + 1024;       // + slack to align the base to 1024
+    static constexpr int kOffMerge = kOffMisc + 64;          // (max, sum) of every row of both lanes
+    static constexpr int kUsed = kOffMerge + kRowTiles * kBM * 8 + 1024;  // + slack to align the base to 1024
     // Never less than 120 KB, more than half of an SM's shared memory: one CTA per SM, so the
     // 512-column TMEM allocation can never wait for a neighbour.
     static constexpr int kBytes = kUsed > 120 * 1024 ? kUsed : 120 * 1024;
@@ -456,6 +534,8 @@ __device__ __forceinline__ constexpr int bar_pfull(int m, int buf) { return kBar
 __device__ __forceinline__ constexpr int bar_pvdone(int m) { return kBar0 + 1 + m * 5 + 4; }
 __device__ __forceinline__ constexpr int bar_item() { return kBar0 + 1 + kRowTiles * 5; }
 __device__ __forceinline__ constexpr int bar_qempty() { return kBar0 + 2 + kRowTiles * 5; }
+// key mode: both softmax warpgroups have their partial result (and its PV completions) behind them
+__device__ __forceinline__ constexpr int bar_merge() { return kBar0 + 3 + kRowTiles * 5; }
 
 template <int D>
 __global__ void __launch_bounds__(kAttnThreads, 1)
@@ -463,7 +543,6 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
                       const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_q) {
     using S = Smem<D>;
     extern __shared__ unsigned char smem_raw[];
-    __shared__ Sched sc;
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     unsigned char* base_ptr = smem_raw + (base - smem_u32(smem_raw));
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -472,6 +551,22 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
     auto bar = [&](int i) { return bars + 8u * i; };
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + S::kOffMisc);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + S::kOffMisc + 8);
+
+    // The work list was written once for the whole step.  From the second layer on it is at least
+    // two kernels old: this kernel can only have started after its predecessor had started, which
+    // can only have started after every CTA of the kernel before that one had passed its own
+    // dependency wait, i.e. after the kernel that wrote the list had completed and flushed.  (Every
+    // kernel of the library signals its dependents only after its own wait, or never.)  So the
+    // list is read before the wait, under the tail of the preceding kernel; only when the list was
+    // written by the kernel immediately before this one does the read have to follow the wait.
+    // Every thread reads the CTA's first item for itself: no role waits for another.
+    int4 head = make_int4(0, 0, 0, 0);
+    Item first_it = {};
+    auto read_plan = [&]() {
+        head = __ldcg(a.plan_head);
+        if (static_cast<int>(blockIdx.x) < head.x) first_it = load_item(a, blockIdx.x, head.y, G);
+    };
+    if (!a.plan_after_wait) read_plan();
 
     // ---- one-time set-up ---------------------------------------------------------------
     if (tid == 0) {
@@ -494,6 +589,7 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
             mbar_init(bar(bar_pvdone(m)), 1);
         }
         mbar_init(bar(bar_item()), kSyncThreads);
+        mbar_init(bar(bar_merge()), kSoftmaxThreads);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == kMmaWarp0) {
@@ -512,15 +608,19 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
     // overlaps the tail of the preceding kernel.
     pdl_wait();
     pdl_launch_dependents();
+    if (a.plan_after_wait) read_plan();
     tc_fence_before();
-    build_sched(a, sc, tid);  // ends with __syncthreads(): barriers, TMEM address and schedule are visible
+    __syncthreads();  // barriers and the TMEM address are visible
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
-    const int total_items = min(sc.item0[a.batch], a.max_items);
-    // Every thread decodes the CTA's first item for itself (a CTA rarely has a second one): no
-    // role waits for another before it starts.
-    Item first_it = {};
-    if (static_cast<int>(blockIdx.x) < total_items) first_it = decode_item(sc, blockIdx.x, G);
+    const int total_items = head.x, group_rows = head.y;
+    // The list must still describe the step parameters it is used with (the caller changes them only
+    // through the library, or asks for a new list): one thread compares its item's sequence.
+    bool stale = false;
+    if (tid == 0 && static_cast<int>(blockIdx.x) < total_items) {
+        const int n_live = min(max(a.n_nodes[first_it.b], 0), a.max_tt), L_live = max(a.steps[first_it.b].prefix_len, 0);
+        stale = (n_live != first_it.n) || (L_live != first_it.L);
+    }
     // The producers issue the first copies of the CTA's first item at once.
     const bool early = (warp == kProducerWarp || warp == kVProducerWarp) && lane == 0 &&
                        static_cast<int>(blockIdx.x) < total_items;
@@ -541,7 +641,7 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
         }
     }
     auto get_item = [&](int item, int local) {  // local = how many items this CTA has started before
-        return local == 0 ? first_it : decode_item(sc, item, G);
+        return local == 0 ? first_it : load_item(a, item, group_rows, G);
     };
 
     // Running use counts of the barrier families.  Every role walks the same items and tiles in
@@ -549,6 +649,7 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
     uint32_t kt_run = 0;     // K/V ring uses (all tiles of all items)
     uint32_t jx = 0;         // tiles this lane has taken (S/P buffers, PV completions)
     uint32_t items_run = 0;
+    uint32_t merges_run = 0;  // key-mode items (uses of the merge barrier)
     bool alive = true;
 
     // Registers follow the roles: the softmax warpgroups hold a tile of S, a tile of P and a row of
@@ -951,80 +1052,122 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
             if (!alive) break;
 
             // ---- epilogue --------------------------------------------------------------
-            const bool direct = row_mode && it.splits == 1;
-            if (!first) {
-                const int t = R / G, h = it.g * G + R % G;
-                const float inv = 1.f / l_run;
-                __nv_bfloat16* dst = a.o + ((static_cast<int64_t>(it.b) * a.max_tt + t) * a.Hq + h) * D;
-                uint4* po = a.part_o + (static_cast<int64_t>(item) * kRowTiles + x) * (D / 8) * kBM + r;
-                while (pv_seen < jx) {
-                    if (!warp_wait(bar(bar_pvdone(x)), pv_seen & 1u, abort_flag)) alive = false;
-                    ++pv_seen;
-                }
+            // Row mode: the lane owns its rows and all their columns.  Key mode: the two lanes hold
+            // partial results over different keys for the same rows; they exchange (max, sum) through
+            // shared memory and each merges one half of the columns, reading the other lane's
+            // accumulator straight from tensor memory (same TMEM lanes, other columns).
+            const bool direct = it.splits == 1;  // the group's only item: the result is final
+            const int nt_oth = row_mode ? 0 : ((it.t_end - it.t_begin + (x ? 1 : 0)) >> 1);  // the other lane's tiles
+            while (pv_seen < jx) {
+                if (!warp_wait(bar(bar_pvdone(x)), pv_seen & 1u, abort_flag)) alive = false;
+                ++pv_seen;
+            }
+            if (!alive) break;
+            const bool use_self = !first, use_oth = nt_oth > 0;
+            float m_tot = (l_run > 0.f) ? m_ref : -INFINITY, l_tot = l_run, w_self = 1.f, w_oth = 0.f;
+            int c_begin = 0, c_end = D / 32;  // 32-column pieces of the row this thread writes
+            if (!row_mode) {
+                float2* xch = reinterpret_cast<float2*>(base_ptr + S::kOffMerge);
+                xch[x * kBM + r] = make_float2(m_tot, l_run);
+                tc_fence_before();
+                mbar_arrive(bar(bar_merge()));
+                alive = warp_wait(bar(bar_merge()), merges_run & 1u, abort_flag);
+                ++merges_run;
                 if (!alive) break;
-                tc_fence_after();
-                if (row_ok && direct && a.lse)
+                const float2 oth = xch[(x ^ 1) * kBM + r];
+                const float m_self = m_tot;
+                m_tot = fmaxf(m_self, oth.x);
+                w_self = (m_self == -INFINITY) ? 0.f : ex2_approx(m_self - m_tot);
+                w_oth = (oth.x == -INFINITY) ? 0.f : ex2_approx(oth.x - m_tot);
+                l_tot = l_run * w_self + oth.y * w_oth;
+                c_begin = x * (D / 64), c_end = c_begin + D / 64;
+            }
+            tc_fence_after();
+            {
+                const int t = R / G, h = it.g * G + R % G;
+                const float inv = (l_tot > 0.f) ? 1.f / l_tot : 0.f;
+                __nv_bfloat16* dst = a.o + ((static_cast<int64_t>(it.b) * a.max_tt + t) * a.Hq + h) * D;
+                const int64_t slot = static_cast<int64_t>(item) * kRowTiles + (row_mode ? x : 0);
+                uint4* po = a.part_o + slot * (D / 8) * kBM + r;
+                const uint32_t oth_t = tmem + lane_sel + (x ^ 1) * 256 + 128;
+                if (row_ok && direct && a.lse && (row_mode || x == 0))
                     a.lse[(static_cast<int64_t>(it.b) * a.max_tt + t) * a.Hq + h] =
-                        (m_ref + log2f(l_run)) * 0.6931471805599453f;
-                {
-                    // The row leaves tensor memory in 32-column pieces (plain loops: the stores, not
-                    // the loads, bound this part, and it runs once per item, so small code wins).
-                    // Partials assume a row scale of 1 and keep the row's largest magnitude; when a
-                    // row of the warp would leave the fp16 range, a second pass writes such rows
-                    // again with their scale.
-                    float am[4] = {0.f, 0.f, 0.f, 0.f};
-                    float scale = 1.f;  // O = Ohat * l * scale
-                    uint32_t orr[32];
+                        (m_tot + log2f(l_tot)) * 0.6931471805599453f;
+                // The row leaves tensor memory in 32-column pieces (plain loops: the stores, not
+                // the loads, bound this part, and it runs once per item, so small code wins).
+                // Partials assume a scale of 1 and keep the largest magnitude; when a row of the
+                // warp would leave the fp16 range, a second pass writes such rows again with
+                // their scale (a scale per half of the columns: the halves may come from
+                // different lanes).
+                float am[4] = {0.f, 0.f, 0.f, 0.f};
+                float scale = 1.f;  // O = Ohat * l * scale
+                uint32_t orr[32];
+                float f[32];
 #pragma unroll 1
-                    for (int pass = 0; pass < 2; ++pass) {
-                        const float mul = (pass == 0) ? ((direct || l_run > 0.f) ? inv : 0.f) : inv / scale;
-                        const bool store = row_ok && (pass == 0 || scale != 1.f);
+                for (int pass = 0; pass < 2; ++pass) {
+                    const float mul = (pass == 0) ? inv : inv / scale;
+                    const bool store = row_ok && (pass == 0 || scale != 1.f);
 #pragma unroll 1
-                        for (int c = 0; c < D / 32; ++c) {
+                    for (int c = c_begin; c < c_end; ++c) {
+                        // (the loads from tensor memory are warp-wide and their conditions warp-uniform)
+                        if (use_self) {
                             tmem_ld32(o_t + c * 32, orr);
                             tmem_wait_ld();
-                            if (store) {
 #pragma unroll
-                                for (int q4 = 0; q4 < 4; ++q4) {
-                                    float f[8];
+                            for (int e = 0; e < 32; ++e) f[e] = __uint_as_float(orr[e]) * w_self;
+                        } else {
 #pragma unroll
-                                    for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(orr[q4 * 8 + e]);
-                                    uint4 v;
-                                    if (direct) {
-                                        v.x = pack_bf16(f[0] * mul, f[1] * mul), v.y = pack_bf16(f[2] * mul, f[3] * mul);
-                                        v.z = pack_bf16(f[4] * mul, f[5] * mul), v.w = pack_bf16(f[6] * mul, f[7] * mul);
-                                        *reinterpret_cast<uint4*>(dst + (c * 4 + q4) * 8) = v;
-                                    } else {
-                                        am[q4] = max3(am[q4], fabsf(f[0]), fabsf(f[1]));
-                                        am[q4] = max3(am[q4], fabsf(f[2]), fabsf(f[3]));
-                                        am[q4] = max3(am[q4], fabsf(f[4]), fabsf(f[5]));
-                                        am[q4] = max3(am[q4], fabsf(f[6]), fabsf(f[7]));
-                                        v.x = pack_half2(f[0] * mul, f[1] * mul), v.y = pack_half2(f[2] * mul, f[3] * mul);
-                                        v.z = pack_half2(f[4] * mul, f[5] * mul), v.w = pack_half2(f[6] * mul, f[7] * mul);
-                                        __stcg(po + (c * 4 + q4) * kBM, v);
-                                    }
+                            for (int e = 0; e < 32; ++e) f[e] = 0.f;
+                        }
+                        if (use_oth) {
+                            tmem_ld32(oth_t + c * 32, orr);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int e = 0; e < 32; ++e) f[e] = fmaf(__uint_as_float(orr[e]), w_oth, f[e]);
+                        }
+                        if (store) {
+#pragma unroll
+                            for (int q4 = 0; q4 < 4; ++q4) {
+                                const float* g8 = f + q4 * 8;
+                                uint4 v;
+                                if (direct) {
+                                    v.x = pack_bf16(g8[0] * mul, g8[1] * mul), v.y = pack_bf16(g8[2] * mul, g8[3] * mul);
+                                    v.z = pack_bf16(g8[4] * mul, g8[5] * mul), v.w = pack_bf16(g8[6] * mul, g8[7] * mul);
+                                    *reinterpret_cast<uint4*>(dst + (c * 4 + q4) * 8) = v;
+                                } else {
+                                    am[q4] = max3(am[q4], fabsf(g8[0]), fabsf(g8[1]));
+                                    am[q4] = max3(am[q4], fabsf(g8[2]), fabsf(g8[3]));
+                                    am[q4] = max3(am[q4], fabsf(g8[4]), fabsf(g8[5]));
+                                    am[q4] = max3(am[q4], fabsf(g8[6]), fabsf(g8[7]));
+                                    v.x = pack_half2(g8[0] * mul, g8[1] * mul), v.y = pack_half2(g8[2] * mul, g8[3] * mul);
+                                    v.z = pack_half2(g8[4] * mul, g8[5] * mul), v.w = pack_half2(g8[6] * mul, g8[7] * mul);
+                                    __stcg(po + (c * 4 + q4) * kBM, v);
                                 }
                             }
                         }
-                        if (direct || pass == 1) break;
-                        // row scale: 1 unless |O / l| would exceed 2^14 (fp16 holds up to 65504)
-                        if (row_ok) {
-                            const float nmax = fmaxf(fmaxf(am[0], am[1]), fmaxf(am[2], am[3])) * inv;
-                            if (nmax > 16384.f && l_run > 0.f) scale = exp2f(ceilf(log2f(nmax)) - 14.f);
-                        }
-                        // (the loads from tensor memory are warp-wide: the whole warp goes round again)
-                        if (!__any_sync(kFull, scale != 1.f)) break;
                     }
-                    if (row_ok && !direct)
-                        __stcg(a.part_ml + (static_cast<int64_t>(item) * kRowTiles + x) * kBM + r,
-                               make_float4(l_run > 0.f ? m_ref : -INFINITY, l_run, l_run * scale, 0.f));
+                    if (direct || pass == 1) break;
+                    // scale: 1 unless |O / l| would exceed 2^14 (fp16 holds up to 65504)
+                    if (row_ok) {
+                        const float nmax = fmaxf(fmaxf(am[0], am[1]), fmaxf(am[2], am[3])) * inv;
+                        if (nmax > 16384.f) scale = exp2f(ceilf(log2f(nmax)) - 14.f);
+                    }
+                    // (the loads from tensor memory are warp-wide: the whole warp goes round again)
+                    if (!__any_sync(kFull, scale != 1.f)) break;
                 }
-                tc_fence_before();
-            } else if (!row_mode && row_ok) {
-                // key mode and no tile for this lane (a one-tile item): an empty partial
-                __stcg(a.part_ml + (static_cast<int64_t>(item) * kRowTiles + x) * kBM + r,
-                       make_float4(-INFINITY, 0.f, 0.f, 0.f));
+                if (row_ok && !direct) {
+                    float* ml = reinterpret_cast<float*>(a.part_ml + slot * kBM + r);
+                    if (row_mode) {
+                        __stcg(a.part_ml + slot * kBM + r, make_float4(m_tot, l_tot, l_tot * scale, l_tot * scale));
+                    } else if (x == 0) {
+                        __stcg(reinterpret_cast<float2*>(ml), make_float2(m_tot, l_tot));
+                        __stcg(ml + 2, l_tot * scale);
+                    } else {
+                        __stcg(ml + 3, l_tot * scale);
+                    }
+                }
             }
+            tc_fence_before();
             mbar_arrive(bar(bar_item()));
             alive = warp_wait(bar(bar_item()), items_run & 1u, abort_flag);
         }
@@ -1035,6 +1178,7 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
         *abort_flag = 1;
         atomicOr(a.status, RESPS_STATUS_WAIT_TIMEOUT);
     }
+    if (stale) atomicOr(a.status, RESPS_STATUS_STALE_PLAN);
     tc_fence_before();
     __syncthreads();
     if (warp == kMmaWarp0) {
@@ -1044,10 +1188,24 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
     }
 }
 
+// The per-sequence part of the work list, from the workspace into shared memory (the list is at
+// least two kernels old when a combine kernel starts: see the note at the attention kernel).
+__device__ __forceinline__ void load_sched(const AttnArgs& a, Sched& sc, int tid, int nthreads) {
+    for (int b = tid; b <= a.batch; b += nthreads) {
+        const int4* src = reinterpret_cast<const int4*>(a.plan_seq + b);
+        const int4 lo = __ldcg(src), hi = __ldcg(src + 1);
+        sc.item0[b] = hi.w;
+        if (b < a.batch)
+            sc.n[b] = lo.x, sc.L[b] = lo.y, sc.mp[b] = lo.z, sc.nfull[b] = lo.w, sc.kt[b] = hi.x, sc.s_row[b] = hi.y,
+            sc.s_key[b] = hi.z;
+    }
+    if (tid == 0) sc.group_rows = __ldcg(a.plan_head).y;
+    __syncthreads();
+}
+
 // Combines the partials of every (sequence, KV head, row-tile pair) group that did not write
-// O directly: O = sum_p w_p O_p / sum_p w_p l_p with w_p = 2^(m_p - max m).  A group in row mode
-// has one partial per split and row tile; a group in key mode (at most 128 rows) has two per
-// split, one from each lane.
+// O directly: O = sum_p w_p O_p / sum_p w_p l_p with w_p = 2^(m_p - max m).  A group has one
+// partial per split and row tile (in key mode the two lanes of a CTA have merged theirs already).
 template <int D>
 __global__ void __launch_bounds__(kCombineThreads) attention_combine_kernel(const AttnArgs a) {
     __shared__ Sched sc;
@@ -1061,12 +1219,12 @@ __global__ void __launch_bounds__(kCombineThreads) attention_combine_kernel(cons
                                              1ll * min(max(a.n_nodes[b], 0), a.max_tt) * a.Hq * (D / 8);
         if (!__syncthreads_or(mine)) return;
     }
-    // The work list is derived again from the step parameters (inputs of the attention kernel,
-    // complete before it ran), and the thread's first piece of work is located, before the wait
+    // The work list is fetched, and the thread's first piece of work located, before the wait
     // for the attention kernel: all of this runs while that kernel drains.
-    build_sched(a, sc, threadIdx.x);  // ends with __syncthreads()
+    load_sched(a, sc, threadIdx.x, kCombineThreads);  // ends with __syncthreads()
     const unsigned G = static_cast<unsigned>(a.Hq / a.Hkv);
     const unsigned stride = gridDim.x * kCombineThreads;
+    const unsigned group_rows = static_cast<unsigned>(sc.group_rows);
     // Work: (sequence, KV head, 8 columns, row) over the valid rows of groups that wrote partials;
     // consecutive threads take consecutive rows.  Every count fits 32 bits (at most 2^11 rows per
     // KV head, 2^4 column pieces, 2^7 heads).
@@ -1081,8 +1239,9 @@ __global__ void __launch_bounds__(kCombineThreads) attention_combine_kernel(cons
         bool key_mode = false;
         int64_t item_first = 0;
         for (; b < a.batch; ++b, idx = blockIdx.x * kCombineThreads + threadIdx.x) {
-            const int nfull = sc.nfull[b], mp_b = sc.mp[b], s_row = sc.s_row[b];
-            if (sc.n[b] == 0 || (s_row <= 1 && nfull == mp_b)) continue;  // every group wrote O directly
+            const int nfull = sc.nfull[b], mp_b = sc.mp[b], s_row = sc.s_row[b], s_key_b = sc.s_key[b];
+            if (sc.n[b] == 0 || ((s_row <= 1 || nfull == 0) && (s_key_b <= 1 || nfull == mp_b)))
+                continue;  // every group wrote O directly
             M = static_cast<unsigned>(sc.n[b]) * G;
             const unsigned per_head = M * (D / 8);
             for (; idx < a.Hkv * per_head; idx += stride) {
@@ -1090,14 +1249,14 @@ __global__ void __launch_bounds__(kCombineThreads) attention_combine_kernel(cons
                 const unsigned rem = idx - g * per_head;
                 c8 = rem / M;
                 R = rem - c8 * M;
-                const int pair = static_cast<int>(R / (kRowTiles * kBM));
+                const int pair = static_cast<int>(R / group_rows);
                 key_mode = pair >= nfull;
-                splits = key_mode ? sc.s_key[b] : s_row;
-                if (!key_mode && splits <= 1) continue;
+                splits = key_mode ? s_key_b : s_row;
+                if (splits <= 1) continue;
                 const int row_items = nfull * s_row;
-                item_first = sc.item0[b] + static_cast<int64_t>(g) * (row_items + (mp_b - nfull) * sc.s_key[b]) +
-                             (key_mode ? row_items : pair * s_row);
-                n_parts = key_mode ? 2 * splits : splits;
+                item_first = sc.item0[b] + static_cast<int64_t>(g) * (row_items + (mp_b - nfull) * s_key_b) +
+                             (key_mode ? row_items + (pair - nfull) * s_key_b : pair * s_row);
+                n_parts = splits;
                 have = true;
                 break;
             }
@@ -1111,8 +1270,8 @@ __global__ void __launch_bounds__(kCombineThreads) attention_combine_kernel(cons
 
         // ---- O = sum_p w_p O_p / sum_p w_p l_p, w_p = 2^(m_p - max m): one pass over the partials,
         // ten at a time so that their loads are in flight together ---------------------------------
-        const unsigned row2 = R % (kRowTiles * kBM);
-        const unsigned mt = row2 / kBM, r = row2 % kBM;
+        const unsigned row2 = R % group_rows;
+        const unsigned mt = row2 / kBM, r = row2 % kBM;  // (a key-mode group is one row tile: mt = 0)
         constexpr int kBatch = 10;
         float Mx = -INFINITY, den = 0.f;
         float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
@@ -1123,8 +1282,7 @@ __global__ void __launch_bounds__(kCombineThreads) attention_combine_kernel(cons
 #pragma unroll
             for (int u = 0; u < kBatch; ++u) {
                 const int p = min(p0 + u, n_parts - 1);
-                const int64_t slot = key_mode ? (item_first + (p >> 1)) * kRowTiles + (p & 1)
-                                              : (item_first + p) * kRowTiles + mt;
+                const int64_t slot = (item_first + p) * kRowTiles + mt;
                 ml[u] = a.part_ml[slot * kBM + r];  // shared by the 16 column pieces of a row: through L1
                 v[u] = __ldcg(a.part_o + (slot * (D / 8) + c8) * kBM + r);
             }
@@ -1143,7 +1301,7 @@ __global__ void __launch_bounds__(kCombineThreads) attention_combine_kernel(cons
                 if (p0 + u >= n_parts || ml[u].x == -INFINITY) continue;  // an empty partial holds no O
                 const float w = ex2_approx(ml[u].x - Mx);
                 den += ml[u].y * w;
-                const float wo = ml[u].z * w;  // O_p = Ohat * l * row scale
+                const float wo = (c8 < D / 16 ? ml[u].z : ml[u].w) * w;  // O_p = Ohat * l * scale of this half of the row
                 const uint32_t hw[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
@@ -1197,11 +1355,11 @@ __global__ void __launch_bounds__(kCombineThreads, 4) attention_combine_flat_ker
         __syncthreads();
         if (static_cast<unsigned long long>(blockIdx.x) * kCombineThreads >= s_bound) return;
     }
-    // The work list is derived again from the step parameters (inputs of the attention kernel,
-    // complete before it ran), and the thread's first piece of work is located, before the wait
+    // The work list is fetched, and the thread's first piece of work located, before the wait
     // for the attention kernel: all of this runs while that kernel drains.
-    build_sched(a, sc, threadIdx.x);  // ends with __syncthreads()
+    load_sched(a, sc, threadIdx.x, kCombineThreads);  // ends with __syncthreads()
     const unsigned G = static_cast<unsigned>(a.Hq / a.Hkv);
+    const unsigned group_rows = static_cast<unsigned>(sc.group_rows);
     if (threadIdx.x < 32) {
         // shares per piece of work and flat offsets (every sequence's range is a multiple of 4,
         // so that the shares of a piece sit in adjacent, aligned lanes)
@@ -1211,7 +1369,7 @@ __global__ void __launch_bounds__(kCombineThreads, 4) attention_combine_flat_ker
             unsigned mine = 0;
             if (b < a.batch && sc.n[b] > 0) {
                 const int nfull = sc.nfull[b], nkey = sc.mp[b] - nfull;
-                const int parts = max(nfull > 0 && sc.s_row[b] > 1 ? sc.s_row[b] : 0, nkey > 0 ? 2 * sc.s_key[b] : 0);
+                const int parts = max(nfull > 0 && sc.s_row[b] > 1 ? sc.s_row[b] : 0, nkey > 0 && sc.s_key[b] > 1 ? sc.s_key[b] : 0);
                 const unsigned shares = parts <= kCombineBatch ? 1u : parts <= 2 * kCombineBatch ? 2u : 4u;
                 s_shares[b] = static_cast<unsigned char>(shares);
                 if (parts > 0) mine = (static_cast<unsigned>(sc.n[b]) * a.Hq * (D / 8) * shares + 3u) & ~3u;
@@ -1258,15 +1416,15 @@ __global__ void __launch_bounds__(kCombineThreads, 4) attention_combine_flat_ker
                 const unsigned rem = piece - g * per_head;
                 c8 = rem / M;
                 R = rem - c8 * M;
-                const int nfull = sc.nfull[b], s_row = sc.s_row[b];
-                const int pair = static_cast<int>(R / (kRowTiles * kBM));
+                const int nfull = sc.nfull[b], s_row = sc.s_row[b], s_key_b = sc.s_key[b];
+                const int pair = static_cast<int>(R / group_rows);
                 key_mode = pair >= nfull;
-                splits = key_mode ? sc.s_key[b] : s_row;
-                if (key_mode || splits > 1) {  // otherwise the group wrote O directly
+                splits = key_mode ? s_key_b : s_row;
+                if (splits > 1) {  // otherwise the group wrote O directly
                     const int row_items = nfull * s_row;
-                    item_first = sc.item0[b] + static_cast<int64_t>(g) * (row_items + (sc.mp[b] - nfull) * sc.s_key[b]) +
-                                 (key_mode ? row_items : pair * s_row);
-                    n_parts = key_mode ? 2 * splits : splits;
+                    item_first = sc.item0[b] + static_cast<int64_t>(g) * (row_items + (sc.mp[b] - nfull) * s_key_b) +
+                                 (key_mode ? row_items + (pair - nfull) * s_key_b : pair * s_row);
+                    n_parts = splits;
                     have = true;
                 }
             }
@@ -1278,7 +1436,7 @@ __global__ void __launch_bounds__(kCombineThreads, 4) attention_combine_flat_ker
         if (!__any_sync(0xFFFFFFFFu, have)) continue;
 
         // ---- this share's partials: p = share, share + shares, ... ------------------------------
-        const unsigned row2 = R % (kRowTiles * kBM);
+        const unsigned row2 = R % group_rows;
         const unsigned mt = row2 / kBM, r = row2 % kBM;
         float Mx = -INFINITY, den = 0.f;
         float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
@@ -1290,8 +1448,7 @@ __global__ void __launch_bounds__(kCombineThreads, 4) attention_combine_flat_ker
 #pragma unroll
                 for (int u = 0; u < kCombineBatch; ++u) {
                     const int p = min(p0 + u * static_cast<int>(shares), n_parts - 1);
-                    const int64_t slot = key_mode ? (item_first + (p >> 1)) * kRowTiles + (p & 1)
-                                                  : (item_first + p) * kRowTiles + mt;
+                    const int64_t slot = (item_first + p) * kRowTiles + mt;
                     ml[u] = a.part_ml[slot * kBM + r];  // shared by the 16 column pieces of a row: through L1
                     v[u] = __ldcg(a.part_o + (slot * (D / 8) + c8) * kBM + r);
                 }
@@ -1310,7 +1467,7 @@ __global__ void __launch_bounds__(kCombineThreads, 4) attention_combine_flat_ker
                     if (p0 + u * static_cast<int>(shares) >= n_parts || ml[u].x == -INFINITY) continue;  // an empty partial holds no O
                     const float wgt = ex2_approx(ml[u].x - Mx);
                     den += ml[u].y * wgt;
-                    const float wo = ml[u].z * wgt;  // O_p = Ohat * l * row scale
+                    const float wo = (c8 < D / 16 ? ml[u].z : ml[u].w) * wgt;  // O_p = Ohat * l * scale of this half of the row
                     const uint32_t hw[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
@@ -1413,6 +1570,54 @@ bool make_q_map(CUtensorMap* map, const void* basep, int D, int G, int Hkv, int 
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Tensor maps are kept per context, keyed by everything that goes into them: a decode loop calls
+// with the same few buffers over and over, and encoding a map is a driver call.
+struct MapKey {
+    const void* base;
+    int64_t a, b, c, d;  // K/V: token, head, sequence strides and capacity; Q: G, max_tt, 0, 0
+    int hkv, batch, kind;  // kind 0: K/V cache, 1: Q
+    bool operator==(const MapKey& o) const {
+        return base == o.base && a == o.a && b == o.b && c == o.c && d == o.d && hkv == o.hkv && batch == o.batch &&
+               kind == o.kind;
+    }
+};
+struct MapKeyHash {
+    size_t operator()(const MapKey& k) const {
+        uint64_t h = reinterpret_cast<uintptr_t>(k.base) * 0x9E3779B97F4A7C15ull;
+        h ^= (static_cast<uint64_t>(k.a) * 31 + k.b) * 0xBF58476D1CE4E5B9ull + k.c + k.d * 7 + k.batch * 131 + k.kind +
+             k.hkv * 8191;
+        return static_cast<size_t>(h ^ (h >> 29));
+    }
+};
+struct HostState {
+    std::mutex mu;
+    std::unordered_map<MapKey, CUtensorMap, MapKeyHash> maps;
+    // The work list in the workspace was made for these arguments ...
+    bool plan_valid = false;
+    const resps_step* plan_steps = nullptr;
+    const int32_t* plan_n_nodes = nullptr;
+    int plan_batch = 0;
+    int64_t plan_capacity = 0;
+    cudaStream_t plan_stream = nullptr;
+    // ... and this many kernels of the library have been enqueued behind the one that wrote it.
+    int plan_age = 0;
+};
+constexpr size_t kMaxCachedMaps = 4096;
+
+HostState* host_state(const resps_ctx* ctx) { return static_cast<HostState*>(ctx->attn_host); }
+
+const CUtensorMap* cached_map(HostState* hs, const MapKey& key, int D) {
+    auto it = hs->maps.find(key);
+    if (it != hs->maps.end()) return &it->second;
+    CUtensorMap m;
+    const bool ok = key.kind == 0 ? make_kv_map(&m, key.base, D, key.d, key.hkv, key.batch, key.a, key.b, key.c)
+                                  : make_q_map(&m, key.base, D, static_cast<int>(key.a), key.hkv,
+                                               static_cast<int>(key.b), key.batch);
+    if (!ok) return nullptr;
+    if (hs->maps.size() >= kMaxCachedMaps) hs->maps.clear();
+    return &hs->maps.emplace(key, m).first->second;
+}
+
 template <int D>
 cudaError_t launch_for_dim(const resps_ctx* ctx, const AttnArgs& a, const CUtensorMap& mk, const CUtensorMap& mv,
                            const CUtensorMap& mq, cudaStream_t st) {
@@ -1436,6 +1641,8 @@ cudaError_t launch_for_dim(const resps_ctx* ctx, const AttnArgs& a, const CUtens
 }  // namespace
 
 cudaError_t attention_setup(resps_ctx* ctx) {
+    ctx->attn_host = new (std::nothrow) HostState();
+    if (!ctx->attn_host) return cudaErrorMemoryAllocation;
     cudaError_t e = cudaFuncSetAttribute(tree_attention_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          Smem<128>::kBytes);
     if (e != cudaSuccess) return e;
@@ -1457,6 +1664,21 @@ cudaError_t attention_setup(resps_ctx* ctx) {
     return cudaSuccess;
 }
 
+void attention_teardown(resps_ctx* ctx) {
+    delete host_state(ctx);
+    ctx->attn_host = nullptr;
+}
+
+// The step parameters or node counts behind `steps` may have changed (or the scheduling knobs
+// have): the next attention call derives its work list anew.
+void attention_plan_invalidate(resps_ctx* ctx, const void* steps_or_null) {
+    HostState* hs = host_state(ctx);
+    if (!hs) return;
+    std::lock_guard<std::mutex> lock(hs->mu);
+    if (steps_or_null == nullptr || steps_or_null == hs->plan_steps || steps_or_null == hs->plan_n_nodes)
+        hs->plan_valid = false;
+}
+
 cudaError_t launch_tree_attention(const resps_ctx* ctx, const resps_step* d_steps,
                                   const int32_t* d_n_nodes, int batch, const __nv_bfloat16* q,
                                   __nv_bfloat16* o, float* lse, const __nv_bfloat16* k_cache,
@@ -1475,23 +1697,47 @@ cudaError_t launch_tree_attention(const resps_ctx* ctx, const resps_step* d_step
     a.min_tiles = ctx->ws.attn_min_tiles, a.status = ctx->ws.status;
     a.rounds = ctx->ws.attn_rounds;
     a.stagger = ctx->ws.attn_stagger;
+    a.plan_head = reinterpret_cast<int4*>(ctx->ws.attn_plan);
+    a.plan_seq = reinterpret_cast<PlanSeq*>(ctx->ws.attn_plan + 16);
+    a.plan_item = reinterpret_cast<PlanItem*>(ctx->ws.attn_plan + 16 + sizeof(PlanSeq) * (ctx->shape.max_batch + 1));
     const int D = ctx->shape.head_dim;
     const int G = a.Hq / a.Hkv;
     a.q_by_tma = (G <= kBM && kBM % G == 0) ? 1 : 0;
-    CUtensorMap mk, mv, mq;
-    if (!make_kv_map(&mk, k_cache, D, capacity, a.Hkv, batch, stride_tok, stride_head, stride_seq) ||
-        !make_kv_map(&mv, v_cache, D, capacity, a.Hkv, batch, stride_tok, stride_head, stride_seq))
-        return cudaErrorInvalidValue;
+    HostState* hs = host_state(ctx);
+    std::lock_guard<std::mutex> lock(hs->mu);
+    MapKey kk = {k_cache, stride_tok, stride_head, stride_seq, capacity, a.Hkv, batch, 0};
+    MapKey kv = kk;
+    kv.base = v_cache;
+    const CUtensorMap* mk = cached_map(hs, kk, D);
+    const CUtensorMap* mv = cached_map(hs, kv, D);
+    if (!mk || !mv) return cudaErrorInvalidValue;
+    const CUtensorMap* mq = mk;  // unused by the kernel unless Q comes by TMA
     if (a.q_by_tma) {
-        if (!make_q_map(&mq, q, D, G, a.Hkv, a.max_tt, batch)) return cudaErrorInvalidValue;
-    } else {
-        mq = mk;  // unused by the kernel
+        MapKey kq = {q, G, a.max_tt, 0, 0, a.Hkv, batch, 1};
+        mq = cached_map(hs, kq, D);
+        if (!mq) return cudaErrorInvalidValue;
     }
-    return D == 128 ? launch_for_dim<128>(ctx, a, mk, mv, mq, st) : launch_for_dim<64>(ctx, a, mk, mv, mq, st);
+    // The work list: made by the first call after anything that may have changed the step, reused
+    // by the calls for the other layers.
+    const bool reuse = hs->plan_valid && hs->plan_steps == d_steps && hs->plan_n_nodes == d_n_nodes &&
+                       hs->plan_batch == batch && hs->plan_capacity == capacity && hs->plan_stream == st;
+    if (!reuse) {
+        cudaError_t e = launch_pdl(attention_plan_kernel, dim3(1), dim3(256), 0, st, a);
+        if (e != cudaSuccess) return e;
+        hs->plan_valid = true, hs->plan_steps = d_steps, hs->plan_n_nodes = d_n_nodes, hs->plan_batch = batch;
+        hs->plan_capacity = capacity, hs->plan_stream = st, hs->plan_age = 0;
+    }
+    a.plan_after_wait = hs->plan_age == 0 ? 1 : 0;
+    cudaError_t e = D == 128 ? launch_for_dim<128>(ctx, a, *mk, *mv, *mq, st) : launch_for_dim<64>(ctx, a, *mk, *mv, *mq, st);
+    hs->plan_age += 2;
+    return e;
 }
 
 int attention_item_rows() { return kRowTiles * kBM; }
 int attention_max_rounds() { return kMaxRounds; }
 int attention_max_batch() { return kMaxBatchSmem; }
+size_t attention_plan_bytes(int max_batch, int max_items) {
+    return 16 + sizeof(PlanSeq) * (max_batch + 1) + sizeof(PlanItem) * static_cast<size_t>(max_items);
+}
 
 }  // namespace resps

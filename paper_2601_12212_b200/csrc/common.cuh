@@ -36,6 +36,7 @@ struct Workspace {
     int attn_stagger = 1000;    // cycles lane 1 starts behind lane 0 (RESPS_ATTN_STAGGER)
     int attn_rounds = 0;        // 0: chosen by the work list; else forced (RESPS_ATTN_ROUNDS, for tests)
     int attn_max_items = 0;     // partial slots
+    unsigned char* attn_plan = nullptr;  // the attention work list: header, per-sequence and per-item entries
     __half* attn_part_o = nullptr;  // [items][item rows][D] fp16
     float4* attn_part_ml = nullptr; // [items][item rows]
     int attn_max_groups = 0;
@@ -52,6 +53,7 @@ struct resps_ctx {
     void* arena;
     int64_t arena_bytes;
     resps::Workspace ws;
+    void* attn_host;  // host-side state of the attention launcher (tensor-map cache, work-list bookkeeping)
 };
 
 namespace resps {
@@ -73,18 +75,22 @@ cudaError_t launch_accept_walk(const resps_ctx* ctx, const resps_step* d_steps,
                                const int32_t* parent, const int32_t* target_argmax,
                                int32_t* accept_path, int32_t* accept_len, int32_t* out_tokens,
                                resps_step* steps_next, cudaStream_t st);
-cudaError_t launch_kv_compact(const resps_ctx* ctx, const resps_step* d_steps, int batch,
+cudaError_t launch_kv_compact(const resps_ctx* ctx, const resps_step* d_steps, int steps_advanced, int batch,
                               const int32_t* accept_path, const int32_t* accept_len,
                               void* const* k_caches, void* const* v_caches, int n_layers,
                               int64_t stride_seq, int64_t stride_head, int64_t stride_tok,
-                              cudaStream_t st);
+                              int64_t capacity, cudaStream_t st);
 cudaError_t launch_tree_attention(const resps_ctx* ctx, const resps_step* d_steps,
                                   const int32_t* d_n_nodes, int batch, const __nv_bfloat16* q,
                                   __nv_bfloat16* o, float* lse, const __nv_bfloat16* k_cache,
                                   const __nv_bfloat16* v_cache, int64_t stride_seq,
                                   int64_t stride_head, int64_t stride_tok, int64_t capacity,
                                   const uint64_t* mask, float scale, cudaStream_t st);
-cudaError_t attention_setup(resps_ctx* ctx);  // one-time function attributes
+cudaError_t attention_setup(resps_ctx* ctx);  // one-time function attributes, host-side state
+void attention_teardown(resps_ctx* ctx);
+// The arrays behind `steps_or_null` (step parameters or node counts; null = any) are about to change.
+void attention_plan_invalidate(resps_ctx* ctx, const void* steps_or_null = nullptr);
+size_t attention_plan_bytes(int max_batch, int max_items);
 
 // Launch with programmatic stream serialization (see pdl_wait above).
 template <typename Kernel, typename... Args>

@@ -234,7 +234,7 @@ class Runner:
 
         # ---- compaction ------------------------------------------------------------------
         binding.resps_kv_compact(self.ctx, self.d_steps, B, self.d_path, self.d_alen, self.k_ptrs,
-                                 self.v_ptrs, self.nl, *self.kv_strides)
+                                 self.v_ptrs, self.nl, *self.kv_strides, self.cap)
         for s, acc in enumerate(accs):
             L = self.L[s]
             for l in range(self.nl):

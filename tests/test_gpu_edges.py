@@ -124,11 +124,14 @@ def test_ragged_batch_and_clamping_sets_status():
 
 
 # ------------------------------------------------------------------------ attention
-def _attention_case(n, Hq, Hkv, D, L, cap, parent=None, poison=False, seed=0, B=1, max_tt=128, v_scale=1.0):
+def _attention_case(n, Hq, Hkv, D, L, cap, parent=None, poison=False, seed=0, B=1, max_tt=128, v_scale=1.0,
+                    debug=()):
     oracle, binding, synth = _imports()
     from harness import check_attention, u16_to_bf16_cuda, bf16_to_f64
     rng = np.random.default_rng(seed)
     ctx = binding.Context(Hq, Hkv, D, 1000, max_batch=B, max_tt=max_tt, max_k=4, max_depth=4)
+    for key, value in debug:
+        ctx.debug_set(key, value)
     ns = [n] * B if isinstance(n, int) else n
     Ls = [L] * B if isinstance(L, int) else L
     q = synth.to_bf16_bits(rng.normal(size=(B, max_tt, Hq, D)).astype(np.float32).ravel()).reshape(B, max_tt, Hq, D)
@@ -195,12 +198,13 @@ def test_attention_large_values_survive_the_split_partials(n, Hq, Hkv):
 
 
 @pytest.mark.parametrize("rounds", [2, 3, 4])
-def test_attention_work_list_of_several_rounds(rounds, monkeypatch):
+def test_attention_work_list_of_several_rounds(rounds):
     """Long sequences may be cut into more items than CTAs (a CTA then takes several, one after the
-    other); the environment variable forces that on a problem small enough for the oracle."""
-    monkeypatch.setenv("RESPS_ATTN_ROUNDS", str(rounds))
-    _attention_case(40, 16, 4, 128, 9000, cap=9300, seed=rounds)
-    _attention_case([9, 70, 33], 8, 8, 128, [5000, 2500, 7777], cap=8192, seed=rounds, B=3)
+    other); the library's test-only override forces that on a problem small enough for the oracle."""
+    _, binding, _ = _imports()
+    dbg = ((binding.RESPS_DEBUG_ATTN_ROUNDS, rounds),)
+    _attention_case(40, 16, 4, 128, 9000, cap=9300, seed=rounds, debug=dbg)
+    _attention_case([9, 70, 33], 8, 8, 128, [5000, 2500, 7777], cap=8192, seed=rounds, B=3, debug=dbg)
 
 
 def test_attention_chain_mask_is_causal():
@@ -285,6 +289,25 @@ def test_attention_overflowing_sequence_is_skipped_and_flagged():
     assert ctx.status() == binding.RESPS_STATUS_KV_OVERFLOW
     assert torch.isnan(o[0].float()).all()                  # skipped
     assert not torch.isnan(o[1, :8].float()).any()          # the other sequence ran
+    # compaction of the same step: the overflowing sequence is left untouched (no slot past the cache
+    # is read or written) and flagged again, the other one is moved
+    path = torch.tensor([[0, 3, 7, -1, -1], [0, 2, 5, -1, -1]], dtype=torch.int32, device="cuda")
+    alen = torch.tensor([2, 2], dtype=torch.int32, device="cuda")
+    k0, v0 = kc.clone(), vc.clone()
+    binding.resps_kv_compact(ctx, steps, 2, path, alen, binding.layer_pointer_table([kc]),
+                             binding.layer_pointer_table([vc]), 1, cap * D, cap * D, D, cap)
+    assert ctx.status() == binding.RESPS_STATUS_KV_OVERFLOW
+    assert torch.equal(kc[0], k0[0]) and torch.equal(vc[0], v0[0])
+    assert torch.equal(kc[1, :, 11], k0[1, :, 12]) and torch.equal(vc[1, :, 12], v0[1, :, 15])
+    # a path entry outside the tree, or a negative prefix that is clamped to 0, is refused or handled too
+    bad = torch.tensor([[0, 99, -1, -1, -1], [0, -3, -1, -1, -1]], dtype=torch.int32, device="cuda")
+    one = torch.tensor([1, 1], dtype=torch.int32, device="cuda")
+    low = torch.tensor([[8, 1, 1, 10], [8, 1, 1, 10]], dtype=torch.int32, device="cuda")
+    k1, v1 = kc.clone(), vc.clone()
+    binding.resps_kv_compact(ctx, low, 2, bad, one, binding.layer_pointer_table([kc]),
+                             binding.layer_pointer_table([vc]), 1, cap * D, cap * D, D, cap)
+    assert ctx.status() == binding.RESPS_STATUS_KV_OVERFLOW
+    assert torch.equal(kc, k1) and torch.equal(vc, v1)
     ctx.close()
 
 
@@ -350,7 +373,7 @@ def test_compaction_in_place_hazard_and_strided_cache():
     steps = torch.tensor([[64, 16, 2, Ls[0]], [64, 16, 2, Ls[1]]], dtype=torch.int32, device="cuda")
     binding.resps_kv_compact(ctx, steps, B, torch.from_numpy(paths).cuda(), torch.from_numpy(alen).cuda(),
                              binding.layer_pointer_table(ks), binding.layer_pointer_table(vs), NL,
-                             Hkv * cap * (D + pad), cap * (D + pad), D + pad)
+                             Hkv * cap * (D + pad), cap * (D + pad), D + pad, cap)
     for l in range(NL):
         for s in range(B):
             hk = np.ascontiguousarray(host[l][s, :, :, :D])

@@ -30,7 +30,7 @@ def test_one_captured_step_graph_serves_changing_tree_shapes():
         binding.resps_verify_accept(r.ctx, r.d_steps, r.d_n_nodes, B, r.d_target, T * V, V, r.d_tokens, r.d_parent,
                                     r.d_argmax, r.d_path, r.d_alen, r.d_out, r.d_steps_next, stream=stream)
         binding.resps_kv_compact(r.ctx, r.d_steps, B, r.d_path, r.d_alen, r.k_ptrs, r.v_ptrs, 1, *r.kv_strides,
-                                 stream=stream)
+                                 r.cap, stream=stream)
 
     graph = None
     shapes = set()
