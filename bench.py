@@ -4,18 +4,22 @@ compaction) on seeded synthetic inputs shaped like the paper's target models.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--config 2] [--impl ours|reference]
 
-Prints ONE JSON line.  `value` is microseconds per speculative step with all inputs resident
-in HBM, measured with CUDA events around K replays of a captured CUDA graph of the step;
-`e2e` is the same step driven from pinned HOST buffers (inputs copied in, results copied out
-inside the timed region); `roofline` describes the dominant kernel (tree attention) from a
-live CUDA-event measurement; `cpu_baseline` is the CPU oracle timed on this machine's host cores.
-`--impl reference` times the CPU oracle alone.
+Prints ONE JSON line.  A step follows the chosen workload as stated: the per-step (TT, d, k) of its
+schedule (each draw held for 4 steps where the workload says so), per-sequence prefixes, the model's
+layer count, and the prefix growing by the accepted length ON THE DEVICE (the host writes no prefix
+between steps).  `value` is microseconds per speculative step with all inputs resident in HBM,
+measured with CUDA events around K replays of captured CUDA graphs of the step; `e2e` is the same
+step driven from pinned HOST buffers (inputs copied in, results copied out inside the timed region);
+`roofline` describes the dominant kernel (tree attention) from a live CUDA-event measurement,
+`roofline_by_kernel` the three bandwidth-bound kernels; `cpu_baseline` is the CPU oracle timed on
+this machine's host cores.  `--impl reference` times the CPU oracle alone.
 """
 from __future__ import annotations
 
 import argparse
 import json
 import os
+import socket
 import subprocess
 import sys
 import threading
@@ -32,17 +36,39 @@ from paper_2601_12212_b200 import synth  # noqa: E402
 METRIC = "us_per_speculative_step"
 UNIT = "us/step"
 NOMINAL_HBM_GBS = 8000.0
-# DRAM bytes of one tree_attention_kernel launch on the benchmarked workload, from the ncu capture
-# summarised in profiles/tree_attention_cfg2_ncu.md (set to None when the kernel changes).
-ATTENTION_TRAFFIC_BYTES = 5018624
+L2_BYTES = 126 * 1024 * 1024
+# DRAM bytes per launch from profiler captures, kept beside their summaries: one record per
+# (kernel, workload) with the bytes and the date of the capture; a record whose "kernel_rev" is not
+# the current revision string of that kernel's source is stale and reported as null.
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "dram_traffic.json")
 
 
 def measured_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
         j = json.load(open(p))
-        return float(j["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
-    return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+        return (float(j["hbm_gbs"]), float(j.get("bf16_tflops_sustained", 1400.0)),
+                "measured (MEASURED_PEAKS.json hbm_gbs / bf16_tflops_sustained)")
+    return 6650.0, 1400.0, "fallback (6.65 TB/s, 1.4 PFLOP/s sustained: earlier measurements on this pool)"
+
+
+def kernel_rev(source: str) -> str:
+    """Short content hash of a kernel source file: ties a stored profiler figure to the code it was taken from."""
+    import hashlib
+    path = os.path.join(ROOT, "paper_2601_12212_b200", "csrc", source)
+    return hashlib.sha1(open(path, "rb").read()).hexdigest()[:12]
+
+
+def recorded_traffic(kernel: str, workload_index: int, source: str):
+    try:
+        for rec in json.load(open(TRAFFIC_FILE))["records"]:
+            if rec["kernel"] == kernel and rec["workload"] == workload_index:
+                if rec.get("kernel_rev") == kernel_rev(source):
+                    return rec["dram_bytes_per_launch"], rec.get("captured")
+                return None, f"stale: taken from another revision of {source}"
+    except (OSError, KeyError, ValueError):
+        pass
+    return None, "no capture on record"
 
 
 # --------------------------------------------------------------------------- clocks
@@ -98,47 +124,58 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------- reference (oracle) arm
-def oracle_step_seconds(w: synth.Workload, attn_layers: int, step: int = 0):
-    """One speculative step of the CPU oracle, with `attn_layers` of the workload's layers
-    computed; returns per-phase seconds.  Single-threaded C++ (see oracle/)."""
+def oracle_step_seconds(w: synth.Workload, attn_layers: int, step: int = 0, seqs=None):
+    """One speculative step of the CPU oracle over the sequences `seqs` of the batch (all by default),
+    with `attn_layers` of the workload's layers computed; returns per-phase seconds summed over those
+    sequences.  Single-threaded C++ (see oracle/)."""
     import oracle
-    tt, d, k = synth.step_params(w, step, 0)
-    L = synth.initial_prefix(w, 0)
-    cap = L + tt + 8
-    dl = synth.draft_logits(w, step, 0, d, k)
-    t0 = time.perf_counter()
-    tree = oracle.tree_expand(synth.root_token(w, step, 0), dl, tt, d, k, L)
-    t_expand = time.perf_counter() - t0
-    n = tree.n_nodes
-    tl = synth.target_logits(w, step, 0, tree.tokens, tree.parent, n, synth.agreement_prob(w, 0))
-    t_attn = 0.0
-    caches = []
-    for l in range(attn_layers):
-        kc = np.zeros((w.n_kv_heads, cap, w.head_dim), np.uint16)
-        vc = np.zeros_like(kc)
-        pk, pv = synth.prefix_kv(w, 0, l, L)
-        tk, tv = synth.tree_kv(w, step, 0, l, n)
-        kc[:, :L], vc[:, :L] = pk, pv
-        kc[:, L:L + n], vc[:, L:L + n] = tk, tv
-        q = synth.queries(w, step, 0, l, n)
+    seqs = range(w.batch) if seqs is None else seqs
+    t_expand = t_attn = t_verify = t_compact = 0.0
+    nodes = []
+    for s in seqs:
+        tt, d, k = synth.step_params(w, step, s)
+        L = synth.initial_prefix(w, s)
+        cap = L + tt + 8
+        dl = synth.draft_logits(w, step, s, d, k)
         t0 = time.perf_counter()
-        oracle.tree_attention(q, kc, vc, L, tree.mask, 1.0 / np.sqrt(w.head_dim))
-        t_attn += time.perf_counter() - t0
-        caches.append((kc, vc))
-    t0 = time.perf_counter()
-    acc = oracle.verify_accept(tl, tree.tokens, tree.parent)
-    t_verify = time.perf_counter() - t0
-    t0 = time.perf_counter()
-    for kc, vc in caches:
-        oracle.kv_compact(kc, vc, L, acc.path)
-    t_compact = time.perf_counter() - t0
+        tree = oracle.tree_expand(synth.root_token(w, step, s), dl, tt, d, k, L)
+        t_expand += time.perf_counter() - t0
+        n = tree.n_nodes
+        nodes.append(n)
+        tl = synth.target_logits(w, step, s, tree.tokens, tree.parent, n, synth.agreement_prob(w, s))
+        caches = []
+        for l in range(attn_layers):
+            kc = np.zeros((w.n_kv_heads, cap, w.head_dim), np.uint16)
+            vc = np.zeros_like(kc)
+            pk, pv = synth.prefix_kv(w, s, l, L)
+            tk, tv = synth.tree_kv(w, step, s, l, n)
+            kc[:, :L], vc[:, :L] = pk, pv
+            kc[:, L:L + n], vc[:, L:L + n] = tk, tv
+            q = synth.queries(w, step, s, l, n)
+            t0 = time.perf_counter()
+            oracle.tree_attention(q, kc, vc, L, tree.mask, 1.0 / np.sqrt(w.head_dim))
+            t_attn += time.perf_counter() - t0
+            caches.append((kc, vc))
+        t0 = time.perf_counter()
+        acc = oracle.verify_accept(tl, tree.tokens, tree.parent)
+        t_verify += time.perf_counter() - t0
+        t0 = time.perf_counter()
+        for kc, vc in caches:
+            oracle.kv_compact(kc, vc, L, acc.path)
+        t_compact += time.perf_counter() - t0
     return {"expand": t_expand, "attn_per_layer": t_attn / max(1, attn_layers), "verify": t_verify,
-            "compact_per_layer": t_compact / max(1, attn_layers), "n_nodes": n}
+            "compact_per_layer": t_compact / max(1, attn_layers), "n_nodes": nodes}
 
 
-def oracle_us_per_step(w, parts):
-    return 1e6 * (parts["expand"] + parts["verify"] +
-                  w.n_layers * (parts["attn_per_layer"] + parts["compact_per_layer"]))
+def oracle_us_per_step(w, parts, seq_scale=1.0):
+    return 1e6 * seq_scale * (parts["expand"] + parts["verify"] +
+                              w.n_layers * (parts["attn_per_layer"] + parts["compact_per_layer"]))
+
+
+def oracle_sample_plan(w):
+    """(layers, sequences) of one step the oracle is timed on: a bounded sample (about 10-30 s of CPU
+    work), scaled to the workload's layer count and batch."""
+    return {1: (1, None), 2: (w.n_layers, None), 3: (4, None), 4: (2, None), 5: (1, (0, 1, 2))}[w.index]
 
 
 def run_reference(args, w):
@@ -147,15 +184,21 @@ def run_reference(args, w):
         return
     import oracle
     oracle.build()
-    layers = 2
+    layers = 2 if w.index != 5 else 1
+    seqs = None if w.index != 5 else (0,)
+    seq_scale = 1.0 if seqs is None else w.batch / len(seqs)
     for i in range(args.warmup):
-        oracle_step_seconds(w, 1, step=i)
+        oracle_step_seconds(w, 1, step=i, seqs=(0,))
     t0 = time.perf_counter()
-    vals = [oracle_us_per_step(w, oracle_step_seconds(w, layers, step=i)) for i in range(args.steps)]
+    vals = [oracle_us_per_step(w, oracle_step_seconds(w, layers, step=i, seqs=seqs), seq_scale)
+            for i in range(args.steps)]
     wall = time.perf_counter() - t0
     v = float(np.mean(vals))
-    sample = (f"per step: tree construction + verification of one full step and {layers} of the "
-              f"{w.n_layers} layers' attention + compaction, layer phases scaled to {w.n_layers} layers")
+    sample = (f"each of the {args.steps} timed steps computes tree construction + verification"
+              f"{'' if seqs is None else f' of {len(seqs)} of the {w.batch} sequences'} in full and {layers} of the "
+              f"{w.n_layers} layers' attention + compaction; the value scales the layer phases to {w.n_layers} layers"
+              f"{'' if seqs is None else f' and everything to {w.batch} sequences'} "
+              f"(measured on the sample: {wall / max(1, args.steps):.2f} s per step)")
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": v / 1e3, "higher_is_better": False,
@@ -163,52 +206,59 @@ def run_reference(args, w):
         "config": workload_config(w),
         "cpu_baseline": {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
         "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
-        "wall_s": wall}))
+        "wall_s": wall, "measured_sample_s_per_step": wall / max(1, args.steps)}))
 
 
-def workload_config(w, extra=None):
-    c = {"workload": f"configs[{w.index - 1}] {w.name}: batch {w.batch}, {w.n_q_heads}q/{w.n_kv_heads}kv heads, "
-                     f"head_dim {w.head_dim}, vocab {w.vocab}, prefix {w.prefix}, TT={w.tt} d={w.d} k={w.k}, "
-                     f"{w.n_layers} layers of attention+compaction per step",
-         "step": "tree_expand + n_layers x tree_attention + verify_accept + kv_compact(all layers)"}
-    if extra:
-        c.update(extra)
-    return c
+def workload_config(w):
+    """The same for both arms: what is run, not how."""
+    sched = (f"TT={w.tt} d={w.d} k={w.k}" if w.schedule == "fixed" else
+             f"(TT,d,k) drawn per sequence from TT in {list(synth.GRID_TT)} x d in 3..8 x k in 4..12, held {w.hold} steps")
+    return {"workload": f"configs[{w.index - 1}] {w.name}: batch {w.batch}, {w.n_q_heads}q/{w.n_kv_heads}kv heads, "
+                        f"head_dim {w.head_dim}, vocab {w.vocab}, prefix {w.prefix} growing by the accepted length, "
+                        f"{sched}, {w.n_layers} layers of attention+compaction per step",
+            "step": "tree_expand + n_layers x tree_attention + verify_accept + kv_compact(all layers)"}
 
 
 # ------------------------------------------------------------------------------ our arm
 class DeviceWorkload:
-    """All device state of one workload: a pool of distinct step inputs (each larger than
-    L2 together with the per-layer KV caches) and the output buffers."""
+    """All device state of one workload: a pool of step inputs (entry i = step i of the workload's
+    schedule), the per-layer KV caches and the output buffers.  The step parameters live in device
+    memory; the prefix length advances there (resps_verify_accept writes it back in place)."""
 
     def __init__(self, w: synth.Workload, pool: int, seq_offset: int = 0):
         import torch
         from paper_2601_12212_b200 import binding
         self.torch, self.binding, self.w = torch, binding, w
         dev = "cuda"
-        B, V, T, NL = w.batch, w.vocab, w.tt, w.n_layers
-        self.B, self.T, self.pool = B, T, pool
+        grid = w.schedule == "grid"
+        self.T = T = max(synth.GRID_TT) if grid else w.tt
+        self.max_k = max(synth.GRID_K) if grid else w.k
+        self.max_d = max(synth.GRID_D) if grid else w.d
+        B, V, NL = w.batch, w.vocab, w.n_layers
+        self.B, self.pool, self.seq_offset = B, pool, seq_offset
         self.ctx = binding.Context(w.n_q_heads, w.n_kv_heads, w.head_dim, V, max_batch=B, max_tt=T,
-                                   max_k=w.k, max_depth=w.d)
+                                   max_k=self.max_k, max_depth=self.max_d)
         i32 = dict(dtype=torch.int32, device=dev)
-        self.L = [synth.initial_prefix(w, seq_offset + s) for s in range(B)]
-        steps = np.array([[w.tt, w.d, w.k, self.L[s]] for s in range(B)], np.int32)
-        self.h_steps = torch.from_numpy(steps).pin_memory()
-        self.d_steps = self.h_steps.to(dev)
-        self.d_steps_next = torch.zeros(B, 4, **i32)
+        self.L0 = [synth.initial_prefix(w, seq_offset + s) for s in range(B)]
+        self.params = [[synth.step_params(w, i, seq_offset + s) for s in range(B)] for i in range(pool)]
+        steps0 = np.array([[*self.params[0][s], self.L0[s]] for s in range(B)], np.int32)
+        self.h_steps0 = torch.from_numpy(steps0).pin_memory()
+        self.d_steps = self.h_steps0.to(dev)
+        self.h_params = [torch.from_numpy(np.array(p, np.int32)).pin_memory() for p in self.params]
+        self.d_params = [h.to(dev) for h in self.h_params]
         self.tokens = torch.zeros(B, T, **i32)
         self.parent = torch.zeros(B, T, **i32)
         self.depth = torch.zeros(B, T, **i32)
         self.pos = torch.zeros(B, T, **i32)
         self.mask = torch.zeros(B, T, 2, dtype=torch.int64, device=dev)
-        self.retrieve = torch.zeros(B, T, w.d + 1, **i32)
+        self.retrieve = torch.zeros(B, T, self.max_d + 1, **i32)
         self.n_leaves = torch.zeros(B, **i32)
         self.n_nodes = torch.zeros(B, **i32)
         self.argmax = torch.zeros(B, T, **i32)
-        self.path = torch.zeros(B, w.d + 1, **i32)
+        self.path = torch.zeros(B, self.max_d + 1, **i32)
         self.alen = torch.zeros(B, **i32)
-        self.out_tokens = torch.zeros(B, w.d + 1, **i32)
-        self.result_host = torch.zeros(B, 2 * (w.d + 1) + 1, dtype=torch.int32).pin_memory()
+        self.out_tokens = torch.zeros(B, self.max_d + 1, **i32)
+        self.result_host = torch.zeros(B, 2 * (self.max_d + 1) + 1, dtype=torch.int32).pin_memory()
         self.o = torch.zeros(B, T, w.n_q_heads, w.head_dim, dtype=torch.bfloat16, device=dev)
         cap = w.kv_capacity
         self.cap = cap
@@ -216,25 +266,32 @@ class DeviceWorkload:
         g = torch.Generator(device=dev)
         g.manual_seed(1234 + seq_offset)
         kv_shape = (B, w.n_kv_heads, cap, w.head_dim)
-        # prefix and tree K/V: bf16 N(0,1).  (Timing only: values do not steer the data path of
+        # prefix and tree K/V: bf16 N(0,1) in every slot, so that whatever the prefix has grown to the
+        # tree tokens' K/V "are already there".  (Timing only: values do not steer the data path of
         # attention; the parity tests use the host-seeded generators.)
-        self.k = [torch.randn(kv_shape, generator=g, device=dev, dtype=torch.float32).bfloat16() for _ in range(NL)]
-        self.v = [torch.randn(kv_shape, generator=g, device=dev, dtype=torch.float32).bfloat16() for _ in range(NL)]
+        self.k = [torch.randn(kv_shape, generator=g, device=dev, dtype=torch.bfloat16) for _ in range(NL)]
+        self.v = [torch.randn(kv_shape, generator=g, device=dev, dtype=torch.bfloat16) for _ in range(NL)]
         self.k_ptrs = binding.layer_pointer_table(self.k)
         self.v_ptrs = binding.layer_pointer_table(self.v)
-        self.q = [torch.randn(B, T, w.n_q_heads, w.head_dim, generator=g, device=dev).bfloat16() for _ in range(NL)]
+        self.q = [torch.randn(B, T, w.n_q_heads, w.head_dim, generator=g, device=dev, dtype=torch.bfloat16)
+                  for _ in range(NL)]
         # the pool of step inputs (host-seeded, pinned for the end-to-end leg)
         self.h_draft, self.h_target, self.h_root = [], [], []
         self.d_draft, self.d_target, self.d_root = [], [], []
+        self.nodes = []
         for i in range(pool):
-            dl = np.stack([synth.draft_logits(w, i, seq_offset + s, w.d, w.k) for s in range(B)])
+            dl = np.zeros((B, self.max_d, self.max_k, V), np.float32)
+            for s in range(B):
+                tt, d, k = self.params[i][s]
+                dl[s, :d, :k] = synth.draft_logits(w, i, seq_offset + s, d, k)
             roots = np.array([synth.root_token(w, i, seq_offset + s) for s in range(B)], np.int32)
             hd = torch.from_numpy(dl).pin_memory()
             hr = torch.from_numpy(roots).pin_memory()
-            dd, dr = hd.to(dev), hr.to(dev)
-            self.h_draft.append(hd), self.h_root.append(hr), self.d_draft.append(dd), self.d_root.append(dr)
+            self.h_draft.append(hd), self.h_root.append(hr)
+            self.d_draft.append(hd.to(dev)), self.d_root.append(hr.to(dev))
             # the tree of this pool entry decides the target logits (the target "agrees" with a
             # child with probability p_agree); build it once with the library itself
+            self.set_params(i)
             self.expand(i)
             torch.cuda.synchronize()
             tok, par, nn = self.tokens.cpu().numpy(), self.parent.cpu().numpy(), self.n_nodes.cpu().numpy()
@@ -244,75 +301,104 @@ class DeviceWorkload:
                                                      synth.agreement_prob(w, seq_offset + s))
             ht = torch.from_numpy(tl).pin_memory()
             self.h_target.append(ht), self.d_target.append(ht.to(dev))
+            self.nodes.append([int(x) for x in nn])
         self.h_q = torch.stack([q.cpu() for q in self.q]).pin_memory()          # [NL][B][T][Hq][D]
-        n0 = int(self.n_nodes[0])
         self.h_tree_kv = torch.randn(2, NL, B, w.n_kv_heads, T, w.head_dim).bfloat16().pin_memory()
-        self.n0 = n0
         self.scale = 1.0 / float(np.sqrt(w.head_dim))
+        self.reset_prefix()
 
-    # -- the four calls of a step ------------------------------------------------------
+    def reset_prefix(self):
+        """Back to step 0's parameters and the initial prefix lengths (outside any timed region)."""
+        self.d_steps.copy_(self.h_steps0)
+        self.host_L = list(self.L0)
+
+    def steps_until_overflow(self):
+        grow = self.max_d + 1
+        return min((self.cap - L - self.T) // grow for L in self.L0)
+
+    # -- the calls of a step ------------------------------------------------------------
+    def set_params(self, i):
+        """(TT, d, k) of pool entry i into the device-resident step array; the prefix column stays."""
+        self.d_steps[:, :3].copy_(self.d_params[i])
+
     def expand(self, i):
-        w, V = self.w, self.w.vocab
+        V = self.w.vocab
         self.binding.resps_tree_expand(
-            self.ctx, self.d_steps, self.B, self.d_draft[i], w.d * w.k * V, w.k * V, V, w.d, w.k,
-            self.d_root[i], self.tokens, self.parent, self.depth, self.pos, self.mask, self.retrieve,
-            self.n_leaves, self.n_nodes)
+            self.ctx, self.d_steps, self.B, self.d_draft[i], self.max_d * self.max_k * V, self.max_k * V, V,
+            self.max_d, self.max_k, self.d_root[i], self.tokens, self.parent, self.depth, self.pos, self.mask,
+            self.retrieve, self.n_leaves, self.n_nodes)
 
     def attention(self, l):
         self.binding.resps_tree_attention(
             self.ctx, self.d_steps, self.n_nodes, self.B, self.q[l], self.o, None, self.k[l], self.v[l],
             *self.kv_strides, self.cap, self.mask, self.scale)
 
-    def verify(self, i):
+    def verify(self, i, advance=True):
         V = self.w.vocab
         self.binding.resps_verify_accept(
             self.ctx, self.d_steps, self.n_nodes, self.B, self.d_target[i], self.T * V, V, self.tokens,
-            self.parent, self.argmax, self.path, self.alen, self.out_tokens, self.d_steps_next)
+            self.parent, self.argmax, self.path, self.alen, self.out_tokens,
+            self.d_steps if advance else None)
 
-    def compact(self):
+    def compact(self, advanced=True):
         self.binding.resps_kv_compact(self.ctx, self.d_steps, self.B, self.path, self.alen, self.k_ptrs,
-                                      self.v_ptrs, self.w.n_layers, *self.kv_strides, self.cap)
+                                      self.v_ptrs, self.w.n_layers, *self.kv_strides, self.cap,
+                                      steps_advanced=advanced)
 
     def step(self, i):
+        self.set_params(i)
         self.expand(i)
         for l in range(self.w.n_layers):
             self.attention(l)
-        self.verify(i)
+        self.verify(i)          # prefix_len += accepted + 1, in place on the device
         self.compact()
 
-    LAUNCHES_PER_STEP = staticmethod(lambda w: 2 + 2 * w.n_layers + 2 + 1)  # scan, tree; attention + combine per layer; argmax, walk; compact
+    def launches_per_step(self):
+        # scan, tree build; the attention work list once; attention + combine per layer; arg-max, walk; compaction
+        return 2 + 1 + 2 * self.w.n_layers + 2 + 1
 
     # -- end to end: host buffers in, host result out ---------------------------------------
     def step_e2e(self, i):
+        """One host-driven step: this step's inputs go up from pinned memory, the kernels run, the
+        accepted tokens and path come back and the host waits for them (it needs them to prepare the
+        next step, here: to know where the next tree's K/V go)."""
         torch, w = self.torch, self.w
-        L = self.L[0]
-        self.d_steps.copy_(self.h_steps, non_blocking=True)
+        self.d_steps[:, :3].copy_(self.h_params[i], non_blocking=True)
         self.d_root[i].copy_(self.h_root[i], non_blocking=True)
         self.d_draft[i].copy_(self.h_draft[i], non_blocking=True)
         self.d_target[i].copy_(self.h_target[i], non_blocking=True)
         for l in range(w.n_layers):
             self.q[l].copy_(self.h_q[l], non_blocking=True)
             for s in range(self.B):
-                Ls = self.L[s]
+                Ls = self.host_L[s]
                 self.k[l][s, :, Ls:Ls + self.T].copy_(self.h_tree_kv[0, l, s], non_blocking=True)
                 self.v[l][s, :, Ls:Ls + self.T].copy_(self.h_tree_kv[1, l, s], non_blocking=True)
-        self.step(i)
-        d1 = w.d + 1
+        self.expand(i)
+        for l in range(w.n_layers):
+            self.attention(l)
+        self.verify(i)
+        self.compact()
+        d1 = self.max_d + 1
         self.result_host[:, :d1].copy_(self.out_tokens, non_blocking=True)
         self.result_host[:, d1:2 * d1].copy_(self.path, non_blocking=True)
         self.result_host[:, 2 * d1].copy_(self.alen, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+        for s in range(self.B):
+            self.host_L[s] += int(self.result_host[s, 2 * d1]) + 1
 
     def e2e_bytes(self):
-        w = self.w
-        h2d = (self.h_steps.numel() * 4 + self.h_root[0].numel() * 4 + self.h_draft[0].numel() * 4 +
+        h2d = (self.h_params[0].numel() * 4 + self.h_root[0].numel() * 4 + self.h_draft[0].numel() * 4 +
                self.h_target[0].numel() * 4 + self.h_q.numel() * 2 + self.h_tree_kv.numel() * 2)
         d2h = self.result_host.numel() * 4
         return int(h2d), int(d2h)
 
 
-def attention_algorithmic_bytes(w, L, n):
-    """Per launch (one layer, one sequence): K and V of the L+n visible slots, Q in and O out."""
-    return 2 * (L + n) * w.n_kv_heads * w.head_dim * 2 + 2 * n * w.n_q_heads * w.head_dim * 2
+def attention_algorithmic(w, Ls, ns):
+    """Per launch (one layer, the whole batch): K and V of the L+n visible slots, Q in and O out (bytes);
+    4 n Hq (L+n) D flop."""
+    by = sum(2 * (L + n) * w.n_kv_heads * w.head_dim * 2 + 2 * n * w.n_q_heads * w.head_dim * 2 for L, n in zip(Ls, ns))
+    fl = sum(4 * n * w.n_q_heads * (L + n) * w.head_dim for L, n in zip(Ls, ns))
+    return by, fl
 
 
 def max_over_ranks(values, world, device):
@@ -331,6 +417,15 @@ def whole_job_value(t_step_us, world):
     return t_step_us / world
 
 
+def pool_size(w):
+    """Distinct step inputs kept on the device: at least 4, and enough logits between two uses of
+    the same entry to exceed L2 several times where memory allows."""
+    grid = w.schedule == "grid"
+    max_d, max_k, T = (max(synth.GRID_D), max(synth.GRID_K), max(synth.GRID_TT)) if grid else (w.d, w.k, w.tt)
+    per_entry = w.batch * (max_d * max_k + T) * w.vocab * 4
+    return int(min(16, max(4, -(-3 * L2_BYTES // per_entry))))
+
+
 def run_ours(args, w):
     import torch
     import torch.distributed as dist
@@ -346,10 +441,12 @@ def run_ours(args, w):
     if world > 1:
         dist.barrier()
 
-    pool = 4
+    pool = pool_size(w)
     dw = DeviceWorkload(w, pool, seq_offset=rank * w.batch)
     stream = torch.cuda.Stream()
-    K, W = args.steps, max(3, args.warmup)
+    W = max(3, args.warmup)
+    K = max(1, min(args.steps, dw.steps_until_overflow() - W - 2))
+    flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device="cuda")
 
     def barrier():
         torch.cuda.synchronize()
@@ -368,10 +465,17 @@ def run_ours(args, w):
             with torch.cuda.graph(g, stream=stream):
                 dw.step(i)
             graphs.append(g)
+        # the dominant kernel alone: all layers of one step, back to back, on the tree of pool entry 0
+        dw.reset_prefix()
+        dw.set_params(0)
+        dw.expand(0)
+        torch.cuda.synchronize()
         attn_graph = torch.cuda.CUDAGraph()
         with torch.cuda.graph(attn_graph, stream=stream):
             for l in range(w.n_layers):
                 dw.attention(l)
+        attn_graph.replay()
+        dw.reset_prefix()
         for i in range(W):
             graphs[i % pool].replay()
         barrier()
@@ -380,26 +484,35 @@ def run_ours(args, w):
         if rank == 0:
             sampler.start()
         ev = [torch.cuda.Event(enable_timing=True) for _ in range(6)]
-        # ---- timed region 1: K whole steps, inputs resident in HBM -----------------------
+        # ---- timed region 1: K whole steps, inputs resident in HBM; the prefix advances on the device ----
         ev[0].record(stream)
         for i in range(K):
-            graphs[i % pool].replay()
+            graphs[(W + i) % pool].replay()
         ev[1].record(stream)
         barrier()
+        prefix_after = [int(x) for x in dw.d_steps[:, 3].cpu()]
         # ---- timed region 2: the dominant kernel alone (all layers, back to back) ----------
+        dw.reset_prefix()
+        dw.set_params(0)
+        dw.expand(0)
+        torch.cuda.synchronize()
+        Ka = max(1, min(K, 2000 // w.n_layers))
         ev[2].record(stream)
-        for i in range(K):
+        for i in range(Ka):
             attn_graph.replay()
         ev[3].record(stream)
         barrier()
+        attn_L = [int(x) for x in dw.d_steps[:, 3].cpu()]
+        attn_n = [int(x) for x in dw.n_nodes.cpu()]
         # ---- timed region 3: end to end from pinned host buffers ---------------------------
+        dw.reset_prefix()
         for i in range(2):
             dw.step_e2e(i % pool)
         barrier()
         Ke = max(3, min(K, 20))
         ev[4].record(stream)
         for i in range(Ke):
-            dw.step_e2e(i % pool)
+            dw.step_e2e((2 + i) % pool)
         ev[5].record(stream)
         barrier()
         if rank == 0:
@@ -407,31 +520,48 @@ def run_ours(args, w):
             # same step keeps running (untimed) until a handful of samples under this load are in
             t_stop = time.perf_counter() + 1.5
             i = 0
+            dw.reset_prefix()
             while len(sampler.lines) < 6 and time.perf_counter() < t_stop:
                 graphs[i % pool].replay()
                 i += 1
                 if i % 32 == 0:
                     torch.cuda.synchronize()
+                    dw.reset_prefix()
             torch.cuda.synchronize()
         clocks = sampler.stop() if rank == 0 else None
 
         t_step = ev[0].elapsed_time(ev[1]) * 1e3 / K            # us
-        t_attn = ev[2].elapsed_time(ev[3]) * 1e3 / (K * w.n_layers)
+        t_attn = ev[2].elapsed_time(ev[3]) * 1e3 / (Ka * w.n_layers)
         t_e2e = ev[4].elapsed_time(ev[5]) * 1e3 / Ke
 
-        # per-phase breakdown (plain launches, not part of `value`)
-        phases = {}
-        for name, fn in (("expand", dw.expand), ("verify", dw.verify), ("compact", lambda r: dw.compact())):
-            reps = 20
+        # per-phase figures (not part of `value`): each call alone between two events, L2 flushed before
+        # it (a 252 MB fill), summed over the pool entries
+        dw.reset_prefix()
+        phases, phase_bytes = {}, {}
+        for name, fn in (("expand", dw.expand), ("verify", lambda i: dw.verify(i, advance=False)),
+                         ("compact", lambda i: dw.compact(advanced=False))):
             fn(0)
             torch.cuda.synchronize()
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(stream)
-            for r in range(reps):
-                fn(r % pool)
-            b.record(stream)
-            torch.cuda.synchronize()
-            phases[name + "_us"] = a.elapsed_time(b) * 1e3 / reps
+            total, reps = 0.0, 0
+            for rep in range(3):
+                for i in range(pool):
+                    if name != "compact":
+                        dw.set_params(i)
+                        if name == "verify":
+                            dw.expand(i)
+                    flush.fill_(rep)
+                    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    a.record(stream)
+                    fn(i)
+                    b.record(stream)
+                    torch.cuda.synchronize()
+                    total += a.elapsed_time(b) * 1e3
+                    reps += 1
+            phases[name + "_us"] = total / reps
+        V = w.vocab
+        phase_bytes["scan"] = float(np.mean([sum((1 + (d - 1) * k) * V * 4 for (_, d, k) in dw.params[i])
+                                             for i in range(pool)]))
+        phase_bytes["argmax"] = float(np.mean([sum(dw.nodes[i]) * V * 4 for i in range(pool)]))
 
     t_step, t_attn, t_e2e = max_over_ranks([t_step, t_attn, t_e2e], world, "cuda")
     status = dw.ctx.status()
@@ -440,58 +570,91 @@ def run_ours(args, w):
             dist.destroy_process_group()
         return
 
-    peak, peak_src = measured_peaks()
-    n = dw.n0
-    L = dw.L[0]
-    alg = attention_algorithmic_bytes(w, L, n) * w.batch
-    achieved = alg / (t_attn * 1e-6) / 1e9
-    V = w.vocab
-    scan_bytes = (1 + (w.d - 1) * w.k) * V * 4 * w.batch
-    argmax_bytes = n * V * 4 * w.batch
+    hbm_peak, tensor_peak, peak_src = measured_peaks()
+    alg_bytes, alg_flop = attention_algorithmic(w, attn_L, attn_n)
+    achieved = alg_bytes / (t_attn * 1e-6) / 1e9
+    tflops = alg_flop / (t_attn * 1e-6) / 1e12
+    # the roof that binds the attention launch: the slower of its HBM time and its tensor-pipe time
+    t_hbm, t_tensor = alg_bytes / (hbm_peak * 1e9), alg_flop / (tensor_peak * 1e12)
+    bound = "hbm" if t_hbm >= t_tensor else "tensor"
     h2d, d2h = dw.e2e_bytes()
+    traffic, traffic_note = recorded_traffic("tree_attention_kernel", w.index, "attention.cu")
+
+    def hbm_entry(kernel, by, us, note):
+        gbs = by / (us * 1e-6) / 1e9
+        return {"kernel": kernel, "bound": "hbm", "algorithmic_bytes": by, "us": us, "achieved": gbs, "unit": "GB/s",
+                "peak": hbm_peak, "frac": gbs / hbm_peak, "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS, "timing": note}
+
+    by_kernel = [
+        dict(hbm_entry("tree_attention_kernel (one resps_tree_attention call, whole batch)", alg_bytes, t_attn,
+                       "CUDA events around a replayed graph of all layers, back to back"),
+             flop=alg_flop, tflops=tflops,
+             binding_roof=bound,
+             frac_of_binding_roof=(achieved / hbm_peak if bound == "hbm" else tflops / tensor_peak),
+             tensor_peak_tflops=tensor_peak),
+        hbm_entry("row_scan_stream_kernel + tree_build_kernel (one resps_tree_expand call)", phase_bytes["scan"],
+                  phases["expand_us"], "one call between two events after an L2 flush, mean over the pool"),
+        hbm_entry("row_argmax_kernel + accept_walk_kernel (one resps_verify_accept call)", phase_bytes["argmax"],
+                  phases["verify_us"], "one call between two events after an L2 flush, mean over the pool"),
+    ]
 
     # CPU baseline: the oracle as it stands, one core, a bounded sample of the same workload
-    cpu_layers = w.n_layers if w.index == 2 else 1
+    cpu_layers, cpu_seqs = oracle_sample_plan(w)
+    seq_scale = 1.0 if cpu_seqs is None else w.batch / len(cpu_seqs)
     t0 = time.perf_counter()
-    parts = oracle_step_seconds(w, cpu_layers)
+    parts = oracle_step_seconds(w, cpu_layers, seqs=cpu_seqs)
     cpu_wall = time.perf_counter() - t0
-    cpu = {"value": oracle_us_per_step(w, parts), "unit": UNIT, "cores": 1, "kind": "oracle",
-           "sample": f"one step: tree construction + verification in full, {cpu_layers} of {w.n_layers} "
-                     f"layers of attention + compaction scaled to {w.n_layers} ({cpu_wall:.1f} s of CPU work)",
+    cpu = {"value": oracle_us_per_step(w, parts, seq_scale), "unit": UNIT, "cores": 1, "kind": "oracle",
+           "sample": f"step 0: tree construction + verification in full"
+                     f"{'' if cpu_seqs is None else f' for {len(cpu_seqs)} of {w.batch} sequences'}, {cpu_layers} of "
+                     f"{w.n_layers} layers of attention + compaction; scaled to {w.n_layers} layers"
+                     f"{'' if cpu_seqs is None else f' and {w.batch} sequences'} ({cpu_wall:.1f} s of CPU work)",
            "host_cores_available": os.cpu_count(),
-           "phases_us": {"expand": parts["expand"] * 1e6, "attention_per_layer": parts["attn_per_layer"] * 1e6,
-                         "verify": parts["verify"] * 1e6, "compact_per_layer": parts["compact_per_layer"] * 1e6}}
+           "phases_us": {"expand": parts["expand"] * 1e6 * seq_scale,
+                         "attention_per_layer": parts["attn_per_layer"] * 1e6 * seq_scale,
+                         "verify": parts["verify"] * 1e6 * seq_scale,
+                         "compact_per_layer": parts["compact_per_layer"] * 1e6 * seq_scale}}
 
     line = {
         "metric": METRIC, "value": whole_job_value(t_step, world), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": t_step / 1e3, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16 attention (fp32 accumulate), fp32 logits", "data": "synthetic (seeded)",
-        "config": workload_config(w, {
-            "l2": f"inputs larger than L2: pool of {pool} distinct logit sets "
-                  f"({(scan_bytes + argmax_bytes) * pool / 1e6:.0f} MB) and {w.n_layers} distinct KV-cache "
-                  f"layers ({alg * w.n_layers / 1e6:.0f} MB read per step)",
-            "launch": "CUDA graph of one whole step, replayed", "replicas": world,
-            "n_nodes": n, "prefix_len": L}),
+        "config": workload_config(w),
+        "run": {"l2": f"inputs larger than L2: pool of {pool} distinct step inputs "
+                      f"({(phase_bytes['scan'] + phase_bytes['argmax']) * pool / 1e6:.0f} MB of logits) and {w.n_layers} "
+                      f"distinct KV-cache layers ({alg_bytes * w.n_layers / 1e6:.0f} MB read per step)",
+                "launch": "one CUDA graph of a whole step per pool entry, replayed; step parameters and prefix "
+                          "lengths live in device memory and the prefix advances there",
+                "replicas": world, "pool": pool, "prefix_start": dw.L0, "prefix_after_timed_steps": prefix_after,
+                "n_nodes_per_pool_entry": dw.nodes[:4]},
         "e2e": {"value": t_e2e / world, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "steps": Ke},
-        "gpu_launches": DeviceWorkload.LAUNCHES_PER_STEP(w) * K,
-        "gpu_launches_per_step": DeviceWorkload.LAUNCHES_PER_STEP(w),
-        "roofline": {"kernel": "tree_attention_kernel (+ attention_combine_kernel, one resps_tree_attention call)",
-                     "bound": "hbm", "achieved": achieved, "peak": peak,
-                     "unit": "GB/s", "frac": achieved / peak, "traffic": ATTENTION_TRAFFIC_BYTES,
-                     "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of tree_attention_kernel, "
-                                       "one launch of this workload (profiles/tree_attention_cfg2_ncu.md)",
-                     "peak_source": peak_src, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
-                     "algorithmic_bytes_per_launch": alg, "us_per_launch": t_attn,
-                     "launches_timed": K * w.n_layers},
-        "phases": dict(phases, attention_per_layer_us=t_attn,
-                       scan_gbs=scan_bytes / (phases["expand_us"] * 1e-6) / 1e9,
-                       argmax_gbs=argmax_bytes / (phases["verify_us"] * 1e-6) / 1e9),
+        "gpu_launches": dw.launches_per_step() * K,
+        "gpu_launches_per_step": dw.launches_per_step(),
+        "roofline": {"kernel": "tree_attention_kernel (one resps_tree_attention call)",
+                     "bound": bound, "achieved": achieved if bound == "hbm" else tflops,
+                     "peak": hbm_peak if bound == "hbm" else tensor_peak,
+                     "unit": "GB/s" if bound == "hbm" else "TFLOP/s",
+                     "frac": achieved / hbm_peak if bound == "hbm" else tflops / tensor_peak,
+                     "traffic": traffic, "traffic_source": traffic_note,
+                     "peak_source": peak_src, "hbm_gbs": achieved, "hbm_frac_of_measured": achieved / hbm_peak,
+                     "hbm_frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS, "tflops": tflops,
+                     "algorithmic_bytes_per_launch": alg_bytes, "algorithmic_flop_per_launch": alg_flop,
+                     "us_per_launch": t_attn, "launches_timed": Ka * w.n_layers,
+                     "prefix_len": attn_L, "n_nodes": attn_n},
+        "roofline_by_kernel": by_kernel,
+        "phases": dict(phases, attention_per_layer_us=t_attn),
         "cpu_baseline": cpu, "clocks": clocks, "device_status": status,
     }
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
+
+
+def free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
 
 
 def main():
@@ -503,6 +666,15 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     args = ap.parse_args()
     w = synth.WORKLOADS[args.config]
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # not under a launcher: start one replica per GPU ourselves
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+               "--master-addr", "127.0.0.1", "--master-port", str(free_port()), os.path.abspath(__file__)] + sys.argv[1:]
+        sys.exit(subprocess.call(cmd))
+    if world != args.gpus:
+        sys.exit(f"bench.py: --gpus {args.gpus} but WORLD_SIZE={world}: start it with one rank per GPU "
+                 f"(or without a launcher, then it starts the ranks itself)")
     if args.impl == "reference":
         run_reference(args, w)
     else:

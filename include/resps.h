@@ -94,7 +94,9 @@ int resps_create(resps_ctx** out, const resps_shape* shape);
 int resps_destroy(resps_ctx* ctx);
 /* Static string for a return code. */
 const char* resps_strerror(int code);
-/* Synchronises `stream`, copies the device status word to *status and clears it. */
+/* Synchronises `stream`, copies the device status word to *status and clears it.  After a
+ * RESPS_STATUS_WAIT_TIMEOUT it also resets the workspace's arrival counters, so that the context
+ * can serve further calls. */
 int resps_status(resps_ctx* ctx, resps_stream stream, int32_t* status);
 /* Bytes of device workspace held by the context. */
 int64_t resps_workspace_bytes(const resps_ctx* ctx);

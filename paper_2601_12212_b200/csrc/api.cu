@@ -178,6 +178,16 @@ int resps_status(resps_ctx* ctx, resps_stream stream, int32_t* status) {
         return RESPS_ERR_CUDA;
     if (cudaMemsetAsync(ctx->ws.status, 0, sizeof(int32_t), stream) != cudaSuccess) return RESPS_ERR_CUDA;
     if (cudaStreamSynchronize(stream) != cudaSuccess) return RESPS_ERR_CUDA;
+    if (*status & RESPS_STATUS_WAIT_TIMEOUT) {
+        // a kernel that gave up may have left arrival counters half-way: start them again from zero
+        const resps::Workspace& w = ctx->ws;
+        const size_t rows = static_cast<size_t>(ctx->shape.max_batch) * w.max_rows;
+        const size_t nodes = static_cast<size_t>(ctx->shape.max_batch) * ctx->shape.max_tt;
+        if (cudaMemsetAsync(w.row_counter, 0, rows * sizeof(unsigned int), stream) != cudaSuccess ||
+            cudaMemsetAsync(w.amax_counter, 0, nodes * sizeof(unsigned int), stream) != cudaSuccess ||
+            cudaStreamSynchronize(stream) != cudaSuccess)
+            return RESPS_ERR_CUDA;
+    }
     return RESPS_OK;
 }
 
