@@ -110,7 +110,6 @@ int resps_create(resps_ctx** out, const resps_shape* shape) {
     const int G = s.n_q_heads / s.n_kv_heads;
     const int item_rows = resps::attention_item_rows();
     w.attn_grid = c->sm_count;
-    w.attn_combine_grid = c->sm_count * 4;
     w.attn_min_tiles = 2;
     w.attn_max_groups = s.max_batch * s.n_kv_heads * ((s.max_tt * G + item_rows / 2 - 1) / (item_rows / 2));  // single row tiles
     w.attn_max_items = resps::attention_max_rounds() * w.attn_grid + w.attn_max_groups;

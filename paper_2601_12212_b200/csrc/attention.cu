@@ -1203,11 +1203,150 @@ __device__ __forceinline__ void load_sched(const AttnArgs& a, Sched& sc, int tid
     __syncthreads();
 }
 
-// Combines the partials of every (sequence, KV head, row-tile pair) group that did not write
-// O directly: O = sum_p w_p O_p / sum_p w_p l_p with w_p = 2^(m_p - max m).  A group has one
-// partial per split and row tile (in key mode the two lanes of a CTA have merged theirs already).
+// Combines the partials of every (sequence, KV head, group of row tiles) that did not write O
+// directly: O = sum_p w_p O_p / sum_p w_p l_p with w_p = 2^(m_p - max m).  A group has one partial
+// per split and row tile (in key mode the two lanes of a CTA have merged theirs already).
+//
+// The kernel is two dependent round trips to L2 (partials in, O out) behind a dependency wait, so
+// what counts is how many memory requests an SM has to issue: with plain loads a warp-load is four
+// 128-byte requests, an SM can only keep so many in flight, and 100 requests per warp made the
+// kernel several round trips long.  Here a CTA takes one row tile x two 8-column pieces and lets
+// the copy engine fetch its share of every partial (one bulk copy per partial and column piece,
+// one for the (max, sum, scales) of the rows) into shared memory: a few dozen requests per CTA, all
+// in flight at once.
+constexpr int kCombChunk = 8;   // partials fetched together
+constexpr int kCombPieces = 2;  // 8-column pieces per CTA
+constexpr int kCombSlotBytes = (kCombPieces + 1) * kBM * 16;  // per partial: the pieces, then (max, sum, scales)
+
 template <int D>
 __global__ void __launch_bounds__(kCombineThreads) attention_combine_kernel(const AttnArgs a) {
+    constexpr int kPieces = D / 8;                    // 16-byte pieces of a row
+    constexpr int kCtasPerTile = kPieces / kCombPieces;
+    static_assert(kCombineThreads == kCombPieces * kBM, "thread = (row, piece)");
+    extern __shared__ __align__(128) unsigned char comb_smem[];  // [kCombChunk][kCombSlotBytes]
+    __shared__ Sched sc;
+    __shared__ __align__(8) unsigned long long s_bar;
+    pdl_launch_dependents();
+    // The work list is fetched and the CTA's share located before the wait for the attention
+    // kernel: all of this runs while that kernel drains.  A CTA without work leaves at once.
+    load_sched(a, sc, threadIdx.x, kCombineThreads);  // ends with __syncthreads()
+    const int tid = threadIdx.x;
+    const int G = a.Hq / a.Hkv;
+    const int group_rows = sc.group_rows;
+    int blk = blockIdx.x, b = 0, tiles = 0;
+    for (; b < a.batch; ++b) {
+        tiles = ceil_div(sc.n[b] * G, kBM);
+        if (blk < a.Hkv * tiles * kCtasPerTile) break;
+        blk -= a.Hkv * tiles * kCtasPerTile;
+    }
+    if (b == a.batch) return;
+    const int M = sc.n[b] * G;
+    const int g = blk / (tiles * kCtasPerTile);
+    const int tile = (blk - g * tiles * kCtasPerTile) / kCtasPerTile;
+    const int c8_0 = (blk % kCtasPerTile) * kCombPieces;
+    const int R0 = tile * kBM;
+    const int nfull = sc.nfull[b], s_row = sc.s_row[b], s_key = sc.s_key[b];
+    const int pair = R0 / group_rows;
+    const bool key_mode = pair >= nfull;
+    const int splits = key_mode ? s_key : s_row;
+    if (splits <= 1) return;  // the group wrote O directly
+    const int row_items = nfull * s_row;
+    const int64_t item_first = sc.item0[b] + static_cast<int64_t>(g) * (row_items + (sc.mp[b] - nfull) * s_key) +
+                               (key_mode ? row_items + (pair - nfull) * s_key : pair * s_row);
+    const int mt = (R0 % group_rows) / kBM;  // row tile inside the group (a key-mode group is one tile)
+    const int nv = min(kBM, M - R0);         // valid rows of the tile
+    const uint32_t bar = smem_u32(&s_bar);
+    if (tid == 0) {
+        mbar_init(bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    const int r = tid % kBM, cc = tid / kBM;
+    pdl_wait();  // the attention kernel has finished and its partials are visible
+
+    float Mx = -INFINITY, den = 0.f;
+    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    bool ok = true;
+    uint32_t phase = 0;
+#pragma unroll 1
+    for (int p0 = 0; p0 < splits; p0 += kCombChunk, phase ^= 1u) {
+        const int np = min(kCombChunk, splits - p0);
+        // one copy per thread, so that they are issued side by side: a partial's column pieces and
+        // its (max, sum, scales), each nv x 16 contiguous bytes
+        if (tid == 0) mbar_expect_tx(bar, static_cast<uint32_t>(np * (kCombPieces + 1) * nv * 16));
+        if (tid < np * (kCombPieces + 1)) {
+            const int u = tid / (kCombPieces + 1), c = tid % (kCombPieces + 1);
+            const int64_t slot = (item_first + p0 + u) * kRowTiles + mt;
+            const uint32_t dst = smem_u32(comb_smem + u * kCombSlotBytes + c * kBM * 16);
+            const void* src = (c < kCombPieces) ? static_cast<const void*>(a.part_o + (slot * kPieces + c8_0 + c) * kBM)
+                                                : static_cast<const void*>(a.part_ml + slot * kBM);
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+                         "l"(src), "r"(nv * 16), "r"(bar)
+                         : "memory");
+        }
+        {
+            // bounded: on expiry the status word is flagged and the CTA leaves without a result
+            const uint32_t t0 = static_cast<uint32_t>(clock());
+            uint32_t spins = 0;
+            while (ok && !mbar_try(bar, phase))
+                if ((++spins & 255u) == 0u && static_cast<uint32_t>(clock()) - t0 > kWaitLimitCycles) ok = false;
+        }
+        if (!__syncthreads_and(ok)) {
+            if (tid == 0) atomicOr(a.status, RESPS_STATUS_WAIT_TIMEOUT);
+            return;
+        }
+        if (r < nv) {
+            float mx = Mx;
+            for (int u = 0; u < np; ++u)
+                mx = fmaxf(mx, reinterpret_cast<const float4*>(comb_smem + u * kCombSlotBytes + kCombPieces * kBM * 16)[r].x);
+            if (mx != -INFINITY) {
+                const float corr = ex2_approx(Mx - mx);  // 0 on the first chunk
+                den *= corr;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc[e] *= corr;
+                Mx = mx;
+#pragma unroll 2
+                for (int u = 0; u < np; ++u) {
+                    const unsigned char* sl = comb_smem + u * kCombSlotBytes;
+                    const float4 ml = reinterpret_cast<const float4*>(sl + kCombPieces * kBM * 16)[r];
+                    if (ml.x == -INFINITY) continue;  // an empty partial holds no O
+                    const float w = ex2_approx(ml.x - Mx);
+                    den += ml.y * w;
+                    const float wo = (c8_0 + cc < kPieces / 2 ? ml.z : ml.w) * w;  // O_p = Ohat * l * scale of this half
+                    const uint4 v = reinterpret_cast<const uint4*>(sl + cc * kBM * 16)[r];
+                    const uint32_t hw[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&hw[e]));
+                        acc[2 * e] += f.x * wo, acc[2 * e + 1] += f.y * wo;
+                    }
+                }
+            }
+        }
+        if (p0 + kCombChunk < splits) __syncthreads();  // the next chunk overwrites the staging area
+    }
+    if (r >= nv) return;
+    const float inv = 1.f / den;
+    const int R = R0 + r;
+    const int t = R / G, h = g * G + (R - t * G);
+    __nv_bfloat16* dst = a.o + ((static_cast<int64_t>(b) * a.max_tt + t) * a.Hq + h) * D + (c8_0 + cc) * 8;
+    uint4 out;
+    out.x = pack_bf16(acc[0] * inv, acc[1] * inv);
+    out.y = pack_bf16(acc[2] * inv, acc[3] * inv);
+    out.z = pack_bf16(acc[4] * inv, acc[5] * inv);
+    out.w = pack_bf16(acc[6] * inv, acc[7] * inv);
+    *reinterpret_cast<uint4*>(dst) = out;
+    if (a.lse && c8_0 + cc == 0)
+        a.lse[(static_cast<int64_t>(b) * a.max_tt + t) * a.Hq + h] = (Mx + log2f(den)) * 0.6931471805599453f;
+}
+
+// The same with plain loads, one thread per (row, 8 columns) over a flat index space: its first
+// data arrives sooner than through the copy engine, which wins when there is little to combine (a
+// single sequence with at most two row tiles per KV head: 12.0 against 13.3 us per call on the
+// 8B-shaped workload); with more rows the copy-engine form is ahead (26.4 against 28.1 us on the
+// 70B-shaped one).
+template <int D>
+__global__ void __launch_bounds__(kCombineThreads) attention_combine_small_kernel(const AttnArgs a) {
     __shared__ Sched sc;
     pdl_launch_dependents();
     // A CTA past the last row of the largest tree has nothing to do.  It learns that from one
@@ -1633,9 +1772,16 @@ cudaError_t launch_for_dim(const resps_ctx* ctx, const AttnArgs& a, const CUtens
         const int grid = static_cast<int>(std::min<long long>(ctx->ws.attn_combine_flat_grid, std::max<long long>(most, 1)));
         return launch_pdl(attention_combine_flat_kernel<D>, dim3(grid), dim3(kCombineThreads), 0, st, a);
     }
-    const long long most = (a.batch * pieces + kCombineThreads - 1) / kCombineThreads;
-    const int grid = static_cast<int>(std::min<long long>(ctx->ws.attn_combine_grid, std::max<long long>(most, 1)));
-    return launch_pdl(attention_combine_kernel<D>, dim3(grid), dim3(kCombineThreads), 0, st, a);
+    const int G = a.Hq / a.Hkv;
+    if (a.max_tt * G <= kRowTiles * kBM) {
+        const long long few = (a.batch * pieces + kCombineThreads - 1) / kCombineThreads;
+        return launch_pdl(attention_combine_small_kernel<D>, dim3(static_cast<unsigned>(std::max<long long>(few, 1))),
+                          dim3(kCombineThreads), 0, st, a);
+    }
+    // one CTA per (row tile, pair of column pieces) of the largest trees (CTAs past the trees at hand leave at once)
+    const long long most = 1ll * a.batch * a.Hkv * ((a.max_tt * G + kBM - 1) / kBM) * (D / 8 / kCombPieces);
+    return launch_pdl(attention_combine_kernel<D>, dim3(static_cast<unsigned>(std::max<long long>(most, 1))),
+                      dim3(kCombineThreads), kCombChunk * kCombSlotBytes, st, a);
 }
 
 }  // namespace
@@ -1648,14 +1794,13 @@ cudaError_t attention_setup(resps_ctx* ctx) {
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(tree_attention_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<64>::kBytes);
     if (e != cudaSuccess) return e;
-    // The combine kernel runs as one resident round: a CTA that has to wait for a free SM pays
-    // its set-up after the attention kernel has ended instead of under its tail.
-    int per_sm = 0;
-    e = (ctx->shape.head_dim == 128)
-            ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, attention_combine_kernel<128>, kCombineThreads, 0)
-            : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, attention_combine_kernel<64>, kCombineThreads, 0);
+    e = cudaFuncSetAttribute(attention_combine_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             kCombChunk * kCombSlotBytes);
     if (e != cudaSuccess) return e;
-    ctx->ws.attn_combine_grid = ctx->sm_count * std::max(per_sm, 1);
+    e = cudaFuncSetAttribute(attention_combine_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             kCombChunk * kCombSlotBytes);
+    if (e != cudaSuccess) return e;
+    int per_sm = 0;
     e = (ctx->shape.head_dim == 128)
             ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, attention_combine_flat_kernel<128>, kCombineThreads, 0)
             : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, attention_combine_flat_kernel<64>, kCombineThreads, 0);

@@ -30,7 +30,6 @@ struct Workspace {
     unsigned int* amax_counter = nullptr;    // [max_batch][max_tt]
     // attention
     int attn_grid = 0;          // persistent CTAs (one per SM)
-    int attn_combine_grid = 0;  // CTAs of the partial-combine kernel
     int attn_combine_flat_grid = 0;  // ... of its variant for batches
     int attn_min_tiles = 0;     // smallest key-tile count a split is given
     int attn_stagger = 1000;    // cycles lane 1 starts behind lane 0 (RESPS_ATTN_STAGGER)
