@@ -23,8 +23,20 @@ def _newer(target: str, deps) -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
+WAIT_TEST_LIB = os.path.join(HERE, "libresps_waittest.so")
+
+
+def build(force: bool = False, verbose: bool = False, wait_test: bool = False) -> str:
+    """Builds the library.  wait_test=True builds the separate test library instead
+    (-DRESPS_WAIT_TEST: millisecond wait limits and a switch that leaves out one copy); it is
+    loaded by the bounded-wait test only, never by the binding."""
     nvcc = os.environ.get("NVCC", "nvcc")
+    if wait_test:
+        return _build_into(nvcc, os.path.join(OBJ, "waittest"), WAIT_TEST_LIB, ["-DRESPS_WAIT_TEST"], force, verbose)
+    return _build_into(nvcc, OBJ, LIB, [], force, verbose)
+
+
+def _build_into(nvcc, OBJ, LIB, extra_flags, force, verbose) -> str:
     os.makedirs(OBJ, exist_ok=True)
     headers = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".cuh", ".h"))]
     headers.append(os.path.join(ROOT, "include", "resps.h"))
@@ -33,7 +45,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         s = os.path.join(CSRC, src)
         o = os.path.join(OBJ, src.replace(".cu", ".o"))
         if force or _newer(o, [s] + headers):
-            cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-c", s, "-o", o]
+            cmd = [nvcc] + NVCC_FLAGS + extra_flags + (["-Xptxas", "-v"] if verbose else []) + ["-c", s, "-o", o]
             jobs.append(cmd)
     if jobs:
         with ThreadPoolExecutor(max_workers=len(jobs)) as ex:

@@ -13,59 +13,14 @@ namespace {
 
 constexpr unsigned kFull = 0xFFFFFFFFu;
 
-struct AcceptArgs {
-    const resps_step* steps;
-    const int32_t* n_nodes;
-    const int32_t *tokens, *parent, *target_argmax;
-    int max_tt, max_depth;
-    int32_t *accept_path, *accept_len, *out_tokens;
-    resps_step* steps_next;
-};
-
-// One CTA of 128 threads per sequence: thread c owns tree node c.
+// One CTA of 128 threads per sequence: thread c owns tree node c.  (Used when the arg-max kernel
+// could not take the walk along: rows that are not 16-byte aligned.)
 __global__ void __launch_bounds__(RESPS_MAX_TT) accept_walk_kernel(const AcceptArgs a) {
     pdl_wait();  // the kernel before this one in the stream has completed
     pdl_launch_dependents();
-    const int b = blockIdx.x, tid = threadIdx.x;
-    const int n = min(max(a.n_nodes[b], 1), a.max_tt);
-    const int64_t ob = static_cast<int64_t>(b) * a.max_tt;
-    const int cap = a.max_depth + 1;
     __shared__ int s_tgt[RESPS_MAX_TT];
     __shared__ int s_next;
-    const int my_tok = (tid < n) ? a.tokens[ob + tid] : -1;
-    const int my_par = (tid < n) ? a.parent[ob + tid] : -2;
-    if (tid < n) s_tgt[tid] = a.target_argmax[ob + tid];
-    if (tid < cap) {
-        a.accept_path[b * cap + tid] = (tid == 0) ? 0 : -1;
-        a.out_tokens[b * cap + tid] = -1;
-    }
-    __syncthreads();
-    int cur = 0, len = 0;
-    for (int hop = 0; hop < a.max_depth; ++hop) {
-        if (tid == 0) s_next = -1;
-        __syncthreads();
-        // children of one node carry distinct tokens, so at most one thread matches
-        if (tid > 0 && tid < n && my_par == cur && my_tok == s_tgt[cur]) s_next = tid;
-        __syncthreads();
-        const int nxt = s_next;
-        __syncthreads();
-        if (nxt < 0) break;
-        cur = nxt;
-        ++len;
-        if (tid == 0) {
-            a.accept_path[b * cap + len] = cur;
-            a.out_tokens[b * cap + len - 1] = a.tokens[ob + cur];
-        }
-    }
-    if (tid == 0) {
-        a.out_tokens[b * cap + len] = s_tgt[cur];
-        a.accept_len[b] = len;
-        if (a.steps_next) {
-            resps_step s = a.steps[b];
-            s.prefix_len += len + 1;
-            a.steps_next[b] = s;
-        }
-    }
+    accept_walk_device(a, blockIdx.x, threadIdx.x, s_tgt, &s_next, [] { __syncthreads(); });
 }
 
 struct CompactArgs {
@@ -131,17 +86,25 @@ __global__ void __launch_bounds__(128) kv_compact_kernel(const CompactArgs a) {
 
 }  // namespace
 
-cudaError_t launch_accept_walk(const resps_ctx* ctx, const resps_step* d_steps,
-                               const int32_t* d_n_nodes, int batch, const int32_t* tokens,
-                               const int32_t* parent, const int32_t* target_argmax,
-                               int32_t* accept_path, int32_t* accept_len, int32_t* out_tokens,
-                               resps_step* steps_next, cudaStream_t st) {
+AcceptArgs make_accept_args(const resps_ctx* ctx, const resps_step* d_steps, const int32_t* d_n_nodes,
+                            const int32_t* tokens, const int32_t* parent, const int32_t* target_argmax,
+                            int32_t* accept_path, int32_t* accept_len, int32_t* out_tokens, resps_step* steps_next) {
     AcceptArgs a;
     a.steps = d_steps, a.n_nodes = d_n_nodes;
     a.tokens = tokens, a.parent = parent, a.target_argmax = target_argmax;
     a.max_tt = ctx->shape.max_tt, a.max_depth = ctx->shape.max_depth;
     a.accept_path = accept_path, a.accept_len = accept_len, a.out_tokens = out_tokens;
     a.steps_next = steps_next;
+    return a;
+}
+
+cudaError_t launch_accept_walk(const resps_ctx* ctx, const resps_step* d_steps,
+                               const int32_t* d_n_nodes, int batch, const int32_t* tokens,
+                               const int32_t* parent, const int32_t* target_argmax,
+                               int32_t* accept_path, int32_t* accept_len, int32_t* out_tokens,
+                               resps_step* steps_next, cudaStream_t st) {
+    const AcceptArgs a = make_accept_args(ctx, d_steps, d_n_nodes, tokens, parent, target_argmax, accept_path,
+                                          accept_len, out_tokens, steps_next);
     return launch_pdl(accept_walk_kernel, dim3(batch), dim3(RESPS_MAX_TT), 0, st, a);
 }
 

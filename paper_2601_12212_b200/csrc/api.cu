@@ -36,6 +36,7 @@ void carve(resps_ctx* c, Carver& cv) {
     cv.take(w.status, 64);
     cv.take(w.row_counter, rows);
     cv.take(w.amax_counter, nodes);
+    cv.take(w.amax_seq_counter, s.max_batch);
     const int64_t zero_end = cv.off;  // everything above must start as zero
     (void)zero_end;
     cv.take(w.part_key, rows * w.scan_splits * s.max_k);
@@ -162,6 +163,9 @@ int resps_debug_set(resps_ctx* ctx, int key, int value) {
         case RESPS_DEBUG_ATTN_MIN_TILES: w.attn_min_tiles = std::max(1, value); break;
         case RESPS_DEBUG_ATTN_STAGGER: w.attn_stagger = std::min(100000, std::max(0, value)); break;
         case RESPS_DEBUG_SCAN_SLICES: w.scan_slices_hint = std::max(0, value); break;
+#ifdef RESPS_WAIT_TEST
+        case 100: w.test_drop = value; break;  // test build only: which copy is left out (see common.cuh)
+#endif
         default: return RESPS_ERR_INVALID_ARG;
     }
     resps::attention_plan_invalidate(ctx);
@@ -184,6 +188,7 @@ int resps_status(resps_ctx* ctx, resps_stream stream, int32_t* status) {
         const size_t nodes = static_cast<size_t>(ctx->shape.max_batch) * ctx->shape.max_tt;
         if (cudaMemsetAsync(w.row_counter, 0, rows * sizeof(unsigned int), stream) != cudaSuccess ||
             cudaMemsetAsync(w.amax_counter, 0, nodes * sizeof(unsigned int), stream) != cudaSuccess ||
+            cudaMemsetAsync(w.amax_seq_counter, 0, ctx->shape.max_batch * sizeof(unsigned int), stream) != cudaSuccess ||
             cudaStreamSynchronize(stream) != cudaSuccess)
             return RESPS_ERR_CUDA;
     }
@@ -272,12 +277,17 @@ int resps_verify_accept(resps_ctx* ctx, const resps_step* d_steps, const int32_t
     if (batch < 1 || ld_row < ctx->shape.vocab || ld_b < 0) return RESPS_ERR_INVALID_ARG;
     if (batch > ctx->shape.max_batch) return RESPS_ERR_CAPACITY;
     if (d_steps_next) resps::attention_plan_invalidate(ctx, d_steps_next);  // prefix lengths move on
-    if (resps::launch_row_argmax(ctx, d_n_nodes, batch, d_target_logits, ld_b, ld_row, d_target_argmax,
-                                 stream) != cudaSuccess)
+    // One kernel where the rows allow the streaming arg-max (the CTA that completes a sequence's last
+    // row walks its tree); otherwise the walk is a second, small kernel.
+    const resps::AcceptArgs walk = resps::make_accept_args(ctx, d_steps, d_n_nodes, d_tokens, d_parent, d_target_argmax,
+                                                           d_accept_path, d_accept_len, d_out_tokens, d_steps_next);
+    bool walked = false;
+    if (resps::launch_row_argmax(ctx, d_n_nodes, batch, d_target_logits, ld_b, ld_row, d_target_argmax, &walk,
+                                 &walked, stream) != cudaSuccess)
         return RESPS_ERR_CUDA;
-    if (resps::launch_accept_walk(ctx, d_steps, d_n_nodes, batch, d_tokens, d_parent, d_target_argmax,
-                                  d_accept_path, d_accept_len, d_out_tokens, d_steps_next,
-                                  stream) != cudaSuccess)
+    if (!walked && resps::launch_accept_walk(ctx, d_steps, d_n_nodes, batch, d_tokens, d_parent, d_target_argmax,
+                                             d_accept_path, d_accept_len, d_out_tokens, d_steps_next,
+                                             stream) != cudaSuccess)
         return RESPS_ERR_CUDA;
     return RESPS_OK;
 }

@@ -69,7 +69,7 @@ constexpr int kMaxBatchSmem = 256;
 constexpr int kTmemCols = 512;
 constexpr int kCombineThreads = 256;
 constexpr int kMaxRounds = 4;      // rounds of items the work list may plan for (long sequences only)
-constexpr uint32_t kWaitLimitCycles = 0x70000000u;  // bounded waits give up after ~1 s of SM clocks
+constexpr uint32_t kWaitLimitCycles = kWaitTest ? 2000000u : 0x70000000u;  // bounded waits give up after ~1 s of SM clocks
 constexpr float kRescaleSlack = 8.0f;  // O is rescaled only when the running max grows by > 2^8
 constexpr unsigned kFull = 0xFFFFFFFFu;
 
@@ -110,6 +110,7 @@ struct AttnArgs {
     int stagger;      // cycles lane 1 starts behind lane 0 in row mode
     int q_by_tma;     // 1: Q tiles come by TMA (128 % (Hq/Hkv) == 0), 0: by plain loads
     int plan_after_wait;  // 1: the work list was written by the kernel just before this one
+    int test_drop;        // test build only: 1 = the CTA's first V copy is left out
     int32_t* status;
     // The work list, written by attention_plan_kernel.
     int4* plan_head;             // (items, rows per group, -, -)
@@ -353,6 +354,15 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         if ((++spins & 255u) == 0u && (*abort_flag || static_cast<uint32_t>(clock()) - t0 > kWaitLimitCycles))
             return false;
     }
+    return true;
+}
+// For the tear-down: a copy this thread issued must have landed before the CTA gives up its shared
+// memory, whatever else went wrong, so this wait looks at nothing but its own barrier and clock.
+__device__ __forceinline__ bool drain_wait(uint32_t bar, uint32_t parity) {
+    const uint32_t t0 = static_cast<uint32_t>(clock());
+    uint32_t spins = 0;
+    while (!mbar_try(bar, parity))
+        if ((++spins & 255u) == 0u && static_cast<uint32_t>(clock()) - t0 > kWaitLimitCycles) return false;
     return true;
 }
 // Same, with a warp-uniform answer (the callers go on to warp-collective TMEM instructions).
@@ -635,7 +645,7 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
                     tma_load_5d(base + S::kOffQ + m * S::kQTile, &map_q, bar(bar_qfull()), 0, 0, it.g,
                                 it.b * a.max_tt + it.tok0 + m * (kBM / G), 0);
             }
-        } else {
+        } else if (!(kWaitTest && (a.test_drop & 1))) {
             mbar_expect_tx(bar(bar_vfull(0)), S::kKVTile);
             tma_load_5d(base + S::kOffV, &map_v, bar(bar_vfull(0)), 0, it.t_begin * kBN, it.g, it.b, 0);
         }
@@ -692,11 +702,12 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
                     }
                 }
             }
-            // Drain: every copy this thread issued has landed before the CTA may exit.
-            bool landed = !(a.q_by_tma && items_run > 0) || mbar_wait(bar(bar_qfull()), (items_run - 1u) & 1u, abort_flag);
+            // Drain: every copy this thread issued has landed before the CTA may exit (each one is
+            // waited for, also after an earlier wait has run out).
+            bool landed = !(a.q_by_tma && items_run > 0) || drain_wait(bar(bar_qfull()), (items_run - 1u) & 1u);
             const uint32_t issued = kt_run;
-            for (uint32_t u = (issued > kStagesK ? issued - kStagesK : 0u); u < issued && landed; ++u)
-                landed = mbar_wait(bar(bar_kfull(u % kStagesK)), (u / kStagesK) & 1u, abort_flag);
+            for (uint32_t u = (issued > kStagesK ? issued - kStagesK : 0u); u < issued; ++u)
+                landed = drain_wait(bar(bar_kfull(u % kStagesK)), (u / kStagesK) & 1u) && landed;
             alive = alive && landed;
         }
     } else if (warp == kVProducerWarp) {
@@ -720,8 +731,8 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
             }
             const uint32_t issued = kt_run;
             bool landed = true;
-            for (uint32_t u = (issued > kStagesV ? issued - kStagesV : 0u); u < issued && landed; ++u)
-                landed = mbar_wait(bar(bar_vfull(u % kStagesV)), (u / kStagesV) & 1u, abort_flag);
+            for (uint32_t u = (issued > kStagesV ? issued - kStagesV : 0u); u < issued; ++u)
+                landed = drain_wait(bar(bar_vfull(u % kStagesV)), (u / kStagesV) & 1u) && landed;
             alive = alive && landed;
         }
     } else if (warp == kMmaWarp0 || warp == kMmaWarp0 + 1) {
@@ -1873,6 +1884,7 @@ cudaError_t launch_tree_attention(const resps_ctx* ctx, const resps_step* d_step
         hs->plan_capacity = capacity, hs->plan_stream = st, hs->plan_age = 0;
     }
     a.plan_after_wait = hs->plan_age == 0 ? 1 : 0;
+    a.test_drop = ctx->ws.test_drop;
     cudaError_t e = D == 128 ? launch_for_dim<128>(ctx, a, *mk, *mv, *mq, st) : launch_for_dim<64>(ctx, a, *mk, *mv, *mq, st);
     hs->plan_age += 2;
     return e;

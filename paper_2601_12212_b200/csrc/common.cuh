@@ -10,6 +10,15 @@
 
 namespace resps {
 
+// The test build (-DRESPS_WAIT_TEST, a separate library that only the bounded-wait test loads) gives
+// every device-side wait a limit of about a millisecond and can leave out one copy, so that a wait
+// really runs out; the product library is built without it.
+#ifdef RESPS_WAIT_TEST
+constexpr bool kWaitTest = true;
+#else
+constexpr bool kWaitTest = false;
+#endif
+
 constexpr int kScanThreads = 256;
 constexpr int kWarp = 32;
 
@@ -28,6 +37,7 @@ struct Workspace {
     double* row_lse = nullptr;               // [max_batch][max_rows]
     unsigned long long* amax_part = nullptr; // [max_batch][max_tt][splits]
     unsigned int* amax_counter = nullptr;    // [max_batch][max_tt]
+    unsigned int* amax_seq_counter = nullptr;  // [max_batch] rows of a sequence whose arg-max is final (self-resetting)
     // attention
     int attn_grid = 0;          // persistent CTAs (one per SM)
     int attn_combine_flat_grid = 0;  // ... of its variant for batches
@@ -39,6 +49,9 @@ struct Workspace {
     __half* attn_part_o = nullptr;  // [items][item rows][D] fp16
     float4* attn_part_ml = nullptr; // [items][item rows]
     int attn_max_groups = 0;
+    // Only read by the test build (RESPS_WAIT_TEST): bit 0 = the attention kernel's first V copy is
+    // never issued, bit 1 = the streaming scan's second chunk copy is never issued.
+    int test_drop = 0;
     // status
     int32_t* status = nullptr;
 };
@@ -57,6 +70,16 @@ struct resps_ctx {
 
 namespace resps {
 
+// Arguments of the greedy acceptance walk (accept_walk_device below).
+struct AcceptArgs {
+    const resps_step* steps;
+    const int32_t* n_nodes;
+    const int32_t *tokens, *parent, *target_argmax;
+    int max_tt, max_depth;
+    int32_t *accept_path, *accept_len, *out_tokens;
+    resps_step* steps_next;
+};
+
 // ---- launchers (one per translation unit) ---------------------------------
 cudaError_t launch_row_scan(const resps_ctx* ctx, const resps_step* d_steps, int batch,
                             const float* logits, int64_t ld_b, int64_t ld_level, int64_t ld_row,
@@ -66,9 +89,14 @@ cudaError_t launch_tree_build(const resps_ctx* ctx, const resps_step* d_steps, i
                               int32_t* tokens, int32_t* parent, int32_t* depth, int32_t* position_ids,
                               uint64_t* mask, int32_t* retrieve, int32_t* n_leaves, int32_t* n_nodes,
                               cudaStream_t st);
+// Arg-max of every target row; with `walk` non-null and rows that allow the streaming kernel the
+// acceptance walk runs in the same kernel (returns true through `walked`).
 cudaError_t launch_row_argmax(const resps_ctx* ctx, const int32_t* d_n_nodes, int batch,
                               const float* logits, int64_t ld_b, int64_t ld_row, int32_t* argmax_out,
-                              cudaStream_t st);
+                              const AcceptArgs* walk, bool* walked, cudaStream_t st);
+AcceptArgs make_accept_args(const resps_ctx* ctx, const resps_step* d_steps, const int32_t* d_n_nodes,
+                            const int32_t* tokens, const int32_t* parent, const int32_t* target_argmax,
+                            int32_t* accept_path, int32_t* accept_len, int32_t* out_tokens, resps_step* steps_next);
 cudaError_t launch_accept_walk(const resps_ctx* ctx, const resps_step* d_steps,
                                const int32_t* d_n_nodes, int batch, const int32_t* tokens,
                                const int32_t* parent, const int32_t* target_argmax,
@@ -141,6 +169,51 @@ __device__ __forceinline__ float ex2_approx(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
+}
+
+// Greedy acceptance walk (Section 3.2, "Acceptance Criterion" at temperature 0; Algorithm 2, "get
+// accepted tokens"): from the root, follow the child whose token equals the target's arg-max at the
+// current node until no child matches.  Run by `nthreads` >= RESPS_MAX_TT threads of one CTA for
+// sequence b (thread c owns tree node c); `sync` is a barrier over exactly those threads.
+template <typename Sync>
+__device__ __forceinline__ void accept_walk_device(const AcceptArgs& a, int b, int tid, int* s_tgt, int* s_next, Sync sync) {
+    const int n = min(max(a.n_nodes[b], 1), a.max_tt);
+    const int64_t ob = static_cast<int64_t>(b) * a.max_tt;
+    const int cap = a.max_depth + 1;
+    const int my_tok = (tid < n) ? a.tokens[ob + tid] : -1;
+    const int my_par = (tid < n) ? a.parent[ob + tid] : -2;
+    if (tid < n) s_tgt[tid] = __ldcg(a.target_argmax + ob + tid);
+    if (tid < cap) {
+        a.accept_path[b * cap + tid] = (tid == 0) ? 0 : -1;
+        a.out_tokens[b * cap + tid] = -1;
+    }
+    sync();
+    int cur = 0, len = 0;
+    for (int hop = 0; hop < a.max_depth; ++hop) {
+        if (tid == 0) *s_next = -1;
+        sync();
+        // children of one node carry distinct tokens, so at most one thread matches
+        if (tid > 0 && tid < n && my_par == cur && my_tok == s_tgt[cur]) *s_next = tid;
+        sync();
+        const int nxt = *s_next;
+        sync();
+        if (nxt < 0) break;
+        cur = nxt;
+        ++len;
+        if (tid == 0) {
+            a.accept_path[b * cap + len] = cur;
+            a.out_tokens[b * cap + len - 1] = a.tokens[ob + cur];
+        }
+    }
+    if (tid == 0) {
+        a.out_tokens[b * cap + len] = s_tgt[cur];
+        a.accept_len[b] = len;
+        if (a.steps_next) {
+            resps_step s = a.steps[b];
+            s.prefix_len += len + 1;
+            a.steps_next[b] = s;
+        }
+    }
 }
 
 // Step parameters clamped into the extents the caller supplied.

@@ -26,6 +26,7 @@ struct ScanArgs {
     int vocab, max_tt, max_k, max_rows;
     int chunk, splits;
     int slices, cps;  // streaming kernel: slices per row, chunks per slice (partials keep the stride `splits`)
+    int test_drop;    // test build only: 2 = the second chunk copy of every slice is left out
     unsigned long long* part_key;
     float2* part_ms;
     unsigned int* counter;
@@ -255,7 +256,7 @@ __global__ void __launch_bounds__(kScanThreads, 4) row_scan_kernel(const ScanArg
 // of its own from its quad maxima, which bounds its candidates by 128 k.
 // ---------------------------------------------------------------------------------------
 constexpr int kStreamStages = 3;
-constexpr long long kScanWaitLimitCycles = 4000000000ll;
+constexpr long long kScanWaitLimitCycles = kWaitTest ? 2000000ll : 4000000000ll;
 
 __device__ __forceinline__ uint32_t scan_smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -279,7 +280,7 @@ __device__ __forceinline__ void scan_mbar_wait(uint32_t bar, uint32_t parity, in
     unsigned spins = 0;
     while (!scan_mbar_try(bar, parity)) {
         if ((++spins & 63u) == 0u && clock64() - t0 > kScanWaitLimitCycles) {
-            atomicOr(status, RESPS_STATUS_WAIT_TIMEOUT);
+            if (status) atomicOr(status, RESPS_STATUS_WAIT_TIMEOUT);
             return;
         }
     }
@@ -351,6 +352,7 @@ __global__ void __launch_bounds__(kStreamThreads, 2) row_scan_stream_kernel(cons
                 scan_mbar_wait(empty_bar(st), ((u / kStreamStages) & 1u) ^ 1u, a.status);
                 const int e0 = c * kScanChunkMax;
                 const uint32_t bytes = static_cast<uint32_t>(min(a.vocab - e0, kScanChunkMax)) * 4u;
+                if (kWaitTest && (a.test_drop & 2) && u == 1) continue;
                 asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(full_bar(st)), "r"(bytes)
                              : "memory");
                 asm volatile(
@@ -584,10 +586,143 @@ struct ArgmaxArgs {
     const float* logits;
     int64_t ld_b, ld_row;
     int vocab, max_tt, chunk, splits;
+    int slices, cps;  // streaming kernel: slices per row, chunks per slice (partials keep the stride `splits`)
     unsigned long long* part;
     unsigned int* counter;
+    unsigned int* seq_counter;  // streaming kernel: rows of a sequence that are final
     int32_t* out;
+    int32_t* status;            // streaming kernel: where a wait that ran out is flagged (may be null)
 };
+
+// Streaming arg-max (16-byte aligned rows): like the streaming scan, a CTA walks a slice of several
+// 8192-logit chunks of one row behind a copy-issuing warp (cp.async.bulk three chunks ahead), a thread
+// keeps 32 logits of the chunk in registers and its best (ordered value, ~id) key across chunks.  The
+// last CTA of a row merges the slices; the CTA that completes the last row of a sequence goes on to
+// the acceptance walk (Section 3.2, "Acceptance Criterion" at temperature 0) when the caller asked
+// for it, so that arg-max and walk are one kernel.
+__global__ void __launch_bounds__(kStreamThreads, 2) row_argmax_stream_kernel(const ArgmaxArgs a, const AcceptArgs w,
+                                                                               const int do_walk) {
+    pdl_wait();  // the kernel before this one in the stream has completed
+    pdl_launch_dependents();
+    extern __shared__ __align__(128) unsigned char s_raw[];
+    float* s_stage = reinterpret_cast<float*>(s_raw);  // [3][8192]
+    __shared__ __align__(8) unsigned long long s_bar[2 * kStreamStages];  // full[3], empty[3]
+    __shared__ unsigned long long s_k[kScanThreads / 32];
+    __shared__ int s_flag;
+    __shared__ int s_tgt[RESPS_MAX_TT];
+    __shared__ int s_next;
+    const int b = blockIdx.z, r = blockIdx.y, sl = blockIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int n = min(max(a.n_nodes[b], 0), a.max_tt);
+    if (r >= n) return;
+    const float* row = a.logits + b * a.ld_b + r * a.ld_row;
+    const int c_begin = sl * a.cps;
+    const int c_end = min(a.splits, c_begin + a.cps);  // chunks [c_begin, c_end) of this row
+    const uint32_t bar0 = scan_smem_u32(s_bar);
+    auto full_bar = [&](int st) { return bar0 + 8u * st; };
+    auto empty_bar = [&](int st) { return bar0 + 8u * (kStreamStages + st); };
+    if (tid == 0) {
+        for (int st = 0; st < kStreamStages; ++st) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(full_bar(st)) : "memory");
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(empty_bar(st)), "r"(kScanThreads) : "memory");
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+
+    if (warp == kScanThreads / 32) {
+        // ---- copy-issuing warp: a stage is refilled as soon as every consumer has read it ----------
+        if (lane == 0) {
+            for (int c = c_begin; c < c_end; ++c) {
+                const int u = c - c_begin, st = u % kStreamStages;
+                scan_mbar_wait(empty_bar(st), ((u / kStreamStages) & 1u) ^ 1u, a.status);
+                const int e0 = c * kScanChunkMax;
+                const uint32_t bytes = static_cast<uint32_t>(min(a.vocab - e0, kScanChunkMax)) * 4u;
+                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(full_bar(st)), "r"(bytes)
+                             : "memory");
+                asm volatile(
+                    "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                        scan_smem_u32(s_stage + st * kScanChunkMax)),
+                    "l"(row + e0), "r"(bytes), "r"(full_bar(st))
+                    : "memory");
+            }
+        }
+        return;  // the consumers wait for every copy that was issued
+    }
+
+    unsigned long long best = 0ull;  // 0 = nothing yet (every real key has a non-zero value part)
+    for (int c = c_begin; c < c_end; ++c) {
+        const int u0 = c - c_begin, st = u0 % kStreamStages;
+        const int begin = c * kScanChunkMax;
+        const int end = min(a.vocab, begin + kScanChunkMax);
+        scan_mbar_wait(full_bar(st), (u0 / kStreamStages) & 1u, a.status);
+        float v[kScanPerThread];
+#pragma unroll
+        for (int u = 0; u < kScanPerThread / 4; ++u) {
+            const int off = (u * kScanThreads + tid) * 4;
+            v[4 * u] = v[4 * u + 1] = v[4 * u + 2] = v[4 * u + 3] = -INFINITY;
+            if (begin + off < end) {  // the vocabulary is a multiple of 4 on this path
+                const float4 x = *reinterpret_cast<const float4*>(s_stage + st * kScanChunkMax + off);
+                v[4 * u] = x.x, v[4 * u + 1] = x.y, v[4 * u + 2] = x.z, v[4 * u + 3] = x.w;
+            }
+        }
+        asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(empty_bar(st)) : "memory");
+        // position i of a thread is logit begin + ((i / 4) * 256 + tid) * 4 + i % 4: ids ascend with i
+        if (begin + tid * 4 < end) {
+            float tmax = v[0];
+#pragma unroll
+            for (int i = 1; i + 1 < kScanPerThread; i += 2) tmax = max3f(tmax, v[i], v[i + 1]);
+            tmax = fmaxf(tmax, v[kScanPerThread - 1]);
+            int tpos = 0;
+#pragma unroll
+            for (int i = kScanPerThread - 1; i >= 0; --i)
+                if (v[i] == tmax) tpos = i;
+            const unsigned long long key = pack_val_id(tmax, begin + ((tpos >> 2) * kScanThreads + tid) * 4 + (tpos & 3));
+            best = key > best ? key : best;  // an equal value later in the row has a higher id: a smaller key
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const unsigned long long other = __shfl_xor_sync(kFull, best, o);
+        best = (other > best) ? other : best;
+    }
+    if (lane == 0) s_k[warp] = best;
+    consumer_sync();
+    const int64_t prow = static_cast<int64_t>(b) * a.max_tt + r;
+    // ---- the row's result: directly, or by the last slice to arrive ----------------------------------
+    if (tid == 0) {
+        for (int wq = 1; wq < kScanThreads / 32; ++wq) best = (s_k[wq] > best) ? s_k[wq] : best;
+        int row_done = 1;
+        if (a.slices > 1) {
+            a.part[prow * a.splits + sl] = best;
+            __threadfence();
+            row_done = (atomicAdd(a.counter + prow, 1u) == static_cast<unsigned>(a.slices - 1));
+            if (row_done) {
+                __threadfence();
+                for (int i = 0; i < a.slices; ++i) {
+                    const unsigned long long p = __ldcg(a.part + prow * a.splits + i);
+                    best = (p > best) ? p : best;
+                }
+                a.counter[prow] = 0u;
+            }
+        }
+        int seq_done = 0;
+        if (row_done) {
+            a.out[prow] = key_id(best);
+            if (do_walk) {
+                __threadfence();
+                seq_done = (atomicAdd(a.seq_counter + b, 1u) == static_cast<unsigned>(n - 1));
+                if (seq_done) a.seq_counter[b] = 0u;
+            }
+        }
+        s_flag = seq_done;
+    }
+    consumer_sync();
+    if (!s_flag) return;
+    // ---- the sequence's last row is final: the acceptance walk, by this CTA's consumer threads ---------
+    __threadfence();
+    accept_walk_device(w, b, tid, s_tgt, &s_next, [] { consumer_sync(); });
+}
 
 template <bool VEC>
 __global__ void __launch_bounds__(kScanThreads, 4) row_argmax_kernel(const ArgmaxArgs a) {
@@ -689,6 +824,9 @@ static size_t stream_smem_bytes(int max_k, int slices) {
 }
 
 cudaError_t scan_setup(resps_ctx* ctx) {
+    cudaError_t e = cudaFuncSetAttribute(row_argmax_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         static_cast<int>(kStreamStages * kScanChunkMax * sizeof(float)));
+    if (e != cudaSuccess) return e;
     return cudaFuncSetAttribute(row_scan_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 static_cast<int>(stream_smem_bytes(ctx->shape.max_k, 128)));
 }
@@ -709,6 +847,7 @@ cudaError_t launch_row_scan(const resps_ctx* ctx, const resps_step* d_steps, int
     const int k_ext = min(n_slots, ctx->shape.max_k);
     const int rows = (n_levels > 1) ? 1 + (n_levels - 1) * k_ext : 1;
     a.slices = w.scan_splits, a.cps = 1;
+    a.test_drop = w.test_drop;
     const size_t smem = sizeof(unsigned long long) * ctx->shape.max_k * max(kQuadElems, w.scan_splits);
     if (vec_ok(logits, ld_b, ld_level, ld_row, a.vocab, a.chunk) && w.scan_chunk == kScanChunkMax) {
         // Slices per row: two CTAs fit an SM, and a slice's first chunk costs about three later ones (the
@@ -730,7 +869,7 @@ cudaError_t launch_row_scan(const resps_ctx* ctx, const resps_step* d_steps, int
 
 cudaError_t launch_row_argmax(const resps_ctx* ctx, const int32_t* d_n_nodes, int batch,
                               const float* logits, int64_t ld_b, int64_t ld_row, int32_t* argmax_out,
-                              cudaStream_t st) {
+                              const AcceptArgs* walk, bool* walked, cudaStream_t st) {
     const Workspace& w = ctx->ws;
     ArgmaxArgs a;
     a.n_nodes = d_n_nodes;
@@ -738,7 +877,23 @@ cudaError_t launch_row_argmax(const resps_ctx* ctx, const int32_t* d_n_nodes, in
     a.ld_b = ld_b, a.ld_row = ld_row;
     a.vocab = ctx->shape.vocab, a.max_tt = ctx->shape.max_tt;
     a.chunk = w.scan_chunk, a.splits = w.scan_splits;
-    a.part = w.amax_part, a.counter = w.amax_counter, a.out = argmax_out;
+    a.slices = w.scan_splits, a.cps = 1;
+    a.part = w.amax_part, a.counter = w.amax_counter, a.seq_counter = w.amax_seq_counter, a.out = argmax_out;
+    a.status = w.status;
+    if (walked) *walked = false;
+    if (vec_ok(logits, ld_b, ld_row, 0, a.vocab, a.chunk) && w.scan_chunk == kScanChunkMax) {
+        // Slices per row as in the scan: a row is cut only as far as all CTAs still run at once.
+        const int want = max(1, 2 * ctx->sm_count / max(ctx->shape.max_tt * batch, 1));
+        const int slices0 = max(1, min(w.scan_splits, want));
+        a.cps = (w.scan_splits + slices0 - 1) / slices0;
+        a.slices = (w.scan_splits + a.cps - 1) / a.cps;
+        AcceptArgs wa = {};
+        if (walk) wa = *walk;
+        if (walked) *walked = walk != nullptr;
+        dim3 grid(a.slices, ctx->shape.max_tt, batch);
+        return launch_pdl(row_argmax_stream_kernel, grid, dim3(kStreamThreads),
+                          kStreamStages * kScanChunkMax * sizeof(float), st, a, wa, walk ? 1 : 0);
+    }
     dim3 grid(w.scan_splits, ctx->shape.max_tt, batch);
     if (vec_ok(logits, ld_b, ld_row, 0, a.vocab, a.chunk))
         return launch_pdl(row_argmax_kernel<true>, grid, dim3(kScanThreads), 0, st, a);
@@ -804,6 +959,7 @@ extern "C" int resps_target_argmax_static(const int32_t* d_n_nodes, int batch, i
     a.logits = d_target_logits;
     a.ld_b = ld_b, a.ld_row = ld_row;
     a.vocab = vocab, a.max_tt = max_tt, a.chunk = chunk, a.splits = splits;
+    a.slices = splits, a.cps = 1, a.seq_counter = nullptr, a.status = nullptr;
     a.part = reinterpret_cast<unsigned long long*>(scratch);
     a.counter = reinterpret_cast<unsigned int*>(scratch + kStaticPartBytes);
     a.out = d_target_argmax;
