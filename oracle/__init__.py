@@ -73,6 +73,21 @@ class Tree:
     frontier: np.ndarray      # int32 [d, k]: candidates expanded after each level
     min_gap: float
     near_pairs: np.ndarray    # int32 [n_near, 2]: boundary pairs (before, after) with a gap below tau
+    node_cand: np.ndarray     # int32 [n]: candidate index of each node (-1 for the root)
+
+    def node_rows(self, d: int, k: int, slots: int) -> np.ndarray:
+        """int32 [n]: for every node the index level * slots + slot of the draft row its children were taken
+        from (the root: row 0; a candidate that is the p-th member of the frontier after level j < d-1:
+        row (j+1, p)), or -1 for a node that was not expanded."""
+        row_of_cand = {}
+        for j in range(d - 1):
+            for p_, c in enumerate(self.frontier[j][:k]):
+                row_of_cand[int(c)] = (j + 1) * slots + p_
+        out = np.full(self.n_nodes, -1, np.int32)
+        out[0] = 0
+        for i in range(1, self.n_nodes):
+            out[i] = row_of_cand.get(int(self.node_cand[i]), -1)
+        return out
 
 
 def tree_expand(root_token: int, logits: np.ndarray, TT: int, d: int, k: int, L: int,
@@ -105,6 +120,7 @@ def tree_expand(root_token: int, logits: np.ndarray, TT: int, d: int, k: int, L:
     max_near = 64
     near = np.zeros((max_near, 2), np.int32)
     n_near = ctypes.c_int32()
+    node_cand = np.full(max_tt, -1, np.int32)
     if order_bias is not None:
         order_bias = _c(order_bias, np.float64)
         assert order_bias.shape == (n_cand,)
@@ -113,12 +129,13 @@ def tree_expand(root_token: int, logits: np.ndarray, TT: int, d: int, k: int, L:
         V, TT, d, k, L, max_tt, ret_stride, _p(tokens), _p(parent), _p(depth), _p(pos), _p(mask),
         _p(retrieve), ctypes.byref(n_leaves), ctypes.byref(n_nodes), _p(cand), _p(ctok), _p(cpar),
         _p(frontier), ctypes.byref(gap), _p(order_bias) if order_bias is not None else None,
-        ctypes.c_double(tau), _p(near), max_near, ctypes.byref(n_near))
+        ctypes.c_double(tau), _p(near), max_near, ctypes.byref(n_near), _p(node_cand))
     if rc != 0:
         raise ValueError(f"oracle_tree_expand rc={rc}")
     n = n_nodes.value
     return Tree(tokens[:n], parent[:n], depth[:n], pos[:n], mask[:n], retrieve[:n_leaves.value],
-                n, n_leaves.value, cand, ctok, cpar, frontier, gap.value, near[:n_near.value].copy())
+                n, n_leaves.value, cand, ctok, cpar, frontier, gap.value, near[:n_near.value].copy(),
+                node_cand[:n].copy())
 
 
 def tree_expand_swapped(root_token: int, logits: np.ndarray, TT: int, d: int, k: int, L: int,
@@ -190,6 +207,42 @@ def verify_accept(target_logits: np.ndarray, tokens: np.ndarray, parent: np.ndar
     if rc != 0:
         raise ValueError(f"oracle_verify_accept rc={rc}")
     return Accept(tgt, path[:a.value + 1].copy(), a.value, out[:a.value + 1].copy())
+
+
+@dataclass
+class SampledAccept:
+    path: np.ndarray        # int32 [a+1]
+    accept_len: int
+    out_tokens: np.ndarray  # int32 [a+1]: the accepted draft tokens, then the drawn token
+    min_margin: float
+
+
+def verify_accept_sampled(target_logits: np.ndarray, draft_rows: np.ndarray, node_row: np.ndarray,
+                          tokens: np.ndarray, parent: np.ndarray, temperature: float,
+                          u_accept: np.ndarray, u_sample: np.ndarray, path_cap: int = 17) -> SampledAccept:
+    """Acceptance under sampling.  target_logits fp32 [n][V]; draft_rows fp32 [R][V];
+    node_row int32 [n]: the draft row a node's children were taken from (-1: none);
+    u_accept fp64 [path_cap][max_children], u_sample fp64 [path_cap]: uniforms in (0, 1)."""
+    target_logits = _c(target_logits, np.float32)
+    draft_rows = _c(draft_rows, np.float32)
+    node_row = _c(node_row, np.int32)
+    tokens = _c(tokens, np.int32)
+    parent = _c(parent, np.int32)
+    u_accept = _c(u_accept, np.float64)
+    u_sample = _c(u_sample, np.float64)
+    n, V = target_logits.shape
+    assert draft_rows.shape[1] == V and u_accept.shape[0] >= path_cap and u_sample.shape[0] >= path_cap
+    path = np.empty(path_cap, np.int32)
+    out = np.empty(path_cap, np.int32)
+    a = ctypes.c_int32()
+    margin = ctypes.c_double()
+    rc = _load().oracle_verify_accept_sampled(
+        n, V, _p(target_logits), ctypes.c_int64(V), _p(draft_rows), ctypes.c_int64(V), _p(node_row), _p(tokens),
+        _p(parent), ctypes.c_double(temperature), _p(u_accept), int(u_accept.shape[1]), _p(u_sample), path_cap,
+        _p(path), ctypes.byref(a), _p(out), ctypes.byref(margin))
+    if rc != 0:
+        raise ValueError(f"oracle_verify_accept_sampled rc={rc}")
+    return SampledAccept(path[:a.value + 1].copy(), a.value, out[:a.value + 1].copy(), margin.value)
 
 
 def kv_compact(k_cache: np.ndarray, v_cache: np.ndarray, L: int, path: np.ndarray) -> int:

@@ -18,13 +18,17 @@
 //   attention      : chain tree == causal attention (library routine),
 //                    one-node tree == plain decode, closed forms, poison slots
 //   accept         : brute force over retrieve rows, chain == longest common prefix
+//   sampled accept : chain of sampled draft tokens keeps the target's distribution (chi-square
+//                    against the exact P_T, acceptance rate = sum min(p, q)); T -> 0 equals greedy
 //   compaction     : gather definition, identity path is a no-op
 //   whole step     : greedy speculative decoding over a tiny random transformer
 //                    reproduces greedy autoregressive decoding token for token
 // Parity unpinned (conventions of this implementation that no external value fixes):
 //   the tie-break orders (equal logits -> lower token id, equal scores -> lower
 //   candidate index), the node order (ascending candidate index), the retrieve
-//   row order, and reading "depth d" as d draft levels.
+//   row order, reading "depth d" as d draft levels, and -- in the sampled
+//   acceptance -- how the siblings of a tree are tried after a rejection (the paper
+//   gives the rule for a chain only).
 //
 // Build: g++ -O2 -std=c++17 -shared -fPIC resps_oracle.cpp -o libresps_oracle.so
 
@@ -141,6 +145,8 @@ int oracle_topk_lse(const float* row, int V, int k, float* out_val, int32_t* out
 // order and may therefore resolve a gap below `tau` the other way):
 //   near_pairs (optional, capacity max_near pairs): every boundary pair (before,
 //   after) as above whose gap is below tau; n_near = their number.
+//   node_cand (optional, [max_tt]): the candidate index each node was made from (-1 for the
+//   root); with frontier[][] it tells which draft row a node's children were taken from.
 //   order_bias (optional, [n_cand]): added to a candidate's score where candidates
 //   are *ordered* (frontier choice and rerank), never to the score its children
 //   inherit.  A bias that lifts `after` just above `before` yields the tree of the
@@ -152,7 +158,7 @@ int oracle_tree_expand(int32_t root_token, const float* logits, int64_t ld_level
                        uint64_t* mask, int32_t* retrieve, int32_t* n_leaves, int32_t* n_nodes,
                        double* cand_score, int32_t* cand_token, int32_t* cand_parent,
                        int32_t* frontier_out, double* min_gap, const double* order_bias, double tau,
-                       int32_t* near_pairs, int max_near, int32_t* n_near) {
+                       int32_t* near_pairs, int max_near, int32_t* n_near, int32_t* node_cand) {
     if (V < 1 || k < 1 || k > V || d < 1 || TT < 1 || TT > max_tt || max_tt > 128) return -1;
     if (ret_stride < d + 1) return -1;
     const int n_cand = k + (d - 1) * k * k;
@@ -225,6 +231,10 @@ int oracle_tree_expand(int32_t root_token, const float* logits, int64_t ld_level
     const int n = m + 1;
     std::vector<int32_t> node_of_cand(n_cand, -1);
     for (int i = 0; i < m; ++i) node_of_cand[kept[i]] = i + 1;
+    if (node_cand) {
+        node_cand[0] = -1;
+        for (int i = 0; i < m; ++i) node_cand[i + 1] = kept[i];
+    }
     tokens[0] = root_token;
     parent[0] = -1;
     depth[0] = 0;
@@ -375,6 +385,128 @@ int oracle_verify_accept(int n, int V, const float* target_logits, int64_t ld_ro
     }
     out_tokens[a] = target_argmax[cur];
     *accept_len = a;
+    return 0;
+}
+
+// ---------------------------------------------------------------------------
+// Verification and acceptance under sampling (temperature T > 0) for one sequence
+// (Section 3.2, "Acceptance Criterion": a draft token y is accepted with probability
+// alpha = min(1, P_T(y | .) / P_d(y | .)); Section 4.1, "Lossless Output Fidelity":
+// speculative sampling with rejection-based correction keeps the target's output
+// distribution).
+//
+// P_T(. | node i) = softmax(target_logits[i] / T); P_d(. | node i) = softmax(draft
+// row of node i / T), the row its children were taken from (node_row[i], -1 for a node
+// that was not expanded).  All arithmetic in fp64.
+//
+// The paper states the rule for a chain of draft tokens.  For a chain this function is
+// that rule, with the correction step of the speculative-sampling papers it cites: on
+// the first rejected token the emitted token is drawn from the normalised residual
+// max(0, P_T - P_d); after the last accepted token of a chain that was accepted in full
+// it is drawn from P_T.  Reading for a tree (the paper is silent): the children of the
+// current node are tried in node order (= the draft's order of preference); after a
+// rejected child x the target-side distribution becomes the normalised residual
+// max(0, p - q) and the draft-side one q with x removed, renormalised, and the next
+// sibling is tried against those; when no child is left the token is drawn from the
+// residual.  (A residual that is zero everywhere leaves p as it is.)
+//
+// Random numbers are inputs: u_accept[level * max_children + j] for the j-th child tried
+// at walk level `level`, u_sample[level] for the token drawn when the walk stops there;
+// all uniform in (0, 1).  A token is drawn by inverse CDF in token-id order: the first v
+// with sum_{w <= v} p[w] > u * sum_w p[w].
+//
+// Outputs as oracle_verify_accept (path, accept_len, out_tokens; no argmax), and
+// min_margin: the smallest distance of any decision from flipping -- |u - alpha| of
+// every acceptance test that was taken with alpha < 1 or u near 1, and the distance of
+// u * total from the two cumulative sums that bracket the drawn token, relative to
+// total.  An implementation that sums in another order must reproduce every decision
+// whose margin exceeds its own rounding error.
+// ---------------------------------------------------------------------------
+int oracle_verify_accept_sampled(int n, int V, const float* target_logits, int64_t ld_row,
+                                 const float* draft_logits, int64_t draft_ld_row, const int32_t* node_row,
+                                 const int32_t* tokens, const int32_t* parent, double temperature,
+                                 const double* u_accept, int max_children, const double* u_sample,
+                                 int path_cap, int32_t* accept_path, int32_t* accept_len,
+                                 int32_t* out_tokens, double* min_margin) {
+    if (n < 1 || V < 1 || !(temperature > 0.0) || path_cap < 1) return -1;
+    auto softmax_t = [&](const float* row, std::vector<double>& out) {
+        double mx = -std::numeric_limits<double>::infinity();
+        for (int v = 0; v < V; ++v) mx = std::max(mx, static_cast<double>(row[v]) / temperature);
+        double sum = 0.0;
+        for (int v = 0; v < V; ++v) {
+            out[v] = std::exp(static_cast<double>(row[v]) / temperature - mx);
+            sum += out[v];
+        }
+        for (int v = 0; v < V; ++v) out[v] /= sum;
+    };
+    double margin = std::numeric_limits<double>::infinity();
+    auto draw = [&](const std::vector<double>& p, double u) {
+        double total = 0.0;
+        for (int v = 0; v < V; ++v) total += p[v];
+        const double target = u * total;
+        double run = 0.0;
+        for (int v = 0; v < V; ++v) {
+            const double before = run;
+            run += p[v];
+            if (run > target || v == V - 1) {
+                margin = std::min(margin, (target - before) / total);
+                if (v < V - 1) margin = std::min(margin, (run - target) / total);
+                return v;
+            }
+        }
+        return V - 1;
+    };
+    for (int t = 0; t < path_cap; ++t) {
+        accept_path[t] = -1;
+        out_tokens[t] = -1;
+    }
+    std::vector<double> p(V), q(V);
+    int cur = 0, a = 0;
+    accept_path[0] = 0;
+    for (;;) {
+        softmax_t(target_logits + cur * ld_row, p);
+        std::vector<int> children;
+        for (int c = 1; c < n; ++c)
+            if (parent[c] == cur) children.push_back(c);
+        int next = -1;
+        if (!children.empty()) {
+            if (node_row[cur] < 0) return -3;  // a node with children must have a draft row
+            softmax_t(draft_logits + node_row[cur] * draft_ld_row, q);
+            for (size_t j = 0; j < children.size(); ++j) {
+                if (static_cast<int>(j) >= max_children) return -4;
+                const int x = tokens[children[j]];
+                // (a draft probability that has underflowed to zero: the ratio is infinite, or 0/0 = reject)
+                const double alpha = q[x] > 0.0 ? std::min(1.0, p[x] / q[x]) : (p[x] > 0.0 ? 1.0 : 0.0);
+                const double u = u_accept[a * max_children + j];
+                margin = std::min(margin, alpha < 1.0 ? std::fabs(u - alpha) : 1.0 - u);
+                if (u < alpha) {
+                    next = children[j];
+                    break;
+                }
+                // rejected: residual on the target side, x removed on the draft side
+                double z = 0.0;
+                for (int v = 0; v < V; ++v) z += std::max(p[v] - q[v], 0.0);
+                if (z > 0.0)
+                    for (int v = 0; v < V; ++v) p[v] = std::max(p[v] - q[v], 0.0) / z;
+                q[x] = 0.0;
+                double rest = 0.0;  // (summed, not 1 - q[x]: a dominant q[x] rounds to 1 and would leave nothing)
+                for (int v = 0; v < V; ++v) rest += q[v];
+                if (rest > 0.0)
+                    for (int v = 0; v < V; ++v) q[v] /= rest;
+            }
+        }
+        if (next < 0) {
+            out_tokens[a] = draw(p, u_sample[a]);
+            break;
+        }
+        if (a + 1 >= path_cap) return -2;
+        cur = next;
+        ++a;
+        accept_path[a] = cur;
+        out_tokens[a - 1] = tokens[cur];
+    }
+    *accept_len = a;
+    if (min_margin) *min_margin = margin;
     return 0;
 }
 
