@@ -305,6 +305,9 @@ class DeviceWorkload:
         self.h_q = torch.stack([q.cpu() for q in self.q]).pin_memory()          # [NL][B][T][Hq][D]
         self.h_tree_kv = torch.randn(2, NL, B, w.n_kv_heads, T, w.head_dim).bfloat16().pin_memory()
         self.scale = 1.0 / float(np.sqrt(w.head_dim))
+        # uniforms for the acceptance under sampling (timed as a phase of its own, not part of the step)
+        self.u_accept = torch.rand(B, self.max_d + 1, self.max_k, generator=g, device=dev, dtype=torch.float64)
+        self.u_sample = torch.rand(B, self.max_d + 1, generator=g, device=dev, dtype=torch.float64)
         self.reset_prefix()
 
     def reset_prefix(self):
@@ -339,6 +342,13 @@ class DeviceWorkload:
             self.ctx, self.d_steps, self.n_nodes, self.B, self.d_target[i], self.T * V, V, self.tokens,
             self.parent, self.argmax, self.path, self.alen, self.out_tokens,
             self.d_steps if advance else None)
+
+    def verify_sampled(self, i, temperature=1.0):
+        V = self.w.vocab
+        self.binding.resps_verify_accept_sampled(
+            self.ctx, self.d_steps, self.n_nodes, self.B, self.d_target[i], self.T * V, V, self.d_draft[i],
+            self.max_d * self.max_k * V, self.max_k * V, V, temperature, self.tokens, self.parent, self.u_accept,
+            self.u_sample, self.path, self.alen, self.out_tokens, None)
 
     def compact(self, advanced=True):
         self.binding.resps_kv_compact(self.ctx, self.d_steps, self.B, self.path, self.alen, self.k_ptrs,
@@ -539,7 +549,7 @@ def run_ours(args, w):
         dw.reset_prefix()
         phases, phase_bytes = {}, {}
         for name, fn in (("expand", dw.expand), ("verify", lambda i: dw.verify(i, advance=False)),
-                         ("compact", lambda i: dw.compact(advanced=False))):
+                         ("verify_sampled_t1", dw.verify_sampled), ("compact", lambda i: dw.compact(advanced=False))):
             fn(0)
             torch.cuda.synchronize()
             total, reps = 0.0, 0
@@ -547,7 +557,7 @@ def run_ours(args, w):
                 for i in range(pool):
                     if name != "compact":
                         dw.set_params(i)
-                        if name == "verify":
+                        if name != "expand":
                             dw.expand(i)
                     flush.fill_(rep)
                     a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)

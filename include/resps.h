@@ -216,6 +216,41 @@ int resps_verify_accept(resps_ctx* ctx, const resps_step* d_steps, const int32_t
                         int32_t* d_out_tokens, resps_step* d_steps_next, resps_stream stream);
 
 /*
+ * Verification and acceptance under sampling, temperature T > 0 (Section 3.2, "Acceptance
+ * Criterion": a draft token y is accepted with probability min(1, P_T(y|.) / P_d(y|.)); Section
+ * 4.1, "Lossless Output Fidelity": speculative sampling with rejection-based correction keeps the
+ * target model's output distribution).  The alternative to resps_verify_accept, which is the same
+ * step at temperature 0.
+ *
+ * P_T(.|node i) = softmax(d_target_logits[b][i] / T); P_d(.|node i) = softmax(r / T) of the draft
+ * row r the node's children were taken from.  From the root: the children of the current node
+ * are tried in node order; child j with token x is accepted when u_accept < min(1, p(x) / q(x)) and
+ * the walk moves on to it; after a rejection p becomes the normalised residual max(0, p - q) and q
+ * loses x (renormalised), and the next sibling is tried against those.  When no child is accepted
+ * (or the node has none) the step's last token is drawn from the current p by inverse CDF in token
+ * order with u_sample.  For a chain this is the paper's rule; how siblings are tried is this
+ * library's reading where the paper is silent.  All arithmetic is fp64.
+ *
+ * d_draft_logits  the same rows (and strides) resps_tree_expand was given for this tree.  Which row
+ *                 stands behind which node is kept in the context by resps_tree_expand: call this
+ *                 for the tree of the last resps_tree_expand on this context.
+ * temperature     T > 0 (INVALID_ARG otherwise)
+ * d_u_accept      DEVICE fp64 [batch][max_depth+1][max_k]: uniform (0,1) numbers, entry (level, j)
+ *                 decides the j-th child tried at the walk's level `level`
+ * d_u_sample      DEVICE fp64 [batch][max_depth+1]: entry `level` draws the token when the walk
+ *                 stops at that level
+ * Outputs as resps_verify_accept (no arg-max): d_accept_path, d_accept_len, d_out_tokens (the
+ * accepted tokens, then the drawn one), d_steps_next (may alias d_steps, see there).
+ */
+int resps_verify_accept_sampled(resps_ctx* ctx, const resps_step* d_steps, const int32_t* d_n_nodes, int batch,
+                                const float* d_target_logits, int64_t ld_b, int64_t ld_row,
+                                const float* d_draft_logits, int64_t draft_ld_b, int64_t draft_ld_level,
+                                int64_t draft_ld_row, float temperature, const int32_t* d_tokens,
+                                const int32_t* d_parent, const double* d_u_accept, const double* d_u_sample,
+                                int32_t* d_accept_path, int32_t* d_accept_len, int32_t* d_out_tokens,
+                                resps_step* d_steps_next, resps_stream stream);
+
+/*
  * In-place KV-cache compaction (Appendix D, "input update": rejected tokens are discarded
  * from the cache).  For every bound layer, KV head and j = 0..a:
  *   slot L+j  <-  slot L+path[j]     (K and V),   L = the prefix length before the step.

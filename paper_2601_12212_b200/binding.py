@@ -30,7 +30,7 @@ RESPS_DEBUG_SCAN_SLICES = 4
 
 EXPORTS = ("resps_create", "resps_destroy", "resps_strerror", "resps_status",
            "resps_workspace_bytes", "resps_debug_set", "resps_attention_replan", "resps_tree_expand", "resps_tree_attention",
-           "resps_verify_accept", "resps_kv_compact", "resps_target_argmax_static")
+           "resps_verify_accept", "resps_verify_accept_sampled", "resps_kv_compact", "resps_target_argmax_static")
 
 
 class RespsShape(ctypes.Structure):
@@ -70,6 +70,8 @@ def load() -> ctypes.CDLL:
     lib.resps_tree_attention.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp, vp, i64, i64, i64, i64,
                                          vp, f32, vp]
     lib.resps_verify_accept.argtypes = [vp, vp, vp, i32, vp, i64, i64, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.resps_verify_accept_sampled.argtypes = [vp, vp, vp, i32, vp, i64, i64, vp, i64, i64, i64, f32, vp, vp, vp, vp,
+                                                vp, vp, vp, vp, vp]
     lib.resps_kv_compact.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp, i32, i64, i64, i64, i64, vp]
     lib.resps_debug_set.argtypes = [vp, i32, i32]
     lib.resps_attention_replan.argtypes = [vp]
@@ -183,6 +185,19 @@ def resps_verify_accept(ctx: Context, steps, n_nodes, batch: int, target_logits,
         ld_b, ld_row, _ptr(tokens, i32), _ptr(parent, i32), _ptr(target_argmax, i32),
         _ptr(accept_path, i32), _ptr(accept_len, i32), _ptr(out_tokens, i32), _ptr(steps_next, i32),
         _stream(stream)), "resps_verify_accept")
+
+
+def resps_verify_accept_sampled(ctx: Context, steps, n_nodes, batch: int, target_logits, ld_b: int, ld_row: int,
+                                draft_logits, draft_ld_b: int, draft_ld_level: int, draft_ld_row: int,
+                                temperature: float, tokens, parent, u_accept, u_sample, accept_path, accept_len,
+                                out_tokens, steps_next=None, stream=None) -> None:
+    """Acceptance under sampling (T > 0) for the tree of the last resps_tree_expand on this context."""
+    i32, f32, f64 = torch.int32, torch.float32, torch.float64
+    _check(load().resps_verify_accept_sampled(
+        ctx.handle, _ptr(steps, i32), _ptr(n_nodes, i32), batch, _ptr(target_logits, f32), ld_b, ld_row,
+        _ptr(draft_logits, f32), draft_ld_b, draft_ld_level, draft_ld_row, float(temperature), _ptr(tokens, i32),
+        _ptr(parent, i32), _ptr(u_accept, f64), _ptr(u_sample, f64), _ptr(accept_path, i32), _ptr(accept_len, i32),
+        _ptr(out_tokens, i32), _ptr(steps_next, i32), _stream(stream)), "resps_verify_accept_sampled")
 
 
 def resps_kv_compact(ctx: Context, steps, batch: int, accept_path, accept_len, k_cache_ptrs,

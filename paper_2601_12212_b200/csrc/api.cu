@@ -39,6 +39,8 @@ void carve(resps_ctx* c, Carver& cv) {
     cv.take(w.amax_seq_counter, s.max_batch);
     const int64_t zero_end = cv.off;  // everything above must start as zero
     (void)zero_end;
+    cv.take(w.node_row, nodes);
+    cv.take(w.samp_scratch, static_cast<int64_t>(resps::sampled_scratch_doubles(s.max_batch)));
     cv.take(w.part_key, rows * w.scan_splits * s.max_k);
     cv.take(w.part_ms, rows * w.scan_splits);
     cv.take(w.row_val, rows * s.max_k);
@@ -288,6 +290,38 @@ int resps_verify_accept(resps_ctx* ctx, const resps_step* d_steps, const int32_t
     if (!walked && resps::launch_accept_walk(ctx, d_steps, d_n_nodes, batch, d_tokens, d_parent, d_target_argmax,
                                              d_accept_path, d_accept_len, d_out_tokens, d_steps_next,
                                              stream) != cudaSuccess)
+        return RESPS_ERR_CUDA;
+    return RESPS_OK;
+}
+
+int resps_verify_accept_sampled(resps_ctx* ctx, const resps_step* d_steps, const int32_t* d_n_nodes, int batch,
+                                const float* d_target_logits, int64_t ld_b, int64_t ld_row,
+                                const float* d_draft_logits, int64_t draft_ld_b, int64_t draft_ld_level,
+                                int64_t draft_ld_row, float temperature, const int32_t* d_tokens,
+                                const int32_t* d_parent, const double* d_u_accept, const double* d_u_sample,
+                                int32_t* d_accept_path, int32_t* d_accept_len, int32_t* d_out_tokens,
+                                resps_step* d_steps_next, resps_stream stream) {
+    RESPS_CHECK_PTR(ctx);
+    RESPS_CHECK_PTR(d_steps);
+    RESPS_CHECK_PTR(d_n_nodes);
+    RESPS_CHECK_PTR(d_target_logits);
+    RESPS_CHECK_PTR(d_draft_logits);
+    RESPS_CHECK_PTR(d_tokens);
+    RESPS_CHECK_PTR(d_parent);
+    RESPS_CHECK_PTR(d_u_accept);
+    RESPS_CHECK_PTR(d_u_sample);
+    RESPS_CHECK_PTR(d_accept_path);
+    RESPS_CHECK_PTR(d_accept_len);
+    RESPS_CHECK_PTR(d_out_tokens);
+    if (batch < 1 || ld_row < ctx->shape.vocab || ld_b < 0 || draft_ld_row < ctx->shape.vocab || draft_ld_level < 0 ||
+        draft_ld_b < 0 || !(temperature > 0.f))
+        return RESPS_ERR_INVALID_ARG;
+    if (batch > ctx->shape.max_batch) return RESPS_ERR_CAPACITY;
+    if (d_steps_next) resps::attention_plan_invalidate(ctx, d_steps_next);  // prefix lengths move on
+    if (resps::launch_accept_sampled(ctx, d_steps, d_n_nodes, batch, d_target_logits, ld_b, ld_row, d_draft_logits,
+                                     draft_ld_b, draft_ld_level, draft_ld_row, static_cast<double>(temperature),
+                                     d_tokens, d_parent, d_u_accept, d_u_sample, d_accept_path, d_accept_len,
+                                     d_out_tokens, d_steps_next, stream) != cudaSuccess)
         return RESPS_ERR_CUDA;
     return RESPS_OK;
 }

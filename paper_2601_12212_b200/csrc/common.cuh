@@ -37,6 +37,8 @@ struct Workspace {
     double* row_lse = nullptr;               // [max_batch][max_rows]
     unsigned long long* amax_part = nullptr; // [max_batch][max_tt][splits]
     unsigned int* amax_counter = nullptr;    // [max_batch][max_tt]
+    int32_t* node_row = nullptr;             // [max_batch][max_tt] draft row behind every node's children (tree build)
+    double* samp_scratch = nullptr;          // acceptance under sampling: a few words per sequence
     unsigned int* amax_seq_counter = nullptr;  // [max_batch] rows of a sequence whose arg-max is final (self-resetting)
     // attention
     int attn_grid = 0;          // persistent CTAs (one per SM)
@@ -130,6 +132,13 @@ cudaError_t launch_pdl(Kernel kernel, dim3 grid, dim3 block, size_t smem, cudaSt
     cfg.attrs = attr, cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, kernel, args...);
 }
+cudaError_t launch_accept_sampled(const resps_ctx* ctx, const resps_step* d_steps, const int32_t* d_n_nodes, int batch,
+                                  const float* target, int64_t ld_b, int64_t ld_row, const float* draft, int64_t dld_b,
+                                  int64_t dld_level, int64_t dld_row, double temperature, const int32_t* tokens,
+                                  const int32_t* parent, const double* u_accept, const double* u_sample,
+                                  int32_t* accept_path, int32_t* accept_len, int32_t* out_tokens, resps_step* steps_next,
+                                  cudaStream_t st);
+size_t sampled_scratch_doubles(int max_batch);
 cudaError_t tree_setup(resps_ctx* ctx);
 cudaError_t scan_setup(resps_ctx* ctx);
 int tree_candidate_limit();

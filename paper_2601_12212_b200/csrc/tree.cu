@@ -28,6 +28,7 @@ struct TreeArgs {
     int32_t *tokens, *parent, *depth, *position_ids;
     uint64_t* mask;
     int32_t *retrieve, *n_leaves, *n_nodes;
+    int32_t* node_row;  // workspace [batch][max_tt]: level * RESPS_MAX_K + slot of the draft row a node's children came from
     int32_t* status;
     int cand_cap;  // candidates the shared-memory arrays hold
 };
@@ -195,6 +196,16 @@ __global__ void __launch_bounds__(kTreeThreads, 1) tree_build_kernel(const TreeA
         }
     }
     __syncthreads();
+    // The draft row every node's children were taken from (kept in the workspace for the acceptance
+    // under sampling, which needs the draft distribution behind every tried child): the root's is row
+    // (0, 0); the p-th member of the frontier after level j < d-1 was given row (j+1, p).
+    for (int i = tid; i < n; i += kTreeThreads) a.node_row[ob + i] = (i == 0) ? 0 : -1;
+    __syncthreads();
+    for (int e = tid; e < (d - 1) * k; e += kTreeThreads) {
+        const int j = e / k, p = e - j * k;
+        const int i = node_of[frontier[j * RESPS_MAX_K + p]];
+        if (i > 0) a.node_row[ob + i] = (j + 1) * RESPS_MAX_K + p;
+    }
     // `total` equals m by construction of the ranks.
     for (int c = tid; c < n_cand; c += kTreeThreads) {
         const int i = node_of[c];
@@ -283,6 +294,7 @@ cudaError_t launch_tree_build(const resps_ctx* ctx, const resps_step* d_steps, i
     a.root_token = root_token;
     a.tokens = tokens, a.parent = parent, a.depth = depth, a.position_ids = position_ids;
     a.mask = mask, a.retrieve = retrieve, a.n_leaves = n_leaves, a.n_nodes = n_nodes;
+    a.node_row = ctx->ws.node_row;
     a.status = ctx->ws.status;
     a.cand_cap = s.max_k + (s.max_depth - 1) * s.max_k * s.max_k;
     const size_t smem = tree_smem_bytes(a.cand_cap);
