@@ -258,3 +258,67 @@ def kv_compact(k_cache: np.ndarray, v_cache: np.ndarray, L: int, path: np.ndarra
     if rc != 0:
         raise ValueError(f"oracle_kv_compact rc={rc}")
     return L + a + 1
+
+
+# ------------------------------------------------------------------------------ controller
+@dataclass
+class ControllerState:
+    """Per-sequence state of the action cache (Algorithm 1)."""
+    cache_step: int = 0        # position inside the cache interval; 0 = the policy is asked at the next step
+    action: int = -1           # index of the cached action
+    reward_sum: float = 0.0    # sum of accepted tokens / second over the steps of the open interval
+    reward_steps: int = 0
+
+
+def policy_logits(state_vec: np.ndarray, w1, b1, w2, b2, w3, b3) -> np.ndarray:
+    """The policy network (Appendix A: two hidden layers of 128 units) in fp64 on the state
+    s_t = concat(h, m, l) (Eq. 4): logits = W3 tanh(W2 tanh(W1 s + b1) + b2) + b3.  (tanh is the
+    default activation of the Stable-Baselines3 policy the paper uses; the paper does not name it.)"""
+    s = np.asarray(state_vec, np.float64)
+    h1 = np.tanh(np.asarray(w1, np.float64) @ s + np.asarray(b1, np.float64))
+    h2 = np.tanh(np.asarray(w2, np.float64) @ h1 + np.asarray(b2, np.float64))
+    return np.asarray(w3, np.float64) @ h2 + np.asarray(b3, np.float64)
+
+
+def controller_step(st: ControllerState, state_vec, weights, actions: np.ndarray, interval: int,
+                    temperature: float, u: float, prev_accept_len, prev_elapsed_s):
+    """One decoding step of Algorithm 1 (action caching) with the reward of Eq. 5.
+
+    prev_accept_len / prev_elapsed_s describe the step that has just finished (None before the first
+    step): its reward, tokens emitted (accepted drafts + 1) per second (Eq. 3), is added to the open
+    interval.  When cache_step is 0 the interval is closed -- r_avg (Eq. 5), the mean of its rewards, is
+    reported -- and the policy is asked: arg-max of its logits at temperature 0, else a draw from
+    softmax(logits / temperature) by inverse CDF with u.  The chosen (TT, d, k) is then used for
+    `interval` consecutive steps.  Returns (new state, (TT, d, k), r_avg or None, logits or None,
+    margin): margin is the distance of the choice from flipping (top-2 logit gap, or the CDF distance)."""
+    st = ControllerState(st.cache_step, st.action, st.reward_sum, st.reward_steps)
+    if prev_accept_len is not None:
+        st.reward_sum += (int(prev_accept_len) + 1) / float(prev_elapsed_s)
+        st.reward_steps += 1
+    r_avg, logits, margin = None, None, float("inf")
+    if st.cache_step == 0 or st.action < 0:
+        if st.reward_steps > 0:
+            r_avg = st.reward_sum / st.reward_steps
+        st.reward_sum, st.reward_steps = 0.0, 0
+        logits = policy_logits(state_vec, *weights)
+        if temperature <= 0.0:
+            order = np.argsort(-logits, kind="stable")
+            st.action = int(order[0])
+            if len(order) > 1:
+                margin = float(logits[order[0]] - logits[order[1]])
+        else:
+            z = logits / temperature
+            p = np.exp(z - z.max())
+            p /= p.sum()
+            cdf = np.cumsum(p)
+            target = u * cdf[-1]
+            st.action = int(min(np.searchsorted(cdf, target, side="right"), len(p) - 1))
+            lo = cdf[st.action - 1] if st.action > 0 else 0.0
+            margin = float(min(target - lo, cdf[st.action] - target)) if st.action < len(p) - 1 else float(target - lo)
+        st.cache_step = 1
+    else:
+        st.cache_step += 1
+    if st.cache_step >= interval:
+        st.cache_step = 0
+    tt, d, k = (int(x) for x in actions[st.action])
+    return st, (tt, d, k), r_avg, logits, margin
