@@ -275,6 +275,51 @@ int resps_kv_compact(resps_ctx* ctx, const resps_step* d_steps, int steps_advanc
                      int64_t kv_capacity, resps_stream stream);
 
 /*
+ * Controller glue: one call per decoding step, before resps_tree_expand (Algorithm 1, "Re-SpS with
+ * Action Caching"; Eq. 4: the state s_t is the concatenation of three hidden layers of the target
+ * model; Eq. 3 and Eq. 5: the reward is tokens per second, averaged over the cache interval; Appendix
+ * A: the policy network has two hidden layers of 128 units over the filtered action grid).
+ *
+ * Per sequence b:
+ *   - the step that has just finished (d_prev_accept_len, d_prev_elapsed_s; both NULL before the first
+ *     step) adds (accepted + 1) / seconds to the open interval;
+ *   - while the cached action is valid (0 < cache_step) it is kept and cache_step advances, wrapping to
+ *     0 after `interval` steps;
+ *   - at cache_step 0 the interval is closed (d_reward_avg[b] = mean reward of its steps, Eq. 5), the
+ *     policy is evaluated on the state, logits = W3 tanh(W2 tanh(W1 s + b1) + b2) + b3, an action is
+ *     chosen (temperature 0: arg-max, ties -> lowest index; else a draw from softmax(logits / T) by
+ *     inverse CDF in action order with d_uniform[b]) and its (TT, d, k) written into d_steps[b].
+ * The library reads (TT, d, k) from d_steps in device memory, so nothing else has to be told.
+ *
+ * policy          HOST struct of DEVICE pointers: fp32 weights, row-major [out][in]; actions int32
+ *                 [n_actions][3] = (TT, d, k); n_features divisible by 3, hidden <= 256, n_actions <= 1024
+ * d_hidden_h/m/l  DEVICE bf16 [batch][n_features / 3], row stride ld_hidden elements: the three layers'
+ *                 hidden states, read where the model left them
+ * d_state         DEVICE resps_controller_state [batch]; zero-initialised by the caller before the first step
+ * d_logits        DEVICE fp32 [batch][n_actions] or NULL; d_action DEVICE int32 [batch] or NULL
+ * The activation (tanh) and "accepted tokens = accepted drafts + 1" are this library's readings.
+ */
+typedef struct {
+    const float *w1, *b1; /* [hidden][n_features], [hidden]   */
+    const float *w2, *b2; /* [hidden][hidden], [hidden]       */
+    const float *w3, *b3; /* [n_actions][hidden], [n_actions] */
+    const int32_t* actions;
+    int32_t n_features, hidden, n_actions;
+} resps_policy;
+typedef struct {
+    int32_t cache_step;   /* position in the cache interval; 0: the policy is asked at this step */
+    int32_t action;       /* cached action index (state starts zeroed: the first step asks anyway) */
+    float reward_sum;     /* sum of tokens / second over the open interval */
+    int32_t reward_steps;
+} resps_controller_state;
+int resps_controller_step(resps_ctx* ctx, const resps_policy* policy, const void* d_hidden_h,
+                          const void* d_hidden_m, const void* d_hidden_l, int64_t ld_hidden, int batch,
+                          int interval, float temperature, const double* d_uniform,
+                          const int32_t* d_prev_accept_len, const float* d_prev_elapsed_s,
+                          resps_controller_state* d_state, resps_step* d_steps, float* d_reward_avg,
+                          float* d_logits, int32_t* d_action, resps_stream stream);
+
+/*
  * Per-node target arg-max for callers that cannot allocate device memory.  (The paper has no
  * counterpart: this is the arg-max step of resps_verify_accept offered without a context.)
  *

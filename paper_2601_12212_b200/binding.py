@@ -30,13 +30,18 @@ RESPS_DEBUG_SCAN_SLICES = 4
 
 EXPORTS = ("resps_create", "resps_destroy", "resps_strerror", "resps_status",
            "resps_workspace_bytes", "resps_debug_set", "resps_attention_replan", "resps_tree_expand", "resps_tree_attention",
-           "resps_verify_accept", "resps_verify_accept_sampled", "resps_kv_compact", "resps_target_argmax_static")
+           "resps_verify_accept", "resps_verify_accept_sampled", "resps_controller_step", "resps_kv_compact", "resps_target_argmax_static")
 
 
 class RespsShape(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in
                 ("n_q_heads", "n_kv_heads", "head_dim", "vocab", "max_batch", "max_tt", "max_k",
                  "max_depth")]
+
+
+class RespsPolicy(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in ("w1", "b1", "w2", "b2", "w3", "b3", "actions")] + \
+               [(n, ctypes.c_int32) for n in ("n_features", "hidden", "n_actions")]
 
 
 class RespsError(RuntimeError):
@@ -72,6 +77,8 @@ def load() -> ctypes.CDLL:
     lib.resps_verify_accept.argtypes = [vp, vp, vp, i32, vp, i64, i64, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.resps_verify_accept_sampled.argtypes = [vp, vp, vp, i32, vp, i64, i64, vp, i64, i64, i64, f32, vp, vp, vp, vp,
                                                 vp, vp, vp, vp, vp]
+    lib.resps_controller_step.argtypes = [vp, ctypes.POINTER(RespsPolicy), vp, vp, vp, i64, i32, i32, f32, vp, vp, vp,
+                                          vp, vp, vp, vp, vp, vp]
     lib.resps_kv_compact.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp, i32, i64, i64, i64, i64, vp]
     lib.resps_debug_set.argtypes = [vp, i32, i32]
     lib.resps_attention_replan.argtypes = [vp]
@@ -198,6 +205,28 @@ def resps_verify_accept_sampled(ctx: Context, steps, n_nodes, batch: int, target
         _ptr(draft_logits, f32), draft_ld_b, draft_ld_level, draft_ld_row, float(temperature), _ptr(tokens, i32),
         _ptr(parent, i32), _ptr(u_accept, f64), _ptr(u_sample, f64), _ptr(accept_path, i32), _ptr(accept_len, i32),
         _ptr(out_tokens, i32), _ptr(steps_next, i32), _stream(stream)), "resps_verify_accept_sampled")
+
+
+CONTROLLER_STATE_DTYPE = torch.int32  # resps_controller_state = (int32, int32, float32, int32): tensors [batch, 4]
+
+
+def make_policy(w1, b1, w2, b2, w3, b3, actions) -> RespsPolicy:
+    """Policy weights (fp32 CUDA tensors, [out][in]) and the action table (int32 [n_actions][3])."""
+    f32 = torch.float32
+    return RespsPolicy(_ptr(w1, f32), _ptr(b1, f32), _ptr(w2, f32), _ptr(b2, f32), _ptr(w3, f32), _ptr(b3, f32),
+                       _ptr(actions, torch.int32), w1.shape[1], w1.shape[0], w3.shape[0])
+
+
+def resps_controller_step(ctx: Context, policy: RespsPolicy, hidden_h, hidden_m, hidden_l, ld_hidden: int, batch: int,
+                          interval: int, temperature: float, uniform, prev_accept_len, prev_elapsed_s, state, steps,
+                          reward_avg, logits=None, action=None, stream=None) -> None:
+    """One controller step (action cache, policy network, averaged reward); writes (TT, d, k) into `steps`."""
+    bf, i32, f32 = torch.bfloat16, torch.int32, torch.float32
+    _check(load().resps_controller_step(
+        ctx.handle, ctypes.byref(policy), _ptr(hidden_h, bf), _ptr(hidden_m, bf), _ptr(hidden_l, bf), ld_hidden, batch,
+        interval, float(temperature), _ptr(uniform, torch.float64), _ptr(prev_accept_len, i32),
+        _ptr(prev_elapsed_s, f32), _ptr(state, i32), _ptr(steps, i32), _ptr(reward_avg, f32), _ptr(logits, f32),
+        _ptr(action, i32), _stream(stream)), "resps_controller_step")
 
 
 def resps_kv_compact(ctx: Context, steps, batch: int, accept_path, accept_len, k_cache_ptrs,

@@ -11,7 +11,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libresps.so")
-SOURCES = ["api.cu", "scan.cu", "tree.cu", "attention.cu", "accept.cu", "sampled.cu"]
+SOURCES = ["api.cu", "scan.cu", "tree.cu", "attention.cu", "accept.cu", "sampled.cu", "controller.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 

@@ -37,9 +37,11 @@ void carve(resps_ctx* c, Carver& cv) {
     cv.take(w.row_counter, rows);
     cv.take(w.amax_counter, nodes);
     cv.take(w.amax_seq_counter, s.max_batch);
+    cv.take(w.ctl_counter, s.max_batch);
     const int64_t zero_end = cv.off;  // everything above must start as zero
     (void)zero_end;
     cv.take(w.node_row, nodes);
+    cv.take(w.ctl_h1, static_cast<int64_t>(s.max_batch) * resps::controller_max_hidden());
     cv.take(w.samp_scratch, static_cast<int64_t>(resps::sampled_scratch_doubles(s.max_batch)));
     cv.take(w.part_key, rows * w.scan_splits * s.max_k);
     cv.take(w.part_ms, rows * w.scan_splits);
@@ -191,6 +193,7 @@ int resps_status(resps_ctx* ctx, resps_stream stream, int32_t* status) {
         if (cudaMemsetAsync(w.row_counter, 0, rows * sizeof(unsigned int), stream) != cudaSuccess ||
             cudaMemsetAsync(w.amax_counter, 0, nodes * sizeof(unsigned int), stream) != cudaSuccess ||
             cudaMemsetAsync(w.amax_seq_counter, 0, ctx->shape.max_batch * sizeof(unsigned int), stream) != cudaSuccess ||
+            cudaMemsetAsync(w.ctl_counter, 0, ctx->shape.max_batch * sizeof(unsigned int), stream) != cudaSuccess ||
             cudaStreamSynchronize(stream) != cudaSuccess)
             return RESPS_ERR_CUDA;
     }
@@ -322,6 +325,42 @@ int resps_verify_accept_sampled(resps_ctx* ctx, const resps_step* d_steps, const
                                      draft_ld_b, draft_ld_level, draft_ld_row, static_cast<double>(temperature),
                                      d_tokens, d_parent, d_u_accept, d_u_sample, d_accept_path, d_accept_len,
                                      d_out_tokens, d_steps_next, stream) != cudaSuccess)
+        return RESPS_ERR_CUDA;
+    return RESPS_OK;
+}
+
+int resps_controller_step(resps_ctx* ctx, const resps_policy* policy, const void* d_hidden_h,
+                          const void* d_hidden_m, const void* d_hidden_l, int64_t ld_hidden, int batch,
+                          int interval, float temperature, const double* d_uniform,
+                          const int32_t* d_prev_accept_len, const float* d_prev_elapsed_s,
+                          resps_controller_state* d_state, resps_step* d_steps, float* d_reward_avg,
+                          float* d_logits, int32_t* d_action, resps_stream stream) {
+    RESPS_CHECK_PTR(ctx);
+    RESPS_CHECK_PTR(policy);
+    RESPS_CHECK_PTR(d_hidden_h);
+    RESPS_CHECK_PTR(d_hidden_m);
+    RESPS_CHECK_PTR(d_hidden_l);
+    RESPS_CHECK_PTR(d_state);
+    RESPS_CHECK_PTR(d_steps);
+    RESPS_CHECK_PTR(d_reward_avg);
+    RESPS_CHECK_PTR(policy->w1);
+    RESPS_CHECK_PTR(policy->b1);
+    RESPS_CHECK_PTR(policy->w2);
+    RESPS_CHECK_PTR(policy->b2);
+    RESPS_CHECK_PTR(policy->w3);
+    RESPS_CHECK_PTR(policy->b3);
+    RESPS_CHECK_PTR(policy->actions);
+    if (batch < 1 || interval < 1 || policy->n_features < 3 || policy->n_features % 3 || policy->hidden < 1 ||
+        policy->n_actions < 1 || ld_hidden < policy->n_features / 3 || temperature < 0.f ||
+        (temperature > 0.f && !d_uniform) || ((d_prev_accept_len == nullptr) != (d_prev_elapsed_s == nullptr)))
+        return RESPS_ERR_INVALID_ARG;
+    if (policy->hidden > resps::controller_max_hidden() || policy->n_actions > resps::controller_max_actions())
+        return RESPS_ERR_UNSUPPORTED_SHAPE;
+    if (batch > ctx->shape.max_batch) return RESPS_ERR_CAPACITY;
+    resps::attention_plan_invalidate(ctx, d_steps);  // (TT, d, k) may change
+    if (resps::launch_controller(ctx, policy, d_hidden_h, d_hidden_m, d_hidden_l, ld_hidden, batch, interval,
+                                 temperature, d_uniform, d_prev_accept_len, d_prev_elapsed_s, d_state, d_steps,
+                                 d_reward_avg, d_logits, d_action, stream) != cudaSuccess)
         return RESPS_ERR_CUDA;
     return RESPS_OK;
 }

@@ -38,6 +38,8 @@ struct Workspace {
     unsigned long long* amax_part = nullptr; // [max_batch][max_tt][splits]
     unsigned int* amax_counter = nullptr;    // [max_batch][max_tt]
     int32_t* node_row = nullptr;             // [max_batch][max_tt] draft row behind every node's children (tree build)
+    float* ctl_h1 = nullptr;                 // controller: first hidden layer [max_batch][256]
+    unsigned int* ctl_counter = nullptr;     // controller: hidden units done per sequence (self-resetting)
     double* samp_scratch = nullptr;          // acceptance under sampling: a few words per sequence
     unsigned int* amax_seq_counter = nullptr;  // [max_batch] rows of a sequence whose arg-max is final (self-resetting)
     // attention
@@ -139,6 +141,13 @@ cudaError_t launch_accept_sampled(const resps_ctx* ctx, const resps_step* d_step
                                   int32_t* accept_path, int32_t* accept_len, int32_t* out_tokens, resps_step* steps_next,
                                   cudaStream_t st);
 size_t sampled_scratch_doubles(int max_batch);
+cudaError_t launch_controller(const resps_ctx* ctx, const resps_policy* pol, const void* h, const void* m, const void* l,
+                              int64_t ld_hidden, int batch, int interval, float temperature, const double* uniform,
+                              const int32_t* accept_len, const float* elapsed_s, resps_controller_state* state,
+                              resps_step* steps, float* reward_avg, float* logits_out, int32_t* action_out,
+                              cudaStream_t st);
+int controller_max_hidden();
+int controller_max_actions();
 cudaError_t tree_setup(resps_ctx* ctx);
 cudaError_t scan_setup(resps_ctx* ctx);
 int tree_candidate_limit();
