@@ -151,6 +151,46 @@ int resps_tree_expand(resps_ctx* ctx, const resps_step* d_steps, int batch,
                       int32_t* d_n_leaves, int32_t* d_n_nodes, resps_stream stream);
 
 /*
+ * The same construction level by level, for a draft model that runs between levels (Section 3.2,
+ * "Draft Tree Expansion": the k best tokens of a layer are expanded to the next layer; Algorithm 2:
+ * the draft model is called inside the tree-building loop).
+ *
+ *   resps_tree_expand_begin(ctx, d_steps, batch, n_slots)
+ *   for level j = 0 .. d-1:
+ *       the draft model produces the rows of level j (level 0: one row, after the root; level j >= 1:
+ *       one row per member of the frontier after level j-1, in slot order)
+ *       resps_tree_expand_level(ctx, d_steps, batch, j, rows, ...)  ->  the frontier after level j
+ *   resps_tree_expand_finish(ctx, d_steps, batch, d_root_token, <outputs of resps_tree_expand>)
+ * yields exactly the tree resps_tree_expand builds from the same rows.  The number of levels given
+ * bounds the depth (a step asking for more is clamped and flagged).
+ *
+ * d_level_logits  DEVICE fp32, element (b, slot, v) at b*ld_b + slot*ld_row + v
+ * Frontier outputs, DEVICE, [batch][max_k], entries >= k untouched.  Member p of the frontier after
+ * level j is "draft node" 1 + j k + p (the root is draft node 0): the order in which a draft model
+ * appends its tokens' K/V behind the prefix.
+ *   d_frontier_tokens         its token
+ *   d_frontier_parent_slot    the slot of its parent in the frontier after level j-1 (-1: the root)
+ *   d_frontier_position_ids   L + j + 1
+ *   d_frontier_node_index     1 + j k + p
+ *   d_frontier_mask   uint64 [batch][max_k][2]: ancestor-or-self bits over draft nodes, in the format
+ *                     of resps_tree_attention (written as zero once 1 + (j+1) k exceeds 128 draft
+ *                     nodes); with the rows collected level by level it lets the draft model run
+ *                     resps_tree_attention over prefix + draft nodes
+ *   d_frontier_score  fp64 [batch][max_k] or NULL: cumulative log-probability (log V_i)
+ * Calls of one expansion must come in order on one stream; levels out of order return INVALID_ARG.
+ */
+int resps_tree_expand_begin(resps_ctx* ctx, const resps_step* d_steps, int batch, int n_slots);
+int resps_tree_expand_level(resps_ctx* ctx, const resps_step* d_steps, int batch, int level,
+                            const float* d_level_logits, int64_t ld_b, int64_t ld_row,
+                            int32_t* d_frontier_tokens, int32_t* d_frontier_parent_slot,
+                            int32_t* d_frontier_position_ids, int32_t* d_frontier_node_index,
+                            uint64_t* d_frontier_mask, double* d_frontier_score, resps_stream stream);
+int resps_tree_expand_finish(resps_ctx* ctx, const resps_step* d_steps, int batch, const int32_t* d_root_token,
+                             int32_t* d_tokens, int32_t* d_parent, int32_t* d_depth, int32_t* d_position_ids,
+                             uint64_t* d_mask, int32_t* d_retrieve, int32_t* d_n_leaves, int32_t* d_n_nodes,
+                             resps_stream stream);
+
+/*
  * Tree-masked verification attention for one layer (Section 3.2, "Verification Phase":
  * the target model scores all tree tokens in a single pass; Appendix D: attention masks
  * follow the tree).

@@ -75,6 +75,29 @@ class Tree:
     near_pairs: np.ndarray    # int32 [n_near, 2]: boundary pairs (before, after) with a gap below tau
     node_cand: np.ndarray     # int32 [n]: candidate index of each node (-1 for the root)
 
+    def level_frontier(self, j: int, k: int, L: int):
+        """The frontier after level j as a draft model needs it (Section 3.2, "Draft Tree Expansion": the k
+        best tokens of a layer are expanded to the next one): per member p its token, the slot of its
+        parent in the previous frontier (-1: the root), position id L + j + 1, its draft-node index
+        1 + j k + p (the root is draft node 0) and the ancestor-or-self mask over draft nodes."""
+        cands = [int(c) for c in self.frontier[j][:k]]
+        tokens = np.array([self.cand_token[c] for c in cands], np.int32)
+        prev = [int(c) for c in self.frontier[j - 1][:k]] if j > 0 else []
+        parent_slot = np.array([prev.index(int(self.cand_parent[c])) if j > 0 else -1 for c in cands], np.int32)
+        mask = np.zeros((k, 2), np.uint64)
+        for p_, c in enumerate(cands):
+            bits, cc, jj = 1, c, j                      # the root
+            while True:
+                slot = [int(x) for x in self.frontier[jj][:k]].index(cc)
+                bits |= 1 << (1 + jj * k + slot)
+                if jj == 0:
+                    break
+                cc, jj = int(self.cand_parent[cc]), jj - 1
+            mask[p_] = (bits & 0xFFFFFFFFFFFFFFFF, bits >> 64)
+        return dict(tokens=tokens, parent_slot=parent_slot, position_ids=np.full(k, L + j + 1, np.int32),
+                    node_index=np.arange(1 + j * k, 1 + j * k + k, dtype=np.int32), mask=mask,
+                    score=np.array([self.cand_score[c] for c in cands]))
+
     def node_rows(self, d: int, k: int, slots: int) -> np.ndarray:
         """int32 [n]: for every node the index level * slots + slot of the draft row its children were taken
         from (the root: row 0; a candidate that is the p-th member of the frontier after level j < d-1:

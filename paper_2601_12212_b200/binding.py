@@ -29,7 +29,8 @@ RESPS_DEBUG_ATTN_STAGGER = 3
 RESPS_DEBUG_SCAN_SLICES = 4
 
 EXPORTS = ("resps_create", "resps_destroy", "resps_strerror", "resps_status",
-           "resps_workspace_bytes", "resps_debug_set", "resps_attention_replan", "resps_tree_expand", "resps_tree_attention",
+           "resps_workspace_bytes", "resps_debug_set", "resps_attention_replan", "resps_tree_expand", "resps_tree_expand_begin", "resps_tree_expand_level",
+           "resps_tree_expand_finish", "resps_tree_attention",
            "resps_verify_accept", "resps_verify_accept_sampled", "resps_controller_step", "resps_kv_compact", "resps_target_argmax_static")
 
 
@@ -72,6 +73,9 @@ def load() -> ctypes.CDLL:
     lib.resps_workspace_bytes.restype = i64
     lib.resps_tree_expand.argtypes = [vp, vp, i32, vp, i64, i64, i64, i32, i32, vp,
                                       vp, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.resps_tree_expand_begin.argtypes = [vp, vp, i32, i32]
+    lib.resps_tree_expand_level.argtypes = [vp, vp, i32, i32, vp, i64, i64, vp, vp, vp, vp, vp, vp, vp]
+    lib.resps_tree_expand_finish.argtypes = [vp, vp, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.resps_tree_attention.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp, vp, i64, i64, i64, i64,
                                          vp, f32, vp]
     lib.resps_verify_accept.argtypes = [vp, vp, vp, i32, vp, i64, i64, vp, vp, vp, vp, vp, vp, vp, vp]
@@ -170,6 +174,30 @@ def resps_tree_expand(ctx: Context, steps, batch: int, draft_logits, ld_b: int, 
         n_levels, n_slots, _ptr(root_token, i32), _ptr(tokens, i32), _ptr(parent, i32),
         _ptr(depth, i32), _ptr(position_ids, i32), _ptr(mask), _ptr(retrieve, i32),
         _ptr(n_leaves, i32), _ptr(n_nodes, i32), _stream(stream)), "resps_tree_expand")
+
+
+def resps_tree_expand_begin(ctx: Context, steps, batch: int, n_slots: int) -> None:
+    _check(load().resps_tree_expand_begin(ctx.handle, _ptr(steps, torch.int32), batch, n_slots), "resps_tree_expand_begin")
+
+
+def resps_tree_expand_level(ctx: Context, steps, batch: int, level: int, level_logits, ld_b: int, ld_row: int,
+                            frontier_tokens, frontier_parent_slot, frontier_position_ids, frontier_node_index,
+                            frontier_mask, frontier_score=None, stream=None) -> None:
+    i32 = torch.int32
+    _check(load().resps_tree_expand_level(
+        ctx.handle, _ptr(steps, i32), batch, level, _ptr(level_logits, torch.float32), ld_b, ld_row,
+        _ptr(frontier_tokens, i32), _ptr(frontier_parent_slot, i32), _ptr(frontier_position_ids, i32),
+        _ptr(frontier_node_index, i32), _ptr(frontier_mask), _ptr(frontier_score, torch.float64), _stream(stream)),
+        "resps_tree_expand_level")
+
+
+def resps_tree_expand_finish(ctx: Context, steps, batch: int, root_token, tokens, parent, depth, position_ids, mask,
+                             retrieve, n_leaves, n_nodes, stream=None) -> None:
+    i32 = torch.int32
+    _check(load().resps_tree_expand_finish(
+        ctx.handle, _ptr(steps, i32), batch, _ptr(root_token, i32), _ptr(tokens, i32), _ptr(parent, i32),
+        _ptr(depth, i32), _ptr(position_ids, i32), _ptr(mask), _ptr(retrieve, i32), _ptr(n_leaves, i32),
+        _ptr(n_nodes, i32), _stream(stream)), "resps_tree_expand_finish")
 
 
 def resps_tree_attention(ctx: Context, steps, n_nodes, batch: int, q, o, lse, k_cache, v_cache,

@@ -99,6 +99,7 @@ int resps_create(resps_ctx** out, const resps_shape* shape) {
     resps_ctx* c = new (std::nothrow) resps_ctx();
     if (!c) return RESPS_ERR_CUDA;
     c->attn_host = nullptr;
+    c->level_next = 0, c->level_slots = 1;
     c->shape = s;
     c->device = dev;
     c->sm_count = prop.multiProcessorCount;
@@ -225,12 +226,79 @@ int resps_tree_expand(resps_ctx* ctx, const resps_step* d_steps, int batch,
     if (n_slots > ctx->shape.max_k) n_slots = ctx->shape.max_k;
     resps::attention_plan_invalidate(ctx);  // a new tree: new node counts, possibly new step parameters
     if (resps::launch_row_scan(ctx, d_steps, batch, d_draft_logits, ld_b, ld_level, ld_row, n_levels,
-                               n_slots, stream) != cudaSuccess)
+                               n_slots, -1, stream) != cudaSuccess)
         return RESPS_ERR_CUDA;
     if (resps::launch_tree_build(ctx, d_steps, batch, n_levels, n_slots, d_root_token, d_tokens, d_parent,
                                  d_depth, d_position_ids, d_mask, d_retrieve, d_n_leaves, d_n_nodes,
                                  stream) != cudaSuccess)
         return RESPS_ERR_CUDA;
+    return RESPS_OK;
+}
+
+// ---- level form of the tree expansion --------------------------------------------------------------
+int resps_tree_expand_begin(resps_ctx* ctx, const resps_step* d_steps, int batch, int n_slots) {
+    RESPS_CHECK_PTR(ctx);
+    RESPS_CHECK_PTR(d_steps);
+    if (batch < 1 || n_slots < 1) return RESPS_ERR_INVALID_ARG;
+    if (batch > ctx->shape.max_batch) return RESPS_ERR_CAPACITY;
+    ctx->level_next = 0;
+    ctx->level_slots = n_slots > ctx->shape.max_k ? ctx->shape.max_k : n_slots;
+    resps::attention_plan_invalidate(ctx);
+    return RESPS_OK;
+}
+
+int resps_tree_expand_level(resps_ctx* ctx, const resps_step* d_steps, int batch, int level,
+                            const float* d_level_logits, int64_t ld_b, int64_t ld_row,
+                            int32_t* d_frontier_tokens, int32_t* d_frontier_parent_slot,
+                            int32_t* d_frontier_position_ids, int32_t* d_frontier_node_index,
+                            uint64_t* d_frontier_mask, double* d_frontier_score, resps_stream stream) {
+    RESPS_CHECK_PTR(ctx);
+    RESPS_CHECK_PTR(d_steps);
+    RESPS_CHECK_PTR(d_level_logits);
+    RESPS_CHECK_PTR(d_frontier_tokens);
+    RESPS_CHECK_PTR(d_frontier_parent_slot);
+    RESPS_CHECK_PTR(d_frontier_position_ids);
+    RESPS_CHECK_PTR(d_frontier_node_index);
+    RESPS_CHECK_PTR(d_frontier_mask);
+    if (batch < 1 || ld_row < ctx->shape.vocab || ld_b < 0 || level < 0) return RESPS_ERR_INVALID_ARG;
+    if (batch > ctx->shape.max_batch) return RESPS_ERR_CAPACITY;
+    if (level != ctx->level_next || level >= ctx->shape.max_depth) return RESPS_ERR_INVALID_ARG;  // levels come in order
+    const int n_levels = ctx->shape.max_depth, n_slots = ctx->level_slots;
+    if (resps::launch_row_scan(ctx, d_steps, batch, d_level_logits, ld_b, 0, ld_row, n_levels, n_slots, level,
+                               stream) != cudaSuccess)
+        return RESPS_ERR_CUDA;
+    resps::FrontierOut out = {d_frontier_tokens, d_frontier_parent_slot, d_frontier_position_ids,
+                              d_frontier_node_index, d_frontier_mask, d_frontier_score};
+    if (resps::launch_tree_level(ctx, d_steps, batch, n_levels, n_slots, level, out, stream) != cudaSuccess)
+        return RESPS_ERR_CUDA;
+    ctx->level_next = level + 1;
+    return RESPS_OK;
+}
+
+int resps_tree_expand_finish(resps_ctx* ctx, const resps_step* d_steps, int batch, const int32_t* d_root_token,
+                             int32_t* d_tokens, int32_t* d_parent, int32_t* d_depth, int32_t* d_position_ids,
+                             uint64_t* d_mask, int32_t* d_retrieve, int32_t* d_n_leaves, int32_t* d_n_nodes,
+                             resps_stream stream) {
+    RESPS_CHECK_PTR(ctx);
+    RESPS_CHECK_PTR(d_steps);
+    RESPS_CHECK_PTR(d_root_token);
+    RESPS_CHECK_PTR(d_tokens);
+    RESPS_CHECK_PTR(d_parent);
+    RESPS_CHECK_PTR(d_depth);
+    RESPS_CHECK_PTR(d_position_ids);
+    RESPS_CHECK_PTR(d_mask);
+    RESPS_CHECK_PTR(d_retrieve);
+    RESPS_CHECK_PTR(d_n_leaves);
+    RESPS_CHECK_PTR(d_n_nodes);
+    if (batch < 1 || ctx->level_next < 1) return RESPS_ERR_INVALID_ARG;  // at least level 0 must have been given
+    if (batch > ctx->shape.max_batch) return RESPS_ERR_CAPACITY;
+    resps::attention_plan_invalidate(ctx);
+    // the levels that were given bound the depth: a step asking for more is clamped (and flagged)
+    if (resps::launch_tree_build(ctx, d_steps, batch, ctx->level_next, ctx->level_slots, d_root_token, d_tokens,
+                                 d_parent, d_depth, d_position_ids, d_mask, d_retrieve, d_n_leaves, d_n_nodes,
+                                 stream) != cudaSuccess)
+        return RESPS_ERR_CUDA;
+    ctx->level_next = 0;
     return RESPS_OK;
 }
 

@@ -69,6 +69,7 @@ struct resps_ctx {
     void* arena;
     int64_t arena_bytes;
     resps::Workspace ws;
+    int level_next, level_slots;  // level form of the tree expansion: the level expected next, the slots per level
     void* attn_host;  // host-side state of the attention launcher (tensor-map cache, work-list bookkeeping)
 };
 
@@ -87,7 +88,15 @@ struct AcceptArgs {
 // ---- launchers (one per translation unit) ---------------------------------
 cudaError_t launch_row_scan(const resps_ctx* ctx, const resps_step* d_steps, int batch,
                             const float* logits, int64_t ld_b, int64_t ld_level, int64_t ld_row,
-                            int n_levels, int n_slots, cudaStream_t st);
+                            int n_levels, int n_slots, int only_level, cudaStream_t st);
+// What the level form of the tree expansion hands back per level: the members of the new frontier.
+struct FrontierOut {
+    int32_t *tokens, *parent_slot, *position_ids, *node_index;  // [batch][max_k]
+    uint64_t* mask;                                              // [batch][max_k][2]
+    double* score;                                               // [batch][max_k] or null
+};
+cudaError_t launch_tree_level(const resps_ctx* ctx, const resps_step* d_steps, int batch, int n_levels, int n_slots,
+                              int level, const FrontierOut& out, cudaStream_t st);
 cudaError_t launch_tree_build(const resps_ctx* ctx, const resps_step* d_steps, int batch,
                               int n_levels, int n_slots, const int32_t* root_token,
                               int32_t* tokens, int32_t* parent, int32_t* depth, int32_t* position_ids,

@@ -27,6 +27,7 @@ struct ScanArgs {
     int chunk, splits;
     int slices, cps;  // streaming kernel: slices per row, chunks per slice (partials keep the stride `splits`)
     int test_drop;    // test build only: 2 = the second chunk copy of every slice is left out
+    int only_level;   // -1: the rows of all levels; j >= 0: only level j's rows (blockIdx.y = slot)
     unsigned long long* part_key;
     float2* part_ms;
     unsigned int* counter;
@@ -89,11 +90,13 @@ __global__ void __launch_bounds__(kScanThreads, 4) row_scan_kernel(const ScanArg
     __shared__ int s_count;
     __shared__ float2 s_ms[kScanThreads / 32];
     __shared__ bool s_last;
-    const int b = blockIdx.z, r = blockIdx.y, sp = blockIdx.x;
+    const int b = blockIdx.z, ry = blockIdx.y, sp = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const StepDims sd = clamp_step(a.steps[b], a.n_levels, a.n_slots, a.max_tt, a.max_k, a.vocab);
     const int k = sd.k;
     const int rows = 1 + (sd.d - 1) * k;
+    if (a.only_level >= 0 && ry >= (a.only_level == 0 ? 1 : k)) return;
+    const int r = (a.only_level < 0) ? ry : (a.only_level == 0 ? 0 : 1 + (a.only_level - 1) * k + ry);
     if (r >= rows) return;
     if (sd.clamped && r == 0 && sp == 0 && tid == 0) atomicOr(a.status, RESPS_STATUS_STEP_CLAMPED);
     const int level = (r == 0) ? 0 : 1 + (r - 1) / k;
@@ -316,11 +319,13 @@ __global__ void __launch_bounds__(kStreamThreads, 2) row_scan_stream_kernel(cons
     __shared__ int s_count;
     __shared__ float2 s_ms[kScanThreads / 32];
     __shared__ bool s_last;
-    const int b = blockIdx.z, r = blockIdx.y, sl = blockIdx.x;
+    const int b = blockIdx.z, ry = blockIdx.y, sl = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const StepDims sd = clamp_step(a.steps[b], a.n_levels, a.n_slots, a.max_tt, a.max_k, a.vocab);
     const int k = sd.k;
     const int rows = 1 + (sd.d - 1) * k;
+    if (a.only_level >= 0 && ry >= (a.only_level == 0 ? 1 : k)) return;
+    const int r = (a.only_level < 0) ? ry : (a.only_level == 0 ? 0 : 1 + (a.only_level - 1) * k + ry);
     if (r >= rows) return;
     if (sd.clamped && r == 0 && sl == 0 && tid == 0) atomicOr(a.status, RESPS_STATUS_STEP_CLAMPED);
     const int level = (r == 0) ? 0 : 1 + (r - 1) / k;
@@ -833,7 +838,7 @@ cudaError_t scan_setup(resps_ctx* ctx) {
 
 cudaError_t launch_row_scan(const resps_ctx* ctx, const resps_step* d_steps, int batch,
                             const float* logits, int64_t ld_b, int64_t ld_level, int64_t ld_row,
-                            int n_levels, int n_slots, cudaStream_t st) {
+                            int n_levels, int n_slots, int only_level, cudaStream_t st) {
     const Workspace& w = ctx->ws;
     ScanArgs a;
     a.steps = d_steps;
@@ -845,7 +850,8 @@ cudaError_t launch_row_scan(const resps_ctx* ctx, const resps_step* d_steps, int
     a.part_key = w.part_key, a.part_ms = w.part_ms, a.counter = w.row_counter;
     a.row_val = w.row_val, a.row_id = w.row_id, a.row_lse = w.row_lse, a.status = w.status;
     const int k_ext = min(n_slots, ctx->shape.max_k);
-    const int rows = (n_levels > 1) ? 1 + (n_levels - 1) * k_ext : 1;
+    a.only_level = only_level;
+    const int rows = (only_level >= 0) ? (only_level == 0 ? 1 : k_ext) : ((n_levels > 1) ? 1 + (n_levels - 1) * k_ext : 1);
     a.slices = w.scan_splits, a.cps = 1;
     a.test_drop = w.test_drop;
     const size_t smem = sizeof(unsigned long long) * ctx->shape.max_k * max(kQuadElems, w.scan_splits);

@@ -31,6 +31,10 @@ struct TreeArgs {
     int32_t* node_row;  // workspace [batch][max_tt]: level * RESPS_MAX_K + slot of the draft row a node's children came from
     int32_t* status;
     int cand_cap;  // candidates the shared-memory arrays hold
+    // Level form: emit_level = j >= 0 ranks the levels up to j from the rows scanned so far, hands out
+    // the frontier after level j and stops; -1 builds the whole tree.
+    int emit_level;
+    FrontierOut fr;
 };
 
 // Candidate order of the method: larger score first, equal scores by lower index.
@@ -87,7 +91,8 @@ __global__ void __launch_bounds__(kTreeThreads, 1) tree_build_kernel(const TreeA
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int b = blockIdx.x, tid = threadIdx.x;
     const StepDims sd = clamp_step(a.steps[b], a.n_levels, a.n_slots, a.max_tt, a.max_k, a.vocab);
-    const int k = sd.k, d = sd.d, kk = k * k;
+    const int k = sd.k, kk = k * k;
+    const int d = (a.emit_level >= 0) ? min(sd.d, a.emit_level + 1) : sd.d;  // levels ranked by this launch
     const int n_cand = k + (d - 1) * kk;
     const int m = min(sd.tt - 1, n_cand);
     const int n = m + 1;
@@ -153,6 +158,45 @@ __global__ void __launch_bounds__(kTreeThreads, 1) tree_build_kernel(const TreeA
             }
         }
         __syncthreads();
+    }
+
+    if (a.emit_level >= 0) {
+        // ---- level form: the frontier after level j, for the draft model's next pass ------------------
+        // Member p is draft node 1 + j k + p (the root is draft node 0, the frontier of level i occupies
+        // 1 + i k .. i k + k): token, the slot of its parent in the previous frontier, position id, the
+        // ancestor-or-self mask over draft nodes (only while they fit 128 bits) and its score.
+        const int j = a.emit_level;
+        if (j < sd.d && tid < k) {
+            const int c = frontier[j * RESPS_MAX_K + tid];
+            const int64_t of = static_cast<int64_t>(b) * a.max_k + tid;
+            a.fr.tokens[of] = a.row_id[(row0 + cand_row(c)) * a.max_k + cand_rank_in_row(c)];
+            a.fr.parent_slot[of] = (j == 0) ? -1 : ((c - (k + (j - 1) * kk)) / k);
+            a.fr.position_ids[of] = sd.L + j + 1;
+            a.fr.node_index[of] = 1 + j * k + tid;
+            if (a.fr.score) a.fr.score[of] = score[c];
+            unsigned long long lo = 1ull, hi = 0ull;  // the root
+            if (1 + (j + 1) * k <= 128) {
+                int cc = c, slot = tid;
+                for (int jj = j; jj >= 0; --jj) {
+                    const int node = 1 + jj * k + slot;
+                    if (node < 64)
+                        lo |= 1ull << node;
+                    else
+                        hi |= 1ull << (node - 64);
+                    if (jj > 0) {
+                        slot = (cc - (k + (jj - 1) * kk)) / k;
+                        cc = frontier[(jj - 1) * RESPS_MAX_K + slot];
+                    }
+                }
+            } else {
+                lo = 0ull;
+            }
+            a.fr.mask[of * 2 + 0] = lo;
+            a.fr.mask[of * 2 + 1] = hi;
+        }
+        // (a sequence whose own d is below j + 1 has nothing at this level: its entries stay untouched)
+        if (tid == 0 && sd.clamped) atomicOr(a.status, RESPS_STATUS_STEP_CLAMPED);
+        return;
     }
 
     // ---- global rerank: keep the m best of all candidates -------------------------
@@ -297,8 +341,27 @@ cudaError_t launch_tree_build(const resps_ctx* ctx, const resps_step* d_steps, i
     a.node_row = ctx->ws.node_row;
     a.status = ctx->ws.status;
     a.cand_cap = s.max_k + (s.max_depth - 1) * s.max_k * s.max_k;
+    a.emit_level = -1;
+    a.fr = FrontierOut{};
     const size_t smem = tree_smem_bytes(a.cand_cap);
     return launch_pdl(tree_build_kernel, dim3(batch), dim3(kTreeThreads), smem, st, a);
+}
+
+cudaError_t launch_tree_level(const resps_ctx* ctx, const resps_step* d_steps, int batch, int n_levels, int n_slots,
+                              int level, const FrontierOut& out, cudaStream_t st) {
+    const resps_shape& s = ctx->shape;
+    TreeArgs a = {};
+    a.steps = d_steps;
+    a.n_levels = n_levels, a.n_slots = n_slots;
+    a.vocab = s.vocab, a.max_tt = s.max_tt, a.max_k = s.max_k, a.max_depth = s.max_depth;
+    a.max_rows = ctx->ws.max_rows;
+    a.row_val = ctx->ws.row_val, a.row_id = ctx->ws.row_id, a.row_lse = ctx->ws.row_lse;
+    a.node_row = ctx->ws.node_row;
+    a.status = ctx->ws.status;
+    a.cand_cap = s.max_k + (s.max_depth - 1) * s.max_k * s.max_k;
+    a.emit_level = level;
+    a.fr = out;
+    return launch_pdl(tree_build_kernel, dim3(batch), dim3(kTreeThreads), tree_smem_bytes(a.cand_cap), st, a);
 }
 
 // Largest k + (d-1)k^2 the shared-memory arrays can hold.

@@ -250,3 +250,24 @@ def test_brute_force_enumeration_on_tiny_inputs(seed):
         assert t.tokens.tolist() == tokens and t.parent.tolist() == parent
     else:  # exact score ties under rounding differences: only sizes are comparable
         assert t.n_nodes == len(tokens)
+
+
+def test_level_frontier_of_the_worked_example():
+    """The per-level view of the hand-worked example: after level 0 the frontier is candidates 0 and 1
+    (tokens 0 and 1, children of the root, draft nodes 1 and 2); after level 1 it is candidates 2 (token 2
+    under candidate 0) and 4 (token 3 under candidate 1): draft nodes 3 and 4 with masks root|1|3 and root|2|4."""
+    g = json.load(open(os.path.join(GOLDEN, "tree_worked_example.json")))
+    logits = np.zeros((2, 2, 4), np.float32)
+    logits[0, 0] = np.log(g["probs_level0_slot0"])
+    logits[1, 0] = np.log(g["probs_level1_slot0"])
+    logits[1, 1] = np.log(g["probs_level1_slot1"])
+    t = oracle.tree_expand(9, logits, 5, 2, 2, 7)
+    f0 = t.level_frontier(0, 2, 7)
+    assert f0["tokens"].tolist() == [0, 1] and f0["parent_slot"].tolist() == [-1, -1]
+    assert f0["position_ids"].tolist() == [8, 8] and f0["node_index"].tolist() == [1, 2]
+    assert f0["mask"][:, 0].tolist() == [0b011, 0b101]
+    f1 = t.level_frontier(1, 2, 7)
+    assert f1["tokens"].tolist() == [2, 3] and f1["parent_slot"].tolist() == [0, 1]
+    assert f1["position_ids"].tolist() == [9, 9] and f1["node_index"].tolist() == [3, 4]
+    assert f1["mask"][:, 0].tolist() == [0b01011, 0b10101]
+    np.testing.assert_allclose(np.exp(f1["score"]), [0.275, 0.27], rtol=1e-6)
