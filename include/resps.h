@@ -360,6 +360,43 @@ int resps_controller_step(resps_ctx* ctx, const resps_policy* policy, const void
                           float* d_logits, int32_t* d_action, resps_stream stream);
 
 /*
+ * Vocabulary sharded over several GPUs (Section 5: the 70B target model needs four GPUs; the paper does
+ * not say how the work is split -- this is the split by vocabulary columns).  Rank p of P holds columns
+ * [offset_p, offset_p + V_p) of every logits row and a context created with vocab = V_p (V_p >= max_k).
+ * A step then is, on every rank:
+ *   resps_row_scan_shard       the rank's columns of the draft rows -> k (value, local id) pairs and one
+ *                              log-sum-exp per row
+ *   (all-gather of those small arrays over the ranks: the caller's, e.g. NCCL)
+ *   resps_tree_expand_merge    merges the P shards' rows (ids become global by d_shard_offset) and builds
+ *                              the tree: identical on every rank, and identical to resps_tree_expand on
+ *                              the whole rows
+ *   resps_tree_attention       per rank on its own KV heads if the heads are sharded too (a context is
+ *                              created with the rank's heads; nothing crosses between ranks)
+ *   resps_target_argmax_shard  the rank's columns of the target rows -> one packed (value, local id) per node
+ *   (all-gather)
+ *   resps_verify_accept_merge  merges and walks: identical to resps_verify_accept on the whole rows
+ * Row arrays are [batch][resps_scan_rows(ctx)][max_k] (values fp32, ids int32) and
+ * [batch][resps_scan_rows(ctx)] (log-sum-exp, fp64); gathered arrays carry a leading [n_shards] dimension
+ * (n_shards <= 16); keys are uint64 [batch][max_tt].  d_shard_offset: DEVICE int32 [n_shards].
+ */
+int64_t resps_scan_rows(const resps_ctx* ctx);
+int resps_row_scan_shard(resps_ctx* ctx, const resps_step* d_steps, int batch, const float* d_draft_logits,
+                         int64_t ld_b, int64_t ld_level, int64_t ld_row, int n_levels, int n_slots,
+                         float* d_part_val, int32_t* d_part_id, double* d_part_lse, resps_stream stream);
+int resps_tree_expand_merge(resps_ctx* ctx, const resps_step* d_steps, int batch, int n_levels, int n_slots,
+                            int n_shards, const float* d_all_val, const int32_t* d_all_id, const double* d_all_lse,
+                            const int32_t* d_shard_offset, const int32_t* d_root_token, int32_t* d_tokens,
+                            int32_t* d_parent, int32_t* d_depth, int32_t* d_position_ids, uint64_t* d_mask,
+                            int32_t* d_retrieve, int32_t* d_n_leaves, int32_t* d_n_nodes, resps_stream stream);
+int resps_target_argmax_shard(resps_ctx* ctx, const int32_t* d_n_nodes, int batch, const float* d_target_logits,
+                              int64_t ld_b, int64_t ld_row, uint64_t* d_part_key, resps_stream stream);
+int resps_verify_accept_merge(resps_ctx* ctx, const resps_step* d_steps, const int32_t* d_n_nodes, int batch,
+                              int n_shards, const uint64_t* d_all_key, const int32_t* d_shard_offset,
+                              const int32_t* d_tokens, const int32_t* d_parent, int32_t* d_target_argmax,
+                              int32_t* d_accept_path, int32_t* d_accept_len, int32_t* d_out_tokens,
+                              resps_step* d_steps_next, resps_stream stream);
+
+/*
  * Per-node target arg-max for callers that cannot allocate device memory.  (The paper has no
  * counterpart: this is the arg-max step of resps_verify_accept offered without a context.)
  *

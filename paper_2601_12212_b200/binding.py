@@ -31,7 +31,8 @@ RESPS_DEBUG_SCAN_SLICES = 4
 EXPORTS = ("resps_create", "resps_destroy", "resps_strerror", "resps_status",
            "resps_workspace_bytes", "resps_debug_set", "resps_attention_replan", "resps_tree_expand", "resps_tree_expand_begin", "resps_tree_expand_level",
            "resps_tree_expand_finish", "resps_tree_attention",
-           "resps_verify_accept", "resps_verify_accept_sampled", "resps_controller_step", "resps_kv_compact", "resps_target_argmax_static")
+           "resps_verify_accept", "resps_verify_accept_sampled", "resps_controller_step", "resps_scan_rows", "resps_row_scan_shard",
+           "resps_tree_expand_merge", "resps_target_argmax_shard", "resps_verify_accept_merge", "resps_kv_compact", "resps_target_argmax_static")
 
 
 class RespsShape(ctypes.Structure):
@@ -83,12 +84,19 @@ def load() -> ctypes.CDLL:
                                                 vp, vp, vp, vp, vp]
     lib.resps_controller_step.argtypes = [vp, ctypes.POINTER(RespsPolicy), vp, vp, vp, i64, i32, i32, f32, vp, vp, vp,
                                           vp, vp, vp, vp, vp, vp]
+    lib.resps_scan_rows.argtypes = [vp]
+    lib.resps_scan_rows.restype = i64
+    lib.resps_row_scan_shard.argtypes = [vp, vp, i32, vp, i64, i64, i64, i32, i32, vp, vp, vp, vp]
+    lib.resps_tree_expand_merge.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp,
+                                            vp, vp]
+    lib.resps_target_argmax_shard.argtypes = [vp, vp, i32, vp, i64, i64, vp, vp]
+    lib.resps_verify_accept_merge.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.resps_kv_compact.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp, i32, i64, i64, i64, i64, vp]
     lib.resps_debug_set.argtypes = [vp, i32, i32]
     lib.resps_attention_replan.argtypes = [vp]
     lib.resps_target_argmax_static.argtypes = [vp, i32, i32, i32, vp, i64, i64, vp, vp]
     for name in EXPORTS:
-        if name not in ("resps_strerror", "resps_workspace_bytes"):
+        if name not in ("resps_strerror", "resps_workspace_bytes", "resps_scan_rows"):
             getattr(lib, name).restype = i32
     _lib = lib
     return lib
@@ -255,6 +263,68 @@ def resps_controller_step(ctx: Context, policy: RespsPolicy, hidden_h, hidden_m,
         interval, float(temperature), _ptr(uniform, torch.float64), _ptr(prev_accept_len, i32),
         _ptr(prev_elapsed_s, f32), _ptr(state, i32), _ptr(steps, i32), _ptr(reward_avg, f32), _ptr(logits, f32),
         _ptr(action, i32), _stream(stream)), "resps_controller_step")
+
+
+def resps_row_scan_shard(ctx: Context, steps, batch: int, draft_logits, ld_b: int, ld_level: int, ld_row: int,
+                         n_levels: int, n_slots: int, part_val, part_id, part_lse, stream=None) -> None:
+    _check(load().resps_row_scan_shard(
+        ctx.handle, _ptr(steps, torch.int32), batch, _ptr(draft_logits, torch.float32), ld_b, ld_level, ld_row,
+        n_levels, n_slots, _ptr(part_val, torch.float32), _ptr(part_id, torch.int32), _ptr(part_lse, torch.float64),
+        _stream(stream)), "resps_row_scan_shard")
+
+
+def resps_tree_expand_merge(ctx: Context, steps, batch: int, n_levels: int, n_slots: int, n_shards: int, all_val,
+                            all_id, all_lse, shard_offset, root_token, tokens, parent, depth, position_ids, mask,
+                            retrieve, n_leaves, n_nodes, stream=None) -> None:
+    i32 = torch.int32
+    _check(load().resps_tree_expand_merge(
+        ctx.handle, _ptr(steps, i32), batch, n_levels, n_slots, n_shards, _ptr(all_val, torch.float32),
+        _ptr(all_id, i32), _ptr(all_lse, torch.float64), _ptr(shard_offset, i32), _ptr(root_token, i32),
+        _ptr(tokens, i32), _ptr(parent, i32), _ptr(depth, i32), _ptr(position_ids, i32), _ptr(mask),
+        _ptr(retrieve, i32), _ptr(n_leaves, i32), _ptr(n_nodes, i32), _stream(stream)), "resps_tree_expand_merge")
+
+
+def resps_target_argmax_shard(ctx: Context, n_nodes, batch: int, target_logits, ld_b: int, ld_row: int, part_key,
+                              stream=None) -> None:
+    _check(load().resps_target_argmax_shard(
+        ctx.handle, _ptr(n_nodes, torch.int32), batch, _ptr(target_logits, torch.float32), ld_b, ld_row,
+        _ptr(part_key, torch.int64), _stream(stream)), "resps_target_argmax_shard")
+
+
+def resps_verify_accept_merge(ctx: Context, steps, n_nodes, batch: int, n_shards: int, all_key, shard_offset, tokens,
+                              parent, target_argmax, accept_path, accept_len, out_tokens, steps_next=None,
+                              stream=None) -> None:
+    i32 = torch.int32
+    _check(load().resps_verify_accept_merge(
+        ctx.handle, _ptr(steps, i32), _ptr(n_nodes, i32), batch, n_shards, _ptr(all_key, torch.int64),
+        _ptr(shard_offset, i32), _ptr(tokens, i32), _ptr(parent, i32), _ptr(target_argmax, i32),
+        _ptr(accept_path, i32), _ptr(accept_len, i32), _ptr(out_tokens, i32), _ptr(steps_next, i32),
+        _stream(stream)), "resps_verify_accept_merge")
+
+
+def shard_columns(vocab: int, n_shards: int, multiple: int = 4):
+    """Column ranges [(offset, width)] of a vocabulary cut into n_shards pieces whose widths are multiples
+    of `multiple` (the vectorised kernels want rows that start 16-byte aligned), the last taking the rest."""
+    base = (vocab // n_shards) // multiple * multiple
+    out, off = [], 0
+    for p in range(n_shards):
+        width = base if p < n_shards - 1 else vocab - off
+        out.append((off, width))
+        off += width
+    return out
+
+
+def all_gather_parts(parts, group=None):
+    """All-gather of a rank's partial results (a list of tensors) over the ranks of a torch.distributed
+    group: returns tensors with a leading [world] dimension, the layout the merge calls take."""
+    import torch.distributed as dist
+    world = dist.get_world_size(group)
+    out = []
+    for t in parts:
+        pieces = [torch.empty_like(t) for _ in range(world)]
+        dist.all_gather(pieces, t.contiguous(), group=group)
+        out.append(torch.stack(pieces))
+    return out
 
 
 def resps_kv_compact(ctx: Context, steps, batch: int, accept_path, accept_len, k_cache_ptrs,

@@ -41,6 +41,7 @@ void carve(resps_ctx* c, Carver& cv) {
     const int64_t zero_end = cv.off;  // everything above must start as zero
     (void)zero_end;
     cv.take(w.node_row, nodes);
+    cv.take(w.amax_local, nodes);
     cv.take(w.ctl_h1, static_cast<int64_t>(s.max_batch) * resps::controller_max_hidden());
     cv.take(w.samp_scratch, static_cast<int64_t>(resps::sampled_scratch_doubles(s.max_batch)));
     cv.take(w.part_key, rows * w.scan_splits * s.max_k);
@@ -231,6 +232,114 @@ int resps_tree_expand(resps_ctx* ctx, const resps_step* d_steps, int batch,
     if (resps::launch_tree_build(ctx, d_steps, batch, n_levels, n_slots, d_root_token, d_tokens, d_parent,
                                  d_depth, d_position_ids, d_mask, d_retrieve, d_n_leaves, d_n_nodes,
                                  stream) != cudaSuccess)
+        return RESPS_ERR_CUDA;
+    return RESPS_OK;
+}
+
+// ---- vocabulary sharded over several GPUs -------------------------------------------------------------
+int64_t resps_scan_rows(const resps_ctx* ctx) { return ctx ? ctx->ws.max_rows : 0; }
+
+int resps_row_scan_shard(resps_ctx* ctx, const resps_step* d_steps, int batch, const float* d_draft_logits,
+                         int64_t ld_b, int64_t ld_level, int64_t ld_row, int n_levels, int n_slots,
+                         float* d_part_val, int32_t* d_part_id, double* d_part_lse, resps_stream stream) {
+    RESPS_CHECK_PTR(ctx);
+    RESPS_CHECK_PTR(d_steps);
+    RESPS_CHECK_PTR(d_draft_logits);
+    RESPS_CHECK_PTR(d_part_val);
+    RESPS_CHECK_PTR(d_part_id);
+    RESPS_CHECK_PTR(d_part_lse);
+    if (batch < 1 || n_levels < 1 || n_slots < 1 || ld_row < ctx->shape.vocab || ld_level < 0 || ld_b < 0)
+        return RESPS_ERR_INVALID_ARG;
+    if (batch > ctx->shape.max_batch) return RESPS_ERR_CAPACITY;
+    if (ctx->shape.vocab < ctx->shape.max_k) return RESPS_ERR_UNSUPPORTED_SHAPE;  // a shard holds at least max_k columns
+    if (n_levels > ctx->shape.max_depth) n_levels = ctx->shape.max_depth;
+    if (n_slots > ctx->shape.max_k) n_slots = ctx->shape.max_k;
+    if (resps::launch_row_scan(ctx, d_steps, batch, d_draft_logits, ld_b, ld_level, ld_row, n_levels, n_slots, -1,
+                               stream) != cudaSuccess)
+        return RESPS_ERR_CUDA;
+    const resps::Workspace& w = ctx->ws;
+    const size_t rows = static_cast<size_t>(batch) * w.max_rows;
+    if (cudaMemcpyAsync(d_part_val, w.row_val, rows * ctx->shape.max_k * sizeof(float), cudaMemcpyDeviceToDevice, stream) != cudaSuccess ||
+        cudaMemcpyAsync(d_part_id, w.row_id, rows * ctx->shape.max_k * sizeof(int32_t), cudaMemcpyDeviceToDevice, stream) != cudaSuccess ||
+        cudaMemcpyAsync(d_part_lse, w.row_lse, rows * sizeof(double), cudaMemcpyDeviceToDevice, stream) != cudaSuccess)
+        return RESPS_ERR_CUDA;
+    return RESPS_OK;
+}
+
+int resps_tree_expand_merge(resps_ctx* ctx, const resps_step* d_steps, int batch, int n_levels, int n_slots,
+                            int n_shards, const float* d_all_val, const int32_t* d_all_id, const double* d_all_lse,
+                            const int32_t* d_shard_offset, const int32_t* d_root_token, int32_t* d_tokens,
+                            int32_t* d_parent, int32_t* d_depth, int32_t* d_position_ids, uint64_t* d_mask,
+                            int32_t* d_retrieve, int32_t* d_n_leaves, int32_t* d_n_nodes, resps_stream stream) {
+    RESPS_CHECK_PTR(ctx);
+    RESPS_CHECK_PTR(d_steps);
+    RESPS_CHECK_PTR(d_all_val);
+    RESPS_CHECK_PTR(d_all_id);
+    RESPS_CHECK_PTR(d_all_lse);
+    RESPS_CHECK_PTR(d_shard_offset);
+    RESPS_CHECK_PTR(d_root_token);
+    RESPS_CHECK_PTR(d_tokens);
+    RESPS_CHECK_PTR(d_parent);
+    RESPS_CHECK_PTR(d_depth);
+    RESPS_CHECK_PTR(d_position_ids);
+    RESPS_CHECK_PTR(d_mask);
+    RESPS_CHECK_PTR(d_retrieve);
+    RESPS_CHECK_PTR(d_n_leaves);
+    RESPS_CHECK_PTR(d_n_nodes);
+    if (batch < 1 || n_levels < 1 || n_slots < 1 || n_shards < 1) return RESPS_ERR_INVALID_ARG;
+    if (n_shards > 16) return RESPS_ERR_UNSUPPORTED_SHAPE;
+    if (batch > ctx->shape.max_batch) return RESPS_ERR_CAPACITY;
+    if (n_levels > ctx->shape.max_depth) n_levels = ctx->shape.max_depth;
+    if (n_slots > ctx->shape.max_k) n_slots = ctx->shape.max_k;
+    resps::attention_plan_invalidate(ctx);
+    if (resps::launch_shard_merge_rows(ctx, d_steps, batch, n_levels, n_slots, n_shards, d_all_val, d_all_id, d_all_lse,
+                                       d_shard_offset, stream) != cudaSuccess)
+        return RESPS_ERR_CUDA;
+    if (resps::launch_tree_build(ctx, d_steps, batch, n_levels, n_slots, d_root_token, d_tokens, d_parent, d_depth,
+                                 d_position_ids, d_mask, d_retrieve, d_n_leaves, d_n_nodes, stream) != cudaSuccess)
+        return RESPS_ERR_CUDA;
+    return RESPS_OK;
+}
+
+int resps_target_argmax_shard(resps_ctx* ctx, const int32_t* d_n_nodes, int batch, const float* d_target_logits,
+                              int64_t ld_b, int64_t ld_row, uint64_t* d_part_key, resps_stream stream) {
+    RESPS_CHECK_PTR(ctx);
+    RESPS_CHECK_PTR(d_n_nodes);
+    RESPS_CHECK_PTR(d_target_logits);
+    RESPS_CHECK_PTR(d_part_key);
+    if (batch < 1 || ld_row < ctx->shape.vocab || ld_b < 0) return RESPS_ERR_INVALID_ARG;
+    if (batch > ctx->shape.max_batch) return RESPS_ERR_CAPACITY;
+    if (resps::launch_row_argmax(ctx, d_n_nodes, batch, d_target_logits, ld_b, ld_row, ctx->ws.amax_local, nullptr,
+                                 nullptr, stream, reinterpret_cast<unsigned long long*>(d_part_key)) != cudaSuccess)
+        return RESPS_ERR_CUDA;
+    return RESPS_OK;
+}
+
+int resps_verify_accept_merge(resps_ctx* ctx, const resps_step* d_steps, const int32_t* d_n_nodes, int batch,
+                              int n_shards, const uint64_t* d_all_key, const int32_t* d_shard_offset,
+                              const int32_t* d_tokens, const int32_t* d_parent, int32_t* d_target_argmax,
+                              int32_t* d_accept_path, int32_t* d_accept_len, int32_t* d_out_tokens,
+                              resps_step* d_steps_next, resps_stream stream) {
+    RESPS_CHECK_PTR(ctx);
+    RESPS_CHECK_PTR(d_steps);
+    RESPS_CHECK_PTR(d_n_nodes);
+    RESPS_CHECK_PTR(d_all_key);
+    RESPS_CHECK_PTR(d_shard_offset);
+    RESPS_CHECK_PTR(d_tokens);
+    RESPS_CHECK_PTR(d_parent);
+    RESPS_CHECK_PTR(d_target_argmax);
+    RESPS_CHECK_PTR(d_accept_path);
+    RESPS_CHECK_PTR(d_accept_len);
+    RESPS_CHECK_PTR(d_out_tokens);
+    if (batch < 1 || n_shards < 1) return RESPS_ERR_INVALID_ARG;
+    if (batch > ctx->shape.max_batch) return RESPS_ERR_CAPACITY;
+    if (d_steps_next) resps::attention_plan_invalidate(ctx, d_steps_next);
+    if (resps::launch_shard_merge_argmax(ctx, d_n_nodes, batch, n_shards,
+                                         reinterpret_cast<const unsigned long long*>(d_all_key), d_shard_offset,
+                                         d_target_argmax, stream) != cudaSuccess)
+        return RESPS_ERR_CUDA;
+    if (resps::launch_accept_walk(ctx, d_steps, d_n_nodes, batch, d_tokens, d_parent, d_target_argmax, d_accept_path,
+                                  d_accept_len, d_out_tokens, d_steps_next, stream) != cudaSuccess)
         return RESPS_ERR_CUDA;
     return RESPS_OK;
 }

@@ -1112,47 +1112,55 @@ tree_attention_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_
                 // different lanes).
                 float am[4] = {0.f, 0.f, 0.f, 0.f};
                 float scale = 1.f;  // O = Ohat * l * scale
-                uint32_t orr[32];
-                float f[32];
+                uint32_t r0[32], r1[32];
 #pragma unroll 1
                 for (int pass = 0; pass < 2; ++pass) {
                     const float mul = (pass == 0) ? inv : inv / scale;
                     const bool store = row_ok && (pass == 0 || scale != 1.f);
+                    // Two loads from tensor memory are in flight together: in key mode a piece of this
+                    // lane's O and the same piece of the other lane's, in row mode two pieces of its own.
+                    // (The loads are warp-wide and their conditions warp-uniform.)
+                    const int c_step = row_mode ? 2 : 1;
 #pragma unroll 1
-                    for (int c = c_begin; c < c_end; ++c) {
-                        // (the loads from tensor memory are warp-wide and their conditions warp-uniform)
-                        if (use_self) {
-                            tmem_ld32(o_t + c * 32, orr);
-                            tmem_wait_ld();
+                    for (int c0 = c_begin; c0 < c_end; c0 += c_step) {
+                        const bool second = row_mode && c0 + 1 < c_end;
+                        if (use_self) tmem_ld32(o_t + c0 * 32, r0);
+                        if (use_oth) tmem_ld32(oth_t + c0 * 32, r1);
+                        if (second) tmem_ld32(o_t + (c0 + 1) * 32, r1);
+                        tmem_wait_ld();
 #pragma unroll
-                            for (int e = 0; e < 32; ++e) f[e] = __uint_as_float(orr[e]) * w_self;
-                        } else {
+                        for (int h2 = 0; h2 < 2; ++h2) {
+                            if (h2 == 1 && !second) break;
+                            const int c = c0 + h2;
+                            if (store) {
 #pragma unroll
-                            for (int e = 0; e < 32; ++e) f[e] = 0.f;
-                        }
-                        if (use_oth) {
-                            tmem_ld32(oth_t + c * 32, orr);
-                            tmem_wait_ld();
+                                for (int q4 = 0; q4 < 4; ++q4) {
+                                    float g8[8];
 #pragma unroll
-                            for (int e = 0; e < 32; ++e) f[e] = fmaf(__uint_as_float(orr[e]), w_oth, f[e]);
-                        }
-                        if (store) {
-#pragma unroll
-                            for (int q4 = 0; q4 < 4; ++q4) {
-                                const float* g8 = f + q4 * 8;
-                                uint4 v;
-                                if (direct) {
-                                    v.x = pack_bf16(g8[0] * mul, g8[1] * mul), v.y = pack_bf16(g8[2] * mul, g8[3] * mul);
-                                    v.z = pack_bf16(g8[4] * mul, g8[5] * mul), v.w = pack_bf16(g8[6] * mul, g8[7] * mul);
-                                    *reinterpret_cast<uint4*>(dst + (c * 4 + q4) * 8) = v;
-                                } else {
-                                    am[q4] = max3(am[q4], fabsf(g8[0]), fabsf(g8[1]));
-                                    am[q4] = max3(am[q4], fabsf(g8[2]), fabsf(g8[3]));
-                                    am[q4] = max3(am[q4], fabsf(g8[4]), fabsf(g8[5]));
-                                    am[q4] = max3(am[q4], fabsf(g8[6]), fabsf(g8[7]));
-                                    v.x = pack_half2(g8[0] * mul, g8[1] * mul), v.y = pack_half2(g8[2] * mul, g8[3] * mul);
-                                    v.z = pack_half2(g8[4] * mul, g8[5] * mul), v.w = pack_half2(g8[6] * mul, g8[7] * mul);
-                                    __stcg(po + (c * 4 + q4) * kBM, v);
+                                    for (int e = 0; e < 8; ++e) {
+                                        float v;
+                                        if (h2 == 1) {
+                                            v = __uint_as_float(r1[q4 * 8 + e]);
+                                        } else {
+                                            v = use_self ? __uint_as_float(r0[q4 * 8 + e]) * w_self : 0.f;
+                                            if (use_oth) v = fmaf(__uint_as_float(r1[q4 * 8 + e]), w_oth, v);
+                                        }
+                                        g8[e] = v;
+                                    }
+                                    uint4 v;
+                                    if (direct) {
+                                        v.x = pack_bf16(g8[0] * mul, g8[1] * mul), v.y = pack_bf16(g8[2] * mul, g8[3] * mul);
+                                        v.z = pack_bf16(g8[4] * mul, g8[5] * mul), v.w = pack_bf16(g8[6] * mul, g8[7] * mul);
+                                        *reinterpret_cast<uint4*>(dst + (c * 4 + q4) * 8) = v;
+                                    } else {
+                                        am[q4] = max3(am[q4], fabsf(g8[0]), fabsf(g8[1]));
+                                        am[q4] = max3(am[q4], fabsf(g8[2]), fabsf(g8[3]));
+                                        am[q4] = max3(am[q4], fabsf(g8[4]), fabsf(g8[5]));
+                                        am[q4] = max3(am[q4], fabsf(g8[6]), fabsf(g8[7]));
+                                        v.x = pack_half2(g8[0] * mul, g8[1] * mul), v.y = pack_half2(g8[2] * mul, g8[3] * mul);
+                                        v.z = pack_half2(g8[4] * mul, g8[5] * mul), v.w = pack_half2(g8[6] * mul, g8[7] * mul);
+                                        __stcg(po + (c * 4 + q4) * kBM, v);
+                                    }
                                 }
                             }
                         }

@@ -37,6 +37,7 @@ struct Workspace {
     double* row_lse = nullptr;               // [max_batch][max_rows]
     unsigned long long* amax_part = nullptr; // [max_batch][max_tt][splits]
     unsigned int* amax_counter = nullptr;    // [max_batch][max_tt]
+    int32_t* amax_local = nullptr;           // [max_batch][max_tt] shard-local arg-max ids (vocabulary sharding)
     int32_t* node_row = nullptr;             // [max_batch][max_tt] draft row behind every node's children (tree build)
     float* ctl_h1 = nullptr;                 // controller: first hidden layer [max_batch][256]
     unsigned int* ctl_counter = nullptr;     // controller: hidden units done per sequence (self-resetting)
@@ -106,7 +107,14 @@ cudaError_t launch_tree_build(const resps_ctx* ctx, const resps_step* d_steps, i
 // acceptance walk runs in the same kernel (returns true through `walked`).
 cudaError_t launch_row_argmax(const resps_ctx* ctx, const int32_t* d_n_nodes, int batch,
                               const float* logits, int64_t ld_b, int64_t ld_row, int32_t* argmax_out,
-                              const AcceptArgs* walk, bool* walked, cudaStream_t st);
+                              const AcceptArgs* walk, bool* walked, cudaStream_t st,
+                              unsigned long long* key_out = nullptr);
+cudaError_t launch_shard_merge_rows(const resps_ctx* ctx, const resps_step* d_steps, int batch, int n_levels, int n_slots,
+                                    int n_shards, const float* all_val, const int32_t* all_id, const double* all_lse,
+                                    const int32_t* shard_offset, cudaStream_t st);
+cudaError_t launch_shard_merge_argmax(const resps_ctx* ctx, const int32_t* d_n_nodes, int batch, int n_shards,
+                                      const unsigned long long* all_key, const int32_t* shard_offset, int32_t* out,
+                                      cudaStream_t st);
 AcceptArgs make_accept_args(const resps_ctx* ctx, const resps_step* d_steps, const int32_t* d_n_nodes,
                             const int32_t* tokens, const int32_t* parent, const int32_t* target_argmax,
                             int32_t* accept_path, int32_t* accept_len, int32_t* out_tokens, resps_step* steps_next);

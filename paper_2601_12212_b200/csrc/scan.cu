@@ -596,6 +596,7 @@ struct ArgmaxArgs {
     unsigned int* counter;
     unsigned int* seq_counter;  // streaming kernel: rows of a sequence that are final
     int32_t* out;
+    unsigned long long* key_out;  // optional [batch][max_tt]: the packed (value, id) of every row's arg-max
     int32_t* status;            // streaming kernel: where a wait that ran out is flagged (may be null)
 };
 
@@ -714,6 +715,7 @@ __global__ void __launch_bounds__(kStreamThreads, 2) row_argmax_stream_kernel(co
         int seq_done = 0;
         if (row_done) {
             a.out[prow] = key_id(best);
+            if (a.key_out) a.key_out[prow] = best;
             if (do_walk) {
                 __threadfence();
                 seq_done = (atomicAdd(a.seq_counter + b, 1u) == static_cast<unsigned>(n - 1));
@@ -788,6 +790,7 @@ __global__ void __launch_bounds__(kScanThreads, 4) row_argmax_kernel(const Argma
         for (int w = 1; w < kScanThreads / 32; ++w) key = (s_k[w] > key) ? s_k[w] : key;
         if (a.splits == 1) {
             a.out[prow] = key_id(key);
+            if (a.key_out) a.key_out[prow] = key;
             s_last = false;
         } else {
             a.part[prow * a.splits + sp] = key;
@@ -810,8 +813,85 @@ __global__ void __launch_bounds__(kScanThreads, 4) row_argmax_kernel(const Argma
     }
     if (lane == 0) {
         a.out[prow] = key_id(m);
+        if (a.key_out) a.key_out[prow] = m;
         a.counter[prow] = 0u;
     }
+}
+
+// ---------------------------------------------------------------------------------------
+// Vocabulary sharded over several GPUs: every rank scans its own columns of every row with the
+// kernels above (its context is created with its shard's width), the ranks exchange what they
+// found -- k (value, id) pairs and one log-sum-exp per draft row, one (value, id) per target row --
+// and every rank merges the shards' results with these two kernels.  Ids become global by the
+// shard's first column; the order (value descending, id ascending) is the method's.
+// ---------------------------------------------------------------------------------------
+struct ShardMergeArgs {
+    const resps_step* steps;
+    int n_levels, n_slots, vocab, max_tt, max_k, max_rows, n_shards, batch;
+    const float* all_val;      // [n_shards][batch][max_rows][max_k]
+    const int32_t* all_id;
+    const double* all_lse;     // [n_shards][batch][max_rows]
+    const int32_t* shard_offset;  // [n_shards]
+    float* row_val;
+    int32_t* row_id;
+    double* row_lse;
+};
+
+__global__ void __launch_bounds__(128) shard_merge_rows_kernel(const ShardMergeArgs a) {
+    pdl_wait();  // the kernel before this one in the stream has completed
+    pdl_launch_dependents();
+    __shared__ unsigned long long s_keys[16 * RESPS_MAX_K];
+    const int b = blockIdx.y, r = blockIdx.x, tid = threadIdx.x;
+    const StepDims sd = clamp_step(a.steps[b], a.n_levels, a.n_slots, a.max_tt, a.max_k, a.vocab);
+    const int k = sd.k;
+    if (r >= 1 + (sd.d - 1) * k) return;
+    const int64_t prow = static_cast<int64_t>(b) * a.max_rows + r;
+    const int n = a.n_shards * k;
+    for (int i = tid; i < n; i += blockDim.x) {
+        const int p = i / k, q = i - p * k;
+        const int64_t src = (static_cast<int64_t>(p) * a.batch * a.max_rows + prow) * a.max_k + q;
+        s_keys[i] = pack_val_id(a.all_val[src], a.all_id[src] + a.shard_offset[p]);
+    }
+    __syncthreads();
+    for (int c = tid; c < n; c += blockDim.x) {
+        const unsigned long long mine = s_keys[c];
+        int rank = 0;
+        for (int j = 0; j < n; ++j) rank += (s_keys[j] > mine) || (s_keys[j] == mine && j < c);
+        if (rank < k) {
+            a.row_val[prow * a.max_k + rank] = key_val(mine);
+            a.row_id[prow * a.max_k + rank] = key_id(mine);
+        }
+    }
+    if (tid == 0) {  // log of the sum over the shards of exp(shard's log-sum-exp), fp64
+        double m = -INFINITY;
+        for (int p = 0; p < a.n_shards; ++p) m = fmax(m, a.all_lse[static_cast<int64_t>(p) * a.batch * a.max_rows + prow]);
+        double sum = 0.0;
+        for (int p = 0; p < a.n_shards; ++p) sum += exp(a.all_lse[static_cast<int64_t>(p) * a.batch * a.max_rows + prow] - m);
+        a.row_lse[prow] = m + log(sum);
+    }
+}
+
+struct ShardArgmaxArgs {
+    const int32_t* n_nodes;
+    int max_tt, n_shards, batch;
+    const unsigned long long* all_key;  // [n_shards][batch][max_tt] packed (value, local id)
+    const int32_t* shard_offset;
+    int32_t* out;
+};
+
+__global__ void __launch_bounds__(RESPS_MAX_TT) shard_merge_argmax_kernel(const ShardArgmaxArgs a) {
+    pdl_wait();  // the kernel before this one in the stream has completed
+    pdl_launch_dependents();
+    const int b = blockIdx.x, i = threadIdx.x;
+    const int n = min(max(a.n_nodes[b], 0), a.max_tt);
+    if (i >= n) return;
+    unsigned long long best = 0ull;
+    for (int p = 0; p < a.n_shards; ++p) {
+        const unsigned long long key = a.all_key[(static_cast<int64_t>(p) * a.batch + b) * a.max_tt + i];
+        const unsigned long long global = pack_val_id(key_val(key), key_id(key) + a.shard_offset[p]);
+        best = global > best ? global : best;
+    }
+    a.out[static_cast<int64_t>(b) * a.max_tt + i] = key_id(best);
 }
 
 inline bool vec_ok(const void* p, int64_t s0, int64_t s1, int64_t s2, int vocab, int chunk) {
@@ -875,7 +955,7 @@ cudaError_t launch_row_scan(const resps_ctx* ctx, const resps_step* d_steps, int
 
 cudaError_t launch_row_argmax(const resps_ctx* ctx, const int32_t* d_n_nodes, int batch,
                               const float* logits, int64_t ld_b, int64_t ld_row, int32_t* argmax_out,
-                              const AcceptArgs* walk, bool* walked, cudaStream_t st) {
+                              const AcceptArgs* walk, bool* walked, cudaStream_t st, unsigned long long* key_out) {
     const Workspace& w = ctx->ws;
     ArgmaxArgs a;
     a.n_nodes = d_n_nodes;
@@ -885,6 +965,7 @@ cudaError_t launch_row_argmax(const resps_ctx* ctx, const int32_t* d_n_nodes, in
     a.chunk = w.scan_chunk, a.splits = w.scan_splits;
     a.slices = w.scan_splits, a.cps = 1;
     a.part = w.amax_part, a.counter = w.amax_counter, a.seq_counter = w.amax_seq_counter, a.out = argmax_out;
+    a.key_out = key_out;
     a.status = w.status;
     if (walked) *walked = false;
     if (vec_ok(logits, ld_b, ld_row, 0, a.vocab, a.chunk) && w.scan_chunk == kScanChunkMax) {
@@ -906,6 +987,30 @@ cudaError_t launch_row_argmax(const resps_ctx* ctx, const int32_t* d_n_nodes, in
     else
         return launch_pdl(row_argmax_kernel<false>, grid, dim3(kScanThreads), 0, st, a);
     return cudaGetLastError();
+}
+
+cudaError_t launch_shard_merge_rows(const resps_ctx* ctx, const resps_step* d_steps, int batch, int n_levels, int n_slots,
+                                    int n_shards, const float* all_val, const int32_t* all_id, const double* all_lse,
+                                    const int32_t* shard_offset, cudaStream_t st) {
+    const Workspace& w = ctx->ws;
+    ShardMergeArgs a;
+    a.steps = d_steps, a.n_levels = n_levels, a.n_slots = n_slots;
+    a.vocab = ctx->shape.vocab, a.max_tt = ctx->shape.max_tt, a.max_k = ctx->shape.max_k, a.max_rows = w.max_rows;
+    a.n_shards = n_shards, a.batch = batch;
+    a.all_val = all_val, a.all_id = all_id, a.all_lse = all_lse, a.shard_offset = shard_offset;
+    a.row_val = w.row_val, a.row_id = w.row_id, a.row_lse = w.row_lse;
+    const int k_ext = min(n_slots, ctx->shape.max_k);
+    const int rows = (n_levels > 1) ? 1 + (n_levels - 1) * k_ext : 1;
+    return launch_pdl(shard_merge_rows_kernel, dim3(rows, batch), dim3(128), 0, st, a);
+}
+
+cudaError_t launch_shard_merge_argmax(const resps_ctx* ctx, const int32_t* d_n_nodes, int batch, int n_shards,
+                                      const unsigned long long* all_key, const int32_t* shard_offset, int32_t* out,
+                                      cudaStream_t st) {
+    ShardArgmaxArgs a;
+    a.n_nodes = d_n_nodes, a.max_tt = ctx->shape.max_tt, a.n_shards = n_shards, a.batch = batch;
+    a.all_key = all_key, a.shard_offset = shard_offset, a.out = out;
+    return launch_pdl(shard_merge_argmax_kernel, dim3(batch), dim3(RESPS_MAX_TT), 0, st, a);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -965,7 +1070,7 @@ extern "C" int resps_target_argmax_static(const int32_t* d_n_nodes, int batch, i
     a.logits = d_target_logits;
     a.ld_b = ld_b, a.ld_row = ld_row;
     a.vocab = vocab, a.max_tt = max_tt, a.chunk = chunk, a.splits = splits;
-    a.slices = splits, a.cps = 1, a.seq_counter = nullptr, a.status = nullptr;
+    a.slices = splits, a.cps = 1, a.seq_counter = nullptr, a.status = nullptr, a.key_out = nullptr;
     a.part = reinterpret_cast<unsigned long long*>(scratch);
     a.counter = reinterpret_cast<unsigned int*>(scratch + kStaticPartBytes);
     a.out = d_target_argmax;

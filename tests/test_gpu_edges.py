@@ -411,3 +411,43 @@ def test_host_side_errors():
     assert e.value.code == binding.RESPS_ERR_INVALID_ARG
     assert ctx.workspace_bytes() > 0
     ctx.close()
+
+
+def test_attention_shards_by_kv_head_without_any_exchange():
+    """Attention is independent per KV head: two "ranks", each with a context for its own half of the
+    heads and its own slices of Q and of the caches, produce the halves of the full result (checked
+    against the oracle on the full problem).  Nothing has to cross between them."""
+    oracle, binding, synth = _imports()
+    from harness import check_attention, u16_to_bf16_cuda, bf16_to_f64
+    rng = np.random.default_rng(21)
+    n, Hq, Hkv, D, L, cap, T = 50, 16, 4, 128, 1500, 1700, 64
+    q = synth.to_bf16_bits(rng.normal(size=(1, T, Hq, D)).astype(np.float32).ravel()).reshape(1, T, Hq, D)
+    kc = synth.to_bf16_bits(rng.normal(size=(1, Hkv, cap, D)).astype(np.float32).ravel()).reshape(1, Hkv, cap, D)
+    vc = synth.to_bf16_bits(rng.normal(size=(1, Hkv, cap, D)).astype(np.float32).ravel()).reshape(1, Hkv, cap, D)
+    masks = np.zeros((1, T, 2), np.uint64)
+    parent = [-1] + [int(rng.integers(max(0, i - 6), i)) for i in range(1, n)]
+    for i in range(n):
+        v, c = 0, i
+        while c >= 0:
+            v |= 1 << c
+            c = parent[c]
+        masks[0, i, 0] = v
+    steps = torch.tensor([[n, 1, 1, L]], dtype=torch.int32, device="cuda")
+    nn = torch.tensor([n], dtype=torch.int32, device="cuda")
+    dm = torch.from_numpy(masks.view(np.int64)).cuda()
+    ref = oracle.tree_attention(q[0, :n], kc[0], vc[0], L, masks[0, :n], 1 / np.sqrt(D))
+    out = np.zeros((n, Hq, D))
+    ranks = 2
+    hq, hkv = Hq // ranks, Hkv // ranks
+    for rank in range(ranks):
+        ctx = binding.Context(hq, hkv, D, 1000, max_batch=1, max_tt=T, max_k=4, max_depth=4)
+        dq = u16_to_bf16_cuda(np.ascontiguousarray(q[:, :, rank * hq:(rank + 1) * hq]))
+        dk = u16_to_bf16_cuda(np.ascontiguousarray(kc[:, rank * hkv:(rank + 1) * hkv]))
+        dv = u16_to_bf16_cuda(np.ascontiguousarray(vc[:, rank * hkv:(rank + 1) * hkv]))
+        do = torch.zeros_like(dq)
+        binding.resps_tree_attention(ctx, steps, nn, 1, dq, do, None, dk, dv, hkv * cap * D, cap * D, D, cap, dm,
+                                     1 / np.sqrt(D))
+        assert ctx.status() == 0
+        out[:, rank * hq:(rank + 1) * hq] = bf16_to_f64(do)[0, :n]
+        ctx.close()
+    check_attention(out, ref)

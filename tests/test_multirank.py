@@ -48,3 +48,35 @@ def test_two_gloo_ranks_report_the_slowest_rank_and_the_whole_job_value():
     assert bench.whole_job_value(110.0, 2) == 55.0
     assert bench.whole_job_value(110.0, 1) == 110.0
     assert bench.max_over_ranks([3.0, 4.0], 1, "cpu") == [3.0, 4.0]
+
+
+def _gather_main(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    from paper_2601_12212_b200 import binding
+    cols = binding.shard_columns(128256, world)
+    # what a rank would hand to the merge calls after scanning its columns: small per-row arrays
+    val = torch.full((2, 5, 3), float(rank))
+    ids = torch.full((2, 5, 3), rank, dtype=torch.int32)
+    all_val, all_id = binding.all_gather_parts([val, ids])
+    out.put((rank, cols, tuple(all_val.shape), all_val[:, 0, 0, 0].tolist(), all_id[:, 1, 2, 1].tolist()))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_two_gloo_ranks_gather_their_vocabulary_shards():
+    """The exchange step of the vocabulary-sharded path: every rank ends up with every rank's partial rows,
+    stacked in rank order, and the ranks agree on the column ranges."""
+    world, port = 2, 31000 + os.getpid() % 2000
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    procs = [ctx.Process(target=_gather_main, args=(r, world, port, out)) for r in range(world)]
+    for p in procs:
+        p.start()
+    res = sorted(out.get(timeout=120) for _ in range(world))
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    for rank, cols, shape, vals, ids in res:
+        assert cols == [(0, 64128), (64128, 64128)]
+        assert shape == (2, 2, 5, 3) and vals == [0.0, 1.0] and ids == [0, 1]
