@@ -604,7 +604,7 @@ def run_ours(args, w):
              tensor_peak_tflops=tensor_peak),
         hbm_entry("row_scan_stream_kernel + tree_build_kernel (one resps_tree_expand call)", phase_bytes["scan"],
                   phases["expand_us"], "one call between two events after an L2 flush, mean over the pool"),
-        hbm_entry("row_argmax_kernel + accept_walk_kernel (one resps_verify_accept call)", phase_bytes["argmax"],
+        hbm_entry("row_argmax_stream_kernel with the acceptance walk in its tail (one resps_verify_accept call)", phase_bytes["argmax"],
                   phases["verify_us"], "one call between two events after an L2 flush, mean over the pool"),
     ]
 
