@@ -573,6 +573,22 @@ def run_ours(args, w):
                                              for i in range(pool)]))
         phase_bytes["argmax"] = float(np.mean([sum(dw.nodes[i]) * V * 4 for i in range(pool)]))
 
+        if args.step_log and rank == 0:
+            # untimed extra pass: every step between its own pair of events, one JSON line per step
+            dw.reset_prefix()
+            torch.cuda.synchronize()
+            pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+            for i, (a, b) in enumerate(pairs):
+                a.record(stream)
+                graphs[(W + i) % pool].replay()
+                b.record(stream)
+            torch.cuda.synchronize()
+            with open(args.step_log, "w") as f:
+                for i, (a, b) in enumerate(pairs):
+                    e = (W + i) % pool
+                    f.write(json.dumps({"step": i, "us": a.elapsed_time(b) * 1e3, "pool_entry": e,
+                                        "tt_d_k": [list(p) for p in dw.params[e]], "n_nodes": list(dw.nodes[e])}) + "\n")
+
     t_step, t_attn, t_e2e = max_over_ranks([t_step, t_attn, t_e2e], world, "cuda")
     status = dw.ctx.status()
     if rank != 0:
@@ -674,6 +690,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--config", type=int, default=2, help="1-based index of the synthetic workload (synth.WORKLOADS)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--step-log", default=None, metavar="FILE",
+                    help="also write one JSON line per step (device time, step parameters, tree sizes) from an "
+                         "untimed extra pass")
     args = ap.parse_args()
     w = synth.WORKLOADS[args.config]
     world = int(os.environ.get("WORLD_SIZE", "1"))

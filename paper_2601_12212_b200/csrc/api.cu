@@ -4,6 +4,8 @@
 #include <cstring>
 #include <new>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "common.cuh"
 
 namespace resps {
@@ -14,6 +16,16 @@ int attention_max_batch();
 }  // namespace resps
 
 namespace {
+
+// A named range around the host side of an entry point (visible in a timeline tool when one is
+// attached, free otherwise).  The names carry the component of the paper's time breakdown
+// (Appendix C, Table 8) the call belongs to.
+struct Range {
+    explicit Range(const char* name) { nvtxRangePushA(name); }
+    ~Range() { nvtxRangePop(); }
+    Range(const Range&) = delete;
+    Range& operator=(const Range&) = delete;
+};
 
 inline int64_t align_up(int64_t x, int64_t a) { return (x + a - 1) / a * a; }
 
@@ -208,6 +220,7 @@ int resps_tree_expand(resps_ctx* ctx, const resps_step* d_steps, int batch,
                       int32_t* d_tokens, int32_t* d_parent, int32_t* d_depth,
                       int32_t* d_position_ids, uint64_t* d_mask, int32_t* d_retrieve,
                       int32_t* d_n_leaves, int32_t* d_n_nodes, resps_stream stream) {
+    Range range("resps_tree_expand [tree_construction]");
     RESPS_CHECK_PTR(ctx);
     RESPS_CHECK_PTR(d_steps);
     RESPS_CHECK_PTR(d_draft_logits);
@@ -242,6 +255,7 @@ int64_t resps_scan_rows(const resps_ctx* ctx) { return ctx ? ctx->ws.max_rows : 
 int resps_row_scan_shard(resps_ctx* ctx, const resps_step* d_steps, int batch, const float* d_draft_logits,
                          int64_t ld_b, int64_t ld_level, int64_t ld_row, int n_levels, int n_slots,
                          float* d_part_val, int32_t* d_part_id, double* d_part_lse, resps_stream stream) {
+    Range range("resps_row_scan_shard [tree_construction]");
     RESPS_CHECK_PTR(ctx);
     RESPS_CHECK_PTR(d_steps);
     RESPS_CHECK_PTR(d_draft_logits);
@@ -271,6 +285,7 @@ int resps_tree_expand_merge(resps_ctx* ctx, const resps_step* d_steps, int batch
                             const int32_t* d_shard_offset, const int32_t* d_root_token, int32_t* d_tokens,
                             int32_t* d_parent, int32_t* d_depth, int32_t* d_position_ids, uint64_t* d_mask,
                             int32_t* d_retrieve, int32_t* d_n_leaves, int32_t* d_n_nodes, resps_stream stream) {
+    Range range("resps_tree_expand_merge [tree_construction]");
     RESPS_CHECK_PTR(ctx);
     RESPS_CHECK_PTR(d_steps);
     RESPS_CHECK_PTR(d_all_val);
@@ -303,6 +318,7 @@ int resps_tree_expand_merge(resps_ctx* ctx, const resps_step* d_steps, int batch
 
 int resps_target_argmax_shard(resps_ctx* ctx, const int32_t* d_n_nodes, int batch, const float* d_target_logits,
                               int64_t ld_b, int64_t ld_row, uint64_t* d_part_key, resps_stream stream) {
+    Range range("resps_target_argmax_shard [verification_process]");
     RESPS_CHECK_PTR(ctx);
     RESPS_CHECK_PTR(d_n_nodes);
     RESPS_CHECK_PTR(d_target_logits);
@@ -320,6 +336,7 @@ int resps_verify_accept_merge(resps_ctx* ctx, const resps_step* d_steps, const i
                               const int32_t* d_tokens, const int32_t* d_parent, int32_t* d_target_argmax,
                               int32_t* d_accept_path, int32_t* d_accept_len, int32_t* d_out_tokens,
                               resps_step* d_steps_next, resps_stream stream) {
+    Range range("resps_verify_accept_merge [verification_process]");
     RESPS_CHECK_PTR(ctx);
     RESPS_CHECK_PTR(d_steps);
     RESPS_CHECK_PTR(d_n_nodes);
@@ -346,6 +363,7 @@ int resps_verify_accept_merge(resps_ctx* ctx, const resps_step* d_steps, const i
 
 // ---- level form of the tree expansion --------------------------------------------------------------
 int resps_tree_expand_begin(resps_ctx* ctx, const resps_step* d_steps, int batch, int n_slots) {
+    Range range("resps_tree_expand_begin [tree_initialization]");
     RESPS_CHECK_PTR(ctx);
     RESPS_CHECK_PTR(d_steps);
     if (batch < 1 || n_slots < 1) return RESPS_ERR_INVALID_ARG;
@@ -361,6 +379,7 @@ int resps_tree_expand_level(resps_ctx* ctx, const resps_step* d_steps, int batch
                             int32_t* d_frontier_tokens, int32_t* d_frontier_parent_slot,
                             int32_t* d_frontier_position_ids, int32_t* d_frontier_node_index,
                             uint64_t* d_frontier_mask, double* d_frontier_score, resps_stream stream) {
+    Range range("resps_tree_expand_level [drafting_process]");
     RESPS_CHECK_PTR(ctx);
     RESPS_CHECK_PTR(d_steps);
     RESPS_CHECK_PTR(d_level_logits);
@@ -388,6 +407,7 @@ int resps_tree_expand_finish(resps_ctx* ctx, const resps_step* d_steps, int batc
                              int32_t* d_tokens, int32_t* d_parent, int32_t* d_depth, int32_t* d_position_ids,
                              uint64_t* d_mask, int32_t* d_retrieve, int32_t* d_n_leaves, int32_t* d_n_nodes,
                              resps_stream stream) {
+    Range range("resps_tree_expand_finish [tree_construction]");
     RESPS_CHECK_PTR(ctx);
     RESPS_CHECK_PTR(d_steps);
     RESPS_CHECK_PTR(d_root_token);
@@ -416,6 +436,7 @@ int resps_tree_attention(resps_ctx* ctx, const resps_step* d_steps, const int32_
                          const void* d_k_cache, const void* d_v_cache, int64_t kv_stride_seq,
                          int64_t kv_stride_head, int64_t kv_stride_tok, int64_t kv_capacity,
                          const uint64_t* d_mask, float softmax_scale, resps_stream stream) {
+    Range range("resps_tree_attention [target forward: tree attention]");
     RESPS_CHECK_PTR(ctx);
     RESPS_CHECK_PTR(d_steps);
     RESPS_CHECK_PTR(d_n_nodes);
@@ -446,6 +467,7 @@ int resps_verify_accept(resps_ctx* ctx, const resps_step* d_steps, const int32_t
                         const int32_t* d_tokens, const int32_t* d_parent,
                         int32_t* d_target_argmax, int32_t* d_accept_path, int32_t* d_accept_len,
                         int32_t* d_out_tokens, resps_step* d_steps_next, resps_stream stream) {
+    Range range("resps_verify_accept [verification_process]");
     RESPS_CHECK_PTR(ctx);
     RESPS_CHECK_PTR(d_steps);
     RESPS_CHECK_PTR(d_n_nodes);
@@ -481,6 +503,7 @@ int resps_verify_accept_sampled(resps_ctx* ctx, const resps_step* d_steps, const
                                 const int32_t* d_parent, const double* d_u_accept, const double* d_u_sample,
                                 int32_t* d_accept_path, int32_t* d_accept_len, int32_t* d_out_tokens,
                                 resps_step* d_steps_next, resps_stream stream) {
+    Range range("resps_verify_accept_sampled [verification_process]");
     RESPS_CHECK_PTR(ctx);
     RESPS_CHECK_PTR(d_steps);
     RESPS_CHECK_PTR(d_n_nodes);
@@ -512,6 +535,7 @@ int resps_controller_step(resps_ctx* ctx, const resps_policy* policy, const void
                           const int32_t* d_prev_accept_len, const float* d_prev_elapsed_s,
                           resps_controller_state* d_state, resps_step* d_steps, float* d_reward_avg,
                           float* d_logits, int32_t* d_action, resps_stream stream) {
+    Range range("resps_controller_step [rl_policy]");
     RESPS_CHECK_PTR(ctx);
     RESPS_CHECK_PTR(policy);
     RESPS_CHECK_PTR(d_hidden_h);
@@ -547,6 +571,7 @@ int resps_kv_compact(resps_ctx* ctx, const resps_step* d_steps, int steps_advanc
                      void* const* d_k_caches, void* const* d_v_caches, int n_layers,
                      int64_t kv_stride_seq, int64_t kv_stride_head, int64_t kv_stride_tok,
                      int64_t kv_capacity, resps_stream stream) {
+    Range range("resps_kv_compact [input_update]");
     RESPS_CHECK_PTR(ctx);
     RESPS_CHECK_PTR(d_steps);
     RESPS_CHECK_PTR(d_accept_path);

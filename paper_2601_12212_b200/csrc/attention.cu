@@ -1368,18 +1368,20 @@ template <int D>
 __global__ void __launch_bounds__(kCombineThreads) attention_combine_small_kernel(const AttnArgs a) {
     __shared__ Sched sc;
     pdl_launch_dependents();
-    // A CTA past the last row of the largest tree has nothing to do.  It learns that from one
-    // load and leaves: it may have started only after the attention kernel ended, and whatever it
-    // does until it exits delays the next kernel in the stream.
-    {
-        const int b = threadIdx.x;  // the batch is at most the CTA's thread count
-        const bool mine = b < a.batch && static_cast<long long>(blockIdx.x) * kCombineThreads <
-                                             1ll * min(max(a.n_nodes[b], 0), a.max_tt) * a.Hq * (D / 8);
-        if (!__syncthreads_or(mine)) return;
-    }
     // The work list is fetched, and the thread's first piece of work located, before the wait
-    // for the attention kernel: all of this runs while that kernel drains.
+    // for the attention kernel: all of this runs while that kernel drains, in one round trip to
+    // memory (the list carries the tree sizes it was planned for, which the attention kernel has
+    // checked against the live ones).
     load_sched(a, sc, threadIdx.x, kCombineThreads);  // ends with __syncthreads()
+    // A CTA past the last row of the largest tree has nothing to do and leaves: it may have started
+    // only after the attention kernel ended, and whatever it does until it exits delays the next
+    // kernel in the stream.
+    {
+        bool mine = false;
+        for (int b = 0; b < a.batch; ++b)
+            mine = mine || static_cast<long long>(blockIdx.x) * kCombineThreads < 1ll * sc.n[b] * a.Hq * (D / 8);
+        if (!mine) return;
+    }
     const unsigned G = static_cast<unsigned>(a.Hq / a.Hkv);
     const unsigned stride = gridDim.x * kCombineThreads;
     const unsigned group_rows = static_cast<unsigned>(sc.group_rows);
@@ -1498,24 +1500,19 @@ __global__ void __launch_bounds__(kCombineThreads, 4) attention_combine_flat_ker
     __shared__ unsigned s_work0[kMaxBatchSmem + 1];  // first flat index of a sequence
     __shared__ unsigned char s_shares[kMaxBatchSmem];
     pdl_launch_dependents();
-    // A CTA past the last piece of work that the trees at hand could need has nothing to do.  It
-    // learns that from one load and leaves: it may have started only after the attention kernel
-    // ended, and whatever it does until it exits delays the next kernel in the stream.
-    {
-        const int b = threadIdx.x;  // the batch is at most the CTA's thread count
-        unsigned long long bound = 0;
-        if (b < a.batch) bound = 4ull * min(max(a.n_nodes[b], 0), a.max_tt) * a.Hq * (D / 8) + 4;
-        // (sum over the CTA's threads: every sequence's bound, four shares each)
-        __shared__ unsigned long long s_bound;
-        if (threadIdx.x == 0) s_bound = 0;
-        __syncthreads();
-        if (bound) atomicAdd(&s_bound, bound);
-        __syncthreads();
-        if (static_cast<unsigned long long>(blockIdx.x) * kCombineThreads >= s_bound) return;
-    }
     // The work list is fetched, and the thread's first piece of work located, before the wait
-    // for the attention kernel: all of this runs while that kernel drains.
+    // for the attention kernel: all of this runs while that kernel drains, in one round trip to
+    // memory (the list carries the tree sizes it was planned for, which the attention kernel has
+    // checked against the live ones).
     load_sched(a, sc, threadIdx.x, kCombineThreads);  // ends with __syncthreads()
+    // A CTA past the last piece of work that the trees at hand could need (four shares each) has
+    // nothing to do and leaves: it may have started only after the attention kernel ended, and
+    // whatever it does until it exits delays the next kernel in the stream.
+    {
+        unsigned long long bound = 0;
+        for (int b = 0; b < a.batch; ++b) bound += 4ull * sc.n[b] * a.Hq * (D / 8) + 4;
+        if (static_cast<unsigned long long>(blockIdx.x) * kCombineThreads >= bound) return;
+    }
     const unsigned G = static_cast<unsigned>(a.Hq / a.Hkv);
     const unsigned group_rows = static_cast<unsigned>(sc.group_rows);
     if (threadIdx.x < 32) {
