@@ -19,8 +19,8 @@ __global__ void __launch_bounds__(RESPS_MAX_TT) accept_walk_kernel(const AcceptA
     pdl_wait();  // the kernel before this one in the stream has completed
     pdl_launch_dependents();
     __shared__ int s_tgt[RESPS_MAX_TT];
-    __shared__ int s_next;
-    accept_walk_device(a, blockIdx.x, threadIdx.x, s_tgt, &s_next, [] { __syncthreads(); });
+    __shared__ int s_next[RESPS_MAX_DEPTH];
+    accept_walk_device(a, blockIdx.x, threadIdx.x, s_tgt, s_next, false, [] { __syncthreads(); });
 }
 
 struct CompactArgs {

@@ -42,7 +42,7 @@ struct Workspace {
     float* ctl_h1 = nullptr;                 // controller: first hidden layer [max_batch][256]
     unsigned int* ctl_counter = nullptr;     // controller: hidden units done per sequence (self-resetting)
     double* samp_scratch = nullptr;          // acceptance under sampling: a few words per sequence
-    unsigned int* amax_seq_counter = nullptr;  // [max_batch] rows of a sequence whose arg-max is final (self-resetting)
+    unsigned int* amax_seq_counter = nullptr;  // [max_batch] arg-max CTAs of a sequence that have delivered (self-resetting)
     // attention
     int attn_grid = 0;          // persistent CTAs (one per SM)
     int attn_combine_flat_grid = 0;  // ... of its variant for batches
@@ -210,43 +210,47 @@ __device__ __forceinline__ float ex2_approx(float x) {
 // accepted tokens"): from the root, follow the child whose token equals the target's arg-max at the
 // current node until no child matches.  Run by `nthreads` >= RESPS_MAX_TT threads of one CTA for
 // sequence b (thread c owns tree node c); `sync` is a barrier over exactly those threads.
+// `s_tgt` [RESPS_MAX_TT] receives the targets' arg-max (the caller has filled it already when
+// `have_targets`), `s_next` [RESPS_MAX_DEPTH] is scratch.  The hops are a chain of barriers over
+// shared memory only: every global load is issued before the first hop, and the thread that owns
+// the accepted node writes its entries itself.
 template <typename Sync>
-__device__ __forceinline__ void accept_walk_device(const AcceptArgs& a, int b, int tid, int* s_tgt, int* s_next, Sync sync) {
+__device__ __forceinline__ void accept_walk_device(const AcceptArgs& a, int b, int tid, int* s_tgt, int* s_next,
+                                                   bool have_targets, Sync sync) {
     const int n = min(max(a.n_nodes[b], 1), a.max_tt);
     const int64_t ob = static_cast<int64_t>(b) * a.max_tt;
     const int cap = a.max_depth + 1;
     const int my_tok = (tid < n) ? a.tokens[ob + tid] : -1;
     const int my_par = (tid < n) ? a.parent[ob + tid] : -2;
-    if (tid < n) s_tgt[tid] = __ldcg(a.target_argmax + ob + tid);
+    resps_step step = {};
+    if (tid == 0 && a.steps_next) step = a.steps[b];
+    if (!have_targets && tid < n) s_tgt[tid] = __ldcg(a.target_argmax + ob + tid);
+    if (tid < RESPS_MAX_DEPTH) s_next[tid] = -1;
     if (tid < cap) {
         a.accept_path[b * cap + tid] = (tid == 0) ? 0 : -1;
         a.out_tokens[b * cap + tid] = -1;
     }
-    sync();
+    sync();  // (also orders the -1 fill above before the entries written below)
     int cur = 0, len = 0;
     for (int hop = 0; hop < a.max_depth; ++hop) {
-        if (tid == 0) *s_next = -1;
-        sync();
         // children of one node carry distinct tokens, so at most one thread matches
-        if (tid > 0 && tid < n && my_par == cur && my_tok == s_tgt[cur]) *s_next = tid;
+        if (tid > 0 && tid < n && my_par == cur && my_tok == s_tgt[cur]) {
+            s_next[hop] = tid;
+            a.accept_path[b * cap + len + 1] = tid;
+            a.out_tokens[b * cap + len] = my_tok;
+        }
         sync();
-        const int nxt = *s_next;
-        sync();
+        const int nxt = s_next[hop];
         if (nxt < 0) break;
         cur = nxt;
         ++len;
-        if (tid == 0) {
-            a.accept_path[b * cap + len] = cur;
-            a.out_tokens[b * cap + len - 1] = a.tokens[ob + cur];
-        }
     }
     if (tid == 0) {
         a.out_tokens[b * cap + len] = s_tgt[cur];
         a.accept_len[b] = len;
         if (a.steps_next) {
-            resps_step s = a.steps[b];
-            s.prefix_len += len + 1;
-            a.steps_next[b] = s;
+            step.prefix_len += len + 1;
+            a.steps_next[b] = step;
         }
     }
 }

@@ -594,7 +594,7 @@ struct ArgmaxArgs {
     int slices, cps;  // streaming kernel: slices per row, chunks per slice (partials keep the stride `splits`)
     unsigned long long* part;
     unsigned int* counter;
-    unsigned int* seq_counter;  // streaming kernel: rows of a sequence that are final
+    unsigned int* seq_counter;  // streaming kernel: CTAs of a sequence that have delivered their slice
     int32_t* out;
     unsigned long long* key_out;  // optional [batch][max_tt]: the packed (value, id) of every row's arg-max
     int32_t* status;            // streaming kernel: where a wait that ran out is flagged (may be null)
@@ -603,9 +603,9 @@ struct ArgmaxArgs {
 // Streaming arg-max (16-byte aligned rows): like the streaming scan, a CTA walks a slice of several
 // 8192-logit chunks of one row behind a copy-issuing warp (cp.async.bulk three chunks ahead), a thread
 // keeps 32 logits of the chunk in registers and its best (ordered value, ~id) key across chunks.  The
-// last CTA of a row merges the slices; the CTA that completes the last row of a sequence goes on to
-// the acceptance walk (Section 3.2, "Acceptance Criterion" at temperature 0) when the caller asked
-// for it, so that arg-max and walk are one kernel.
+// last CTA of a sequence to deliver its slice merges the slices of all rows and goes on to the
+// acceptance walk (Section 3.2, "Acceptance Criterion" at temperature 0) when the caller asked for
+// it, so that arg-max and walk are one kernel.
 __global__ void __launch_bounds__(kStreamThreads, 2) row_argmax_stream_kernel(const ArgmaxArgs a, const AcceptArgs w,
                                                                                const int do_walk) {
     pdl_wait();  // the kernel before this one in the stream has completed
@@ -616,7 +616,7 @@ __global__ void __launch_bounds__(kStreamThreads, 2) row_argmax_stream_kernel(co
     __shared__ unsigned long long s_k[kScanThreads / 32];
     __shared__ int s_flag;
     __shared__ int s_tgt[RESPS_MAX_TT];
-    __shared__ int s_next;
+    __shared__ int s_next[RESPS_MAX_DEPTH];
     const int b = blockIdx.z, r = blockIdx.y, sl = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int n = min(max(a.n_nodes[b], 0), a.max_tt);
@@ -695,40 +695,44 @@ __global__ void __launch_bounds__(kStreamThreads, 2) row_argmax_stream_kernel(co
     if (lane == 0) s_k[warp] = best;
     consumer_sync();
     const int64_t prow = static_cast<int64_t>(b) * a.max_tt + r;
-    // ---- the row's result: directly, or by the last slice to arrive ----------------------------------
-    if (tid == 0) {
-        for (int wq = 1; wq < kScanThreads / 32; ++wq) best = (s_k[wq] > best) ? s_k[wq] : best;
-        int row_done = 1;
-        if (a.slices > 1) {
-            a.part[prow * a.splits + sl] = best;
-            __threadfence();
-            row_done = (atomicAdd(a.counter + prow, 1u) == static_cast<unsigned>(a.slices - 1));
-            if (row_done) {
-                __threadfence();
-                for (int i = 0; i < a.slices; ++i) {
-                    const unsigned long long p = __ldcg(a.part + prow * a.splits + i);
-                    best = (p > best) ? p : best;
-                }
-                a.counter[prow] = 0u;
-            }
-        }
-        int seq_done = 0;
-        if (row_done) {
+    const int64_t ob = static_cast<int64_t>(b) * a.max_tt;
+    // ---- a row in one slice and no walk: the CTA's result is the row's -------------------------------
+    if (a.slices == 1 && !do_walk) {
+        if (tid == 0) {
+            for (int wq = 1; wq < kScanThreads / 32; ++wq) best = (s_k[wq] > best) ? s_k[wq] : best;
             a.out[prow] = key_id(best);
             if (a.key_out) a.key_out[prow] = best;
-            if (do_walk) {
-                __threadfence();
-                seq_done = (atomicAdd(a.seq_counter + b, 1u) == static_cast<unsigned>(n - 1));
-                if (seq_done) a.seq_counter[b] = 0u;
-            }
         }
-        s_flag = seq_done;
+        return;
+    }
+    // ---- otherwise the last CTA of the whole sequence to arrive merges the slices of every row (one
+    // counter per sequence: one fence and one atomic on every CTA's way out) and, when asked, goes
+    // on to the acceptance walk with the targets already in shared memory ---------------------------
+    if (tid == 0) {
+        for (int wq = 1; wq < kScanThreads / 32; ++wq) best = (s_k[wq] > best) ? s_k[wq] : best;
+        a.part[prow * a.splits + sl] = best;
+        __threadfence();
+        const unsigned arrivals = static_cast<unsigned>(n) * static_cast<unsigned>(a.slices);
+        const int last = (atomicAdd(a.seq_counter + b, 1u) == arrivals - 1u);
+        if (last) a.seq_counter[b] = 0u;
+        s_flag = last;
     }
     consumer_sync();
     if (!s_flag) return;
-    // ---- the sequence's last row is final: the acceptance walk, by this CTA's consumer threads ---------
     __threadfence();
-    accept_walk_device(w, b, tid, s_tgt, &s_next, [] { consumer_sync(); });
+    for (int t = tid; t < n; t += kScanThreads) {
+        unsigned long long top = 0ull;
+        for (int i = 0; i < a.slices; ++i) {
+            const unsigned long long p = __ldcg(a.part + (ob + t) * a.splits + i);
+            top = (p > top) ? p : top;
+        }
+        a.out[ob + t] = key_id(top);
+        if (a.key_out) a.key_out[ob + t] = top;
+        if (t < RESPS_MAX_TT) s_tgt[t] = key_id(top);
+    }
+    if (!do_walk) return;
+    // (the walk's first barrier orders s_tgt; Section 3.2, "Acceptance Criterion" at temperature 0)
+    accept_walk_device(w, b, tid, s_tgt, s_next, true, [] { consumer_sync(); });
 }
 
 template <bool VEC>
