@@ -55,7 +55,7 @@ void carve(resps_ctx* c, Carver& cv) {
     cv.take(w.node_row, nodes);
     cv.take(w.amax_local, nodes);
     cv.take(w.ctl_h1, static_cast<int64_t>(s.max_batch) * resps::controller_max_hidden());
-    cv.take(w.samp_scratch, static_cast<int64_t>(resps::sampled_scratch_doubles(s.max_batch)));
+    cv.take(w.samp_scratch, static_cast<int64_t>(resps::sampled_scratch_doubles(s.max_batch, s.vocab)));
     cv.take(w.part_key, rows * w.scan_splits * s.max_k);
     cv.take(w.part_ms, rows * w.scan_splits);
     cv.take(w.row_val, rows * s.max_k);
@@ -149,7 +149,7 @@ int resps_create(resps_ctx** out, const resps_shape* shape) {
     real.base = static_cast<char*>(c->arena);
     carve(c, real);
     if (resps::attention_setup(c) != cudaSuccess || resps::tree_setup(c) != cudaSuccess ||
-        resps::scan_setup(c) != cudaSuccess) {
+        resps::scan_setup(c) != cudaSuccess || resps::sampled_setup(c) != cudaSuccess) {
         cudaFree(c->arena);
         resps::attention_teardown(c);
         delete c;

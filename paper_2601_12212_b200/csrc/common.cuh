@@ -41,7 +41,7 @@ struct Workspace {
     int32_t* node_row = nullptr;             // [max_batch][max_tt] draft row behind every node's children (tree build)
     float* ctl_h1 = nullptr;                 // controller: first hidden layer [max_batch][256]
     unsigned int* ctl_counter = nullptr;     // controller: hidden units done per sequence (self-resetting)
-    double* samp_scratch = nullptr;          // acceptance under sampling: a few words per sequence
+    double* samp_scratch = nullptr;          // acceptance under sampling: partial sums, then (p, q) of every token and sequence
     unsigned int* amax_seq_counter = nullptr;  // [max_batch] arg-max CTAs of a sequence that have delivered (self-resetting)
     // attention
     int attn_grid = 0;          // persistent CTAs (one per SM)
@@ -157,7 +157,7 @@ cudaError_t launch_accept_sampled(const resps_ctx* ctx, const resps_step* d_step
                                   const int32_t* parent, const double* u_accept, const double* u_sample,
                                   int32_t* accept_path, int32_t* accept_len, int32_t* out_tokens, resps_step* steps_next,
                                   cudaStream_t st);
-size_t sampled_scratch_doubles(int max_batch);
+size_t sampled_scratch_doubles(int max_batch, int vocab);
 cudaError_t launch_controller(const resps_ctx* ctx, const resps_policy* pol, const void* h, const void* m, const void* l,
                               int64_t ld_hidden, int batch, int interval, float temperature, const double* uniform,
                               const int32_t* accept_len, const float* elapsed_s, resps_controller_state* state,
@@ -167,6 +167,7 @@ int controller_max_hidden();
 int controller_max_actions();
 cudaError_t tree_setup(resps_ctx* ctx);
 cudaError_t scan_setup(resps_ctx* ctx);
+cudaError_t sampled_setup(resps_ctx* ctx);
 int tree_candidate_limit();
 
 // ---- device helpers --------------------------------------------------------

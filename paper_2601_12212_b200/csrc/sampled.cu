@@ -16,6 +16,14 @@
 // barrier (no spinning anywhere), and every CTA then takes the same decision from the same numbers.
 // Arithmetic is fp64 throughout: a decision (accept or not, which token) is a comparison of sums over
 // 10^5 terms, and only at fp64 is the order of summation immaterial to it.
+//
+// The exponentials dominate, so each is taken once per visited node: the pair (p, q) of every token
+// lives in a scratch array (16 bytes per token and sequence, L2-resident) and is brought up to date
+// in place by the pass that needs it next -- first the division by the softmax sums, then one
+// rejection round per pass -- so a pass costs two divisions per token, never an exponential.  Only
+// the thread that owns a token touches its pair; the pairs of the current node's children, which
+// every CTA needs for the decisions, are copied by their owners into a small table behind the same
+// barrier that carries the sums (two tables in turn, so that a pass never writes the one being read).
 #include <cmath>
 
 #include "common.cuh"
@@ -25,7 +33,6 @@ namespace {
 
 constexpr int kClu = 8;             // CTAs per sequence
 constexpr int kSampThreads = 1024;
-constexpr int kMaxRounds = RESPS_MAX_K;  // rejected siblings at one node
 constexpr unsigned kFull = 0xFFFFFFFFu;
 
 struct SampledArgs {
@@ -43,9 +50,13 @@ struct SampledArgs {
     int vocab, max_tt, max_depth, max_k;
     int32_t *accept_path, *accept_len, *out_tokens;
     resps_step* steps_next;
-    double* scratch;  // [batch][kScratchPerSeq]
+    double* scratch;  // [batch][kScratchPerSeq] partial sums, then [batch][kClu][2][per_thr * kSampThreads] (p, q)
+    int64_t state_per_cta;  // doubles of one CTA's p (or q) array
+    int staged;             // 1: the rows' slices fit the staging area in shared memory
 };
-constexpr int kScratchPerSeq = 2 * kClu + 8;  // two alternating sets of partials, then the drawn token
+constexpr int kTableAt = 4 * kClu + 8;
+constexpr int kScratchPerSeq = kTableAt + 2 * 2 * RESPS_MAX_K;  // two alternating sets of pairs of partials, the
+                                                                // drawn token, two alternating tables of the children's (p, q)
 
 __device__ __forceinline__ unsigned cluster_rank() {
     unsigned r;
@@ -56,48 +67,91 @@ __device__ __forceinline__ void cluster_barrier() {
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
-// Sum (or maximum) over the CTA, result in every thread.
+struct Pair {
+    double x, y;
+};
+
+// Two sums (or two maxima) over the CTA at once, result in every thread.
 template <bool MAX>
-__device__ __forceinline__ double block_reduce(double v, double* s_red) {
+__device__ __forceinline__ Pair block_reduce2(Pair v, double* s_red) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
-        const double w = __shfl_xor_sync(kFull, v, o);
-        v = MAX ? fmax(v, w) : v + w;
+        const double wx = __shfl_xor_sync(kFull, v.x, o), wy = __shfl_xor_sync(kFull, v.y, o);
+        v.x = MAX ? fmax(v.x, wx) : v.x + wx;
+        v.y = MAX ? fmax(v.y, wy) : v.y + wy;
     }
     __syncthreads();  // s_red is free again
-    if (lane == 0) s_red[warp] = v;
+    if (lane == 0) s_red[2 * warp] = v.x, s_red[2 * warp + 1] = v.y;
     __syncthreads();
-    double r = s_red[0];
-    for (int w = 1; w < kSampThreads / 32; ++w) r = MAX ? fmax(r, s_red[w]) : r + s_red[w];
+    Pair r = {s_red[0], s_red[1]};
+    for (int w = 1; w < kSampThreads / 32; ++w) {
+        r.x = MAX ? fmax(r.x, s_red[2 * w]) : r.x + s_red[2 * w];
+        r.y = MAX ? fmax(r.y, s_red[2 * w + 1]) : r.y + s_red[2 * w + 1];
+    }
     return r;
 }
 
-// The same over the cluster: the CTAs' results meet in global memory behind the cluster barrier and
-// every thread adds them up in rank order, so all CTAs hold the same bits.  `set` alternates between
-// consecutive reductions (a set is written again only after everyone has read it).
+// Store one double into the shared memory of CTA `peer` of the cluster, at the address `local` has here.
+__device__ __forceinline__ void store_to_peer(double* local, unsigned peer, double v) {
+    const uint32_t mine = static_cast<uint32_t>(__cvta_generic_to_shared(local));
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(mine), "r"(peer));
+    asm volatile("st.shared::cluster.f64 [%0], %1;" ::"r"(remote), "d"(v) : "memory");
+}
+
+// The same over the cluster: every CTA writes its result into every peer's shared memory (slot
+// `rank` of `s_peer[set]`), the hardware cluster barrier orders the writes, and every thread adds the
+// eight up in rank order, so all CTAs hold the same bits.  `set` alternates between consecutive
+// reductions (a set is written again only after everyone has read it: the barrier of the reduction
+// in between).  The barrier also makes the children's table a pass has written visible to the cluster.
 template <bool MAX>
-__device__ __forceinline__ double cluster_reduce(double v, double* s_red, double* scratch, int& set, unsigned rank) {
-    const double mine = block_reduce<MAX>(v, s_red);
-    double* slot = scratch + set * kClu;
-    if (threadIdx.x == 0) __stcg(slot + rank, mine);
+__device__ __forceinline__ Pair cluster_reduce2(Pair v, double* s_red, double (*s_peer)[kClu][2], int& set, unsigned rank) {
+    const Pair mine = block_reduce2<MAX>(v, s_red);
+    if (threadIdx.x < kClu) {
+        store_to_peer(&s_peer[set][rank][0], threadIdx.x, mine.x);
+        store_to_peer(&s_peer[set][rank][1], threadIdx.x, mine.y);
+    }
     cluster_barrier();
-    double r = __ldcg(slot);
-    for (int c = 1; c < kClu; ++c) r = MAX ? fmax(r, __ldcg(slot + c)) : r + __ldcg(slot + c);
+    Pair r = {s_peer[set][0][0], s_peer[set][0][1]};
+    for (int c = 1; c < kClu; ++c) {
+        r.x = MAX ? fmax(r.x, s_peer[set][c][0]) : r.x + s_peer[set][c][0];
+        r.y = MAX ? fmax(r.y, s_peer[set][c][1]) : r.y + s_peer[set][c][1];
+    }
     set ^= 1;
     return r;
+}
+
+// What the stored (p, q) of a token still lack: the division by the softmax sums, or one rejection
+// round (Section 3.2, "Acceptance Criterion": target side -> normalised max(0, p - q), draft side
+// without the rejected token x, renormalised).
+struct Pending {
+    int kind;      // 0 nothing, 1 softmax sums, 2 a rejection round
+    double a, b;   // reciprocals: kind 1 of the target's and the draft's sum (b = 0: no draft row); kind 2 of the
+                   // residual's normaliser (0: residual empty, p is kept) and of the draft mass left (0: q is kept)
+    int x;         // kind 2: the rejected token
+};
+// A division by a normaliser is a multiplication by its fp64 reciprocal (one rounding more than the
+// quotient; the decisions compare sums of 10^5 such terms and are taken with a margin far above that).
+__device__ __forceinline__ double recip_or_zero(double s) { return s > 0.0 ? 1.0 / s : 0.0; }
+__device__ __forceinline__ void apply(const Pending& pd, int v, double& p, double& q) {
+    if (pd.kind == 1) {
+        p = p * pd.a;
+        q = q * pd.b;
+    } else if (pd.kind == 2) {
+        if (pd.a > 0.0) p = fmax(p - q, 0.0) * pd.a;
+        q = (v == pd.x) ? 0.0 : (pd.b > 0.0 ? q * pd.b : q);
+    }
 }
 
 __global__ void __launch_bounds__(kSampThreads, 1) accept_sampled_kernel(const SampledArgs a) {
     pdl_wait();  // the kernel before this one in the stream has completed
     pdl_launch_dependents();
-    __shared__ double s_red[kSampThreads / 32];
+    __shared__ double s_red[2 * (kSampThreads / 32)];
     __shared__ double s_scan[kSampThreads / 32];
+    __shared__ double s_peer[2][kClu][2];  // the cluster's partial results, written by the peers
     __shared__ int s_tok[RESPS_MAX_TT], s_par[RESPS_MAX_TT];
     __shared__ int s_children[RESPS_MAX_TT];
-    __shared__ int s_removed[kMaxRounds];       // tokens of the rejected siblings, in order
-    __shared__ double s_z[kMaxRounds];          // normaliser of the residual after each rejection (0: residual kept)
-    __shared__ double s_rest[kMaxRounds];       // draft mass left after each removal
     __shared__ int s_decision;                  // accepted child, or -1
     __shared__ int s_nchild;
     const unsigned rank = cluster_rank();
@@ -119,6 +173,33 @@ __global__ void __launch_bounds__(kSampThreads, 1) accept_sampled_kernel(const S
     const int c_lo = min(V, static_cast<int>(rank) * per_cta), c_hi = min(V, c_lo + per_cta);
     const int per_thr = (per_cta + kSampThreads - 1) / kSampThreads;
     const int t_lo = min(c_hi, c_lo + tid * per_thr), t_hi = min(c_hi, t_lo + per_thr);
+    // (p, q) of token v: arrays of the CTA that owns v, element (v - its run's start) * threads + its thread,
+    // so that a warp's accesses of one pass are contiguous
+    double* state0 = a.scratch + static_cast<int64_t>(gridDim.x / kClu) * kScratchPerSeq +
+                     static_cast<int64_t>(b) * kClu * 2 * a.state_per_cta;
+    auto p_of = [&](int v) -> double* {
+        const int r = v / per_cta, in_cta = v - r * per_cta;
+        const int t = in_cta / per_thr, i = in_cta - t * per_thr;
+        return state0 + static_cast<int64_t>(r) * 2 * a.state_per_cta + static_cast<int64_t>(i) * kSampThreads + t;
+    };
+    double* my_p = state0 + static_cast<int64_t>(rank) * 2 * a.state_per_cta + tid;  // + i * kSampThreads
+    double* my_q = my_p + a.state_per_cta;
+    double* table = scratch + kTableAt;  // [2][RESPS_MAX_K][2]
+    extern __shared__ float s_stage[];   // [2][kSampThreads][per_thr + 1] when a.staged
+    const int stage_row = kSampThreads * (per_thr + 1);
+    // After a pass (and a CTA barrier): the owners copy the children's pairs into table `par`.
+    auto publish_children = [&](int par, int n_child) {
+        __syncthreads();
+        if (tid < n_child && tid < RESPS_MAX_K) {
+            const int x = s_tok[s_children[tid]];
+            if (x / per_cta == static_cast<int>(rank)) {
+                const double* at = p_of(x);
+                double* dst = table + (par * RESPS_MAX_K + tid) * 2;
+                __stcg(dst, __ldcg(at));
+                __stcg(dst + 1, __ldcg(at + a.state_per_cta));
+            }
+        }
+    };
 
     int cur = 0, acc = 0;
     for (;;) {
@@ -131,43 +212,103 @@ __global__ void __launch_bounds__(kSampThreads, 1) accept_sampled_kernel(const S
                     if (s_par[c] == cur) s_children[m++] = c;
             s_nchild = m;
         }
-        // ---- P_T(. | cur) = softmax(row / T): maximum, then the sum of exponentials ------------------
-        float fm = -INFINITY;
-        for (int v = t_lo; v < t_hi; ++v) fm = fmaxf(fm, __ldg(trow + v));
-        const double mx_t = cluster_reduce<true>(static_cast<double>(fm), s_red, scratch, set, rank) * a.inv_t;
-        double sum = 0.0;
-        for (int v = t_lo; v < t_hi; ++v) sum += exp(static_cast<double>(__ldg(trow + v)) * a.inv_t - mx_t);
-        const double s_t = cluster_reduce<false>(sum, s_red, scratch, set, rank);
-        const int n_child = s_nchild;  // (the reductions above synchronised the CTA)
+        __syncthreads();
+        const int n_child = s_nchild;
         const float* drow = nullptr;
-        double mx_d = 0.0, s_d = 1.0;
         if (n_child > 0) {
             const int row = a.node_row[ob + cur];  // >= 0 for a node with children
             drow = a.draft + b * a.dld_b + (row / RESPS_MAX_K) * a.dld_level + (row % RESPS_MAX_K) * a.dld_row;
-            fm = -INFINITY;
-            for (int v = t_lo; v < t_hi; ++v) fm = fmaxf(fm, __ldg(drow + v));
-            mx_d = cluster_reduce<true>(static_cast<double>(fm), s_red, scratch, set, rank) * a.inv_t;
-            sum = 0.0;
-            for (int v = t_lo; v < t_hi; ++v) sum += exp(static_cast<double>(__ldg(drow + v)) * a.inv_t - mx_d);
-            s_d = cluster_reduce<false>(sum, s_red, scratch, set, rank);
         }
-        // p and q of one token after `rounds` rejections at this node
-        auto eval = [&](int v, int rounds, double& p, double& q) {
-            p = exp(static_cast<double>(__ldg(trow + v)) * a.inv_t - mx_t) / s_t;
-            q = drow ? exp(static_cast<double>(__ldg(drow + v)) * a.inv_t - mx_d) / s_d : 0.0;
-            for (int i = 0; i < rounds; ++i) {
-                if (s_z[i] > 0.0) p = fmax(p - q, 0.0) / s_z[i];
-                q = (v == s_removed[i]) ? 0.0 : (s_rest[i] > 0.0 ? q / s_rest[i] : q);
+        // ---- P_T(. | cur) = softmax(row / T) and the draft's P_d: maxima, then the exponentials (stored)
+        // and their sums -------------------------------------------------------------------------------
+        // The CTA's slice of both rows comes in with coalesced loads (consecutive threads, consecutive
+        // tokens) and is parked in shared memory, token e of the slice at [e / per_thr][e % per_thr] with a
+        // padded row, from where every thread reads its own run without bank conflicts.  (A vocabulary
+        // too large for that is read in place, run by run.)
+        float fm_t = -INFINITY, fm_d = -INFINITY;
+        if (a.staged) {
+            __syncthreads();  // the previous node's readers are done with the staging area
+            constexpr int kGroup = 8;  // loads in flight per thread and row
+            const int n_cta = c_hi - c_lo;
+            for (int e0 = tid; e0 < n_cta; e0 += kGroup * kSampThreads) {
+                float xt[kGroup], xd[kGroup];
+#pragma unroll
+                for (int u = 0; u < kGroup; ++u) {
+                    const int e = e0 + u * kSampThreads;
+                    xt[u] = (e < n_cta) ? __ldg(trow + c_lo + e) : -INFINITY;
+                    xd[u] = (e < n_cta && drow) ? __ldg(drow + c_lo + e) : -INFINITY;
+                }
+#pragma unroll
+                for (int u = 0; u < kGroup; ++u) {
+                    const int e = e0 + u * kSampThreads;
+                    if (e >= n_cta) break;
+                    const int t = e / per_thr, i = e - t * per_thr;
+                    s_stage[t * (per_thr + 1) + i] = xt[u];
+                    s_stage[stage_row + t * (per_thr + 1) + i] = xd[u];
+                    fm_t = fmaxf(fm_t, xt[u]);
+                    fm_d = fmaxf(fm_d, xd[u]);
+                }
+            }
+        } else {
+            for (int v = t_lo; v < t_hi; ++v) {
+                fm_t = fmaxf(fm_t, __ldg(trow + v));
+                if (drow) fm_d = fmaxf(fm_d, __ldg(drow + v));
+            }
+        }
+        // (the reduction's barriers also order the staging area)
+        const Pair mx = cluster_reduce2<true>(Pair{static_cast<double>(fm_t), static_cast<double>(fm_d)}, s_red, s_peer,
+                                              set, rank);
+        const double mx_t = mx.x * a.inv_t, mx_d = mx.y * a.inv_t;
+        Pair sum = {0.0, 0.0};
+        for (int v = t_lo, i = 0; v < t_hi; ++v, ++i) {
+            const float xt = a.staged ? s_stage[tid * (per_thr + 1) + i] : __ldg(trow + v);
+            const float xd = !drow ? 0.f : (a.staged ? s_stage[stage_row + tid * (per_thr + 1) + i] : __ldg(drow + v));
+            const double wt = exp(static_cast<double>(xt) * a.inv_t - mx_t);
+            const double wd = drow ? exp(static_cast<double>(xd) * a.inv_t - mx_d) : 0.0;
+            __stcg(my_p + static_cast<int64_t>(i) * kSampThreads, wt);
+            __stcg(my_q + static_cast<int64_t>(i) * kSampThreads, wd);
+            sum.x += wt, sum.y += wd;
+        }
+        publish_children(0, n_child);
+        sum = cluster_reduce2<false>(sum, s_red, s_peer, set, rank);
+        Pending pend = {1, recip_or_zero(sum.x), drow ? recip_or_zero(sum.y) : 0.0, -1};
+        // p and q of child j's token as they stand at trial j
+        auto eval = [&](int j, int v, double& p, double& q) {
+            const double* at = table + ((j & 1) * RESPS_MAX_K + j) * 2;
+            p = __ldcg(at), q = __ldcg(at + 1);
+            apply(pend, v, p, q);
+        };
+        // one pass over this thread's tokens: bring (p, q) up to date in place, hand each to `f`
+        auto pass = [&](auto&& f) {
+            constexpr int kGroup = 4;  // pairs fetched together: their loads are in flight at once
+            for (int v0 = t_lo, i0 = 0; v0 < t_hi; v0 += kGroup, i0 += kGroup) {
+                double p[kGroup], q[kGroup];
+#pragma unroll
+                for (int u = 0; u < kGroup; ++u) {
+                    const bool live = v0 + u < t_hi;
+                    p[u] = live ? __ldcg(my_p + static_cast<int64_t>(i0 + u) * kSampThreads) : 0.0;
+                    q[u] = live ? __ldcg(my_q + static_cast<int64_t>(i0 + u) * kSampThreads) : 0.0;
+                }
+#pragma unroll
+                for (int u = 0; u < kGroup; ++u) {
+                    if (v0 + u >= t_hi) break;
+                    if (pend.kind) {
+                        apply(pend, v0 + u, p[u], q[u]);
+                        __stcg(my_p + static_cast<int64_t>(i0 + u) * kSampThreads, p[u]);
+                        __stcg(my_q + static_cast<int64_t>(i0 + u) * kSampThreads, q[u]);
+                    }
+                    f(v0 + u, p[u], q[u]);
+                }
             }
         };
         // ---- try the children ---------------------------------------------------------------------
-        int rounds = 0, next = -1;
+        int next = -1;
         for (int j = 0; j < n_child && j < a.max_k; ++j) {
             const int child = s_children[j];
             const int x = s_tok[child];
             if (tid == 0) {
                 double p, q;
-                eval(x, rounds, p, q);
+                eval(j, x, p, q);
                 const double alpha = q > 0.0 ? fmin(1.0, p / q) : (p > 0.0 ? 1.0 : 0.0);
                 const double u = a.u_accept[(static_cast<int64_t>(b) * cap + acc) * a.max_k + j];
                 s_decision = (u < alpha) ? child : -1;
@@ -176,18 +317,14 @@ __global__ void __launch_bounds__(kSampThreads, 1) accept_sampled_kernel(const S
             next = s_decision;
             if (next >= 0) break;
             // rejected: the residual's normaliser and the draft mass that is left without x
-            double z = 0.0, rest = 0.0;
-            for (int v = t_lo; v < t_hi; ++v) {
-                double p, q;
-                eval(v, rounds, p, q);
-                z += fmax(p - q, 0.0);
-                if (v != x) rest += q;
-            }
-            z = cluster_reduce<false>(z, s_red, scratch, set, rank);
-            rest = cluster_reduce<false>(rest, s_red, scratch, set, rank);
-            if (tid == 0) s_removed[rounds] = x, s_z[rounds] = z, s_rest[rounds] = rest;
-            __syncthreads();
-            ++rounds;
+            Pair zr = {0.0, 0.0};
+            pass([&](int v, double p, double q) {
+                zr.x += fmax(p - q, 0.0);
+                if (v != x) zr.y += q;
+            });
+            publish_children((j + 1) & 1, n_child);
+            zr = cluster_reduce2<false>(zr, s_red, s_peer, set, rank);
+            pend = Pending{2, recip_or_zero(zr.x), recip_or_zero(zr.y), x};
         }
         if (next >= 0) {
             cur = next;
@@ -196,16 +333,13 @@ __global__ void __launch_bounds__(kSampThreads, 1) accept_sampled_kernel(const S
                 a.accept_path[b * cap + acc] = cur;
                 a.out_tokens[b * cap + acc - 1] = s_tok[cur];
             }
-            continue;
+            continue;  // (the next node's first reduction is a cluster barrier before anything is overwritten)
         }
         // ---- nobody accepted (or a leaf): draw from the current target-side distribution --------------
         // inverse CDF in token order: this thread's run, the runs before it in the CTA, the CTAs before it
         double run = 0.0;
-        for (int v = t_lo; v < t_hi; ++v) {
-            double p, q;
-            eval(v, rounds, p, q);
-            run += p;
-        }
+        pass([&](int, double p, double) { run += p; });
+        pend.kind = 0;
         // exclusive prefix of the runs over the CTA's threads
         const int lane = tid & 31, warp = tid >> 5;
         double inc = run;
@@ -223,13 +357,12 @@ __global__ void __launch_bounds__(kSampThreads, 1) accept_sampled_kernel(const S
             cta_total += s_scan[w];
         }
         const double excl = before + inc - run;
-        double* slot = scratch + set * kClu;
-        if (tid == 0) __stcg(slot + rank, cta_total);
-        if (rank == 0 && tid == 0) __stcg(scratch + 2 * kClu, -1.0);
+        if (tid < kClu) store_to_peer(&s_peer[set][rank][0], tid, cta_total);
+        if (rank == 0 && tid == 0) __stcg(scratch + 4 * kClu, -1.0);
         cluster_barrier();
         double offset = 0.0, total = 0.0;
         for (int c = 0; c < kClu; ++c) {
-            const double t = __ldcg(slot + c);
+            const double t = s_peer[set][c][0];
             if (c < static_cast<int>(rank)) offset += t;
             total += t;
         }
@@ -241,20 +374,18 @@ __global__ void __launch_bounds__(kSampThreads, 1) accept_sampled_kernel(const S
         if (t_lo < t_hi && start <= target && (start + run > target || last_run)) {
             double cum = start;
             int pick = t_hi - 1;
-            for (int v = t_lo; v < t_hi; ++v) {
-                double p, q;
-                eval(v, rounds, p, q);
-                cum += p;
+            for (int v = t_lo, i = 0; v < t_hi; ++v, ++i) {
+                cum += __ldcg(my_p + static_cast<int64_t>(i) * kSampThreads);  // (up to date since the pass above)
                 if (cum > target) {
                     pick = v;
                     break;
                 }
             }
-            __stcg(scratch + 2 * kClu, static_cast<double>(pick));
+            __stcg(scratch + 4 * kClu, static_cast<double>(pick));
         }
         cluster_barrier();
         if (rank == 0 && tid == 0) {
-            int tok = static_cast<int>(__ldcg(scratch + 2 * kClu));
+            int tok = static_cast<int>(__ldcg(scratch + 4 * kClu));
             if (tok < 0) tok = V - 1;  // rounding left the target past every run: the last token
             a.out_tokens[b * cap + acc] = tok;
             a.accept_len[b] = acc;
@@ -271,7 +402,27 @@ __global__ void __launch_bounds__(kSampThreads, 1) accept_sampled_kernel(const S
 
 }  // namespace
 
-size_t sampled_scratch_doubles(int max_batch) { return static_cast<size_t>(max_batch) * kScratchPerSeq; }
+constexpr size_t kStageCap = 200 * 1024;
+static size_t sampled_stage_bytes(int vocab) {
+    const int per_cta = (vocab + kClu - 1) / kClu;
+    const int per_thr = (per_cta + kSampThreads - 1) / kSampThreads;
+    return 2 * sizeof(float) * kSampThreads * static_cast<size_t>(per_thr + 1);
+}
+
+cudaError_t sampled_setup(resps_ctx*) {
+    return cudaFuncSetAttribute(accept_sampled_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                static_cast<int>(kStageCap));
+}
+
+static int64_t sampled_state_per_cta(int vocab) {
+    const int per_cta = (vocab + kClu - 1) / kClu;
+    const int per_thr = (per_cta + kSampThreads - 1) / kSampThreads;
+    return static_cast<int64_t>(per_thr) * kSampThreads;
+}
+
+size_t sampled_scratch_doubles(int max_batch, int vocab) {
+    return static_cast<size_t>(max_batch) * (kScratchPerSeq + kClu * 2 * sampled_state_per_cta(vocab));
+}
 
 cudaError_t launch_accept_sampled(const resps_ctx* ctx, const resps_step* d_steps, const int32_t* d_n_nodes, int batch,
                                   const float* target, int64_t ld_b, int64_t ld_row, const float* draft, int64_t dld_b,
@@ -290,8 +441,11 @@ cudaError_t launch_accept_sampled(const resps_ctx* ctx, const resps_step* d_step
     a.max_k = ctx->shape.max_k;
     a.accept_path = accept_path, a.accept_len = accept_len, a.out_tokens = out_tokens, a.steps_next = steps_next;
     a.scratch = ctx->ws.samp_scratch;
+    a.state_per_cta = sampled_state_per_cta(ctx->shape.vocab);
+    const size_t stage_bytes = sampled_stage_bytes(ctx->shape.vocab);
+    a.staged = stage_bytes <= kStageCap ? 1 : 0;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(batch * kClu), cfg.blockDim = dim3(kSampThreads), cfg.dynamicSmemBytes = 0, cfg.stream = st;
+    cfg.gridDim = dim3(batch * kClu), cfg.blockDim = dim3(kSampThreads), cfg.dynamicSmemBytes = a.staged ? stage_bytes : 0, cfg.stream = st;
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
