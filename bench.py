@@ -568,6 +568,33 @@ def run_ours(args, w):
                     total += a.elapsed_time(b) * 1e3
                     reps += 1
             phases[name + "_us"] = total / reps
+        # the same calls as they run inside a step: a replayed graph of one call per pool entry, back to
+        # back (distinct logits every call, more than L2 in total; no flush, no host launch in between)
+        in_sequence = {}
+        same_params = all(dw.params[i] == dw.params[0] for i in range(pool))
+        for name in ("expand", "verify"):
+            dw.reset_prefix()
+            dw.set_params(0)
+            dw.expand(0)
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                for i in range(pool):
+                    if name == "expand":
+                        if not same_params:
+                            dw.set_params(i)
+                        dw.expand(i)
+                    else:
+                        dw.verify(i, advance=False)  # the tree of entry 0 against the target rows of entry i
+            for _ in range(2):
+                g.replay()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for _ in range(3):
+                g.replay()
+            b.record(stream)
+            torch.cuda.synchronize()
+            in_sequence[name + "_us"] = a.elapsed_time(b) * 1e3 / (3 * pool)
         V = w.vocab
         phase_bytes["scan"] = float(np.mean([sum((1 + (d - 1) * k) * V * 4 for (_, d, k) in dw.params[i])
                                              for i in range(pool)]))
@@ -622,6 +649,10 @@ def run_ours(args, w):
                   phases["expand_us"], "one call between two events after an L2 flush, mean over the pool"),
         hbm_entry("row_argmax_stream_kernel with the acceptance walk in its tail (one resps_verify_accept call)", phase_bytes["argmax"],
                   phases["verify_us"], "one call between two events after an L2 flush, mean over the pool"),
+        hbm_entry("row_scan_stream_kernel + tree_build_kernel (one resps_tree_expand call)", phase_bytes["scan"],
+                  in_sequence["expand_us"], "replayed graph of one call per pool entry, back to back"),
+        hbm_entry("row_argmax_stream_kernel with the acceptance walk in its tail (one resps_verify_accept call)", phase_bytes["argmax"],
+                  in_sequence["verify_us"], "replayed graph of one call per pool entry, back to back"),
     ]
 
     # CPU baseline: the oracle as it stands, one core, a bounded sample of the same workload
@@ -670,6 +701,8 @@ def run_ours(args, w):
                      "prefix_len": attn_L, "n_nodes": attn_n},
         "roofline_by_kernel": by_kernel,
         "phases": dict(phases, attention_per_layer_us=t_attn),
+        "phases_in_sequence": dict(in_sequence, note="one call per pool entry in a replayed graph, back to back: "
+                                   "the cost of the call inside a step; `phases` times single cold calls"),
         "cpu_baseline": cpu, "clocks": clocks, "device_status": status,
     }
     print(json.dumps(line))
