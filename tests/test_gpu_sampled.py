@@ -99,3 +99,13 @@ def test_sampled_acceptance_llama8b_shape():
     from paper_2601_12212_b200 import synth
     lens, checked = _run(synth.WORKLOADS[2], 1.0, 3, seed=3)
     assert checked >= 3
+
+
+def test_sampled_acceptance_wide_vocabulary():
+    """Vocabulary 200 000: a CTA's slice of two rows no longer fits the staging area in shared memory, so
+    the rows are read in place (the other path of the kernel); two sequences, small trees."""
+    from paper_2601_12212_b200 import synth
+    w = synth.Workload(10, "sampled-wide", 2, 8, 2, 128, 200000, 1, 1024, 16, "gumbel_peaked", "fixed", 12, 3, 4,
+                       (100, 300), 0.7)
+    lens, checked = _run(w, 1.0, 3, seed=5)
+    assert checked >= 5
