@@ -12,18 +12,21 @@
 // All of it is a walk of at most max_depth + 1 nodes, but each step of the walk needs sums over the
 // whole vocabulary (normalisers of softmax and of residuals, the cumulative sum the token is drawn
 // from).  A thread-block cluster of 8 CTAs serves one sequence: every CTA takes an eighth of the
-// vocabulary, partial sums meet through a few words of global memory behind the hardware cluster
-// barrier (no spinning anywhere), and every CTA then takes the same decision from the same numbers.
-// Arithmetic is fp64 throughout: a decision (accept or not, which token) is a comparison of sums over
-// 10^5 terms, and only at fp64 is the order of summation immaterial to it.
+// vocabulary, every CTA writes its partial sums into every peer's shared memory behind the hardware
+// cluster barrier (no spinning anywhere), and every CTA then takes the same decision from the same
+// numbers.  Arithmetic is fp64 throughout: a decision (accept or not, which token) is a comparison of
+// sums over 10^5 terms, and only at fp64 is the order of summation immaterial to it.
 //
-// The exponentials dominate, so each is taken once per visited node: the pair (p, q) of every token
-// lives in a scratch array (16 bytes per token and sequence, L2-resident) and is brought up to date
-// in place by the pass that needs it next -- first the division by the softmax sums, then one
-// rejection round per pass -- so a pass costs two divisions per token, never an exponential.  Only
-// the thread that owns a token touches its pair; the pairs of the current node's children, which
-// every CTA needs for the decisions, are copied by their owners into a small table behind the same
-// barrier that carries the sums (two tables in turn, so that a pass never writes the one being read).
+// The exponentials dominate, so each is taken once per visited node.  The target-side value P of
+// every token of the CTA's slice lives in shared memory (in an L2-resident scratch when the slice is
+// too large) and is brought up to date in place by the pass that needs it next -- first the division
+// by the softmax sum, then one rejection round per pass.  The draft side is the raw exponentials Q in
+// the scratch times one scalar (softmax sum and renormalisations are the same factor for every
+// token; a removed token's entry is set to zero), so a pass reads 8 bytes per token from L2 and
+// multiplies.  Only the thread that owns a token touches its values; (P, Q) of the current node's
+// children, which every CTA needs for the decisions, are copied by their owners into a small table
+// behind the same barrier that carries the sums (two tables in turn, so that a pass never writes the
+// one being read).
 #include <cmath>
 
 #include "common.cuh"
@@ -50,9 +53,10 @@ struct SampledArgs {
     int vocab, max_tt, max_depth, max_k;
     int32_t *accept_path, *accept_len, *out_tokens;
     resps_step* steps_next;
-    double* scratch;  // [batch][kScratchPerSeq] partial sums, then [batch][kClu][2][per_thr * kSampThreads] (p, q)
+    double* scratch;  // [batch][kScratchPerSeq] small words, then [batch][kClu][2][per_thr * kSampThreads] (P, Q)
     int64_t state_per_cta;  // doubles of one CTA's p (or q) array
-    int staged;             // 1: the rows' slices fit the staging area in shared memory
+    int staged;             // 1: a row's slice fits the staging area in shared memory
+    int p_in_smem;          // 1: the target-side values live in shared memory (else in the scratch)
 };
 constexpr int kTableAt = 4 * kClu + 8;
 constexpr int kScratchPerSeq = kTableAt + 2 * 2 * RESPS_MAX_K;  // two alternating sets of pairs of partials, the
@@ -122,26 +126,24 @@ __device__ __forceinline__ Pair cluster_reduce2(Pair v, double* s_red, double (*
     return r;
 }
 
-// What the stored (p, q) of a token still lack: the division by the softmax sums, or one rejection
-// round (Section 3.2, "Acceptance Criterion": target side -> normalised max(0, p - q), draft side
-// without the rejected token x, renormalised).
+// What the stored target-side value of a token still lacks: the division by the softmax sum, or one
+// rejection round (Section 3.2, "Acceptance Criterion": target side -> normalised max(0, p - q)).  The
+// draft side is kept as the raw exponentials times one scalar for the whole row (the softmax sum and
+// the renormalisations after every removal are the same factor for every token), with the entry of
+// a removed token set to zero.
 struct Pending {
-    int kind;      // 0 nothing, 1 softmax sums, 2 a rejection round
-    double a, b;   // reciprocals: kind 1 of the target's and the draft's sum (b = 0: no draft row); kind 2 of the
-                   // residual's normaliser (0: residual empty, p is kept) and of the draft mass left (0: q is kept)
+    int kind;      // 0 nothing, 1 softmax sum, 2 a rejection round
+    double a;      // reciprocal of the target's sum (kind 1) / of the residual's normaliser (kind 2; 0: residual empty, p is kept)
+    double sq_old; // kind 2: the draft side's scalar as it was when the round's child was tried
     int x;         // kind 2: the rejected token
 };
 // A division by a normaliser is a multiplication by its fp64 reciprocal (one rounding more than the
 // quotient; the decisions compare sums of 10^5 such terms and are taken with a margin far above that).
 __device__ __forceinline__ double recip_or_zero(double s) { return s > 0.0 ? 1.0 / s : 0.0; }
-__device__ __forceinline__ void apply(const Pending& pd, int v, double& p, double& q) {
-    if (pd.kind == 1) {
-        p = p * pd.a;
-        q = q * pd.b;
-    } else if (pd.kind == 2) {
-        if (pd.a > 0.0) p = fmax(p - q, 0.0) * pd.a;
-        q = (v == pd.x) ? 0.0 : (pd.b > 0.0 ? q * pd.b : q);
-    }
+__device__ __forceinline__ double apply(const Pending& pd, double p, double q_raw) {
+    if (pd.kind == 1) return p * pd.a;
+    if (pd.kind == 2 && pd.a > 0.0) return fmax(p - q_raw * pd.sq_old, 0.0) * pd.a;
+    return p;
 }
 
 __global__ void __launch_bounds__(kSampThreads, 1) accept_sampled_kernel(const SampledArgs a) {
@@ -173,32 +175,55 @@ __global__ void __launch_bounds__(kSampThreads, 1) accept_sampled_kernel(const S
     const int c_lo = min(V, static_cast<int>(rank) * per_cta), c_hi = min(V, c_lo + per_cta);
     const int per_thr = (per_cta + kSampThreads - 1) / kSampThreads;
     const int t_lo = min(c_hi, c_lo + tid * per_thr), t_hi = min(c_hi, t_lo + per_thr);
-    // (p, q) of token v: arrays of the CTA that owns v, element (v - its run's start) * threads + its thread,
-    // so that a warp's accesses of one pass are contiguous
+    // Target-side value P and raw draft-side weight Q of the token at place i of thread t's run: element
+    // i * threads + t of the owning CTA's arrays, so that a warp's accesses of one pass are contiguous.
+    // Q lives in the L2-resident scratch; P in shared memory when the slice fits, else in the scratch too.
+    extern __shared__ __align__(16) unsigned char s_dyn[];
     double* state0 = a.scratch + static_cast<int64_t>(gridDim.x / kClu) * kScratchPerSeq +
-                     static_cast<int64_t>(b) * kClu * 2 * a.state_per_cta;
-    auto p_of = [&](int v) -> double* {
-        const int r = v / per_cta, in_cta = v - r * per_cta;
-        const int t = in_cta / per_thr, i = in_cta - t * per_thr;
-        return state0 + static_cast<int64_t>(r) * 2 * a.state_per_cta + static_cast<int64_t>(i) * kSampThreads + t;
-    };
-    double* my_p = state0 + static_cast<int64_t>(rank) * 2 * a.state_per_cta + tid;  // + i * kSampThreads
-    double* my_q = my_p + a.state_per_cta;
+                     (static_cast<int64_t>(b) * kClu + rank) * 2 * a.state_per_cta;
+    double* P = a.p_in_smem ? reinterpret_cast<double*>(s_dyn) : state0;
+    double* Q = state0 + a.state_per_cta;
+    float* s_stage = reinterpret_cast<float*>(s_dyn + (a.p_in_smem ? sizeof(double) * a.state_per_cta : 0));  // [threads][per_thr + 1]
     double* table = scratch + kTableAt;  // [2][RESPS_MAX_K][2]
-    extern __shared__ float s_stage[];   // [2][kSampThreads][per_thr + 1] when a.staged
-    const int stage_row = kSampThreads * (per_thr + 1);
-    // After a pass (and a CTA barrier): the owners copy the children's pairs into table `par`.
+    // After a pass (and a CTA barrier): the owners copy (P, Q) of the children's tokens into table `par`.
     auto publish_children = [&](int par, int n_child) {
         __syncthreads();
         if (tid < n_child && tid < RESPS_MAX_K) {
             const int x = s_tok[s_children[tid]];
-            if (x / per_cta == static_cast<int>(rank)) {
-                const double* at = p_of(x);
+            if (x >= c_lo && x < c_hi) {
+                const int in_cta = x - c_lo, t = in_cta / per_thr, i = in_cta - t * per_thr;
                 double* dst = table + (par * RESPS_MAX_K + tid) * 2;
-                __stcg(dst, __ldcg(at));
-                __stcg(dst + 1, __ldcg(at + a.state_per_cta));
+                __stcg(dst, P[static_cast<int64_t>(i) * kSampThreads + t]);
+                __stcg(dst + 1, __ldcg(Q + static_cast<int64_t>(i) * kSampThreads + t));
             }
         }
+    };
+    // The CTA's slice of a row through the staging area: coalesced loads (consecutive threads, consecutive
+    // tokens), token e of the slice parked at [e / per_thr][e % per_thr] with a padded row, from where
+    // every thread reads its own run without bank conflicts.  Returns the maximum this thread saw.
+    auto stage_row = [&](const float* row, bool store) {
+        constexpr int kGroup = 8;  // loads in flight per thread
+        const int n_cta = c_hi - c_lo;
+        float fm = -INFINITY;
+        for (int e0 = tid; e0 < n_cta; e0 += kGroup * kSampThreads) {
+            float x[kGroup];
+#pragma unroll
+            for (int u = 0; u < kGroup; ++u) {
+                const int e = e0 + u * kSampThreads;
+                x[u] = (e < n_cta) ? __ldg(row + c_lo + e) : -INFINITY;
+            }
+#pragma unroll
+            for (int u = 0; u < kGroup; ++u) {
+                const int e = e0 + u * kSampThreads;
+                if (e >= n_cta) break;
+                if (store) {
+                    const int t = e / per_thr, i = e - t * per_thr;
+                    s_stage[t * (per_thr + 1) + i] = x[u];
+                }
+                fm = fmaxf(fm, x[u]);
+            }
+        }
+        return fm;
     };
 
     int cur = 0, acc = 0;
@@ -212,7 +237,7 @@ __global__ void __launch_bounds__(kSampThreads, 1) accept_sampled_kernel(const S
                     if (s_par[c] == cur) s_children[m++] = c;
             s_nchild = m;
         }
-        __syncthreads();
+        __syncthreads();  // (also: the previous node's readers are done with the staging area)
         const int n_child = s_nchild;
         const float* drow = nullptr;
         if (n_child > 0) {
@@ -220,35 +245,12 @@ __global__ void __launch_bounds__(kSampThreads, 1) accept_sampled_kernel(const S
             drow = a.draft + b * a.dld_b + (row / RESPS_MAX_K) * a.dld_level + (row % RESPS_MAX_K) * a.dld_row;
         }
         // ---- P_T(. | cur) = softmax(row / T) and the draft's P_d: maxima, then the exponentials (stored)
-        // and their sums -------------------------------------------------------------------------------
-        // The CTA's slice of both rows comes in with coalesced loads (consecutive threads, consecutive
-        // tokens) and is parked in shared memory, token e of the slice at [e / per_thr][e % per_thr] with a
-        // padded row, from where every thread reads its own run without bank conflicts.  (A vocabulary
-        // too large for that is read in place, run by run.)
+        // and their sums.  The staging area holds one row at a time: the target's while the maxima are
+        // taken (the draft row is only looked at), then the draft's (read again, from L2) -------------
         float fm_t = -INFINITY, fm_d = -INFINITY;
         if (a.staged) {
-            __syncthreads();  // the previous node's readers are done with the staging area
-            constexpr int kGroup = 8;  // loads in flight per thread and row
-            const int n_cta = c_hi - c_lo;
-            for (int e0 = tid; e0 < n_cta; e0 += kGroup * kSampThreads) {
-                float xt[kGroup], xd[kGroup];
-#pragma unroll
-                for (int u = 0; u < kGroup; ++u) {
-                    const int e = e0 + u * kSampThreads;
-                    xt[u] = (e < n_cta) ? __ldg(trow + c_lo + e) : -INFINITY;
-                    xd[u] = (e < n_cta && drow) ? __ldg(drow + c_lo + e) : -INFINITY;
-                }
-#pragma unroll
-                for (int u = 0; u < kGroup; ++u) {
-                    const int e = e0 + u * kSampThreads;
-                    if (e >= n_cta) break;
-                    const int t = e / per_thr, i = e - t * per_thr;
-                    s_stage[t * (per_thr + 1) + i] = xt[u];
-                    s_stage[stage_row + t * (per_thr + 1) + i] = xd[u];
-                    fm_t = fmaxf(fm_t, xt[u]);
-                    fm_d = fmaxf(fm_d, xd[u]);
-                }
-            }
+            fm_t = stage_row(trow, true);
+            if (drow) fm_d = stage_row(drow, false);
         } else {
             for (int v = t_lo; v < t_hi; ++v) {
                 fm_t = fmaxf(fm_t, __ldg(trow + v));
@@ -262,42 +264,52 @@ __global__ void __launch_bounds__(kSampThreads, 1) accept_sampled_kernel(const S
         Pair sum = {0.0, 0.0};
         for (int v = t_lo, i = 0; v < t_hi; ++v, ++i) {
             const float xt = a.staged ? s_stage[tid * (per_thr + 1) + i] : __ldg(trow + v);
-            const float xd = !drow ? 0.f : (a.staged ? s_stage[stage_row + tid * (per_thr + 1) + i] : __ldg(drow + v));
             const double wt = exp(static_cast<double>(xt) * a.inv_t - mx_t);
-            const double wd = drow ? exp(static_cast<double>(xd) * a.inv_t - mx_d) : 0.0;
-            __stcg(my_p + static_cast<int64_t>(i) * kSampThreads, wt);
-            __stcg(my_q + static_cast<int64_t>(i) * kSampThreads, wd);
-            sum.x += wt, sum.y += wd;
+            P[static_cast<int64_t>(i) * kSampThreads + tid] = wt;
+            sum.x += wt;
+        }
+        if (drow) {
+            if (a.staged) {
+                __syncthreads();  // everyone has read the target row
+                stage_row(drow, true);
+                __syncthreads();
+            }
+            for (int v = t_lo, i = 0; v < t_hi; ++v, ++i) {
+                const float xd = a.staged ? s_stage[tid * (per_thr + 1) + i] : __ldg(drow + v);
+                const double wd = exp(static_cast<double>(xd) * a.inv_t - mx_d);
+                __stcg(Q + static_cast<int64_t>(i) * kSampThreads + tid, wd);
+                sum.y += wd;
+            }
         }
         publish_children(0, n_child);
         sum = cluster_reduce2<false>(sum, s_red, s_peer, set, rank);
-        Pending pend = {1, recip_or_zero(sum.x), drow ? recip_or_zero(sum.y) : 0.0, -1};
-        // p and q of child j's token as they stand at trial j
-        auto eval = [&](int j, int v, double& p, double& q) {
-            const double* at = table + ((j & 1) * RESPS_MAX_K + j) * 2;
-            p = __ldcg(at), q = __ldcg(at + 1);
-            apply(pend, v, p, q);
-        };
-        // one pass over this thread's tokens: bring (p, q) up to date in place, hand each to `f`
-        auto pass = [&](auto&& f) {
-            constexpr int kGroup = 4;  // pairs fetched together: their loads are in flight at once
+        Pending pend = {1, recip_or_zero(sum.x), 0.0, -1};
+        double sq = drow ? recip_or_zero(sum.y) : 0.0;  // draft side: q = Q * sq
+        // One pass over this thread's tokens: bring P up to date in place (and retire the token the pending
+        // round removed), hand the current (p, q) of each token to `f`.  The draft side is only read at
+        // nodes that have children (`with_q`); a leaf has no draft row.
+        auto pass = [&](bool with_q, auto&& f) {
+            constexpr int kGroup = 4;  // draft-side values fetched together: their loads are in flight at once
             for (int v0 = t_lo, i0 = 0; v0 < t_hi; v0 += kGroup, i0 += kGroup) {
-                double p[kGroup], q[kGroup];
+                double q_raw[kGroup];
+#pragma unroll
+                for (int u = 0; u < kGroup; ++u)
+                    q_raw[u] = (with_q && v0 + u < t_hi) ? __ldcg(Q + static_cast<int64_t>(i0 + u) * kSampThreads + tid) : 0.0;
 #pragma unroll
                 for (int u = 0; u < kGroup; ++u) {
-                    const bool live = v0 + u < t_hi;
-                    p[u] = live ? __ldcg(my_p + static_cast<int64_t>(i0 + u) * kSampThreads) : 0.0;
-                    q[u] = live ? __ldcg(my_q + static_cast<int64_t>(i0 + u) * kSampThreads) : 0.0;
-                }
-#pragma unroll
-                for (int u = 0; u < kGroup; ++u) {
-                    if (v0 + u >= t_hi) break;
+                    const int v = v0 + u;
+                    if (v >= t_hi) break;
+                    double* pp = P + static_cast<int64_t>(i0 + u) * kSampThreads + tid;
+                    double p = *pp;
                     if (pend.kind) {
-                        apply(pend, v0 + u, p[u], q[u]);
-                        __stcg(my_p + static_cast<int64_t>(i0 + u) * kSampThreads, p[u]);
-                        __stcg(my_q + static_cast<int64_t>(i0 + u) * kSampThreads, q[u]);
+                        p = apply(pend, p, q_raw[u]);
+                        *pp = p;
+                        if (pend.kind == 2 && v == pend.x) {
+                            __stcg(Q + static_cast<int64_t>(i0 + u) * kSampThreads + tid, 0.0);
+                            q_raw[u] = 0.0;
+                        }
                     }
-                    f(v0 + u, p[u], q[u]);
+                    f(v, p, q_raw[u] * sq);
                 }
             }
         };
@@ -307,8 +319,10 @@ __global__ void __launch_bounds__(kSampThreads, 1) accept_sampled_kernel(const S
             const int child = s_children[j];
             const int x = s_tok[child];
             if (tid == 0) {
-                double p, q;
-                eval(j, x, p, q);
+                // (P, Q) of child j's token as the last pass left them, brought up to date here
+                const double* at = table + ((j & 1) * RESPS_MAX_K + j) * 2;
+                const double q_raw = __ldcg(at + 1);
+                const double p = apply(pend, __ldcg(at), q_raw), q = q_raw * sq;
                 const double alpha = q > 0.0 ? fmin(1.0, p / q) : (p > 0.0 ? 1.0 : 0.0);
                 const double u = a.u_accept[(static_cast<int64_t>(b) * cap + acc) * a.max_k + j];
                 s_decision = (u < alpha) ? child : -1;
@@ -318,13 +332,14 @@ __global__ void __launch_bounds__(kSampThreads, 1) accept_sampled_kernel(const S
             if (next >= 0) break;
             // rejected: the residual's normaliser and the draft mass that is left without x
             Pair zr = {0.0, 0.0};
-            pass([&](int v, double p, double q) {
+            pass(true, [&](int v, double p, double q) {
                 zr.x += fmax(p - q, 0.0);
                 if (v != x) zr.y += q;
             });
             publish_children((j + 1) & 1, n_child);
             zr = cluster_reduce2<false>(zr, s_red, s_peer, set, rank);
-            pend = Pending{2, recip_or_zero(zr.x), recip_or_zero(zr.y), x};
+            pend = Pending{2, recip_or_zero(zr.x), sq, x};
+            if (zr.y > 0.0) sq = sq * (1.0 / zr.y);
         }
         if (next >= 0) {
             cur = next;
@@ -338,7 +353,7 @@ __global__ void __launch_bounds__(kSampThreads, 1) accept_sampled_kernel(const S
         // ---- nobody accepted (or a leaf): draw from the current target-side distribution --------------
         // inverse CDF in token order: this thread's run, the runs before it in the CTA, the CTAs before it
         double run = 0.0;
-        pass([&](int, double p, double) { run += p; });
+        pass(drow != nullptr, [&](int, double p, double) { run += p; });
         pend.kind = 0;
         // exclusive prefix of the runs over the CTA's threads
         const int lane = tid & 31, warp = tid >> 5;
@@ -375,7 +390,7 @@ __global__ void __launch_bounds__(kSampThreads, 1) accept_sampled_kernel(const S
             double cum = start;
             int pick = t_hi - 1;
             for (int v = t_lo, i = 0; v < t_hi; ++v, ++i) {
-                cum += __ldcg(my_p + static_cast<int64_t>(i) * kSampThreads);  // (up to date since the pass above)
+                cum += P[static_cast<int64_t>(i) * kSampThreads + tid];  // (up to date since the pass above)
                 if (cum > target) {
                     pick = v;
                     break;
@@ -402,16 +417,19 @@ __global__ void __launch_bounds__(kSampThreads, 1) accept_sampled_kernel(const S
 
 }  // namespace
 
-constexpr size_t kStageCap = 200 * 1024;
-static size_t sampled_stage_bytes(int vocab) {
+constexpr size_t kDynSmemCap = 220 * 1024;
+static int sampled_per_thr(int vocab) {
     const int per_cta = (vocab + kClu - 1) / kClu;
-    const int per_thr = (per_cta + kSampThreads - 1) / kSampThreads;
-    return 2 * sizeof(float) * kSampThreads * static_cast<size_t>(per_thr + 1);
+    return (per_cta + kSampThreads - 1) / kSampThreads;
 }
+static size_t sampled_stage_bytes(int vocab) {  // one row's slice, padded rows
+    return sizeof(float) * kSampThreads * static_cast<size_t>(sampled_per_thr(vocab) + 1);
+}
+static size_t sampled_p_bytes(int vocab) { return sizeof(double) * kSampThreads * static_cast<size_t>(sampled_per_thr(vocab)); }
 
 cudaError_t sampled_setup(resps_ctx*) {
     return cudaFuncSetAttribute(accept_sampled_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                static_cast<int>(kStageCap));
+                                static_cast<int>(kDynSmemCap));
 }
 
 static int64_t sampled_state_per_cta(int vocab) {
@@ -442,10 +460,12 @@ cudaError_t launch_accept_sampled(const resps_ctx* ctx, const resps_step* d_step
     a.accept_path = accept_path, a.accept_len = accept_len, a.out_tokens = out_tokens, a.steps_next = steps_next;
     a.scratch = ctx->ws.samp_scratch;
     a.state_per_cta = sampled_state_per_cta(ctx->shape.vocab);
-    const size_t stage_bytes = sampled_stage_bytes(ctx->shape.vocab);
-    a.staged = stage_bytes <= kStageCap ? 1 : 0;
+    const size_t stage_bytes = sampled_stage_bytes(ctx->shape.vocab), p_bytes = sampled_p_bytes(ctx->shape.vocab);
+    a.p_in_smem = (p_bytes + stage_bytes <= kDynSmemCap) ? 1 : 0;
+    a.staged = ((a.p_in_smem ? p_bytes : 0) + stage_bytes <= kDynSmemCap) ? 1 : 0;
+    const size_t dyn_bytes = (a.p_in_smem ? p_bytes : 0) + (a.staged ? stage_bytes : 0);
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(batch * kClu), cfg.blockDim = dim3(kSampThreads), cfg.dynamicSmemBytes = a.staged ? stage_bytes : 0, cfg.stream = st;
+    cfg.gridDim = dim3(batch * kClu), cfg.blockDim = dim3(kSampThreads), cfg.dynamicSmemBytes = dyn_bytes, cfg.stream = st;
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
