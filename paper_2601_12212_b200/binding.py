@@ -27,6 +27,7 @@ RESPS_DEBUG_ATTN_ROUNDS = 1
 RESPS_DEBUG_ATTN_MIN_TILES = 2
 RESPS_DEBUG_ATTN_STAGGER = 3
 RESPS_DEBUG_SCAN_SLICES = 4
+RESPS_DEBUG_ATTN_SINGLE = 5
 
 EXPORTS = ("resps_create", "resps_destroy", "resps_strerror", "resps_status",
            "resps_workspace_bytes", "resps_debug_set", "resps_attention_replan", "resps_tree_expand", "resps_tree_expand_begin", "resps_tree_expand_level",

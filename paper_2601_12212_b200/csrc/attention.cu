@@ -106,6 +106,7 @@ struct AttnArgs {
     int max_items;
     int sched_grid;   // CTAs of the attention grid (the work list is balanced for it)
     int min_tiles;    // smallest key-tile count worth a split of its own
+    int single_units; // single row tiles while the call costs at most this many units per CTA of the grid
     int rounds;       // 0: the work list chooses its number of rounds; 1..kMaxRounds: as told (tests)
     int stagger;      // cycles lane 1 starts behind lane 0 in row mode
     int q_by_tma;     // 1: Q tiles come by TMA (128 % (Hq/Hkv) == 0), 0: by plain loads
@@ -124,9 +125,14 @@ struct AttnArgs {
 // in key mode and costs one.  Every group is cut into splits of at most T units, with the smallest
 // T for which the items fit one round of the grid (found by a short search; steps of 1/16), so
 // that the CTAs finish together whatever the mix of tree sizes and prefix lengths.
-// When even the shortest row-mode items would leave half of the grid idle (a single short
-// sequence), groups are single row tiles instead, all in key mode: twice the items, each with
-// half the key tiles per lane, for the price of reading K and V through L2 once more.
+// While the whole call is small -- at most `single_units` units per CTA of the grid (8: a single
+// sequence of a few thousand tokens) -- groups are single row tiles instead, all in key mode: items of
+// half the size fill the grid where row-mode items (at least two key tiles for each of two row tiles)
+// cannot, the two halves of a CTA merge into one partial, and K and V pass through L2 once more,
+// which costs nothing at that size.  Measured on the 8B-shaped workload with the prefix growing from
+// 1024 to 3010: 480 us per step against 506 (limit 4), 527 (limit 3) and 510 with the former limit of
+// 2 at 1837; on the 70B-shaped workload (21 units per CTA and more, tensor-pipe-bound) single tiles
+// are 4 % slower (27.4 against 26.3 us per call), so the limit stays below that.
 struct Sched {
     int group_rows;             // rows of a group: 256 (pairs of row tiles) or 128 (single tiles)
     int n[kMaxBatchSmem];       // tree nodes (0 = sequence skipped)
@@ -171,9 +177,8 @@ __device__ __forceinline__ void build_sched(const AttnArgs& a, Sched& sc, int ti
             }
         }
         cost = __reduce_add_sync(0xFFFFFFFFu, min(cost, 1u << 26));
-        // Row-mode items of mt key tiles cost 2 mt units each: if the whole call is worth no more than
-        // half a grid of those, single tiles in key mode fill the grid better.
-        const bool single = cost <= static_cast<unsigned>(mt * a.sched_grid);
+        // a small call is cut into single row tiles (see above)
+        const bool single = cost <= static_cast<unsigned>(a.single_units) * static_cast<unsigned>(a.sched_grid);
         const int group_rows = single ? kBM : kRowTiles * kBM;
         if (tid == 0) sc.group_rows = group_rows;
 #pragma unroll 1
@@ -1856,6 +1861,7 @@ cudaError_t launch_tree_attention(const resps_ctx* ctx, const resps_step* d_step
     a.part_o = reinterpret_cast<uint4*>(ctx->ws.attn_part_o), a.part_ml = ctx->ws.attn_part_ml;
     a.max_items = ctx->ws.attn_max_items, a.sched_grid = ctx->ws.attn_grid;
     a.min_tiles = ctx->ws.attn_min_tiles, a.status = ctx->ws.status;
+    a.single_units = ctx->ws.attn_single;
     a.rounds = ctx->ws.attn_rounds;
     a.stagger = ctx->ws.attn_stagger;
     a.plan_head = reinterpret_cast<int4*>(ctx->ws.attn_plan);
