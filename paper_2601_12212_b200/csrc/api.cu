@@ -245,7 +245,7 @@ int resps_tree_expand(resps_ctx* ctx, const resps_step* d_steps, int batch,
         return RESPS_ERR_CUDA;
     if (resps::launch_tree_build(ctx, d_steps, batch, n_levels, n_slots, d_root_token, d_tokens, d_parent,
                                  d_depth, d_position_ids, d_mask, d_retrieve, d_n_leaves, d_n_nodes,
-                                 stream) != cudaSuccess)
+                                 stream, true) != cudaSuccess)
         return RESPS_ERR_CUDA;
     return RESPS_OK;
 }
@@ -312,7 +312,7 @@ int resps_tree_expand_merge(resps_ctx* ctx, const resps_step* d_steps, int batch
                                        d_shard_offset, stream) != cudaSuccess)
         return RESPS_ERR_CUDA;
     if (resps::launch_tree_build(ctx, d_steps, batch, n_levels, n_slots, d_root_token, d_tokens, d_parent, d_depth,
-                                 d_position_ids, d_mask, d_retrieve, d_n_leaves, d_n_nodes, stream) != cudaSuccess)
+                                 d_position_ids, d_mask, d_retrieve, d_n_leaves, d_n_nodes, stream, true) != cudaSuccess)
         return RESPS_ERR_CUDA;
     return RESPS_OK;
 }
@@ -426,7 +426,7 @@ int resps_tree_expand_finish(resps_ctx* ctx, const resps_step* d_steps, int batc
     // the levels that were given bound the depth: a step asking for more is clamped (and flagged)
     if (resps::launch_tree_build(ctx, d_steps, batch, ctx->level_next, ctx->level_slots, d_root_token, d_tokens,
                                  d_parent, d_depth, d_position_ids, d_mask, d_retrieve, d_n_leaves, d_n_nodes,
-                                 stream) != cudaSuccess)
+                                 stream, false) != cudaSuccess)
         return RESPS_ERR_CUDA;
     ctx->level_next = 0;
     return RESPS_OK;

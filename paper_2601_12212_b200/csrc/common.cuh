@@ -103,7 +103,7 @@ cudaError_t launch_tree_build(const resps_ctx* ctx, const resps_step* d_steps, i
                               int n_levels, int n_slots, const int32_t* root_token,
                               int32_t* tokens, int32_t* parent, int32_t* depth, int32_t* position_ids,
                               uint64_t* mask, int32_t* retrieve, int32_t* n_leaves, int32_t* n_nodes,
-                              cudaStream_t st);
+                              cudaStream_t st, bool after_scan);  // after_scan: a scan or merge kernel of the same call precedes it
 // Arg-max of every target row; with `walk` non-null and rows that allow the streaming kernel the
 // acceptance walk runs in the same kernel (returns true through `walked`).
 cudaError_t launch_row_argmax(const resps_ctx* ctx, const int32_t* d_n_nodes, int batch,

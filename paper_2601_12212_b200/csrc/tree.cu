@@ -41,6 +41,7 @@ struct TreeArgs {
     // the frontier after level j and stops; -1 builds the whole tree.
     int emit_level;
     FrontierOut fr;
+    int setup_before_wait;  // 1: a scan or merge kernel of the same call runs directly before this kernel
 };
 
 // Path scores are compared as integers: the map below keeps the order of finite doubles (and their
@@ -80,8 +81,12 @@ __device__ __forceinline__ int count_above(const long long* keys, int n, int top
 __device__ __forceinline__ int pow2_floor(int n) { return (n > 0) ? (1 << (31 - __clz(n))) : 0; }
 
 __global__ void __launch_bounds__(kTreeThreads, 1) tree_build_kernel(const TreeArgs a) {
-    pdl_wait();  // the kernel before this one in the stream has completed
-    pdl_launch_dependents();
+    // The step parameters were written at least two kernels ago (a scan or a merge kernel of the same
+    // call always sits between their writer and this kernel, and every kernel of the library signals its
+    // dependents only after its own wait), so they are read, and everything that follows from them is
+    // set up, before the wait for the rows: under the tail of the kernel that scans them.  (Where no such
+    // kernel precedes this one -- the last call of the level form -- the wait comes first.)
+    if (!a.setup_before_wait) pdl_wait();
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int b = blockIdx.x, tid = threadIdx.x;
     const StepDims sd = clamp_step(a.steps[b], a.n_levels, a.n_slots, a.max_tt, a.max_k, a.vocab);
@@ -132,6 +137,12 @@ __global__ void __launch_bounds__(kTreeThreads, 1) tree_build_kernel(const TreeA
     int tok_pre[kTokPrefetch];
 #pragma unroll
     for (int i = 0; i < kTokPrefetch; ++i) tok_pre[i] = 0;
+    for (int i = tid; i < RESPS_MAX_DEPTH * (kProbes + kStride + 2); i += kTreeThreads) probe[i] = 0;
+    // the first pass of the per-level loops below has the same index arithmetic at every level
+    const int pair_i = by_k.div(tid), pair_p2 = tid - pair_i * k, pair_p = by_k.div(pair_i);  // pair tid = (candidate, list)
+    const int k_top = pow2_floor(k);
+    if (a.setup_before_wait) pdl_wait();  // the kernel before this one in the stream has completed: the scanned rows are there
+    pdl_launch_dependents();
     for (int c = tid, i = 0; c < n_cand; c += kTreeThreads, ++i) {
         const Cand r = (i == 0) ? own : decode(c);
         const int64_t row = row0 + cand_row(r);
@@ -146,10 +157,6 @@ __global__ void __launch_bounds__(kTreeThreads, 1) tree_build_kernel(const TreeA
         skey[c] = (c < k) ? score_key(lp) : __double_as_longlong(lp);
         node_of[c] = (c < k) ? c : 0;  // level 0 is ranked as scanned; the other levels count from 0
     }
-    for (int i = tid; i < RESPS_MAX_DEPTH * (kProbes + kStride + 2); i += kTreeThreads) probe[i] = 0;
-    // the first pass of the per-level loops below has the same index arithmetic at every level
-    const int pair_i = by_k.div(tid), pair_p2 = tid - pair_i * k, pair_p = by_k.div(pair_i);  // pair tid = (candidate, list)
-    const int k_top = pow2_floor(k);
     __syncthreads();
     // ---- level 0 ---------------------------------------------------------------
     if (tid < k) {
@@ -408,7 +415,7 @@ cudaError_t launch_tree_build(const resps_ctx* ctx, const resps_step* d_steps, i
                               int n_levels, int n_slots, const int32_t* root_token,
                               int32_t* tokens, int32_t* parent, int32_t* depth, int32_t* position_ids,
                               uint64_t* mask, int32_t* retrieve, int32_t* n_leaves, int32_t* n_nodes,
-                              cudaStream_t st) {
+                              cudaStream_t st, bool after_scan) {
     const resps_shape& s = ctx->shape;
     TreeArgs a;
     a.steps = d_steps;
@@ -423,6 +430,7 @@ cudaError_t launch_tree_build(const resps_ctx* ctx, const resps_step* d_steps, i
     a.status = ctx->ws.status;
     a.cand_cap = s.max_k + (s.max_depth - 1) * s.max_k * s.max_k;
     a.emit_level = -1;
+    a.setup_before_wait = after_scan ? 1 : 0;
     a.fr = FrontierOut{};
     const size_t smem = tree_smem_bytes(a.cand_cap);
     return launch_pdl(tree_build_kernel, dim3(batch), dim3(kTreeThreads), smem, st, a);
@@ -441,6 +449,7 @@ cudaError_t launch_tree_level(const resps_ctx* ctx, const resps_step* d_steps, i
     a.status = ctx->ws.status;
     a.cand_cap = s.max_k + (s.max_depth - 1) * s.max_k * s.max_k;
     a.emit_level = level;
+    a.setup_before_wait = 1;  // the scan of this level's rows runs directly before
     a.fr = out;
     return launch_pdl(tree_build_kernel, dim3(batch), dim3(kTreeThreads), tree_smem_bytes(a.cand_cap), st, a);
 }
