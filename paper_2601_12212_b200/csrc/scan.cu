@@ -306,8 +306,6 @@ __device__ __forceinline__ bool consumer_any(bool pred) {  // barrier over the c
 }
 
 __global__ void __launch_bounds__(kStreamThreads, 2) row_scan_stream_kernel(const ScanArgs a) {
-    pdl_wait();  // the kernel before this one in the stream has completed
-    pdl_launch_dependents();
     extern __shared__ __align__(128) unsigned char s_raw[];
     float* s_stage = reinterpret_cast<float*>(s_raw);                                    // [3][8192]
     unsigned long long* s_keys =
@@ -321,6 +319,22 @@ __global__ void __launch_bounds__(kStreamThreads, 2) row_scan_stream_kernel(cons
     __shared__ bool s_last;
     const int b = blockIdx.z, ry = blockIdx.y, sl = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t bar0 = scan_smem_u32(s_bar);
+    auto full_bar = [&](int st) { return bar0 + 8u * st; };
+    auto empty_bar = [&](int st) { return bar0 + 8u * (kStreamStages + st); };
+    // the barriers are set up under the tail of the preceding kernel: nothing here touches global memory
+    if (tid == 0) {
+        for (int st = 0; st < kStreamStages; ++st) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(full_bar(st)) : "memory");
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(empty_bar(st)), "r"(kScanThreads) : "memory");
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        s_count = 0;
+        s_tau = 0ull;
+    }
+    __syncthreads();
+    pdl_wait();  // the kernel before this one in the stream has completed
+    pdl_launch_dependents();
     const StepDims sd = clamp_step(a.steps[b], a.n_levels, a.n_slots, a.max_tt, a.max_k, a.vocab);
     const int k = sd.k;
     const int rows = 1 + (sd.d - 1) * k;
@@ -334,20 +348,6 @@ __global__ void __launch_bounds__(kStreamThreads, 2) row_scan_stream_kernel(cons
     const int c_begin = sl * a.cps;
     const int c_end = min(a.splits, c_begin + a.cps);  // chunks [c_begin, c_end) of this row
     const int list_cap = (kQuadElems + 1) * a.max_k;
-    const uint32_t bar0 = scan_smem_u32(s_bar);
-    auto full_bar = [&](int st) { return bar0 + 8u * st; };
-    auto empty_bar = [&](int st) { return bar0 + 8u * (kStreamStages + st); };
-
-    if (tid == 0) {
-        for (int st = 0; st < kStreamStages; ++st) {
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(full_bar(st)) : "memory");
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(empty_bar(st)), "r"(kScanThreads) : "memory");
-        }
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        s_count = 0;
-        s_tau = 0ull;
-    }
-    __syncthreads();
 
     if (warp == kScanThreads / 32) {
         // ---- copy-issuing warp: a stage is refilled as soon as every consumer has read it ----------
@@ -608,8 +608,6 @@ struct ArgmaxArgs {
 // it, so that arg-max and walk are one kernel.
 __global__ void __launch_bounds__(kStreamThreads, 2) row_argmax_stream_kernel(const ArgmaxArgs a, const AcceptArgs w,
                                                                                const int do_walk) {
-    pdl_wait();  // the kernel before this one in the stream has completed
-    pdl_launch_dependents();
     extern __shared__ __align__(128) unsigned char s_raw[];
     float* s_stage = reinterpret_cast<float*>(s_raw);  // [3][8192]
     __shared__ __align__(8) unsigned long long s_bar[2 * kStreamStages];  // full[3], empty[3]
@@ -619,14 +617,10 @@ __global__ void __launch_bounds__(kStreamThreads, 2) row_argmax_stream_kernel(co
     __shared__ int s_next[RESPS_MAX_DEPTH];
     const int b = blockIdx.z, r = blockIdx.y, sl = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int n = min(max(a.n_nodes[b], 0), a.max_tt);
-    if (r >= n) return;
-    const float* row = a.logits + b * a.ld_b + r * a.ld_row;
-    const int c_begin = sl * a.cps;
-    const int c_end = min(a.splits, c_begin + a.cps);  // chunks [c_begin, c_end) of this row
     const uint32_t bar0 = scan_smem_u32(s_bar);
     auto full_bar = [&](int st) { return bar0 + 8u * st; };
     auto empty_bar = [&](int st) { return bar0 + 8u * (kStreamStages + st); };
+    // the barriers are set up under the tail of the preceding kernel: nothing here touches global memory
     if (tid == 0) {
         for (int st = 0; st < kStreamStages; ++st) {
             asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(full_bar(st)) : "memory");
@@ -635,6 +629,13 @@ __global__ void __launch_bounds__(kStreamThreads, 2) row_argmax_stream_kernel(co
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
+    pdl_wait();  // the kernel before this one in the stream has completed
+    pdl_launch_dependents();
+    const int n = min(max(a.n_nodes[b], 0), a.max_tt);
+    if (r >= n) return;
+    const float* row = a.logits + b * a.ld_b + r * a.ld_row;
+    const int c_begin = sl * a.cps;
+    const int c_end = min(a.splits, c_begin + a.cps);  // chunks [c_begin, c_end) of this row
 
     if (warp == kScanThreads / 32) {
         // ---- copy-issuing warp: a stage is refilled as soon as every consumer has read it ----------
