@@ -410,6 +410,100 @@ class DeviceWorkload:
         return int(h2d), int(d2h)
 
 
+def measure_widened_rows(dw, w, stream, flush):
+    """Device time of the calls beyond the four of a step (not part of `value`): the level form of the tree
+    expansion, the vocabulary split over two ranks (one rank's calls; the two small all-gathers are the caller's
+    and are not timed) and the controller step.  Each figure is the mean of three cold calls after an L2 flush."""
+    import torch
+    binding = dw.binding
+    B, V, T, MK, MD = dw.B, w.vocab, dw.T, dw.max_k, dw.max_d
+    i32 = dict(dtype=torch.int32, device="cuda")
+    out = {}
+
+    def timed(fn, reps=3):
+        fn()
+        torch.cuda.synchronize()
+        total = 0.0
+        for rep in range(reps):
+            flush.fill_(rep)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            fn()
+            b.record(stream)
+            torch.cuda.synchronize()
+            total += a.elapsed_time(b) * 1e3
+        return total / reps
+
+    dw.reset_prefix()
+    dw.set_params(0)
+    d_max = max(d for (_, d, _) in dw.params[0])
+    tree_out = (dw.tokens, dw.parent, dw.depth, dw.pos, dw.mask, dw.retrieve, dw.n_leaves, dw.n_nodes)
+    # ---- level form: begin, one call per level (the draft model would run in between), finish ----------
+    f_tok, f_par, f_pos, f_idx = (torch.zeros(B, MK, **i32) for _ in range(4))
+    f_mask = torch.zeros(B, MK, 2, dtype=torch.int64, device="cuda")
+    dflat, tflat = dw.d_draft[0].view(-1), dw.d_target[0].view(-1)
+
+    def level_form():
+        binding.resps_tree_expand_begin(dw.ctx, dw.d_steps, B, MK)
+        for j in range(d_max):
+            binding.resps_tree_expand_level(dw.ctx, dw.d_steps, B, j, dflat[j * MK * V:], MD * MK * V, V,
+                                            f_tok, f_par, f_pos, f_idx, f_mask, None)
+        binding.resps_tree_expand_finish(dw.ctx, dw.d_steps, B, dw.d_root[0], *tree_out)
+    out["expand_level_form_us"] = timed(level_form)
+    out["expand_level_form_calls"] = d_max + 2
+    # ---- vocabulary split over two ranks: what rank 0 runs ------------------------------------------------
+    P = 2
+    cols = binding.shard_columns(V, P)
+    ctxs = [binding.Context(w.n_q_heads, w.n_kv_heads, w.head_dim, wd, max_batch=B, max_tt=T, max_k=MK, max_depth=MD)
+            for _, wd in cols]
+    rows = int(binding.load().resps_scan_rows(ctxs[0].handle))
+    d_off = torch.tensor([off for off, _ in cols], **i32)
+    parts = [(torch.zeros(B, rows, MK, device="cuda"), torch.zeros(B, rows, MK, **i32),
+              torch.zeros(B, rows, dtype=torch.float64, device="cuda")) for _ in range(P)]
+    keys = [torch.zeros(B, T, dtype=torch.int64, device="cuda") for _ in range(P)]
+    for p_, (off, wd) in enumerate(cols):          # the other rank's share, outside the timing
+        binding.resps_row_scan_shard(ctxs[p_], dw.d_steps, B, dflat[off:], MD * MK * V, MK * V, V, MD, MK, *parts[p_])
+    all_parts = [torch.stack([parts[p_][i] for p_ in range(P)]) for i in range(3)]
+
+    def sharded_expand():
+        binding.resps_row_scan_shard(ctxs[0], dw.d_steps, B, dflat, MD * MK * V, MK * V, V, MD, MK, *parts[0])
+        binding.resps_tree_expand_merge(ctxs[0], dw.d_steps, B, MD, MK, P, *all_parts, d_off, dw.d_root[0], *tree_out)
+    out["expand_vocab_2way_rank_us"] = timed(sharded_expand)
+    for p_, (off, wd) in enumerate(cols):
+        binding.resps_target_argmax_shard(ctxs[p_], dw.n_nodes, B, tflat[off:], T * V, V, keys[p_])
+    all_keys = torch.stack(keys)
+
+    def sharded_verify():
+        binding.resps_target_argmax_shard(ctxs[0], dw.n_nodes, B, tflat, T * V, V, keys[0])
+        binding.resps_verify_accept_merge(ctxs[0], dw.d_steps, dw.n_nodes, B, P, all_keys, d_off, dw.tokens, dw.parent,
+                                          dw.argmax, dw.path, dw.alen, dw.out_tokens, None)
+    out["verify_vocab_2way_rank_us"] = timed(sharded_verify)
+    for c in ctxs:
+        c.close()
+    # ---- controller step: the [128,128] policy on three hidden layers of the model's width, asked every call ------
+    hidden = w.n_q_heads * w.head_dim
+    actions = torch.tensor(synth.action_space(filtered=True), **i32)
+    A, H, F = actions.shape[0], 128, 3 * hidden
+    g = torch.Generator(device="cuda").manual_seed(1)
+    rnd = lambda *shape: torch.randn(*shape, device="cuda", generator=g)
+    pol = binding.make_policy(rnd(H, F) / F ** 0.5, rnd(H) * 0.1, rnd(H, H) / H ** 0.5, rnd(H) * 0.1, rnd(A, H) * 0.5,
+                              rnd(A) * 0.1, actions)
+    hid = [rnd(B, hidden).bfloat16() for _ in range(3)]
+    c_state = torch.zeros(B, 4, **i32)
+    c_steps = dw.d_steps.clone()
+    c_reward = torch.zeros(B, device="cuda")
+    c_u = torch.full((B,), 0.5, dtype=torch.float64, device="cuda")
+    c_ctx = binding.Context(w.n_q_heads, w.n_kv_heads, w.head_dim, 1024, max_batch=B, max_tt=128, max_k=32, max_depth=8)
+
+    def controller():
+        binding.resps_controller_step(c_ctx, pol, *hid, hidden, B, 1, 0.0, c_u, None, None, c_state, c_steps, c_reward)
+    out["controller_step_us"] = timed(controller)
+    out["controller_step_bytes"] = H * F * 4 + 3 * B * hidden * 2
+    c_ctx.close()
+    dw.reset_prefix()
+    return out
+
+
 def attention_algorithmic(w, Ls, ns):
     """Per launch (one layer, the whole batch): K and V of the L+n visible slots, Q in and O out (bytes);
     4 n Hq (L+n) D flop."""
@@ -614,6 +708,12 @@ def run_ours(args, w):
             b.record(stream)
             torch.cuda.synchronize()
             in_sequence[name + "_us"] = a.elapsed_time(b) * 1e3 / (3 * pool)
+        widened = None
+        if rank == 0:
+            try:
+                widened = measure_widened_rows(dw, w, stream, flush)
+            except Exception as e:  # these figures are extras: the line is printed without them
+                widened = {"error": f"{type(e).__name__}: {e}"}
         V = w.vocab
         phase_bytes["scan"] = float(np.mean([sum((1 + (d - 1) * k) * V * 4 for (_, d, k) in dw.params[i])
                                              for i in range(pool)]))
@@ -724,6 +824,7 @@ def run_ours(args, w):
         "phases": dict(phases, attention_per_layer_us=t_attn),
         "phases_in_sequence": dict(in_sequence, note="one call per pool entry in a replayed graph, back to back: "
                                    "the cost of the call inside a step; `phases` times single cold calls"),
+        "widened_rows": widened,
         "cpu_baseline": cpu, "clocks": clocks, "device_status": status,
     }
     print(json.dumps(line))
