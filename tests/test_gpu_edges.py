@@ -207,6 +207,18 @@ def test_attention_work_list_of_several_rounds(rounds):
     _attention_case([9, 70, 33], 8, 8, 128, [5000, 2500, 7777], cap=8192, seed=rounds, B=3, debug=dbg)
 
 
+@pytest.mark.parametrize("single_units", [0, 100000])
+def test_attention_both_groupings_of_the_work_list(single_units):
+    """The work list cuts a call into single row tiles (both halves of a CTA on one tile) while it is small and
+    into pairs of row tiles otherwise; the test-only override forces each grouping on shapes that take the
+    other one by themselves: a short GQA sequence with several row tiles per KV head, a long one, a ragged batch."""
+    _, binding, _ = _imports()
+    dbg = ((binding.RESPS_DEBUG_ATTN_SINGLE, single_units),)
+    _attention_case(60, 32, 8, 128, 700, cap=1024, seed=11, debug=dbg)
+    _attention_case(96, 16, 2, 128, 6000, cap=6400, seed=12, debug=dbg)
+    _attention_case([16, 80, 47], 8, 2, 128, [300, 4000, 1500], cap=4608, seed=13, B=3, debug=dbg)
+
+
 def test_attention_chain_mask_is_causal():
     n = 100
     _attention_case(n, 8, 2, 128, 50, cap=300, parent=list(range(-1, n - 1)), poison=True)
