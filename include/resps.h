@@ -111,8 +111,8 @@ enum {
     RESPS_DEBUG_ATTN_MIN_TILES = 2, /* fewest 64-key tiles a split of the keys is given (default 2)           */
     RESPS_DEBUG_ATTN_STAGGER = 3,   /* SM cycles the second half of a CTA starts behind the first (default 1000) */
     RESPS_DEBUG_SCAN_SLICES = 4,    /* slices a logits row is cut into by the streaming scan: 0 = its own choice */
-    RESPS_DEBUG_ATTN_SINGLE = 5     /* single row tiles (both halves of a CTA on one tile) while the sum over sequences
-                                       of KV heads x row tiles^2 x key tiles is at most this many per CTA (default 100) */
+    RESPS_DEBUG_ATTN_SINGLE = 5     /* single row tiles (both halves of a CTA on one tile) while no sequence has more
+                                       than this many (row tiles per KV head)^2 x key tiles (default 2000)           */
 };
 int resps_debug_set(resps_ctx* ctx, int key, int value);
 

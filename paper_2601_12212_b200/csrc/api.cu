@@ -179,7 +179,7 @@ int resps_debug_set(resps_ctx* ctx, int key, int value) {
     switch (key) {
         case RESPS_DEBUG_ATTN_ROUNDS: w.attn_rounds = std::max(0, value); break;
         case RESPS_DEBUG_ATTN_MIN_TILES: w.attn_min_tiles = std::max(1, value); break;
-        case RESPS_DEBUG_ATTN_SINGLE: w.attn_single = std::min(1 << 16, std::max(0, value)); break;
+        case RESPS_DEBUG_ATTN_SINGLE: w.attn_single = std::min(1 << 26, std::max(0, value)); break;
         case RESPS_DEBUG_ATTN_STAGGER: w.attn_stagger = std::min(100000, std::max(0, value)); break;
         case RESPS_DEBUG_SCAN_SLICES: w.scan_slices_hint = std::max(0, value); break;
 #ifdef RESPS_WAIT_TEST

@@ -106,7 +106,7 @@ struct AttnArgs {
     int max_items;
     int sched_grid;   // CTAs of the attention grid (the work list is balanced for it)
     int min_tiles;    // smallest key-tile count worth a split of its own
-    int single_units; // single row tiles while sum(Hkv tiles^2 key tiles) is at most this many per CTA of the grid
+    int single_units; // single row tiles while no sequence has more than this many (row tiles)^2 x key tiles
     int rounds;       // 0: the work list chooses its number of rounds; 1..kMaxRounds: as told (tests)
     int stagger;      // cycles lane 1 starts behind lane 0 in row mode
     int q_by_tma;     // 1: Q tiles come by TMA (128 % (Hq/Hkv) == 0), 0: by plain loads
@@ -125,16 +125,17 @@ struct AttnArgs {
 // in key mode and costs one.  Every group is cut into splits of at most T units, with the smallest
 // T for which the items fit one round of the grid (found by a short search; steps of 1/16), so
 // that the CTAs finish together whatever the mix of tree sizes and prefix lengths.
-// While the call is small, groups are single row tiles instead, all in key mode: items of half the
-// size fill the grid where row-mode items (at least two key tiles for each of two row tiles) cannot,
-// and the two halves of a CTA merge into one partial; the price is that K and V pass through L2 once
-// per row tile instead of once per pair.  Measured crossover (per-call time against the prefix length,
-// both groupings forced): 2 row tiles per KV head (8B shape, 60 nodes) -- single tiles ahead up to a
-// prefix of 24 000, level at 32 000; 6 row tiles (70B shape, 96 nodes) -- ahead up to 3 000, 1.5 % behind
-// from 4 000.  Both sit near sum over sequences of (KV heads x row tiles^2 x key tiles) = 100 per CTA of
-// the grid, which is the rule (`single_units`).  On the 8B-shaped workload with the prefix growing from
-// 1024 to 3010 this gives 480 us per step, against 510 already at 1837 with the first rule (units <= 2
-// per CTA).
+// Groups are single row tiles instead, all in key mode, while no sequence has many row tiles per KV
+// head over a long prefix: items of half the size fill the grid where row-mode items (at least two key
+// tiles for each of two row tiles) cannot, and the two halves of a CTA merge into one partial; the
+// price is that K and V pass through L2 once per row tile instead of once per pair.  Measured
+// crossovers (per-call time, both groupings forced): 2 row tiles per KV head (8B shape, 60 nodes) --
+// single tiles ahead up to a prefix of 24 000, level at 32 000; 6 row tiles (70B shape, 96 nodes) --
+// ahead up to 3 000, 1.5 % behind from 4 000; ragged batch of 8 with up to 3 row tiles and prefixes up
+// to 8 000 -- ahead by 3 %.  All of them sit near (row tiles)^2 x key tiles = 2000 for the largest
+// sequence, which is the rule (`single_units`).  On the 8B-shaped workload with the prefix growing from
+// 1024 to 3010 this gives 480 us per step, against 510 already at 1837 with the first rule (at most two
+// units of work per CTA).
 struct Sched {
     int group_rows;             // rows of a group: 256 (pairs of row tiles) or 128 (single tiles)
     int n[kMaxBatchSmem];       // tree nodes (0 = sequence skipped)
@@ -162,7 +163,7 @@ __device__ __forceinline__ void build_sched(const AttnArgs& a, Sched& sc, int ti
         // ---- pass 1: sizes, and the cost in row-tile x key-tile units (the same for both groupings:
         // a row-mode pair costs two units per key tile, a single tile one) ----------------------------
         unsigned cost = 0;   // saturates: it only seeds the search below
-        unsigned cost2 = 0;  // the same weighted once more by the row tiles: decides the grouping
+        unsigned cost2 = 0;  // largest (row tiles)^2 x key tiles of a sequence: decides the grouping
 #pragma unroll 1
         for (int i = 0; i < nblk; ++i) {
             const int b = i * 32 + tid;
@@ -177,13 +178,13 @@ __device__ __forceinline__ void build_sched(const AttnArgs& a, Sched& sc, int ti
                 const int kt = (n > 0) ? (L + n + kBN - 1) / kBN : 0;
                 sc.n[b] = n, sc.L[b] = L, sc.kt[b] = kt;
                 cost += min(static_cast<unsigned>(a.Hkv * tiles) * static_cast<unsigned>(kt), 1u << 23);
-                cost2 += min(static_cast<unsigned>(a.Hkv * tiles * tiles) * static_cast<unsigned>(kt), 1u << 23);
+                cost2 = max(cost2, min(static_cast<unsigned>(tiles * tiles) * static_cast<unsigned>(kt), 1u << 26));
             }
         }
         cost = __reduce_add_sync(0xFFFFFFFFu, min(cost, 1u << 26));
-        cost2 = __reduce_add_sync(0xFFFFFFFFu, min(cost2, 1u << 26));
+        cost2 = __reduce_max_sync(0xFFFFFFFFu, cost2);
         // a small call is cut into single row tiles (see above)
-        const bool single = cost2 <= static_cast<unsigned>(a.single_units) * static_cast<unsigned>(a.sched_grid);
+        const bool single = cost2 <= static_cast<unsigned>(a.single_units);
         const int group_rows = single ? kBM : kRowTiles * kBM;
         if (tid == 0) sc.group_rows = group_rows;
 #pragma unroll 1

@@ -47,7 +47,7 @@ struct Workspace {
     int attn_grid = 0;          // persistent CTAs (one per SM)
     int attn_combine_flat_grid = 0;  // ... of its variant for batches
     int attn_min_tiles = 0;     // smallest key-tile count a split is given
-    int attn_single = 100;      // single row tiles while sum(Hkv tiles^2 key tiles) is at most this many per CTA
+    int attn_single = 2000;     // single row tiles while no sequence has more than this many row tiles^2 x key tiles
     int attn_stagger = 1000;    // cycles lane 1 starts behind lane 0 (RESPS_ATTN_STAGGER)
     int attn_rounds = 0;        // 0: chosen by the work list; else forced (RESPS_ATTN_ROUNDS, for tests)
     int attn_max_items = 0;     // partial slots
