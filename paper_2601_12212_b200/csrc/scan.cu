@@ -416,8 +416,10 @@ __global__ void __launch_bounds__(kStreamThreads, 2) row_scan_stream_kernel(cons
         // (branch-free bit mask; the few hits are then re-read from the stage by index)
         uint32_t hits = 0u;
         if (!first) {
+            if (tmax >= tau_v) {  // only a thread whose best logit qualifies has anything to mark
 #pragma unroll
-            for (int i = 0; i < kScanPerThread; ++i) hits |= (v[i] >= tau_v) ? (1u << i) : 0u;
+                for (int i = 0; i < kScanPerThread; ++i) hits |= (v[i] >= tau_v) ? (1u << i) : 0u;
+            }
             if (!consumer_any(hits != 0u)) {
                 release_stage();
                 continue;
